@@ -1,0 +1,187 @@
+/*
+ * shadowsync.h — C boundary of the ShadowSync hot path on one B200 (sm_100a).
+ *
+ * The path is the CTR training step of a DLRM-style model run by R trainer
+ * replicas that live on one GPU (paper Section 3.1, Fig. 1, Algorithm 1) and
+ * the paper's background synchronisation of the replicated dense parameters
+ * (Algorithms 2, 3 and 4).  Every call below enqueues hand-written CUDA kernels
+ * on the stream it is given and returns; nothing here runs on the CPU and there
+ * is no fallback: a device that is not sm_100 gives SS_ERR_ARCH.
+ *
+ * General conventions
+ *   - All data pointers are DEVICE pointers into caller-owned memory unless a
+ *     parameter says "host".  The library allocates nothing and keeps no state
+ *     besides the last CUDA error code and cached driver entry points.
+ *   - Calls validate their arguments on the host, enqueue on `stream`
+ *     (a cudaStream_t passed as void*, 0 = the legacy default stream) and
+ *     return without synchronising.  Buffers must stay alive until the stream
+ *     has run the work.
+ *   - Return value: SS_OK or a negative ss_status.  Nothing aborts; no kernel
+ *     traps.  Malformed *data* seen on the device (an index outside [0,N), a
+ *     decreasing offset) ORs a bit into *d_status and that lookup is skipped.
+ *   - Row-major everywhere.  float = IEEE binary32, bf16 = bfloat16 stored as
+ *     uint16_t.  "ld" = leading dimension in elements.
+ *   - Pointers that are read or written with 128-bit accesses must be 16-byte
+ *     aligned and their ld a multiple of 4 floats / 8 bf16 (SS_ERR_ALIGN).
+ */
+#ifndef SHADOWSYNC_H_
+#define SHADOWSYNC_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef int32_t ss_status;
+enum {
+  SS_OK = 0,
+  SS_ERR_NULL = -1,      /* a required pointer is NULL                                   */
+  SS_ERR_SHAPE = -2,     /* a size is negative, zero where it must not be, or too large  */
+  SS_ERR_ALIGN = -3,     /* pointer or leading dimension not aligned for 128-bit access  */
+  SS_ERR_DTYPE = -4,     /* unsupported gemm_dtype, or a bf16 buffer missing in bf16 mode */
+  SS_ERR_WORKSPACE = -5, /* workspace smaller than the matching *_workspace_bytes query  */
+  SS_ERR_ARCH = -6,      /* current device is not compute capability 10.x                */
+  SS_ERR_CUDA = -7,      /* a CUDA call failed; see ss_last_cuda_error()                 */
+  SS_ERR_RANGE = -8      /* a scalar is outside its domain (alpha not in [0,1], ...)     */
+};
+
+/* bits ORed into *d_status by kernels */
+enum {
+  SS_DEV_BAD_INDEX = 1,  /* a row index outside [0, N): lookup skipped                   */
+  SS_DEV_BAD_OFFSET = 2  /* offsets not non-decreasing or beyond L: bag treated as empty */
+};
+
+typedef void* ss_stream;
+
+const char* ss_status_str(ss_status s);
+int ss_last_cuda_error(void);      /* cudaError_t of the last failed CUDA call of this thread */
+int ss_num_sms(void);              /* multiprocessor count of the current device, <0 on error */
+
+/* ------------------------------------------------------------------------------------------
+ * Embedding lookup + sum pooling (Section 3.1 "Embedding PS": several rows of a feature are
+ * pooled next to the table and only the pooled vector goes to the trainer).
+ *
+ *   out[b, col0 + t*D + d] = sum_{j in [offsets[t*B+b], offsets[t*B+b+1])} tables[t, indices[j], d]
+ *
+ * tables   float [T, N, D]   shared by all replicas (the paper's h)
+ * indices  int32 [L]         row ids, all bags of table 0 first, then table 1, ...
+ * offsets  int32 [T*B + 1]   CSR bag boundaries, bag id = t*B + b, offsets[T*B] = L
+ * out_f32  float [B, ld_f32] nullable; out_bf16 bf16 [B, ld_bf16] nullable; at least one given.
+ *          Both are the replica's concat buffer; col0 is the first pooled column (= D when the
+ *          bottom MLP output occupies columns 0..D-1).
+ * D must be a multiple of 4 and at most 1024.  A row occurring twice in a bag counts twice.
+ * ---------------------------------------------------------------------------------------- */
+ss_status ss_embbag_fwd(const float* tables, int T, int64_t N, int D,
+                        const int32_t* indices, const int32_t* offsets, int B,
+                        float* out_f32, int64_t ld_f32, void* out_bf16, int64_t ld_bf16, int col0,
+                        int32_t* d_status, ss_stream stream);
+
+/* ------------------------------------------------------------------------------------------
+ * Embedding backward fused with the row-wise sparse Adagrad update (Section 3.2 "Embedding
+ * Tables": lock-free updates of the single table copy, optimizer state stored with the rows).
+ * Deterministic: the result does not depend on thread scheduling.
+ *
+ *   1. key = t*N + row for each of the L lookups; stable sort by key
+ *        -> perm[L] (lookup positions, ascending key, equal keys in ascending position)
+ *   2. distinct keys -> uniq_keys[U]; seg_off[U+1] (segment u = perm[seg_off[u] .. seg_off[u+1]))
+ *   3. g_u[d] = sum over the lookups of segment u of grad[b, col0 + t*D + d]  (b = the lookup's sample)
+ *   4. s_u = row_state[key_u] + mean_d g_u[d]^2;  row_state[key_u] = s_u;
+ *      tables[key_u, d] -= lr * g_u[d] / (sqrt(s_u) + eps)
+ *
+ * row_state float [T*N]; grad float [B, ld_grad].  uniq_keys / seg_off / perm are optional
+ * outputs (NULL = keep them in the workspace only); sizes L, L+1, L.  *d_num_unique receives U.
+ * T*N must be below 2^31.  The workspace holds the sort buffers; query its size first.
+ * ---------------------------------------------------------------------------------------- */
+size_t ss_embbag_bwd_workspace_bytes(int T, int64_t N, int D, int B, int64_t L);
+ss_status ss_embbag_bwd_adagrad(float* tables, float* row_state, int T, int64_t N, int D,
+                                const int32_t* indices, const int32_t* offsets, int B, int64_t L,
+                                const float* grad, int64_t ld_grad, int col0, float lr, float eps,
+                                void* workspace, size_t workspace_bytes,
+                                int32_t* uniq_keys, int32_t* seg_off, int32_t* perm,
+                                int32_t* d_num_unique, int32_t* d_status, ss_stream stream);
+
+/* ------------------------------------------------------------------------------------------
+ * Bottom MLP, concat interaction, top MLP, sigmoid + binary cross-entropy (Section 3.1, Fig. 1;
+ * "Trainer": forward pass, then gradients for all parameters, local parameters updated directly).
+ *
+ * ss_mlp_desc (host struct, host int arrays):
+ *   bottom_dims[n_bottom+1]  e.g. {13, 512, 256, 64}: Linear+ReLU for every bottom layer
+ *   top_dims[n_top+1]        e.g. {1728, 512, 256, 1}: Linear+ReLU, the last layer linear -> logit
+ *   top_dims[0] is the concat width W; columns 0..bottom_dims[n_bottom]-1 of the concat buffer are
+ *   the bottom output, the remaining columns are the pooled embeddings written by ss_embbag_fwd.
+ *   gemm_dtype 0: float operands.  1: bf16 operands with float accumulation, float master weights.
+ *
+ * Parameter vector w^(i): ONE flat float array per replica.  Layers in order (bottom first), for
+ * each layer the weight matrix [out, in] row-major, then the bias [out]; every tensor starts on a
+ * multiple of 32 floats (pads are zero and stay zero under all updates).  ss_mlp_param_offsets
+ * writes the start of each tensor.  The Adagrad accumulator, the optional raw-gradient output and
+ * the bf16 mirror (gemm_dtype 1; mirror[k] = bf16(w[k])) share this layout.
+ * ---------------------------------------------------------------------------------------- */
+typedef struct {
+  int n_bottom, n_top;
+  const int* bottom_dims;
+  const int* top_dims;
+  int gemm_dtype;
+} ss_mlp_desc;
+
+int64_t ss_mlp_param_count(const ss_mlp_desc* desc);  /* padded length of the flat vector, <0 on error */
+ss_status ss_mlp_param_offsets(const ss_mlp_desc* desc, int64_t* w_off, int64_t* b_off); /* host arrays [n_bottom+n_top] */
+size_t ss_mlp_workspace_bytes(const ss_mlp_desc* desc, int B);
+
+/* Forward.  dense float [B, bottom_dims[0]]; labels float [B] in {0,1}.
+ * concat_f32 [B, W] (gemm_dtype 0) / concat_bf16 [B, W] (gemm_dtype 1) must already hold the pooled
+ * columns; the call fills columns 0..D0-1.  Outputs: logit[B], prob[B] = sigmoid(logit),
+ * loss[1] = mean_b( max(z,0) - z*y + log(1+exp(-|z|)) ).  The workspace keeps the activations
+ * that ss_mlp_bwd needs: call bwd with the same workspace before the next fwd on it. */
+ss_status ss_mlp_fwd(const ss_mlp_desc* desc, const float* w, const void* w_bf16,
+                     const float* dense, float* concat_f32, void* concat_bf16, int B,
+                     const float* labels, float* logit, float* prob, float* loss,
+                     void* workspace, size_t workspace_bytes, ss_stream stream);
+
+/* Backward + local update.  dz = (prob - y)/B; back-propagation through top and bottom MLP.
+ * grad_pooled float [B, ld_grad] receives d loss / d concat[:, D0:] (column j = concat column D0+j).
+ * grads (nullable) receives the raw dW, db in the flat layout.
+ * If apply_update: element-wise Adagrad on every parameter,
+ *     acc += g*g;  w -= lr * g / (sqrt(acc) + eps);  w_bf16 = bf16(w)   (acc per replica, never synced). */
+ss_status ss_mlp_bwd(const ss_mlp_desc* desc, float* w, void* w_bf16, float* adagrad_acc, float* grads,
+                     const float* dense, const float* concat_f32, const void* concat_bf16,
+                     const float* labels, const float* prob, int B, float lr, float eps, int apply_update,
+                     float* grad_pooled, int64_t ld_grad,
+                     void* workspace, size_t workspace_bytes, ss_stream stream);
+
+/* ------------------------------------------------------------------------------------------
+ * Background synchronisation of the replicated dense parameters (Algorithms 2, 3, 4).  Each call
+ * is ONE kernel that reads all R replica vectors and the centre/global copy once and writes them
+ * back.  w: HOST array of R device pointers to float[n]; w_bf16: NULL or HOST array of R device
+ * pointers to the bf16 mirrors, refreshed from the new values.  1 <= R <= 16, 0 <= alpha <= 1.
+ * The kernels take no lock: run concurrently with training they race with it element by element,
+ * as the paper's shadow thread does with its worker threads (Section 3.2).
+ * ---------------------------------------------------------------------------------------- */
+enum {
+  SS_SYNC_EASGD_LITERAL = 1  /* Algorithm 2 line by line: the replica interpolates toward the updated centre */
+};
+
+/* Shadow EASGD (Algorithm 2), the R trainers visiting the centre in turn, r = 0..R-1:
+ *   d = alpha*(w_r - c);  w_r -= d;  c += d. */
+ss_status ss_sync_easgd(float* const* w, int R, float* center, int64_t n, float alpha, int flags,
+                        void* const* w_bf16, ss_stream stream);
+
+/* Shadow MA (Algorithm 3): m = (1/R) sum_r w_r;  w_r = (1-alpha) w_r + alpha m;  global_out (nullable) = m. */
+ss_status ss_sync_ma(float* const* w, int R, float* global_out, int64_t n, float alpha, int flags,
+                     void* const* w_bf16, ss_stream stream);
+
+/* Shadow BMUF (Algorithm 4) with block momentum: m = mean_r w_r;  delta = mu*delta + eta*(m - g);
+ *   g += delta;  w_r = (1-alpha) w_r + alpha g.   mu = 0 is the algorithm as printed. */
+ss_status ss_sync_bmuf(float* const* w, int R, float* global, float* delta, int64_t n,
+                       float alpha, float eta, float mu, int flags,
+                       void* const* w_bf16, ss_stream stream);
+
+/* float -> bf16 (round to nearest even) of n elements; used to initialise a bf16 mirror. */
+ss_status ss_to_bf16(const float* src, void* dst_bf16, int64_t n, ss_stream stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SHADOWSYNC_H_ */

@@ -1,0 +1,640 @@
+// Embedding-bag forward (sum pooling) and the deterministic backward fused with row-wise Adagrad.
+//
+// Forward: a group of G = D/4 lanes owns one bag; every lane keeps one float4 column slice of the
+// pooled vector in registers and walks the bag's rows with 128-bit loads (rows are D*4 contiguous
+// bytes, so a group reads whole rows, fully coalesced).  Row loads of four lookups are issued
+// together so several gathers are in flight per lane.
+//
+// Backward: (1) keys t*N+row, (2) stable LSD radix sort of (key, position) with a hand-written
+// histogram / scan / ranked-scatter pass per digit, (3) head flags + scan -> unique keys and segment
+// offsets, (4) the sorted lookups are cut into windows of 32 consecutive positions; a lane group
+// sums the gradients of each run of equal keys inside its window in position order.  A run that
+// lies inside one window is final and is updated at once; a run that crosses a window edge leaves a
+// partial sum, and a second kernel adds the partials of such a row in window order and updates it.
+// Work per group is the same whatever the skew of the row distribution, and every sum has a fixed
+// association, so results do not depend on scheduling.
+#include "common.cuh"
+
+namespace ss {
+
+// ======================================================================================
+// forward
+// ======================================================================================
+__device__ __forceinline__ float4 add4(float4 a, float4 b) {
+  return make_float4(a.x + b.x, a.y + b.y, a.z + b.z, a.w + b.w);
+}
+
+__device__ __forceinline__ uint2 bf16x4(float4 v) {
+  __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y);
+  __nv_bfloat162 hi = __floats2bfloat162_rn(v.z, v.w);
+  uint2 r;
+  r.x = *reinterpret_cast<uint32_t*>(&lo);
+  r.y = *reinterpret_cast<uint32_t*>(&hi);
+  return r;
+}
+
+// G lanes per bag (power of two <= 32); NV float4 slices per lane (NV*G*4 >= D).
+template <int G, int NV>
+__global__ void __launch_bounds__(256)
+embbag_fwd_kernel(const float* __restrict__ tables, int T, int64_t N, int D,
+                  const int32_t* __restrict__ indices, const int32_t* __restrict__ offsets, int B,
+                  float* __restrict__ out_f32, int64_t ld_f32,
+                  __nv_bfloat16* __restrict__ out_bf16, int64_t ld_bf16, int col0,
+                  int32_t* __restrict__ d_status) {
+  const int64_t bag = (int64_t)blockIdx.x * (256 / G) + threadIdx.x / G;
+  const int lane = threadIdx.x % G;
+  if (bag >= (int64_t)T * B) return;
+  const int t = (int)(bag / B);
+  const int b = (int)(bag - (int64_t)t * B);
+  int lo = offsets[bag], hi = offsets[bag + 1];
+  int bad = 0;
+  if (lo < 0 || hi < lo) { bad |= SS_DEV_BAD_OFFSET; hi = lo; }
+  const float4* tab = reinterpret_cast<const float4*>(tables + (int64_t)t * N * D);
+  const int nvec = D >> 2;
+
+  float4 acc[NV];
+#pragma unroll
+  for (int v = 0; v < NV; ++v) acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
+
+  for (int j = lo; j < hi; j += 4) {
+    int idx[4];
+    bool ok[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      idx[u] = (j + u < hi) ? indices[j + u] : -1;
+      ok[u] = (idx[u] >= 0) && (idx[u] < N);
+      if (j + u < hi && !ok[u]) bad |= SS_DEV_BAD_INDEX;
+    }
+    float4 rowv[4][NV];
+#pragma unroll
+    for (int u = 0; u < 4; ++u)
+#pragma unroll
+      for (int v = 0; v < NV; ++v) {
+        const int c = lane + v * G;
+        rowv[u][v] = (ok[u] && c < nvec) ? tab[(int64_t)idx[u] * nvec + c] : make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+#pragma unroll
+    for (int u = 0; u < 4; ++u)          // lookups are added in bag order
+#pragma unroll
+      for (int v = 0; v < NV; ++v) acc[v] = add4(acc[v], rowv[u][v]);
+  }
+
+#pragma unroll
+  for (int v = 0; v < NV; ++v) {
+    const int c = lane + v * G;
+    if (c < nvec) {
+      const int64_t col = (int64_t)col0 + (int64_t)t * D + 4 * c;
+      if (out_f32) *reinterpret_cast<float4*>(out_f32 + (int64_t)b * ld_f32 + col) = acc[v];
+      if (out_bf16) *reinterpret_cast<uint2*>(out_bf16 + (int64_t)b * ld_bf16 + col) = bf16x4(acc[v]);
+    }
+  }
+  if (bad && d_status) atomicOr(d_status, bad);
+}
+
+template <int G, int NV>
+static void launch_fwd(const float* tables, int T, int64_t N, int D, const int32_t* indices,
+                       const int32_t* offsets, int B, float* out_f32, int64_t ld_f32, __nv_bfloat16* out_bf16,
+                       int64_t ld_bf16, int col0, int32_t* d_status, cudaStream_t st) {
+  const int64_t bags = (int64_t)T * B;
+  const int per_block = 256 / G;
+  const unsigned blocks = (unsigned)((bags + per_block - 1) / per_block);
+  embbag_fwd_kernel<G, NV><<<blocks, 256, 0, st>>>(tables, T, N, D, indices, offsets, B, out_f32, ld_f32,
+                                                    out_bf16, ld_bf16, col0, d_status);
+}
+
+// ======================================================================================
+// backward: keys, radix sort, unique, windowed segment reduction + row-wise Adagrad
+// ======================================================================================
+constexpr int kSortThreads = 256;
+constexpr int kSortWarps = kSortThreads / 32;
+constexpr int kSortIPT = 16;                              // items per thread
+constexpr int kSortTile = kSortThreads * kSortIPT;        // 4096 items per block
+constexpr int kMaxBins = 512;
+constexpr int kWin = 32;                                  // sorted positions per reduction window
+constexpr int kScanThreads = 1024;
+
+struct BwdPlan {
+  int64_t L;
+  int nblk;          // sort tiles
+  int bits, passes, digit_bits, bins;
+  int nwin;
+  int nblk_u;        // blocks of the unique pass (1024 items each)
+  size_t off_keys_a, off_keys_b, off_pos_a, off_pos_b, off_bag, off_hist, off_usum, off_uniq, off_seg,
+      off_partial, off_scalars, total;
+};
+
+static inline size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
+
+static BwdPlan make_plan(int T, int64_t N, int D, int64_t L) {
+  BwdPlan p{};
+  p.L = L;
+  p.nblk = (int)((L + kSortTile - 1) / kSortTile);
+  if (p.nblk < 1) p.nblk = 1;
+  const uint64_t maxkey = (uint64_t)T * (uint64_t)N;     // sentinel for skipped lookups
+  p.bits = 1;
+  while ((maxkey >> p.bits) != 0) ++p.bits;
+  p.passes = (p.bits + 8) / 9;
+  p.digit_bits = (p.bits + p.passes - 1) / p.passes;
+  p.bins = 1 << p.digit_bits;
+  p.nwin = (int)((L + kWin - 1) / kWin);
+  if (p.nwin < 1) p.nwin = 1;
+  p.nblk_u = (int)((L + kScanThreads - 1) / kScanThreads);
+  if (p.nblk_u < 1) p.nblk_u = 1;
+  size_t o = 0;
+  const size_t l4 = align256((size_t)(L > 0 ? L : 1) * 4);
+  p.off_keys_a = o; o += l4;
+  p.off_keys_b = o; o += l4;
+  p.off_pos_a = o; o += l4;
+  p.off_pos_b = o; o += l4;
+  p.off_bag = o; o += l4;
+  p.off_hist = o; o += align256((size_t)p.nblk * p.bins * 4);
+  p.off_usum = o; o += align256((size_t)(p.nblk_u + 1) * 4);
+  p.off_uniq = o; o += l4;
+  p.off_seg = o; o += align256((size_t)(L + 1) * 4);
+  p.off_partial = o; o += align256((size_t)p.nwin * 2 * (size_t)D * 4);
+  p.off_scalars = o; o += 256;
+  p.total = o;
+  return p;
+}
+
+// ---- (1) keys ---------------------------------------------------------------------------
+// One thread per bag: key = t*N + row for each of its lookups, and the bag id of each position.
+__global__ void __launch_bounds__(256)
+build_keys_kernel(const int32_t* __restrict__ indices, const int32_t* __restrict__ offsets, int T, int64_t N,
+                  int B, int64_t L, uint32_t* __restrict__ keys, int32_t* __restrict__ bag_of,
+                  int32_t* __restrict__ d_status) {
+  const int64_t bag = (int64_t)blockIdx.x * 256 + threadIdx.x;
+  if (bag >= (int64_t)T * B) return;
+  const uint32_t sentinel = (uint32_t)((uint64_t)T * (uint64_t)N);
+  const int t = (int)(bag / B);
+  int lo = offsets[bag], hi = offsets[bag + 1];
+  int bad = 0;
+  if (lo < 0 || hi < lo || hi > L) {
+    // a malformed bag owns no positions; positions nobody owns keep the sentinel written by the fill
+    bad = SS_DEV_BAD_OFFSET;
+    hi = lo = 0;
+  }
+  for (int j = lo; j < hi; ++j) {
+    const int idx = indices[j];
+    uint32_t key = sentinel;
+    if (idx >= 0 && idx < N) key = (uint32_t)((uint64_t)t * (uint64_t)N + (uint64_t)idx);
+    else bad |= SS_DEV_BAD_INDEX;
+    keys[j] = key;
+    bag_of[j] = (int32_t)bag;
+  }
+  if (bad && d_status) atomicOr(d_status, bad);
+}
+
+__global__ void fill_u32_kernel(uint32_t* __restrict__ p, int64_t n, uint32_t v) {
+  int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) p[i] = v;
+}
+
+// ---- (2) radix sort pass ----------------------------------------------------------------
+// hist[bin * nblk + blk] = number of keys of tile blk whose digit is bin.
+__global__ void __launch_bounds__(kSortThreads)
+sort_hist_kernel(const uint32_t* __restrict__ keys, int64_t L, int shift, int bins, int nblk,
+                 uint32_t* __restrict__ hist) {
+  __shared__ uint32_t cnt[kMaxBins];
+  for (int i = threadIdx.x; i < bins; i += kSortThreads) cnt[i] = 0;
+  __syncthreads();
+  const int64_t base = (int64_t)blockIdx.x * kSortTile;
+  const uint32_t mask = (uint32_t)bins - 1u;
+#pragma unroll 4
+  for (int k = 0; k < kSortIPT; ++k) {
+    const int64_t i = base + (int64_t)k * kSortThreads + threadIdx.x;
+    if (i < L) atomicAdd(&cnt[(keys[i] >> shift) & mask], 1u);   // integer counts: order-independent
+  }
+  __syncthreads();
+  for (int i = threadIdx.x; i < bins; i += kSortThreads) hist[(int64_t)i * nblk + blockIdx.x] = cnt[i];
+}
+
+// Exclusive scan of m values in place by one block (m is a few hundred thousand at most).
+__global__ void __launch_bounds__(kScanThreads)
+scan_exclusive_kernel(uint32_t* __restrict__ data, int64_t m, uint32_t* __restrict__ total_out) {
+  __shared__ uint32_t part[kScanThreads];
+  const int64_t chunk = (m + kScanThreads - 1) / kScanThreads;
+  const int64_t lo = (int64_t)threadIdx.x * chunk;
+  const int64_t hi = (lo + chunk < m) ? lo + chunk : m;
+  uint32_t s = 0;
+  for (int64_t i = lo; i < hi; ++i) s += data[i];
+  part[threadIdx.x] = s;
+  __syncthreads();
+  for (int off = 1; off < kScanThreads; off <<= 1) {     // Hillis-Steele inclusive scan of the partials
+    uint32_t v = (threadIdx.x >= off) ? part[threadIdx.x - off] : 0u;
+    __syncthreads();
+    part[threadIdx.x] += v;
+    __syncthreads();
+  }
+  uint32_t run = (threadIdx.x == 0) ? 0u : part[threadIdx.x - 1];
+  for (int64_t i = lo; i < hi; ++i) {
+    const uint32_t v = data[i];
+    data[i] = run;
+    run += v;
+  }
+  if (total_out && threadIdx.x == kScanThreads - 1) *total_out = part[kScanThreads - 1];
+}
+
+// Stable scatter: warp w of the block owns the contiguous items [w*512, (w+1)*512) of the tile and
+// walks them 32 at a time; rank inside a round comes from match_any, across rounds and warps from
+// per-warp running counters that start at the scanned global offset of (digit, tile).
+__global__ void __launch_bounds__(kSortThreads)
+sort_scatter_kernel(const uint32_t* __restrict__ keys_in, const int32_t* __restrict__ pos_in,
+                    uint32_t* __restrict__ keys_out, int32_t* __restrict__ pos_out, int64_t L, int shift,
+                    int bins, int nblk, const uint32_t* __restrict__ hist_scanned) {
+  extern __shared__ uint32_t cnt[];                       // [kSortWarps][bins]
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  for (int i = threadIdx.x; i < kSortWarps * bins; i += kSortThreads) cnt[i] = 0;
+  __syncthreads();
+  const uint32_t mask = (uint32_t)bins - 1u;
+  const int64_t wbase = (int64_t)blockIdx.x * kSortTile + (int64_t)warp * (32 * kSortIPT);
+  uint32_t key[kSortIPT];
+  uint32_t* mycnt = cnt + warp * bins;
+#pragma unroll
+  for (int k = 0; k < kSortIPT; ++k) {
+    const int64_t i = wbase + k * 32 + lane;
+    const bool valid = i < L;
+    key[k] = valid ? keys_in[i] : 0u;
+    const uint32_t digit = valid ? ((key[k] >> shift) & mask) : (uint32_t)bins;   // invalid lanes pair up apart
+    const uint32_t peers = __match_any_sync(0xffffffffu, digit);
+    if (valid && lane == (__ffs(peers) - 1)) mycnt[digit] += __popc(peers);
+    __syncwarp();
+  }
+  __syncthreads();
+  for (int bin = threadIdx.x; bin < bins; bin += kSortThreads) {
+    uint32_t run = hist_scanned[(int64_t)bin * nblk + blockIdx.x];
+#pragma unroll
+    for (int w = 0; w < kSortWarps; ++w) {
+      const uint32_t c = cnt[w * bins + bin];
+      cnt[w * bins + bin] = run;
+      run += c;
+    }
+  }
+  __syncthreads();
+#pragma unroll
+  for (int k = 0; k < kSortIPT; ++k) {
+    const int64_t i = wbase + k * 32 + lane;
+    const bool valid = i < L;
+    const uint32_t digit = valid ? ((key[k] >> shift) & mask) : (uint32_t)bins;
+    const uint32_t peers = __match_any_sync(0xffffffffu, digit);
+    uint32_t dst = 0;
+    if (valid) dst = mycnt[digit] + __popc(peers & ((1u << lane) - 1u));
+    __syncwarp();
+    if (valid && lane == (__ffs(peers) - 1)) mycnt[digit] += __popc(peers);
+    __syncwarp();
+    if (valid) {
+      keys_out[dst] = key[k];
+      pos_out[dst] = pos_in ? pos_in[i] : (int32_t)i;
+    }
+  }
+}
+
+// ---- (3) unique -------------------------------------------------------------------------
+__device__ __forceinline__ bool is_head(const uint32_t* keys, int64_t i, uint32_t sentinel) {
+  const uint32_t k = keys[i];
+  return k < sentinel && (i == 0 || keys[i - 1] != k);
+}
+
+__global__ void __launch_bounds__(kScanThreads)
+unique_count_kernel(const uint32_t* __restrict__ keys, int64_t L, uint32_t sentinel, uint32_t* __restrict__ usum) {
+  const int64_t i = (int64_t)blockIdx.x * kScanThreads + threadIdx.x;
+  const int h = (i < L) && is_head(keys, i, sentinel);
+  const int c = __syncthreads_count(h);
+  if (threadIdx.x == 0) usum[blockIdx.x] = (uint32_t)c;
+}
+
+__global__ void __launch_bounds__(kScanThreads)
+unique_write_kernel(const uint32_t* __restrict__ keys, int64_t L, uint32_t sentinel,
+                    const uint32_t* __restrict__ ubase, int32_t* __restrict__ uniq, int32_t* __restrict__ seg,
+                    int32_t* __restrict__ uniq_out, int32_t* __restrict__ seg_out) {
+  __shared__ uint32_t wsum[32];
+  const int64_t i = (int64_t)blockIdx.x * kScanThreads + threadIdx.x;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const bool in = i < L;
+  const uint32_t k = in ? keys[i] : sentinel;
+  const bool h = in && k < sentinel && (i == 0 || keys[i - 1] != k);
+  const uint32_t ballot = __ballot_sync(0xffffffffu, h);
+  if (lane == 0) wsum[warp] = __popc(ballot);
+  __syncthreads();
+  if (warp == 0) {
+    uint32_t v = wsum[lane];
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+      const uint32_t n = __shfl_up_sync(0xffffffffu, v, off);
+      if (lane >= off) v += n;
+    }
+    wsum[lane] = v;                                        // inclusive over warps
+  }
+  __syncthreads();
+  const uint32_t before = ubase[blockIdx.x] + (warp ? wsum[warp - 1] : 0u) + __popc(ballot & ((1u << lane) - 1u));
+  if (h) {
+    uniq[before] = (int32_t)k;
+    seg[before] = (int32_t)i;
+    if (uniq_out) uniq_out[before] = (int32_t)k;
+    if (seg_out) seg_out[before] = (int32_t)i;
+  }
+  // the last valid position closes the last segment: seg[U] = number of valid lookups
+  if (in && k < sentinel && (i == L - 1 || keys[i + 1] >= sentinel)) {
+    const uint32_t u_end = before + (h ? 1u : 0u);
+    seg[u_end] = (int32_t)(i + 1);
+    if (seg_out) seg_out[u_end] = (int32_t)(i + 1);
+  }
+}
+
+__global__ void unique_finish_kernel(const uint32_t* __restrict__ total, int32_t* __restrict__ seg,
+                                     int32_t* __restrict__ seg_out, int32_t* __restrict__ d_num_unique,
+                                     int32_t* __restrict__ scalars) {
+  const uint32_t U = total ? *total : 0u;
+  if (U == 0) { seg[0] = 0; if (seg_out) seg_out[0] = 0; }
+  if (d_num_unique) *d_num_unique = (int32_t)U;
+  scalars[0] = (int32_t)U;
+}
+
+// ---- (4) windowed reduction + row-wise Adagrad -------------------------------------------
+template <int G, int NV>
+struct RowGrad {
+  float4 v[NV];
+  __device__ __forceinline__ void zero() {
+#pragma unroll
+    for (int i = 0; i < NV; ++i) v[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+  }
+};
+
+// s = state + mean_d g^2;  row -= lr * g / (sqrt(s) + eps).  All G lanes of the group call this.
+template <int G, int NV>
+__device__ __forceinline__ void rowwise_adagrad(const RowGrad<G, NV>& g, uint32_t key, int D, int lane,
+                                                unsigned gmask, float* __restrict__ tables,
+                                                float* __restrict__ row_state, float lr, float eps) {
+  const int nvec = D >> 2;
+  float ss = 0.f;
+#pragma unroll
+  for (int i = 0; i < NV; ++i) {
+    if (lane + i * G < nvec) ss += g.v[i].x * g.v[i].x + g.v[i].y * g.v[i].y + g.v[i].z * g.v[i].z + g.v[i].w * g.v[i].w;
+  }
+#pragma unroll
+  for (int off = G / 2; off >= 1; off >>= 1) ss += __shfl_down_sync(gmask, ss, off, G);
+  ss = __shfl_sync(gmask, ss, 0, G);                       // every lane uses lane 0's sum
+  const float s = row_state[key] + ss / (float)D;
+  const float scale = lr / (sqrtf(s) + eps);
+  float4* row = reinterpret_cast<float4*>(tables + (int64_t)key * D);
+#pragma unroll
+  for (int i = 0; i < NV; ++i) {
+    const int c = lane + i * G;
+    if (c < nvec) {
+      float4 r = row[c];
+      r.x -= scale * g.v[i].x; r.y -= scale * g.v[i].y; r.z -= scale * g.v[i].z; r.w -= scale * g.v[i].w;
+      row[c] = r;
+    }
+  }
+  __syncwarp(gmask);
+  if (lane == 0) row_state[key] = s;
+}
+
+template <int G, int NV>
+__global__ void __launch_bounds__(256)
+window_reduce_kernel(const uint32_t* __restrict__ keys, const int32_t* __restrict__ perm,
+                     const int32_t* __restrict__ bag_of, int64_t L, uint32_t sentinel, int64_t N, int D, int B,
+                     const float* __restrict__ grad, int64_t ld_grad, int col0,
+                     float* __restrict__ tables, float* __restrict__ row_state, float lr, float eps,
+                     float* __restrict__ partial, int nwin) {
+  constexpr int kGroups = 256 / G;
+  __shared__ uint32_t s_key[kGroups][kWin + 2];            // [0] = key before the window, [kWin+1] = key after
+  __shared__ int32_t s_bag[kGroups][kWin];
+  const int grp = threadIdx.x / G, lane = threadIdx.x % G;
+  const int64_t win = (int64_t)blockIdx.x * kGroups + grp;
+  // lanes of a group sit in one warp; mask of this group's lanes
+  const unsigned gmask = (G == 32) ? 0xffffffffu : (((1u << G) - 1u) << ((threadIdx.x & 31) / G * G));
+  if (win >= nwin) return;
+  const int64_t w0 = win * kWin;
+  for (int i = lane; i < kWin + 2; i += G) {
+    const int64_t j = w0 - 1 + i;
+    s_key[grp][i] = (j >= 0 && j < L) ? keys[j] : sentinel;
+  }
+  for (int i = lane; i < kWin; i += G) {
+    const int64_t j = w0 + i;
+    s_bag[grp][i] = (j < L) ? bag_of[perm[j]] : 0;
+  }
+  __syncwarp(gmask);
+  const int nvec = D >> 2;
+  const float4* grad4 = reinterpret_cast<const float4*>(grad + col0);  // col0 multiple of 4
+  const int64_t ld4 = ld_grad >> 2;
+
+  RowGrad<G, NV> acc;
+  acc.zero();
+  int run_start = 0;
+  for (int i0 = 0; i0 < kWin; i0 += 4) {
+    float4 gv[4][NV];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const uint32_t key = s_key[grp][1 + i0 + u];
+      const bool ok = key < sentinel;
+      const int t = ok ? (int)(key / (uint64_t)N) : 0;
+      const int b = s_bag[grp][i0 + u] - t * B;
+#pragma unroll
+      for (int v = 0; v < NV; ++v) {
+        const int c = lane + v * G;
+        gv[u][v] = (ok && c < nvec) ? __ldg(grad4 + (int64_t)b * ld4 + (int64_t)t * nvec + c)
+                                    : make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int i = i0 + u;
+      const uint32_t key = s_key[grp][1 + i];
+      if (key >= sentinel) continue;                       // skipped lookups sort last; nothing follows them
+#pragma unroll
+      for (int v = 0; v < NV; ++v) acc.v[v] = add4(acc.v[v], gv[u][v]);
+      const uint32_t next = s_key[grp][2 + i];
+      const bool last_in_window = (i == kWin - 1);
+      if (next != key || last_in_window) {
+        const bool head_open = (run_start == 0) && (s_key[grp][0] == key);
+        const bool tail_open = (next == key);              // only possible at the window's last position
+        if (!head_open && !tail_open) {
+          rowwise_adagrad<G, NV>(acc, key, D, lane, gmask, tables, row_state, lr, eps);
+        } else {
+          float4* p = reinterpret_cast<float4*>(partial + ((int64_t)win * 2 + (run_start == 0 ? 0 : 1)) * D);
+#pragma unroll
+          for (int v = 0; v < NV; ++v) {
+            const int c = lane + v * G;
+            if (c < nvec) p[c] = acc.v[v];
+          }
+        }
+        acc.zero();
+        run_start = i + 1;
+      }
+    }
+  }
+}
+
+// Rows whose run crosses window edges: add the partial sums in window order, then update.
+template <int G, int NV>
+__global__ void __launch_bounds__(256)
+combine_kernel(const int32_t* __restrict__ uniq, const int32_t* __restrict__ seg, const int32_t* __restrict__ scalars,
+               int D, const float* __restrict__ partial, float* __restrict__ tables, float* __restrict__ row_state,
+               float lr, float eps) {
+  constexpr int kGroups = 256 / G;
+  const int grp = threadIdx.x / G, lane = threadIdx.x % G;
+  const unsigned gmask = (G == 32) ? 0xffffffffu : (((1u << G) - 1u) << ((threadIdx.x & 31) / G * G));
+  const int U = scalars[0];
+  const int nvec = D >> 2;
+  for (int64_t u = (int64_t)blockIdx.x * kGroups + grp; u < U; u += (int64_t)gridDim.x * kGroups) {
+    const int s0 = seg[u], s1 = seg[u + 1];
+    const int k0 = s0 / kWin, k1 = (s1 - 1) / kWin;
+    if (k0 == k1) continue;
+    RowGrad<G, NV> acc;
+    acc.zero();
+    for (int k = k0; k <= k1; ++k) {
+      const int slot = (s0 <= k * kWin) ? 0 : 1;           // the run covers the window's first position -> slot 0
+      const float4* p = reinterpret_cast<const float4*>(partial + ((int64_t)k * 2 + slot) * D);
+#pragma unroll
+      for (int v = 0; v < NV; ++v) {
+        const int c = lane + v * G;
+        if (c < nvec) acc.v[v] = add4(acc.v[v], p[c]);
+      }
+    }
+    rowwise_adagrad<G, NV>(acc, (uint32_t)uniq[u], D, lane, gmask, tables, row_state, lr, eps);
+  }
+}
+
+template <int G, int NV>
+static void launch_reduce(const BwdPlan& p, char* ws, const uint32_t* keys, const int32_t* perm, int T, int64_t N,
+                          int D, int B, const float* grad, int64_t ld_grad, int col0, float* tables,
+                          float* row_state, float lr, float eps, cudaStream_t st) {
+  constexpr int kGroups = 256 / G;
+  const uint32_t sentinel = (uint32_t)((uint64_t)T * (uint64_t)N);
+  float* partial = reinterpret_cast<float*>(ws + p.off_partial);
+  const unsigned blocks = (unsigned)((p.nwin + kGroups - 1) / kGroups);
+  window_reduce_kernel<G, NV><<<blocks, 256, 0, st>>>(keys, perm, reinterpret_cast<int32_t*>(ws + p.off_bag), p.L,
+                                                      sentinel, N, D, B, grad, ld_grad, col0, tables, row_state,
+                                                      lr, eps, partial, p.nwin);
+  const int sms = num_sms();
+  combine_kernel<G, NV><<<sms * 4, 256, 0, st>>>(reinterpret_cast<int32_t*>(ws + p.off_uniq),
+                                                 reinterpret_cast<int32_t*>(ws + p.off_seg),
+                                                 reinterpret_cast<int32_t*>(ws + p.off_scalars), D, partial, tables,
+                                                 row_state, lr, eps);
+}
+
+#define SS_DISPATCH_GNV(D_, CALL)                                                 \
+  do {                                                                            \
+    const int nvec__ = (D_) / 4;                                                  \
+    if (nvec__ <= 4) { CALL(4, 1); }                                              \
+    else if (nvec__ <= 8) { CALL(8, 1); }                                         \
+    else if (nvec__ <= 16) { CALL(16, 1); }                                       \
+    else if (nvec__ <= 32) { CALL(32, 1); }                                       \
+    else if (nvec__ <= 64) { CALL(32, 2); }                                       \
+    else if (nvec__ <= 128) { CALL(32, 4); }                                      \
+    else { CALL(32, 8); }                                                         \
+  } while (0)
+
+}  // namespace ss
+
+extern "C" {
+
+ss_status ss_embbag_fwd(const float* tables, int T, int64_t N, int D, const int32_t* indices,
+                        const int32_t* offsets, int B, float* out_f32, int64_t ld_f32, void* out_bf16,
+                        int64_t ld_bf16, int col0, int32_t* d_status, ss_stream stream) {
+  if (!tables || !indices || !offsets) return SS_ERR_NULL;
+  if (!out_f32 && !out_bf16) return SS_ERR_NULL;
+  if (T < 0 || B < 0 || N <= 0 || D <= 0 || D > 1024 || (D & 3) || col0 < 0) return SS_ERR_SHAPE;
+  if ((uint64_t)T * (uint64_t)N >= (1ull << 31)) return SS_ERR_SHAPE;
+  if (!ss::aligned16(tables) || (col0 & 3)) return SS_ERR_ALIGN;
+  if (out_f32 && (!ss::aligned16(out_f32) || (ld_f32 & 3) || ld_f32 < col0 + (int64_t)T * D)) return SS_ERR_ALIGN;
+  if (out_bf16 && ((reinterpret_cast<uintptr_t>(out_bf16) & 7u) || (ld_bf16 & 3) || ld_bf16 < col0 + (int64_t)T * D))
+    return SS_ERR_ALIGN;
+  ss_status st = ss::check_arch();
+  if (st != SS_OK) return st;
+  if ((int64_t)T * B == 0) return SS_OK;
+  cudaStream_t cs = ss::as_stream(stream);
+#define SS_FWD(G_, NV_)                                                                                     \
+  ss::launch_fwd<G_, NV_>(tables, T, N, D, indices, offsets, B, out_f32, ld_f32, (__nv_bfloat16*)out_bf16, \
+                          ld_bf16, col0, d_status, cs)
+  SS_DISPATCH_GNV(D, SS_FWD);
+#undef SS_FWD
+  SS_LAUNCH_OK();
+  return SS_OK;
+}
+
+size_t ss_embbag_bwd_workspace_bytes(int T, int64_t N, int D, int B, int64_t L) {
+  (void)B;
+  if (T < 0 || N <= 0 || D <= 0 || L < 0) return 0;
+  return ss::make_plan(T, N, D, L).total;
+}
+
+ss_status ss_embbag_bwd_adagrad(float* tables, float* row_state, int T, int64_t N, int D, const int32_t* indices,
+                                const int32_t* offsets, int B, int64_t L, const float* grad, int64_t ld_grad,
+                                int col0, float lr, float eps, void* workspace, size_t workspace_bytes,
+                                int32_t* uniq_keys, int32_t* seg_off, int32_t* perm, int32_t* d_num_unique,
+                                int32_t* d_status, ss_stream stream) {
+  using namespace ss;
+  if (!tables || !row_state || !indices || !offsets || !grad || !workspace) return SS_ERR_NULL;
+  if (T < 0 || B < 0 || N <= 0 || D <= 0 || D > 1024 || (D & 3) || col0 < 0 || L < 0) return SS_ERR_SHAPE;
+  if ((uint64_t)T * (uint64_t)N >= (1ull << 31) || L >= (1ll << 31) - kSortTile) return SS_ERR_SHAPE;
+  if (!aligned16(tables) || !aligned16(grad) || (ld_grad & 3) || (col0 & 3) || !aligned16(workspace)) return SS_ERR_ALIGN;
+  if (ld_grad < col0 + (int64_t)T * D) return SS_ERR_SHAPE;
+  const BwdPlan p = make_plan(T, N, D, L);
+  if (workspace_bytes < p.total) return SS_ERR_WORKSPACE;
+  ss_status stt = check_arch();
+  if (stt != SS_OK) return stt;
+  cudaStream_t cs = as_stream(stream);
+  char* ws = reinterpret_cast<char*>(workspace);
+  uint32_t* keys_a = reinterpret_cast<uint32_t*>(ws + p.off_keys_a);
+  uint32_t* keys_b = reinterpret_cast<uint32_t*>(ws + p.off_keys_b);
+  int32_t* pos_a = reinterpret_cast<int32_t*>(ws + p.off_pos_a);
+  int32_t* pos_b = reinterpret_cast<int32_t*>(ws + p.off_pos_b);
+  int32_t* bag_of = reinterpret_cast<int32_t*>(ws + p.off_bag);
+  uint32_t* hist = reinterpret_cast<uint32_t*>(ws + p.off_hist);
+  uint32_t* usum = reinterpret_cast<uint32_t*>(ws + p.off_usum);
+  int32_t* uniq = reinterpret_cast<int32_t*>(ws + p.off_uniq);
+  int32_t* seg = reinterpret_cast<int32_t*>(ws + p.off_seg);
+  int32_t* scalars = reinterpret_cast<int32_t*>(ws + p.off_scalars);
+  const uint32_t sentinel = (uint32_t)((uint64_t)T * (uint64_t)N);
+
+  if (L == 0 || (int64_t)T * B == 0) {
+    unique_finish_kernel<<<1, 1, 0, cs>>>(nullptr, seg, seg_off, d_num_unique, scalars);
+    SS_LAUNCH_OK();
+    return SS_OK;
+  }
+
+  // (1) keys; positions no bag owns (malformed offsets) keep the sentinel
+  fill_u32_kernel<<<(unsigned)((L + 255) / 256), 256, 0, cs>>>(keys_a, L, sentinel);
+  fill_u32_kernel<<<(unsigned)((L + 255) / 256), 256, 0, cs>>>(reinterpret_cast<uint32_t*>(bag_of), L, 0u);
+  build_keys_kernel<<<(unsigned)(((int64_t)T * B + 255) / 256), 256, 0, cs>>>(indices, offsets, T, N, B, L, keys_a,
+                                                                                bag_of, d_status);
+  SS_LAUNCH_OK();
+
+  // (2) LSD radix sort, `passes` digits of `digit_bits` bits
+  uint32_t* kin = keys_a; uint32_t* kout = keys_b;
+  int32_t* pin = nullptr;  // first pass: position = index
+  int32_t* pout = pos_b;
+  int32_t* pnext = pos_a;
+  const size_t smem = (size_t)kSortWarps * p.bins * 4;
+  for (int pass = 0; pass < p.passes; ++pass) {
+    const int shift = pass * p.digit_bits;
+    sort_hist_kernel<<<p.nblk, kSortThreads, 0, cs>>>(kin, L, shift, p.bins, p.nblk, hist);
+    scan_exclusive_kernel<<<1, kScanThreads, 0, cs>>>(hist, (int64_t)p.nblk * p.bins, nullptr);
+    sort_scatter_kernel<<<p.nblk, kSortThreads, smem, cs>>>(kin, pin, kout, pout, L, shift, p.bins, p.nblk, hist);
+    SS_LAUNCH_OK();
+    uint32_t* tk = kin; kin = kout; kout = tk;
+    pin = pout; pout = pnext; pnext = pin;
+  }
+  const uint32_t* keys_sorted = kin;
+  const int32_t* perm_sorted = pin;
+  if (perm) SS_CUDA(cudaMemcpyAsync(perm, perm_sorted, (size_t)L * 4, cudaMemcpyDeviceToDevice, cs));
+
+  // (3) unique keys and segment offsets
+  unique_count_kernel<<<p.nblk_u, kScanThreads, 0, cs>>>(keys_sorted, L, sentinel, usum);
+  scan_exclusive_kernel<<<1, kScanThreads, 0, cs>>>(usum, p.nblk_u, usum + p.nblk_u);
+  unique_write_kernel<<<p.nblk_u, kScanThreads, 0, cs>>>(keys_sorted, L, sentinel, usum, uniq, seg, uniq_keys, seg_off);
+  unique_finish_kernel<<<1, 1, 0, cs>>>(usum + p.nblk_u, seg, seg_off, d_num_unique, scalars);
+  SS_LAUNCH_OK();
+
+  // (4) windowed segment reduction + row-wise Adagrad
+#define SS_RED(G_, NV_) \
+  launch_reduce<G_, NV_>(p, ws, keys_sorted, perm_sorted, T, N, D, B, grad, ld_grad, col0, tables, row_state, lr, eps, cs)
+  SS_DISPATCH_GNV(D, SS_RED);
+#undef SS_RED
+  SS_LAUNCH_OK();
+  return SS_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,248 @@
+// Bottom MLP -> concat -> top MLP -> sigmoid/BCE, its backward pass and the dense Adagrad update.
+#include "gemm.cuh"
+#include "mlp_plan.cuh"
+
+namespace ss {
+
+// prob = sigmoid(z); loss = mean_b( max(z,0) - z*y + log(1+exp(-|z|)) ); one block, fixed reduction tree.
+__global__ void __launch_bounds__(1024)
+bce_loss_kernel(const float* __restrict__ logit, const float* __restrict__ labels, int B,
+                float* __restrict__ prob, float* __restrict__ loss) {
+  __shared__ float red[1024];
+  float s = 0.f;
+  for (int b = threadIdx.x; b < B; b += 1024) {
+    const float z = logit[b], y = labels[b];
+    const float e = expf(-fabsf(z));
+    prob[b] = (z >= 0.f) ? 1.f / (1.f + e) : e / (1.f + e);
+    s += fmaxf(z, 0.f) - z * y + log1pf(e);
+  }
+  red[threadIdx.x] = s;
+  __syncthreads();
+  for (int off = 512; off >= 1; off >>= 1) {
+    if (threadIdx.x < off) red[threadIdx.x] += red[threadIdx.x + off];
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) loss[0] = red[0] / (float)B;
+}
+
+// dz[b] = (prob[b] - y[b]) / B, stored as float or bf16 (a [B,1] gradient matrix).
+__global__ void dz_kernel(const float* __restrict__ prob, const float* __restrict__ labels, int B, void* __restrict__ dz,
+                          int as_bf16) {
+  const int b = blockIdx.x * blockDim.x + threadIdx.x;
+  if (b >= B) return;
+  const float v = (prob[b] - labels[b]) / (float)B;
+  if (as_bf16) reinterpret_cast<__nv_bfloat16*>(dz)[b] = __float2bfloat16_rn(v);
+  else reinterpret_cast<float*>(dz)[b] = v;
+}
+
+// db[o] = sum_b G[b, o].  Block = 32 columns x 8 row groups; each group adds its rows in ascending
+// order, the 8 partial sums are added in group order.
+__global__ void __launch_bounds__(256)
+bias_grad_kernel(const void* __restrict__ G, int g_bf16, int B, int out, float* __restrict__ db) {
+  __shared__ float part[8][33];
+  const int cx = threadIdx.x & 31, ry = threadIdx.x >> 5;
+  const int o = blockIdx.x * 32 + cx;
+  float s = 0.f;
+  if (o < out) {
+    for (int b = ry; b < B; b += 8) {
+      const int64_t i = (int64_t)b * out + o;
+      s += g_bf16 ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(G)[i]) : reinterpret_cast<const float*>(G)[i];
+    }
+  }
+  part[ry][cx] = s;
+  __syncthreads();
+  if (ry == 0 && o < out) {
+    float t = 0.f;
+#pragma unroll
+    for (int r = 0; r < 8; ++r) t += part[r][cx];
+    db[o] = t;
+  }
+}
+
+// Element-wise Adagrad over the flat parameter vector; refreshes the bf16 mirror.  A zero gradient
+// (pads, dead units) leaves the element untouched.
+__global__ void __launch_bounds__(256)
+adagrad_kernel(float* __restrict__ w, float* __restrict__ acc, const float* __restrict__ g,
+               __nv_bfloat16* __restrict__ mirror, int64_t n4, float lr, float eps) {
+  const int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x;
+  if (i >= n4) return;
+  const float4 gv = reinterpret_cast<const float4*>(g)[i];
+  float4 wv = reinterpret_cast<float4*>(w)[i];
+  float4 av = reinterpret_cast<float4*>(acc)[i];
+#define SS_UPD(F)                                  \
+  if (gv.F != 0.f) {                               \
+    av.F = fmaf(gv.F, gv.F, av.F);                 \
+    wv.F -= lr * gv.F / (sqrtf(av.F) + eps);       \
+  }
+  SS_UPD(x) SS_UPD(y) SS_UPD(z) SS_UPD(w)
+#undef SS_UPD
+  reinterpret_cast<float4*>(w)[i] = wv;
+  reinterpret_cast<float4*>(acc)[i] = av;
+  if (mirror) {
+    __nv_bfloat162 lo = __floats2bfloat162_rn(wv.x, wv.y), hi = __floats2bfloat162_rn(wv.z, wv.w);
+    uint2 r;
+    r.x = *reinterpret_cast<uint32_t*>(&lo);
+    r.y = *reinterpret_cast<uint32_t*>(&hi);
+    reinterpret_cast<uint2*>(mirror)[i] = r;
+  }
+}
+
+static ss_status check_common(const MlpPlan& p, int B, const void* concat_f32, const void* concat_bf16,
+                              const void* w_bf16, void* ws, size_t ws_bytes) {
+  if (B < 1) return SS_ERR_SHAPE;
+  if (!ws) return SS_ERR_NULL;
+  if (p.bf16 && (!concat_bf16 || !w_bf16)) return SS_ERR_DTYPE;
+  if (!p.bf16 && !concat_f32) return SS_ERR_NULL;
+  if (!aligned16(ws) || (concat_f32 && !aligned16(concat_f32)) || (concat_bf16 && !aligned16(concat_bf16)) ||
+      (w_bf16 && !aligned16(w_bf16)))
+    return SS_ERR_ALIGN;
+  if (ws_bytes < p.total) return SS_ERR_WORKSPACE;
+  return check_arch();
+}
+
+}  // namespace ss
+
+extern "C" {
+
+int64_t ss_mlp_param_count(const ss_mlp_desc* desc) {
+  ss::MlpPlan p;
+  if (ss::make_mlp_plan(desc, 0, &p) != SS_OK) return -1;
+  return p.P;
+}
+
+ss_status ss_mlp_param_offsets(const ss_mlp_desc* desc, int64_t* w_off, int64_t* b_off) {
+  if (!w_off || !b_off) return SS_ERR_NULL;
+  ss::MlpPlan p;
+  ss_status st = ss::make_mlp_plan(desc, 0, &p);
+  if (st != SS_OK) return st;
+  for (int l = 0; l < p.nl; ++l) { w_off[l] = p.layer[l].w_off; b_off[l] = p.layer[l].b_off; }
+  return SS_OK;
+}
+
+size_t ss_mlp_workspace_bytes(const ss_mlp_desc* desc, int B) {
+  ss::MlpPlan p;
+  if (ss::make_mlp_plan(desc, B, &p) != SS_OK) return 0;
+  return p.total;
+}
+
+ss_status ss_mlp_fwd(const ss_mlp_desc* desc, const float* w, const void* w_bf16, const float* dense,
+                     float* concat_f32, void* concat_bf16, int B, const float* labels, float* logit, float* prob,
+                     float* loss, void* workspace, size_t workspace_bytes, ss_stream stream) {
+  using namespace ss;
+  if (!w || !dense || !labels || !logit || !prob || !loss) return SS_ERR_NULL;
+  MlpPlan p;
+  ss_status st = make_mlp_plan(desc, B, &p);
+  if (st != SS_OK) return st;
+  st = check_common(p, B, concat_f32, concat_bf16, w_bf16, workspace, workspace_bytes);
+  if (st != SS_OK) return st;
+  if (!aligned16(w)) return SS_ERR_ALIGN;
+  cudaStream_t cs = as_stream(stream);
+  char* ws = reinterpret_cast<char*>(workspace);
+  const int act_kind = p.bf16 ? OP_BF16 : OP_F32;
+
+  for (int l = 0; l < p.nl; ++l) {
+    const LayerInfo& L = p.layer[l];
+    Operand A, Bm;
+    if (l == 0) A = Operand{dense, p.bf16 ? OP_F32_ROUND_BF16 : OP_F32, p.n_dense, 1};
+    else if (l == p.nb) A = Operand{p.bf16 ? (const void*)concat_bf16 : (const void*)concat_f32, act_kind, p.W, 1};
+    else A = Operand{ws + p.act[l - 1], act_kind, L.in, 1};
+    Bm = p.bf16 ? Operand{reinterpret_cast<const __nv_bfloat16*>(w_bf16) + L.w_off, OP_BF16, L.in, 1}
+                : Operand{w + L.w_off, OP_F32, L.in, 1};
+    Epilogue ep;
+    ep.bias = w + L.b_off;
+    ep.relu = L.relu;
+    ep.lo_cols = L.out;
+    if (l == p.nl - 1) {
+      ep.out_lo = logit; ep.lo_bf16 = 0; ep.ld_lo = 1;
+    } else if (l == p.nb - 1) {
+      ep.out_lo = p.bf16 ? concat_bf16 : (void*)concat_f32; ep.lo_bf16 = p.bf16; ep.ld_lo = p.W;
+      if (p.bf16) { ep.out_lo_t = ws + p.concat_t; ep.ld_lo_t = B; }
+    } else {
+      ep.out_lo = ws + p.act[l]; ep.lo_bf16 = p.bf16; ep.ld_lo = L.out;
+      if (p.bf16) { ep.out_lo_t = ws + p.act_t[l]; ep.ld_lo_t = B; }
+    }
+    st = gemm_simt(B, L.out, L.in, A, Bm, ep, cs);
+    if (st != SS_OK) return st;
+  }
+  bce_loss_kernel<<<1, 1024, 0, cs>>>(logit, labels, B, prob, loss);
+  SS_LAUNCH_OK();
+  return SS_OK;
+}
+
+ss_status ss_mlp_bwd(const ss_mlp_desc* desc, float* w, void* w_bf16, float* adagrad_acc, float* grads,
+                     const float* dense, const float* concat_f32, const void* concat_bf16, const float* labels,
+                     const float* prob, int B, float lr, float eps, int apply_update, float* grad_pooled,
+                     int64_t ld_grad, void* workspace, size_t workspace_bytes, ss_stream stream) {
+  using namespace ss;
+  if (!w || !dense || !labels || !prob || !grad_pooled) return SS_ERR_NULL;
+  if (apply_update && !adagrad_acc) return SS_ERR_NULL;
+  MlpPlan p;
+  ss_status st = make_mlp_plan(desc, B, &p);
+  if (st != SS_OK) return st;
+  st = check_common(p, B, concat_f32, concat_bf16, w_bf16, workspace, workspace_bytes);
+  if (st != SS_OK) return st;
+  if (!aligned16(w) || (adagrad_acc && !aligned16(adagrad_acc)) || (grads && !aligned16(grads)) ||
+      !aligned16(grad_pooled) || (ld_grad & 3))
+    return SS_ERR_ALIGN;
+  if (ld_grad < p.W - p.D0) return SS_ERR_SHAPE;
+  if (!(lr >= 0.f) || !(eps >= 0.f)) return SS_ERR_RANGE;
+  cudaStream_t cs = as_stream(stream);
+  char* ws = reinterpret_cast<char*>(workspace);
+  const int act_kind = p.bf16 ? OP_BF16 : OP_F32;
+  float* g = grads ? grads : reinterpret_cast<float*>(ws + p.grads);
+  SS_CUDA(cudaMemsetAsync(g, 0, (size_t)p.P * 4, cs));   // pads of the flat layout carry zero gradient
+
+  dz_kernel<<<(B + 255) / 256, 256, 0, cs>>>(prob, labels, B, ws + p.dact[p.nl - 1], p.bf16);
+  SS_LAUNCH_OK();
+
+  for (int l = p.nl - 1; l >= 0; --l) {
+    const LayerInfo& L = p.layer[l];
+    const void* G = ws + p.dact[l];
+    // input of layer l
+    Operand X;
+    if (l == 0) X = Operand{dense, p.bf16 ? OP_F32_ROUND_BF16 : OP_F32, 1, p.n_dense};
+    else if (l == p.nb) X = Operand{p.bf16 ? concat_bf16 : (const void*)concat_f32, act_kind, 1, p.W};
+    else X = Operand{ws + p.act[l - 1], act_kind, 1, L.in};
+    // dW[o, i] = sum_b G[b, o] * X[b, i]
+    {
+      Operand A{G, act_kind, 1, L.out};
+      Epilogue ep;
+      ep.out_lo = g + L.w_off; ep.lo_bf16 = 0; ep.ld_lo = L.in; ep.lo_cols = L.in;
+      st = gemm_simt(L.out, L.in, B, A, X, ep, cs);
+      if (st != SS_OK) return st;
+    }
+    bias_grad_kernel<<<(L.out + 31) / 32, 256, 0, cs>>>(G, p.bf16, B, L.out, g + L.b_off);
+    SS_LAUNCH_OK();
+    if (l == 0) break;
+    // dX[b, i] = sum_o G[b, o] * W[o, i], gated by the ReLU of the producing layer
+    {
+      Operand A{G, act_kind, L.out, 1};
+      Operand Wt = p.bf16 ? Operand{reinterpret_cast<const __nv_bfloat16*>(w_bf16) + L.w_off, OP_BF16, 1, L.in}
+                          : Operand{w + L.w_off, OP_F32, 1, L.in};
+      Epilogue ep;
+      ep.mask_bf16 = p.bf16;
+      ep.out_lo = ws + p.dact[l - 1]; ep.lo_bf16 = p.bf16;
+      if (l == p.nb) {
+        ep.mask = p.bf16 ? concat_bf16 : (const void*)concat_f32; ep.ld_mask = p.W; ep.mask_cols = p.D0;
+        ep.ld_lo = p.D0; ep.lo_cols = p.D0;
+        ep.out_hi = grad_pooled; ep.ld_hi = ld_grad;
+      } else {
+        ep.mask = ws + p.act[l - 1]; ep.ld_mask = L.in; ep.mask_cols = L.in;
+        ep.ld_lo = L.in; ep.lo_cols = L.in;
+      }
+      if (p.bf16) { ep.out_lo_t = ws + p.dact_t[l - 1]; ep.ld_lo_t = B; }
+      st = gemm_simt(B, L.in, L.out, A, Wt, ep, cs);
+      if (st != SS_OK) return st;
+    }
+  }
+
+  if (apply_update) {
+    const int64_t n4 = p.P / 4;
+    adagrad_kernel<<<(unsigned)((n4 + 255) / 256), 256, 0, cs>>>(w, adagrad_acc, g,
+                                                                 reinterpret_cast<__nv_bfloat16*>(w_bf16), n4, lr, eps);
+    SS_LAUNCH_OK();
+  }
+  return SS_OK;
+}
+
+}  // extern "C"

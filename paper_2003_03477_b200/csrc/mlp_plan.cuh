@@ -1,0 +1,74 @@
+// Host-side description of one replica's MLP: layer list, flat parameter layout, workspace layout.
+#pragma once
+#include "common.cuh"
+
+namespace ss {
+
+constexpr int kMaxLayers = 16;
+
+struct LayerInfo {
+  int in, out;
+  int64_t w_off, b_off;   // element offsets into the flat parameter vector (multiples of 32)
+  bool relu;              // ReLU after the Linear (all but the last top layer)
+};
+
+struct MlpPlan {
+  int nl, nb;             // layers in total, bottom layers
+  int n_dense, D0, W;     // dense features, bottom output width, concat width
+  bool bf16;
+  LayerInfo layer[kMaxLayers];
+  int64_t P;              // padded parameter count
+  // workspace byte offsets; act[l] = output of layer l ([B,out]), dact[l] = gradient of the loss with
+  // respect to it after the ReLU mask.  The last bottom layer's output lives in the concat buffer and
+  // the last top layer's in logit[], so act[] is unused for those two.
+  size_t act[kMaxLayers], act_t[kMaxLayers], dact[kMaxLayers], dact_t[kMaxLayers];
+  size_t concat_t, w_t, grads, dz, total;
+};
+
+inline int64_t pad32(int64_t x) { return (x + 31) & ~(int64_t)31; }
+
+// Returns SS_OK and fills `p` (workspace offsets for batch B; pass B = 0 when only the layout is wanted).
+inline ss_status make_mlp_plan(const ss_mlp_desc* d, int B, MlpPlan* p) {
+  if (!d || !d->bottom_dims || !d->top_dims) return SS_ERR_NULL;
+  if (d->n_bottom < 1 || d->n_top < 1 || d->n_bottom + d->n_top > kMaxLayers || B < 0) return SS_ERR_SHAPE;
+  if (d->gemm_dtype != 0 && d->gemm_dtype != 1) return SS_ERR_DTYPE;
+  p->nb = d->n_bottom;
+  p->nl = d->n_bottom + d->n_top;
+  p->bf16 = d->gemm_dtype == 1;
+  p->n_dense = d->bottom_dims[0];
+  p->D0 = d->bottom_dims[d->n_bottom];
+  p->W = d->top_dims[0];
+  if (d->top_dims[d->n_top] != 1 || p->W < p->D0 || (p->W & 7) || (p->D0 & 7)) return SS_ERR_SHAPE;
+  int64_t off = 0;
+  for (int l = 0; l < p->nl; ++l) {
+    const int* dims = l < p->nb ? d->bottom_dims + l : d->top_dims + (l - p->nb);
+    LayerInfo& L = p->layer[l];
+    L.in = dims[0];
+    L.out = dims[1];
+    if (L.in < 1 || L.out < 1 || L.in > (1 << 20) || L.out > (1 << 20)) return SS_ERR_SHAPE;
+    // hidden widths feed 128-bit accesses: multiples of 8 (the first input and the logit are exempt)
+    if (l != p->nl - 1 && (L.out & 7)) return SS_ERR_SHAPE;
+    L.relu = l != p->nl - 1;
+    L.w_off = off; off += pad32((int64_t)L.in * L.out);
+    L.b_off = off; off += pad32(L.out);
+  }
+  p->P = off;
+  const size_t es = p->bf16 ? 2 : 4;
+  size_t o = 0;
+  auto take = [&](size_t bytes) { size_t r = o; o += (bytes + 255) & ~(size_t)255; return r; };
+  for (int l = 0; l < p->nl; ++l) {
+    const size_t bytes = (size_t)B * p->layer[l].out * es;
+    p->act[l] = take(bytes);
+    p->dact[l] = take(bytes);
+    p->act_t[l] = p->bf16 ? take(bytes) : 0;
+    p->dact_t[l] = p->bf16 ? take(bytes) : 0;
+  }
+  p->concat_t = p->bf16 ? take((size_t)B * p->W * 2) : 0;
+  p->w_t = p->bf16 ? take((size_t)p->P * 2) : 0;
+  p->grads = take((size_t)p->P * 4);
+  p->dz = take((size_t)B * 4);
+  p->total = o;
+  return SS_OK;
+}
+
+}  // namespace ss

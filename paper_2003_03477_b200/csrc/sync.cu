@@ -1,0 +1,204 @@
+// Background synchronisation kernels: Shadow EASGD, Shadow MA, Shadow BMUF (Algorithms 2, 3, 4).
+//
+// Each rule is one element-wise pass: a thread owns one float4 position, loads that position from
+// all R replicas and from the centre/global copy (R+1 independent 128-bit loads in flight), applies
+// the rule in registers and stores everything back.  Traffic is exactly one read and one write of
+// every vector, which is what bounds the kernel (HBM for vectors beyond L2).  The replica pointers
+// travel in the kernel parameter block, so there is no pointer table in device memory.
+#include "common.cuh"
+
+namespace ss {
+
+constexpr int kMaxR = 16;
+
+struct SyncPtrs {
+  float* w[kMaxR];
+  __nv_bfloat16* m[kMaxR];   // bf16 mirrors, only read when MIRROR
+};
+
+__device__ __forceinline__ uint2 pack_bf16x4(float4 v) {
+  __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y);
+  __nv_bfloat162 hi = __floats2bfloat162_rn(v.z, v.w);
+  uint2 r;
+  r.x = *reinterpret_cast<uint32_t*>(&lo);
+  r.y = *reinterpret_cast<uint32_t*>(&hi);
+  return r;
+}
+
+enum { RULE_EASGD = 0, RULE_EASGD_LITERAL = 1, RULE_MA = 2, RULE_BMUF = 3 };
+
+struct SyncScalars {
+  float alpha, eta, mu, inv_r;
+};
+
+// One scalar position of a rule.  w[0..R) in/out; c = centre (EASGD) or global (BMUF/MA out); dl = BMUF delta.
+template <int RULE, int R>
+__device__ __forceinline__ void apply_rule(float (&w)[R], float& c, float& dl, const SyncScalars& s) {
+  if (RULE == RULE_EASGD) {
+#pragma unroll
+    for (int r = 0; r < R; ++r) {          // trainers visit the centre in turn
+      float d = s.alpha * (w[r] - c);
+      w[r] -= d;
+      c += d;
+    }
+  } else if (RULE == RULE_EASGD_LITERAL) {
+#pragma unroll
+    for (int r = 0; r < R; ++r) {          // Algorithm 2 line by line: centre first, replica toward the new centre
+      c = c + s.alpha * (w[r] - c);
+      w[r] = w[r] + s.alpha * (c - w[r]);
+    }
+  } else {
+    float sum = 0.f;
+#pragma unroll
+    for (int r = 0; r < R; ++r) sum += w[r];
+    float m = sum * s.inv_r;
+    if (RULE == RULE_MA) {
+      c = m;
+    } else {
+      dl = s.mu * dl + s.eta * (m - c);
+      c = c + dl;
+    }
+#pragma unroll
+    for (int r = 0; r < R; ++r) w[r] = w[r] + s.alpha * (c - w[r]);
+  }
+}
+
+template <int RULE, int R, bool MIRROR>
+__global__ void __launch_bounds__(256)
+sync_kernel(SyncPtrs p, float* __restrict__ c, float* __restrict__ delta, int64_t n4, int64_t n, SyncScalars s) {
+  const int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x;
+  constexpr bool kReadC = (RULE != RULE_MA);
+  if (i < n4) {
+    float4 wv[R];
+#pragma unroll
+    for (int r = 0; r < R; ++r) wv[r] = reinterpret_cast<const float4*>(p.w[r])[i];
+    float4 cv = make_float4(0.f, 0.f, 0.f, 0.f), dv = cv;
+    if (kReadC) cv = reinterpret_cast<const float4*>(c)[i];
+    if (RULE == RULE_BMUF) dv = reinterpret_cast<const float4*>(delta)[i];
+
+    float a[R];
+#define SS_LANE(F)                                         \
+    {                                                      \
+      _Pragma("unroll") for (int r = 0; r < R; ++r) a[r] = wv[r].F; \
+      apply_rule<RULE, R>(a, cv.F, dv.F, s);               \
+      _Pragma("unroll") for (int r = 0; r < R; ++r) wv[r].F = a[r]; \
+    }
+    SS_LANE(x) SS_LANE(y) SS_LANE(z) SS_LANE(w)
+#undef SS_LANE
+
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+      reinterpret_cast<float4*>(p.w[r])[i] = wv[r];
+      if (MIRROR) reinterpret_cast<uint2*>(p.m[r])[i] = pack_bf16x4(wv[r]);
+    }
+    if (c != nullptr) reinterpret_cast<float4*>(c)[i] = cv;
+    if (RULE == RULE_BMUF) reinterpret_cast<float4*>(delta)[i] = dv;
+  }
+  // ragged tail (n not a multiple of 4): the first threads of block 0 take one scalar each
+  if (blockIdx.x == 0 && threadIdx.x < (int)(n - n4 * 4)) {
+    const int64_t k = n4 * 4 + threadIdx.x;
+    float a[R];
+#pragma unroll
+    for (int r = 0; r < R; ++r) a[r] = p.w[r][k];
+    float cs = (kReadC ? c[k] : 0.f), ds = (RULE == RULE_BMUF ? delta[k] : 0.f);
+    apply_rule<RULE, R>(a, cs, ds, s);
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+      p.w[r][k] = a[r];
+      if (MIRROR) p.m[r][k] = __float2bfloat16_rn(a[r]);
+    }
+    if (c != nullptr) c[k] = cs;
+    if (RULE == RULE_BMUF) delta[k] = ds;
+  }
+}
+
+template <int RULE, int R>
+static ss_status launch_r(const SyncPtrs& p, bool mirror, float* c, float* delta, int64_t n,
+                          const SyncScalars& s, cudaStream_t st) {
+  const int64_t n4 = n / 4;
+  int64_t blocks = (n4 + 255) / 256;
+  if (blocks == 0) blocks = 1;
+  if (blocks > 0x7fffffffLL) return SS_ERR_SHAPE;
+  if (mirror)
+    sync_kernel<RULE, R, true><<<(unsigned)blocks, 256, 0, st>>>(p, c, delta, n4, n, s);
+  else
+    sync_kernel<RULE, R, false><<<(unsigned)blocks, 256, 0, st>>>(p, c, delta, n4, n, s);
+  SS_LAUNCH_OK();
+  return SS_OK;
+}
+
+template <int RULE>
+static ss_status launch(int R, const SyncPtrs& p, bool mirror, float* c, float* delta, int64_t n,
+                        const SyncScalars& s, cudaStream_t st) {
+  switch (R) {
+#define SS_CASE(K) case K: return launch_r<RULE, K>(p, mirror, c, delta, n, s, st);
+    SS_CASE(1) SS_CASE(2) SS_CASE(3) SS_CASE(4) SS_CASE(5) SS_CASE(6) SS_CASE(7) SS_CASE(8)
+    SS_CASE(9) SS_CASE(10) SS_CASE(11) SS_CASE(12) SS_CASE(13) SS_CASE(14) SS_CASE(15) SS_CASE(16)
+#undef SS_CASE
+  }
+  return SS_ERR_SHAPE;
+}
+
+static ss_status collect(float* const* w, int R, int64_t n, void* const* w_bf16, float alpha, SyncPtrs* p) {
+  if (!w) return SS_ERR_NULL;
+  if (R < 1 || R > kMaxR || n < 0) return SS_ERR_SHAPE;
+  if (!(alpha >= 0.f && alpha <= 1.f)) return SS_ERR_RANGE;
+  for (int r = 0; r < kMaxR; ++r) { p->w[r] = nullptr; p->m[r] = nullptr; }
+  for (int r = 0; r < R; ++r) {
+    if (!w[r]) return SS_ERR_NULL;
+    if (!aligned16(w[r])) return SS_ERR_ALIGN;
+    p->w[r] = w[r];
+    if (w_bf16) {
+      if (!w_bf16[r]) return SS_ERR_NULL;
+      if ((reinterpret_cast<uintptr_t>(w_bf16[r]) & 7u) != 0) return SS_ERR_ALIGN;
+      p->m[r] = reinterpret_cast<__nv_bfloat16*>(w_bf16[r]);
+    }
+  }
+  return check_arch();
+}
+
+}  // namespace ss
+
+extern "C" {
+
+ss_status ss_sync_easgd(float* const* w, int R, float* center, int64_t n, float alpha, int flags,
+                        void* const* w_bf16, ss_stream stream) {
+  ss::SyncPtrs p;
+  if (!center) return SS_ERR_NULL;
+  ss_status st = ss::collect(w, R, n, w_bf16, alpha, &p);
+  if (st != SS_OK) return st;
+  if (!ss::aligned16(center)) return SS_ERR_ALIGN;
+  if (n == 0) return SS_OK;
+  ss::SyncScalars s{alpha, 0.f, 0.f, 1.f / (float)R};
+  if (flags & SS_SYNC_EASGD_LITERAL)
+    return ss::launch<ss::RULE_EASGD_LITERAL>(R, p, w_bf16 != nullptr, center, nullptr, n, s, ss::as_stream(stream));
+  return ss::launch<ss::RULE_EASGD>(R, p, w_bf16 != nullptr, center, nullptr, n, s, ss::as_stream(stream));
+}
+
+ss_status ss_sync_ma(float* const* w, int R, float* global_out, int64_t n, float alpha, int flags,
+                     void* const* w_bf16, ss_stream stream) {
+  (void)flags;
+  ss::SyncPtrs p;
+  ss_status st = ss::collect(w, R, n, w_bf16, alpha, &p);
+  if (st != SS_OK) return st;
+  if (global_out && !ss::aligned16(global_out)) return SS_ERR_ALIGN;
+  if (n == 0) return SS_OK;
+  ss::SyncScalars s{alpha, 0.f, 0.f, 1.f / (float)R};
+  return ss::launch<ss::RULE_MA>(R, p, w_bf16 != nullptr, global_out, nullptr, n, s, ss::as_stream(stream));
+}
+
+ss_status ss_sync_bmuf(float* const* w, int R, float* global, float* delta, int64_t n,
+                       float alpha, float eta, float mu, int flags, void* const* w_bf16, ss_stream stream) {
+  (void)flags;
+  ss::SyncPtrs p;
+  if (!global || !delta) return SS_ERR_NULL;
+  ss_status st = ss::collect(w, R, n, w_bf16, alpha, &p);
+  if (st != SS_OK) return st;
+  if (!ss::aligned16(global) || !ss::aligned16(delta)) return SS_ERR_ALIGN;
+  if (!(mu >= 0.f && mu < 1.f) || !(eta >= 0.f)) return SS_ERR_RANGE;
+  if (n == 0) return SS_OK;
+  ss::SyncScalars s{alpha, eta, mu, 1.f / (float)R};
+  return ss::launch<ss::RULE_BMUF>(R, p, w_bf16 != nullptr, global, delta, n, s, ss::as_stream(stream));
+}
+
+}  // extern "C"

@@ -1,0 +1,203 @@
+"""Host-side schedule of the ShadowSync hot path on one GPU (Algorithm 1).
+
+R trainer replicas live on the device as separate buffers.  Each replica owns a high-priority CUDA
+stream on which its training step is enqueued (four library calls: embedding forward, MLP forward,
+MLP backward + dense Adagrad, embedding backward + row-wise Adagrad).  The shadow thread of the
+paper (Section 3.2) is a host thread that keeps enqueuing one synchronisation kernel after another
+on a separate lowest-priority stream; it shares no event or dependency with the training streams.
+
+This module allocates torch tensors and calls the binding; it computes nothing itself.
+"""
+from __future__ import annotations
+
+import threading
+import time
+from typing import List, Optional, Sequence
+
+import numpy as np
+import torch
+
+from . import binding as ss
+
+
+class DeviceBatch:
+    """One batch resident on the device."""
+
+    def __init__(self, indices, offsets, dense, labels, device="cuda"):
+        def dev(a, dt):
+            if isinstance(a, torch.Tensor):
+                return a.to(device=device, dtype=dt, non_blocking=True)
+            return torch.from_numpy(np.ascontiguousarray(a)).to(device=device, dtype=dt)
+        self.indices = dev(indices, torch.int32)
+        self.offsets = dev(offsets, torch.int32)
+        self.dense = dev(dense, torch.float32)
+        self.labels = dev(labels, torch.float32)
+        self.L = int(self.indices.numel())
+
+
+class Replica:
+    """Buffers of one trainer replica: w^(i), its Adagrad accumulator, bf16 mirror, activations, stream."""
+
+    def __init__(self, model: "Model", w0_flat: torch.Tensor, priority: int, max_L: int, keep_sort_outputs: bool):
+        m, dev = model, model.device
+        B, spec = m.B, m.spec
+        self.w = w0_flat.clone()
+        self.acc = torch.zeros_like(self.w)
+        self.w_bf16 = torch.empty(spec.param_count, dtype=torch.bfloat16, device=dev) if spec.bf16 else None
+        if spec.bf16:
+            ss.ss_to_bf16(self.w, self.w_bf16, spec.param_count)
+        self.concat_f32 = torch.zeros(B, spec.W, dtype=torch.float32, device=dev) if (not spec.bf16 or m.keep_f32_concat) else None
+        self.concat_bf16 = torch.zeros(B, spec.W, dtype=torch.bfloat16, device=dev) if spec.bf16 else None
+        self.logit = torch.empty(B, dtype=torch.float32, device=dev)
+        self.prob = torch.empty(B, dtype=torch.float32, device=dev)
+        self.loss = torch.zeros(1, dtype=torch.float32, device=dev)
+        self.grad_pooled = torch.empty(B, m.T * m.D, dtype=torch.float32, device=dev)
+        self.mlp_ws = torch.empty(ss.ss_mlp_workspace_bytes(spec, B), dtype=torch.uint8, device=dev)
+        self.emb_ws = torch.empty(ss.ss_embbag_bwd_workspace_bytes(m.T, m.N, m.D, B, max_L), dtype=torch.uint8, device=dev)
+        self.num_unique = torch.zeros(1, dtype=torch.int32, device=dev)
+        self.uniq_keys = self.seg_off = self.perm = None
+        if keep_sort_outputs:
+            self.uniq_keys = torch.empty(max_L, dtype=torch.int32, device=dev)
+            self.seg_off = torch.empty(max_L + 1, dtype=torch.int32, device=dev)
+            self.perm = torch.empty(max_L, dtype=torch.int32, device=dev)
+        self.stream = torch.cuda.Stream(device=dev, priority=priority)
+        self.steps_done = 0
+
+
+class Model:
+    """Shared embedding tables h, R replicas of the dense parameters, and the centre/global copy."""
+
+    def __init__(self, T: int, N: int, D: int, B: int, bottom: Sequence[int], top: Sequence[int], bf16: bool,
+                 R: int, w0_flat: torch.Tensor, tables: torch.Tensor, lr: float = 0.01, eps: float = 1e-8,
+                 max_L: int = 0, keep_sort_outputs: bool = False, keep_f32_concat: bool = False, device="cuda"):
+        self.T, self.N, self.D, self.B, self.R = T, N, D, B, R
+        self.lr, self.eps = lr, eps
+        self.device = device
+        self.keep_f32_concat = keep_f32_concat
+        self.spec = ss.MlpSpec(bottom, top, bf16)
+        assert self.spec.W == (1 + T) * D and self.spec.D0 == D, "concat = [bottom_out | T pooled vectors]"
+        assert w0_flat.numel() == self.spec.param_count
+        self.tables = tables                       # float32 [T, N, D]
+        self.row_state = torch.zeros(T * N, dtype=torch.float32, device=device)
+        self.d_status = torch.zeros(1, dtype=torch.int32, device=device)
+        lo, hi = torch.cuda.Stream.priority_range()   # (lowest priority value, highest), e.g. (0, -5)
+        self.prio_low, self.prio_high = lo, hi
+        self.replicas: List[Replica] = [Replica(self, w0_flat, hi, max_L, keep_sort_outputs) for _ in range(R)]
+        self.center = w0_flat.clone()              # w^PS (EASGD) / w^global (MA, BMUF), initialised to w0
+        self.delta = torch.zeros_like(self.center)  # BMUF block momentum
+        self.sync_stream = torch.cuda.Stream(device=device, priority=lo)
+        torch.cuda.synchronize()
+
+    # ---------------------------------------------------------------- training step of one replica
+    def step(self, r: int, batch: DeviceBatch, stream: Optional[torch.cuda.Stream] = None) -> None:
+        """Enqueue one worker iteration of Algorithm 1 for replica r on its stream (no synchronisation)."""
+        rep, sp = self.replicas[r], self.spec
+        s = stream or rep.stream
+        T, N, D, B = self.T, self.N, self.D, self.B
+        ss.ss_embbag_fwd(self.tables, T, N, D, batch.indices, batch.offsets, B, rep.concat_f32, sp.W,
+                         rep.concat_bf16, sp.W, D, self.d_status, s)
+        ss.ss_mlp_fwd(sp, rep.w, rep.w_bf16, batch.dense, rep.concat_f32, rep.concat_bf16, B, batch.labels,
+                      rep.logit, rep.prob, rep.loss, rep.mlp_ws, s)
+        ss.ss_mlp_bwd(sp, rep.w, rep.w_bf16, rep.acc, None, batch.dense, rep.concat_f32, rep.concat_bf16,
+                      batch.labels, rep.prob, B, self.lr, self.eps, 1, rep.grad_pooled, T * D, rep.mlp_ws, s)
+        ss.ss_embbag_bwd_adagrad(self.tables, self.row_state, T, N, D, batch.indices, batch.offsets, B, batch.L,
+                                 rep.grad_pooled, T * D, 0, self.lr, self.eps, rep.emb_ws, rep.uniq_keys,
+                                 rep.seg_off, rep.perm, rep.num_unique, self.d_status, s)
+        rep.steps_done += 1
+
+    # ---------------------------------------------------------------- one synchronisation pass
+    def sync(self, rule: str, alpha: float, eta: float = 1.0, mu: float = 0.0, stream=None, flags: int = 0) -> None:
+        """Enqueue one pass of Algorithm 2 ("easgd"), 3 ("ma") or 4 ("bmuf") over all replicas."""
+        s = stream or self.sync_stream
+        ws = [rep.w for rep in self.replicas]
+        mirrors = [rep.w_bf16 for rep in self.replicas] if self.spec.bf16 else None
+        n = self.spec.param_count
+        if rule == "easgd":
+            ss.ss_sync_easgd(ws, self.center, n, alpha, flags, mirrors, s)
+        elif rule == "ma":
+            ss.ss_sync_ma(ws, self.center, n, alpha, flags, mirrors, s)
+        elif rule == "bmuf":
+            ss.ss_sync_bmuf(ws, self.center, self.delta, n, alpha, eta, mu, flags, mirrors, s)
+        else:
+            raise ValueError(rule)
+
+    def status(self) -> int:
+        return int(self.d_status.item())
+
+
+class ShadowLoop:
+    """The shadow thread: loops the synchronisation on the low-priority stream, unaware of training.
+
+    At most `max_in_flight` sync kernels are queued ahead of the device; `pause_s` > 0 paces the loop.
+    """
+
+    def __init__(self, model: Model, rule: str, alpha: float, eta: float = 1.0, mu: float = 0.0,
+                 max_in_flight: int = 2, pause_s: float = 0.0, max_rounds: int = 1 << 30):
+        self.model, self.rule, self.alpha, self.eta, self.mu = model, rule, alpha, eta, mu
+        self.max_in_flight, self.pause_s, self.max_rounds = max_in_flight, pause_s, max_rounds
+        self.rounds = 0
+        self._stop = threading.Event()
+        self._thread: Optional[threading.Thread] = None
+        self.error: Optional[BaseException] = None
+
+    def _run(self) -> None:
+        try:
+            torch.cuda.set_device(self.model.tables.device)
+            pending: List[torch.cuda.Event] = []
+            while not self._stop.is_set() and self.rounds < self.max_rounds:
+                if len(pending) >= self.max_in_flight:
+                    pending.pop(0).synchronize()
+                self.model.sync(self.rule, self.alpha, self.eta, self.mu)
+                ev = torch.cuda.Event()
+                ev.record(self.model.sync_stream)
+                pending.append(ev)
+                self.rounds += 1
+                if self.pause_s > 0:
+                    time.sleep(self.pause_s)
+            for ev in pending:
+                ev.synchronize()
+        except BaseException as e:  # surfaced by stop()
+            self.error = e
+
+    def start(self) -> "ShadowLoop":
+        self._thread = threading.Thread(target=self._run, name="shadow", daemon=True)
+        self._thread.start()
+        return self
+
+    def stop(self) -> int:
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+        if self.error is not None:
+            raise self.error
+        return self.rounds
+
+
+# ------------------------------------------------------------------------------------------
+def pack_params(spec: ss.MlpSpec, layers) -> np.ndarray:
+    """Per-layer (W [out,in], b [out]) float32 arrays -> the flat padded vector of the library's layout."""
+    flat = np.zeros(spec.param_count, dtype=np.float32)
+    for l, (W, b) in enumerate(layers):
+        fin, fout = spec.layer_dims[l]
+        assert W.shape == (fout, fin) and b.shape == (fout,)
+        flat[spec.w_off[l]: spec.w_off[l] + fin * fout] = W.ravel()
+        flat[spec.b_off[l]: spec.b_off[l] + fout] = b
+    return flat
+
+
+def unpack_params(spec: ss.MlpSpec, flat: np.ndarray):
+    out = []
+    for l, (fin, fout) in enumerate(spec.layer_dims):
+        W = flat[spec.w_off[l]: spec.w_off[l] + fin * fout].reshape(fout, fin).copy()
+        b = flat[spec.b_off[l]: spec.b_off[l] + fout].copy()
+        out.append((W, b))
+    return out
+
+
+def device_tables(cfg, device="cuda") -> torch.Tensor:
+    """Fill the synthetic tables of a workload configuration on the device: float32 [T, N, D]."""
+    from . import synth
+    t = torch.empty(cfg.T, cfg.N, cfg.D, dtype=torch.float32, device=device)
+    ss.ssh_fill_uniform(t, t.numel(), int(synth.table_key(cfg)), 0, float(np.float32(synth.TABLE_HI - synth.TABLE_LO)),
+                        float(np.float32(0.5 * (synth.TABLE_HI + synth.TABLE_LO))))
+    return t

@@ -1,0 +1,26 @@
+"""Shared helpers of the GPU parity tests: tolerance rule, oracle <-> flat-layout conversion."""
+import numpy as np
+
+RTOL_F32 = 1e-5     # pooled embeddings, MLP outputs, updated parameters on the float path
+RTOL_BF16 = 2e-2    # outputs of bf16 GEMMs
+RTOL_SYNC = 1e-6    # outputs of the synchronisation kernels
+
+
+def assert_close(got, want, rtol, what=""):
+    """|got - want| <= rtol * max(|want|, rms(want)) element-wise.
+
+    A pure element-wise relative error is undefined at exact zeros (ReLU outputs, pads) and meaningless
+    for elements far below the tensor's scale, so the tensor's RMS is the floor of the reference scale.
+    """
+    got = np.asarray(got, dtype=np.float64)
+    want = np.asarray(want, dtype=np.float64)
+    assert got.shape == want.shape, (what, got.shape, want.shape)
+    assert np.isfinite(got).all(), f"{what}: non-finite values"
+    rms = float(np.sqrt(np.mean(want * want))) if want.size else 0.0
+    scale = np.maximum(np.abs(want), rms)
+    err = np.abs(got - want)
+    bad = err > rtol * scale + 1e-30
+    if bad.any():
+        i = np.unravel_index(np.argmax(err / (scale + 1e-30)), err.shape)
+        raise AssertionError(f"{what}: {int(bad.sum())}/{bad.size} beyond rtol={rtol}; worst at {i}: "
+                             f"got {got[i]!r} want {want[i]!r} (scale {scale[i]:.3e})")
