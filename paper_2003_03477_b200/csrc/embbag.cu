@@ -566,7 +566,7 @@ ss_status ss_embbag_bwd_adagrad(float* tables, float* row_state, int T, int64_t 
                                 int32_t* uniq_keys, int32_t* seg_off, int32_t* perm, int32_t* d_num_unique,
                                 int32_t* d_status, ss_stream stream) {
   using namespace ss;
-  if (!tables || !row_state || !indices || !offsets || !grad || !workspace) return SS_ERR_NULL;
+  if (!tables || !row_state || (!indices && L > 0) || !offsets || !grad || !workspace) return SS_ERR_NULL;
   if (T < 0 || B < 0 || N <= 0 || D <= 0 || D > 1024 || (D & 3) || col0 < 0 || L < 0) return SS_ERR_SHAPE;
   if ((uint64_t)T * (uint64_t)N >= (1ull << 31) || L >= (1ll << 31) - kSortTile) return SS_ERR_SHAPE;
   if (!aligned16(tables) || !aligned16(grad) || (ld_grad & 3) || (col0 & 3) || !aligned16(workspace)) return SS_ERR_ALIGN;

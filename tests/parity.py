@@ -6,18 +6,20 @@ RTOL_BF16 = 2e-2    # outputs of bf16 GEMMs
 RTOL_SYNC = 1e-6    # outputs of the synchronisation kernels
 
 
-def assert_close(got, want, rtol, what=""):
+def assert_close(got, want, rtol, what="", floor=0.0):
     """|got - want| <= rtol * max(|want|, rms(want)) element-wise.
 
     A pure element-wise relative error is undefined at exact zeros (ReLU outputs, pads) and meaningless
     for elements far below the tensor's scale, so the tensor's RMS is the floor of the reference scale.
+    `floor` raises that floor to the magnitude of the operands when a tensor is too short for its RMS to
+    say anything (rounding error scales with the operands, not with a result that cancelled).
     """
     got = np.asarray(got, dtype=np.float64)
     want = np.asarray(want, dtype=np.float64)
     assert got.shape == want.shape, (what, got.shape, want.shape)
     assert np.isfinite(got).all(), f"{what}: non-finite values"
     rms = float(np.sqrt(np.mean(want * want))) if want.size else 0.0
-    scale = np.maximum(np.abs(want), rms)
+    scale = np.maximum(np.abs(want), max(rms, floor))
     err = np.abs(got - want)
     bad = err > rtol * scale + 1e-30
     if bad.any():

@@ -15,7 +15,7 @@ def _dev(vs):
     return [torch.from_numpy(v.copy()).cuda() for v in vs]
 
 
-def _run(rule, R, n, alpha, eta=1.0, mu=0.0, flags=0, mirror=False, seed=1):
+def _run(rule, R, n, alpha, eta=1.0, mu=0.0, flags=0, mirror=False, seed=1, floor=0.0):
     ws = synth.sync_vectors(n, R, seed)
     c = synth.sync_vectors(n, 1, seed + 100)[0]
     d = synth.sync_vectors(n, 1, seed + 200)[0] if rule == "bmuf" else None
@@ -33,12 +33,12 @@ def _run(rule, R, n, alpha, eta=1.0, mu=0.0, flags=0, mirror=False, seed=1):
         O.sync_bmuf(ws, c, d, alpha, eta, mu)
     torch.cuda.synchronize()
     for r in range(R):
-        assert_close(dw[r].cpu().numpy(), ws[r], RTOL_SYNC, f"{rule} w[{r}]")
+        assert_close(dw[r].cpu().numpy(), ws[r], RTOL_SYNC, f"{rule} w[{r}]", floor)
         if mirror:
             assert torch.equal(mir[r], dw[r].to(torch.bfloat16)), "bf16 mirror must be the rounded new value"
-    assert_close(dc.cpu().numpy(), c, RTOL_SYNC, f"{rule} centre")
+    assert_close(dc.cpu().numpy(), c, RTOL_SYNC, f"{rule} centre", floor)
     if d is not None:
-        assert_close(dd.cpu().numpy(), d, RTOL_SYNC, "bmuf delta")
+        assert_close(dd.cpu().numpy(), d, RTOL_SYNC, "bmuf delta", floor)
     return dw, dc
 
 
@@ -60,8 +60,9 @@ def test_sync_tiny_and_empty():
             w = [torch.zeros(4, device="cuda")]
             ss.ss_sync_easgd(w, torch.zeros(4, device="cuda"), 0, 0.1)
         else:
-            _run("easgd", 2, n, 0.3)
-            _run("bmuf", 2, n, 0.3, 0.5, 0.9)
+            # a handful of elements: the operands' scale (std 0.02) is the reference, not a cancelled result
+            _run("easgd", 2, n, 0.3, floor=0.02)
+            _run("bmuf", 2, n, 0.3, 0.5, 0.9, floor=0.02)
 
 
 def test_easgd_literal_flag():
@@ -85,7 +86,8 @@ def test_alpha_limits_and_invariants_on_device():
     dw = _dev(ws)
     g = torch.zeros(n, device="cuda")
     ss.ss_sync_ma(dw, g, n, 1.0)                          # alpha = 1: every replica becomes the mean
-    assert all(torch.equal(a, g) for a in dw)
+    for a in dw:                                          # (w + 1*(m - w) rounds once more than m itself)
+        assert_close(a.cpu().numpy(), g.cpu().numpy(), RTOL_SYNC, "ma alpha=1")
     # BMUF with mu = 0, eta = 1 equals MA
     a, b = _dev(ws), _dev(ws)
     gg, dl = torch.from_numpy(c.copy()).cuda(), torch.zeros(n, device="cuda")
