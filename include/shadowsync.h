@@ -178,6 +178,22 @@ ss_status ss_sync_bmuf(float* const* w, int R, float* global, float* delta, int6
                        float alpha, float eta, float mu, int flags,
                        void* const* w_bf16, ss_stream stream);
 
+/* ------------------------------------------------------------------------------------------
+ * The tensor-core building block of ss_mlp_fwd / ss_mlp_bwd, exposed for testing and timing:
+ *   C[m, n] = sum_k A(m, k) * B(n, k),  bf16 operands, float accumulation, float C [M, ldc].
+ * a_mn_major = 0: A is stored [M, lda] with k contiguous (activations, weights in the forward pass).
+ * a_mn_major = 1: A is stored [K, lda] with m contiguous (the same buffers read transposed in the
+ * backward pass: dW = dY^T X, dX = dY W).  Likewise for B with n.  lda, ldb multiples of 8, N a
+ * multiple of 8, K >= 16, pointers 16-byte aligned, else SS_ERR_ALIGN.  force_simt = 1 runs the
+ * same product on the SIMT kernel instead (any shape).
+ * ss_device_error returns the device-side error flag (0 = none; k > 0 = the k-th kind of bounded
+ * wait in a tensor-core kernel ran out: 1 producer, 2 MMA issuer, 3 epilogue) after synchronising
+ * the device, and clears it if clear != 0.  A negative value means the flag could not be read.
+ * ---------------------------------------------------------------------------------------- */
+ss_status ss_gemm_bf16(const void* a, int a_mn_major, int64_t lda, const void* b, int b_mn_major, int64_t ldb,
+                       float* c, int64_t ldc, int M, int N, int K, int force_simt, ss_stream stream);
+int ss_device_error(int clear);
+
 /* float -> bf16 (round to nearest even) of n elements; used to initialise a bf16 mirror. */
 ss_status ss_to_bf16(const float* src, void* dst_bf16, int64_t n, ss_stream stream);
 

@@ -25,7 +25,7 @@ SS_SYNC_EASGD_LITERAL = 1
 EXPORTS = ["ss_status_str", "ss_last_cuda_error", "ss_num_sms", "ss_embbag_fwd", "ss_embbag_bwd_workspace_bytes",
            "ss_embbag_bwd_adagrad", "ss_mlp_param_count", "ss_mlp_param_offsets", "ss_mlp_workspace_bytes",
            "ss_mlp_fwd", "ss_mlp_bwd", "ss_sync_easgd", "ss_sync_ma", "ss_sync_bmuf", "ss_to_bf16",
-           "ssh_fill_uniform"]
+           "ss_gemm_bf16", "ss_device_error", "ssh_fill_uniform"]
 
 
 class SsError(RuntimeError):
@@ -76,6 +76,8 @@ def lib() -> C.CDLL:
         L.ss_sync_ma.argtypes = [C.POINTER(vp), i32, vp, i64, f32, i32, C.POINTER(vp), vp]
         L.ss_sync_bmuf.argtypes = [C.POINTER(vp), i32, vp, vp, i64, f32, f32, f32, i32, C.POINTER(vp), vp]
         L.ss_to_bf16.argtypes = [vp, vp, i64, vp]
+        L.ss_gemm_bf16.argtypes = [vp, i32, i64, vp, i32, i64, vp, i64, i32, i32, i32, i32, vp]
+        L.ss_device_error.argtypes = [i32]
         L.ssh_fill_uniform.argtypes = [vp, i64, C.c_uint64, C.c_uint64, f32, f32, vp]
         for name in EXPORTS:
             if name not in ("ss_status_str", "ss_last_cuda_error", "ss_num_sms", "ss_embbag_bwd_workspace_bytes",
@@ -208,6 +210,15 @@ def ss_sync_bmuf(w: Sequence[torch.Tensor], global_, delta, n, alpha, eta, mu, f
                  stream=None) -> None:
     _check("ss_sync_bmuf", lib().ss_sync_bmuf(_ptr_array(w), len(w), _ptr(global_), _ptr(delta), n, alpha, eta, mu,
                                                flags, _ptr_array(w_bf16), _stream(stream)))
+
+
+def ss_gemm_bf16(a, a_mn_major, lda, b, b_mn_major, ldb, c, ldc, M, N, K, force_simt=0, stream=None) -> None:
+    _check("ss_gemm_bf16", lib().ss_gemm_bf16(_ptr(a), int(a_mn_major), lda, _ptr(b), int(b_mn_major), ldb, _ptr(c),
+                                               ldc, M, N, K, int(force_simt), _stream(stream)))
+
+
+def ss_device_error(clear: bool = True) -> int:
+    return lib().ss_device_error(1 if clear else 0)
 
 
 def ss_to_bf16(src, dst_bf16, n, stream=None) -> None:

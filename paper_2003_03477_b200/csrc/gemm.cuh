@@ -25,8 +25,6 @@ struct Epilogue {
   int lo_cols = 0;
   float* out_hi = nullptr;
   int64_t ld_hi = 0;
-  void* out_lo_t = nullptr;     // optional transposed bf16 copy of the out_lo block: [lo_cols, ld_lo_t]
-  int64_t ld_lo_t = 0;
 };
 
 struct Operand {
@@ -37,6 +35,13 @@ struct Operand {
 
 // Any shape, any strides; fp32 FMA accumulation in ascending k.
 ss_status gemm_simt(int M, int N, int K, const Operand& A, const Operand& B, const Epilogue& ep, cudaStream_t st);
+// bf16 operands on the tensor cores (tcgen05); see gemm_tc_eligible for what it accepts.
+bool gemm_tc_eligible(int M, int N, int K, const Operand& A, const Operand& B, const Epilogue& ep);
+ss_status gemm_tc(int M, int N, int K, const Operand& A, const Operand& B, const Epilogue& ep, cudaStream_t st);
+// Tensor cores when eligible, SIMT otherwise.
+ss_status gemm(int M, int N, int K, const Operand& A, const Operand& B, const Epilogue& ep, cudaStream_t st);
+// The device error flag raised by a bounded wait that ran out (0 = none); synchronises the device.
+int read_device_error(bool clear);
 
 __device__ __forceinline__ float epilogue_value(const Epilogue& ep, float v, int64_t m, int n) {
   if (ep.bias) v += ep.bias[n];
@@ -52,9 +57,7 @@ __device__ __forceinline__ float epilogue_value(const Epilogue& ep, float v, int
 __device__ __forceinline__ void epilogue_store(const Epilogue& ep, float v, int64_t m, int n) {
   if (n < ep.lo_cols) {
     if (ep.lo_bf16) {
-      const __nv_bfloat16 h = __float2bfloat16_rn(v);
-      reinterpret_cast<__nv_bfloat16*>(ep.out_lo)[m * ep.ld_lo + n] = h;
-      if (ep.out_lo_t) reinterpret_cast<__nv_bfloat16*>(ep.out_lo_t)[(int64_t)n * ep.ld_lo_t + m] = h;
+      reinterpret_cast<__nv_bfloat16*>(ep.out_lo)[m * ep.ld_lo + n] = __float2bfloat16_rn(v);
     } else {
       reinterpret_cast<float*>(ep.out_lo)[m * ep.ld_lo + n] = v;
     }

@@ -1,0 +1,397 @@
+// bf16 x bf16 -> fp32 GEMM on the 5th-generation tensor cores (tcgen05) of sm_100a.
+//
+//   C[m, n] = sum_k A(m, k) * B(n, k)
+//
+// One CTA computes a 128 x 128 tile.  Warp 0 (one lane) streams 128 x 64 / 64 x 128 operand tiles
+// into a ring of shared-memory stages with TMA (128-byte swizzle); warp 1 (one lane) issues
+// tcgen05.mma (M = 128, N = 128, K = 16, accumulators in tensor memory) and releases stages with
+// tcgen05.commit; warps 2-5 wait for the accumulator, read it with tcgen05.ld (one row per thread)
+// and apply the epilogue (bias, ReLU, ReLU-gradient mask, bf16 / fp32 stores).
+//
+// Either operand may be K-major (k contiguous in memory: the forward pass reads activations [B, in]
+// and weights [out, in] this way) or MN-major (m or n contiguous: the backward pass reads the same
+// buffers transposed, dW = dY^T X and dX = dY W), so no transposed copy of any matrix is ever made.
+// K-major tiles are one TMA box of 128 rows x 64 k; MN-major tiles are two boxes of 64 k x 64 m, the
+// canonical 128-byte-swizzle layouts of the shared-memory matrix descriptor in both cases.
+//
+// Every mbarrier wait is bounded: when it runs out the kernel raises a device error flag, stops
+// waiting, drains, frees its tensor memory and returns; the host reads the flag (ss_device_error).
+#include <cuda.h>
+#include <cudaTypedefs.h>
+#include "gemm.cuh"
+
+namespace ss {
+
+constexpr int kBM = 128, kBN = 128, kBK = 64;
+constexpr int kStages = 5;
+constexpr int kTileBytes = kBM * kBK * 2;                 // 16 KiB per operand tile
+constexpr int kStageBytes = 2 * kTileBytes;
+constexpr int kTcThreads = 192;
+constexpr int kTmemCols = 128;
+constexpr size_t kTcSmem = (size_t)kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr long long kWaitCycles = 400ll * 1000 * 1000;    // ~0.2 s: far beyond any legitimate wait
+constexpr long long kWaitCyclesAborted = 2ll * 1000 * 1000;
+
+__device__ int g_device_error = 0;   // 0 ok; otherwise the code of the first wait that ran out
+
+struct TcParams {
+  int M, N, K;
+  int a_mn, b_mn;          // 1 = MN-major operand
+  Epilogue ep;
+  int* err;
+};
+
+// ---------------------------------------------------------------------------------------- PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok;
+}
+// Bounded wait.  Returns false (and records `code`) when the limit is reached.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* aborted, int* err, int code) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  const long long limit = *aborted ? kWaitCyclesAborted : kWaitCycles;
+  while (!mbar_try_wait(bar, parity)) {
+    if (clock64() - t0 > limit) {
+      *aborted = 1;
+      atomicCAS(err, 0, code);
+      return false;
+    }
+  }
+  return true;
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(x), "r"(y) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr) : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+// Shared-memory matrix descriptor, 128-byte swizzle, descriptor version 1 (sm_100).
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  uint64_t d = (uint64_t)((addr & 0x3FFFFu) >> 4);
+  d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;
+  d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32;
+  d |= 1ull << 46;
+  d |= 2ull << 61;
+  return d;
+}
+
+__device__ __forceinline__ uint32_t pack2(float a, float b) {
+  __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
+  return *reinterpret_cast<uint32_t*>(&h);
+}
+
+// ---------------------------------------------------------------------------------------- kernel
+__global__ void __launch_bounds__(kTcThreads, 1)
+gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, TcParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t tiles = (raw + 1023u) & ~1023u;                 // 1024-byte aligned swizzle atoms
+  uint8_t* gen = smem_raw + (tiles - raw);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(gen + (size_t)kStages * kStageBytes);
+  const uint32_t bar0 = tiles + kStages * kStageBytes;
+  // bars: [0,S) full, [S,2S) empty, [2S] accumulator ready; then tmem base and the abort flag
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kStages + 1);
+  volatile int* aborted = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  auto full = [&](int s) { return bar0 + 8u * s; };
+  auto empty = [&](int s) { return bar0 + 8u * (kStages + s); };
+  const uint32_t acc_bar = bar0 + 8u * (2 * kStages);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int m0 = blockIdx.y * kBM, n0 = blockIdx.x * kBN;
+  const int nk = (p.K + kBK - 1) / kBK;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kStages; ++s) { mbar_init(full(s), 1); mbar_init(empty(s), 1); }
+    mbar_init(acc_bar, 1);
+    *aborted = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(kTmemCols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      for (int kb = 0; kb < nk; ++kb) {
+        const int s = kb % kStages;
+        const uint32_t ph = (kb / kStages) & 1;
+        mbar_wait(empty(s), ph ^ 1u, aborted, p.err, 1);
+        mbar_expect_tx(full(s), kStageBytes);
+        const uint32_t sa = tiles + s * kStageBytes, sb = sa + kTileBytes;
+        const int k0 = kb * kBK;
+        if (p.a_mn) {                       // A stored [K, M]: two boxes of 64 k-rows x 64 m
+          tma_load_2d(sa, &map_a, full(s), m0, k0);
+          tma_load_2d(sa + kTileBytes / 2, &map_a, full(s), m0 + 64, k0);
+        } else {                            // A stored [M, K]: one box of 128 rows x 64 k
+          tma_load_2d(sa, &map_a, full(s), k0, m0);
+        }
+        if (p.b_mn) {
+          tma_load_2d(sb, &map_b, full(s), n0, k0);
+          tma_load_2d(sb + kTileBytes / 2, &map_b, full(s), n0 + 64, k0);
+        } else {
+          tma_load_2d(sb, &map_b, full(s), k0, n0);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      // instruction descriptor: D = f32, A = B = bf16, majors, N >> 3, M >> 4
+      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)p.a_mn << 15) | ((uint32_t)p.b_mn << 16) |
+                             ((uint32_t)(kBN >> 3) << 17) | ((uint32_t)(kBM >> 4) << 24);
+      // K-major: 8-row groups 1024 B apart (SBO), K step of 16 elements = 32 B inside the swizzle span.
+      // MN-major: 64-wide m atoms 8192 B apart (LBO), 8-k groups 1024 B apart (SBO), K step of 16 = 2048 B.
+      const uint32_t a_lbo = p.a_mn ? 8192u : 16u, a_step = p.a_mn ? 2048u : 32u;
+      const uint32_t b_lbo = p.b_mn ? 8192u : 16u, b_step = p.b_mn ? 2048u : 32u;
+      for (int kb = 0; kb < nk; ++kb) {
+        const int s = kb % kStages;
+        const uint32_t ph = (kb / kStages) & 1;
+        mbar_wait(full(s), ph, aborted, p.err, 2);
+        tc_fence_after();
+        const uint32_t sa = tiles + s * kStageBytes, sb = sa + kTileBytes;
+#pragma unroll
+        for (int k = 0; k < kBK / 16; ++k) {
+          const uint64_t ad = smem_desc(sa + k * a_step, a_lbo, 1024u);
+          const uint64_t bd = smem_desc(sb + k * b_step, b_lbo, 1024u);
+          tc_mma(tmem, ad, bd, idesc, (kb > 0 || k > 0) ? 1u : 0u);
+        }
+        tc_commit(empty(s));              // frees the stage when these MMAs have read it
+      }
+      tc_commit(acc_bar);                 // accumulator complete
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue warps 2..5
+    const int q = warp & 3;               // tensor-memory lane quadrant this warp may read
+    const int64_t m = (int64_t)m0 + 32 * q + lane;
+    const bool m_ok = m < p.M;
+    const Epilogue& ep = p.ep;
+    mbar_wait(acc_bar, 0, aborted, p.err, 3);
+    tc_fence_after();
+#pragma unroll 1
+    for (int c = 0; c < kBN / 32; ++c) {
+      const int nb = n0 + 32 * c;
+      if (nb >= p.N) break;
+      uint32_t r[32];
+      tc_ld32(tmem + ((uint32_t)(32 * q) << 16) + (uint32_t)(32 * c), r);
+      float v[32];
+#pragma unroll
+      for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
+      if (ep.bias) {
+#pragma unroll
+        for (int j = 0; j < 32; ++j) if (nb + j < p.N) v[j] += __ldg(ep.bias + nb + j);
+      }
+      if (ep.relu) {
+#pragma unroll
+        for (int j = 0; j < 32; ++j) v[j] = fmaxf(v[j], 0.f);
+      }
+      if (!m_ok) continue;
+#pragma unroll
+      for (int g = 0; g < 4; ++g) {
+        const int n = nb + 8 * g;
+        if (n >= p.N) break;
+        float* x = v + 8 * g;
+        if (ep.mask && n < ep.mask_cols) {                       // bf16 activation of the producing layer
+          const uint4 mk = *reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(ep.mask) + m * ep.ld_mask + n);
+          const uint32_t w[4] = {mk.x, mk.y, mk.z, mk.w};
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            // a bf16 is positive iff its sign bit is clear and it is not zero
+            const uint32_t lo = w[j] & 0xFFFFu, hi = w[j] >> 16;
+            if (!((lo & 0x8000u) == 0 && (lo & 0x7FFFu) != 0)) x[2 * j] = 0.f;
+            if (!((hi & 0x8000u) == 0 && (hi & 0x7FFFu) != 0)) x[2 * j + 1] = 0.f;
+          }
+        }
+        if (n < ep.lo_cols) {
+          if (ep.lo_bf16) {
+            uint4 o;
+            o.x = pack2(x[0], x[1]); o.y = pack2(x[2], x[3]); o.z = pack2(x[4], x[5]); o.w = pack2(x[6], x[7]);
+            *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(ep.out_lo) + m * ep.ld_lo + n) = o;
+          } else {
+            float4* o = reinterpret_cast<float4*>(reinterpret_cast<float*>(ep.out_lo) + m * ep.ld_lo + n);
+            o[0] = make_float4(x[0], x[1], x[2], x[3]);
+            o[1] = make_float4(x[4], x[5], x[6], x[7]);
+          }
+        } else if (ep.out_hi) {
+          float4* o = reinterpret_cast<float4*>(ep.out_hi + m * ep.ld_hi + (n - ep.lo_cols));
+          o[0] = make_float4(x[0], x[1], x[2], x[3]);
+          o[1] = make_float4(x[4], x[5], x[6], x[7]);
+        }
+      }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
+  }
+}
+
+// ---------------------------------------------------------------------------------------- host side
+static PFN_cuTensorMapEncodeTiled_v12000 encode_fn() {
+  static PFN_cuTensorMapEncodeTiled_v12000 fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<PFN_cuTensorMapEncodeTiled_v12000>(p);
+  }
+  return fn;
+}
+
+// bf16 matrix with `inner` contiguous elements per row, `outer` rows, row pitch ld elements.
+static bool make_map(CUtensorMap* map, const void* base, int64_t inner, int64_t outer, int64_t ld, int box_inner,
+                     int box_outer) {
+  PFN_cuTensorMapEncodeTiled_v12000 fn = encode_fn();
+  if (!fn) return false;
+  cuuint64_t dims[2] = {(cuuint64_t)inner, (cuuint64_t)outer};
+  cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
+  cuuint32_t box[2] = {(cuuint32_t)box_inner, (cuuint32_t)box_outer};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
+static int* device_error_ptr() {
+  static int* ptr[64];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  if (!ptr[dev]) {
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_device_error) != cudaSuccess) return nullptr;
+    ptr[dev] = reinterpret_cast<int*>(p);
+  }
+  return ptr[dev];
+}
+
+bool gemm_tc_eligible(int M, int N, int K, const Operand& A, const Operand& B, const Epilogue& ep) {
+  if (A.kind != OP_BF16 || B.kind != OP_BF16) return false;
+  if (M < 1 || N < 8 || K < 16 || (N & 7)) return false;
+  auto ok = [](const Operand& o) {
+    const bool kmaj = o.s_k == 1, mnmaj = o.s_row == 1 && o.s_k != 1;
+    if (!kmaj && !mnmaj) return false;
+    const int64_t ld = kmaj ? o.s_row : o.s_k;
+    return (ld & 7) == 0 && aligned16(o.p);
+  };
+  if (!ok(A) || !ok(B)) return false;
+  if ((ep.lo_cols & 7) || (ep.mask && ((ep.mask_cols & 7) || !ep.mask_bf16 || (ep.ld_mask & 7) || !aligned16(ep.mask))))
+    return false;
+  if (ep.out_lo && (!aligned16(ep.out_lo) || (ep.ld_lo & (ep.lo_bf16 ? 7 : 3)))) return false;
+  if (ep.out_hi && (!aligned16(ep.out_hi) || (ep.ld_hi & 3))) return false;
+  if (ep.lo_cols < N && !ep.out_hi) return false;
+  return true;
+}
+
+ss_status gemm_tc(int M, int N, int K, const Operand& A, const Operand& B, const Epilogue& ep, cudaStream_t st) {
+  static bool attr_set[64];
+  int dev = 0;
+  SS_CUDA(cudaGetDevice(&dev));
+  if (dev >= 0 && dev < 64 && !attr_set[dev]) {
+    SS_CUDA(cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTcSmem));
+    attr_set[dev] = true;
+  }
+  TcParams p;
+  p.M = M; p.N = N; p.K = K;
+  p.a_mn = (A.s_k != 1);
+  p.b_mn = (B.s_k != 1);
+  p.ep = ep;
+  p.err = device_error_ptr();
+  if (!p.err) return SS_ERR_CUDA;
+  alignas(64) CUtensorMap ma, mb;
+  const bool oka = p.a_mn ? make_map(&ma, A.p, M, K, A.s_k, 64, 64) : make_map(&ma, A.p, K, M, A.s_row, 64, kBM);
+  const bool okb = p.b_mn ? make_map(&mb, B.p, N, K, B.s_k, 64, 64) : make_map(&mb, B.p, K, N, B.s_row, 64, kBN);
+  if (!oka || !okb) return SS_ERR_CUDA;
+  dim3 grid((N + kBN - 1) / kBN, (M + kBM - 1) / kBM);
+  gemm_tc_kernel<<<grid, kTcThreads, kTcSmem, st>>>(ma, mb, p);
+  SS_LAUNCH_OK();
+  return SS_OK;
+}
+
+int read_device_error(bool clear) {
+  int* d = device_error_ptr();
+  if (!d) return -1;
+  int v = 0;
+  if (cudaMemcpy(&v, d, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return -1;
+  if (clear && v != 0) {
+    int z = 0;
+    cudaMemcpy(d, &z, sizeof(int), cudaMemcpyHostToDevice);
+  }
+  return v;
+}
+
+ss_status gemm(int M, int N, int K, const Operand& A, const Operand& B, const Epilogue& ep, cudaStream_t st) {
+  if (gemm_tc_eligible(M, N, K, A, B, ep)) return gemm_tc(M, N, K, A, B, ep, st);
+  return gemm_simt(M, N, K, A, B, ep, st);
+}
+
+}  // namespace ss
+
+extern "C" {
+
+int ss_device_error(int clear) { return ss::read_device_error(clear != 0); }
+
+ss_status ss_gemm_bf16(const void* a, int a_mn_major, int64_t lda, const void* b, int b_mn_major, int64_t ldb,
+                       float* c, int64_t ldc, int M, int N, int K, int force_simt, ss_stream stream) {
+  using namespace ss;
+  if (!a || !b || !c) return SS_ERR_NULL;
+  if (M < 1 || N < 1 || K < 1 || lda < 1 || ldb < 1 || ldc < N) return SS_ERR_SHAPE;
+  ss_status stt = check_arch();
+  if (stt != SS_OK) return stt;
+  Operand A{a, OP_BF16, a_mn_major ? 1 : lda, a_mn_major ? lda : 1};
+  Operand B{b, OP_BF16, b_mn_major ? 1 : ldb, b_mn_major ? ldb : 1};
+  Epilogue ep;
+  ep.out_lo = c; ep.lo_bf16 = 0; ep.ld_lo = ldc; ep.lo_cols = N;
+  if (force_simt) return gemm_simt(M, N, K, A, B, ep, as_stream(stream));
+  if (!gemm_tc_eligible(M, N, K, A, B, ep)) return SS_ERR_ALIGN;
+  return gemm_tc(M, N, K, A, B, ep, as_stream(stream));
+}
+
+}  // extern "C"

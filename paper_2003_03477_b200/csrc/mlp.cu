@@ -156,12 +156,10 @@ ss_status ss_mlp_fwd(const ss_mlp_desc* desc, const float* w, const void* w_bf16
       ep.out_lo = logit; ep.lo_bf16 = 0; ep.ld_lo = 1;
     } else if (l == p.nb - 1) {
       ep.out_lo = p.bf16 ? concat_bf16 : (void*)concat_f32; ep.lo_bf16 = p.bf16; ep.ld_lo = p.W;
-      if (p.bf16) { ep.out_lo_t = ws + p.concat_t; ep.ld_lo_t = B; }
     } else {
       ep.out_lo = ws + p.act[l]; ep.lo_bf16 = p.bf16; ep.ld_lo = L.out;
-      if (p.bf16) { ep.out_lo_t = ws + p.act_t[l]; ep.ld_lo_t = B; }
     }
-    st = gemm_simt(B, L.out, L.in, A, Bm, ep, cs);
+    st = gemm(B, L.out, L.in, A, Bm, ep, cs);
     if (st != SS_OK) return st;
   }
   bce_loss_kernel<<<1, 1024, 0, cs>>>(logit, labels, B, prob, loss);
@@ -208,7 +206,7 @@ ss_status ss_mlp_bwd(const ss_mlp_desc* desc, float* w, void* w_bf16, float* ada
       Operand A{G, act_kind, 1, L.out};
       Epilogue ep;
       ep.out_lo = g + L.w_off; ep.lo_bf16 = 0; ep.ld_lo = L.in; ep.lo_cols = L.in;
-      st = gemm_simt(L.out, L.in, B, A, X, ep, cs);
+      st = gemm(L.out, L.in, B, A, X, ep, cs);
       if (st != SS_OK) return st;
     }
     bias_grad_kernel<<<(L.out + 31) / 32, 256, 0, cs>>>(G, p.bf16, B, L.out, g + L.b_off);
@@ -230,8 +228,7 @@ ss_status ss_mlp_bwd(const ss_mlp_desc* desc, float* w, void* w_bf16, float* ada
         ep.mask = ws + p.act[l - 1]; ep.ld_mask = L.in; ep.mask_cols = L.in;
         ep.ld_lo = L.in; ep.lo_cols = L.in;
       }
-      if (p.bf16) { ep.out_lo_t = ws + p.dact_t[l - 1]; ep.ld_lo_t = B; }
-      st = gemm_simt(B, L.in, L.out, A, Wt, ep, cs);
+      st = gemm(B, L.in, L.out, A, Wt, ep, cs);
       if (st != SS_OK) return st;
     }
   }

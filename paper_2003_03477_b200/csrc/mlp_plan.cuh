@@ -21,8 +21,8 @@ struct MlpPlan {
   // workspace byte offsets; act[l] = output of layer l ([B,out]), dact[l] = gradient of the loss with
   // respect to it after the ReLU mask.  The last bottom layer's output lives in the concat buffer and
   // the last top layer's in logit[], so act[] is unused for those two.
-  size_t act[kMaxLayers], act_t[kMaxLayers], dact[kMaxLayers], dact_t[kMaxLayers];
-  size_t concat_t, w_t, grads, dz, total;
+  size_t act[kMaxLayers], dact[kMaxLayers];
+  size_t grads, total;
 };
 
 inline int64_t pad32(int64_t x) { return (x + 31) & ~(int64_t)31; }
@@ -60,13 +60,8 @@ inline ss_status make_mlp_plan(const ss_mlp_desc* d, int B, MlpPlan* p) {
     const size_t bytes = (size_t)B * p->layer[l].out * es;
     p->act[l] = take(bytes);
     p->dact[l] = take(bytes);
-    p->act_t[l] = p->bf16 ? take(bytes) : 0;
-    p->dact_t[l] = p->bf16 ? take(bytes) : 0;
   }
-  p->concat_t = p->bf16 ? take((size_t)B * p->W * 2) : 0;
-  p->w_t = p->bf16 ? take((size_t)p->P * 2) : 0;
   p->grads = take((size_t)p->P * 4);
-  p->dz = take((size_t)B * 4);
   p->total = o;
   return SS_OK;
 }
