@@ -103,7 +103,7 @@ static void launch_fwd(const float* tables, int T, int64_t N, int D, const int32
 }
 
 // ======================================================================================
-// backward: keys, radix sort, unique, windowed segment reduction + row-wise Adagrad
+// backward: keys, radix sort, unique, windowed segment reduction, row-wise Adagrad
 // ======================================================================================
 constexpr int kSortThreads = 256;
 constexpr int kSortWarps = kSortThreads / 32;
@@ -119,8 +119,8 @@ struct BwdPlan {
   int bits, passes, digit_bits, bins;
   int nwin;
   int nblk_u;        // blocks of the unique pass (1024 items each)
-  size_t off_keys_a, off_keys_b, off_pos_a, off_pos_b, off_bag, off_hist, off_usum, off_uniq, off_seg,
-      off_partial, off_scalars, total;
+  size_t off_keys_a, off_keys_b, off_pos_a, off_pos_b, off_bag, off_hist, off_bintot, off_usum, off_uniq, off_seg,
+      off_uidx, off_partial, off_gsum, off_scalars, total;
 };
 
 static inline size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
@@ -148,10 +148,14 @@ static BwdPlan make_plan(int T, int64_t N, int D, int64_t L) {
   p.off_pos_b = o; o += l4;
   p.off_bag = o; o += l4;
   p.off_hist = o; o += align256((size_t)p.nblk * p.bins * 4);
+  p.off_bintot = o; o += align256((size_t)kMaxBins * 4);
   p.off_usum = o; o += align256((size_t)(p.nblk_u + 1) * 4);
   p.off_uniq = o; o += l4;
   p.off_seg = o; o += align256((size_t)(L + 1) * 4);
+  p.off_uidx = o; o += l4;
   p.off_partial = o; o += align256((size_t)p.nwin * 2 * (size_t)D * 4);
+  const uint64_t umax = (uint64_t)L < maxkey ? (uint64_t)L : maxkey;   // distinct rows cannot exceed either
+  p.off_gsum = o; o += align256((size_t)(umax > 0 ? umax : 1) * (size_t)D * 4);
   p.off_scalars = o; o += 256;
   p.total = o;
   return p;
@@ -185,31 +189,60 @@ build_keys_kernel(const int32_t* __restrict__ indices, const int32_t* __restrict
   if (bad && d_status) atomicOr(d_status, bad);
 }
 
-__global__ void fill_u32_kernel(uint32_t* __restrict__ p, int64_t n, uint32_t v) {
+// keys <- sentinel, bag_of <- 0 for all positions (those no well-formed bag owns stay that way)
+__global__ void fill_keys_kernel(uint32_t* __restrict__ keys, int32_t* __restrict__ bag_of, int64_t n, uint32_t v) {
   int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (i < n) p[i] = v;
+  if (i < n) { keys[i] = v; bag_of[i] = 0; }
 }
 
 // ---- (2) radix sort pass ----------------------------------------------------------------
-// hist[bin * nblk + blk] = number of keys of tile blk whose digit is bin.
+// hist[bin * nblk + blk] = number of keys of tile blk whose digit is bin.  Lanes holding the same
+// digit are counted together (match_any), so a hot row does not serialise on one counter.
 __global__ void __launch_bounds__(kSortThreads)
 sort_hist_kernel(const uint32_t* __restrict__ keys, int64_t L, int shift, int bins, int nblk,
                  uint32_t* __restrict__ hist) {
   __shared__ uint32_t cnt[kMaxBins];
   for (int i = threadIdx.x; i < bins; i += kSortThreads) cnt[i] = 0;
   __syncthreads();
+  const int lane = threadIdx.x & 31;
   const int64_t base = (int64_t)blockIdx.x * kSortTile;
   const uint32_t mask = (uint32_t)bins - 1u;
 #pragma unroll 4
   for (int k = 0; k < kSortIPT; ++k) {
     const int64_t i = base + (int64_t)k * kSortThreads + threadIdx.x;
-    if (i < L) atomicAdd(&cnt[(keys[i] >> shift) & mask], 1u);   // integer counts: order-independent
+    const bool valid = i < L;
+    const uint32_t digit = valid ? ((keys[i] >> shift) & mask) : (uint32_t)bins;
+    const uint32_t peers = __match_any_sync(0xffffffffu, digit);
+    if (valid && lane == (__ffs(peers) - 1)) atomicAdd(&cnt[digit], (uint32_t)__popc(peers));  // integer: order-free
   }
   __syncthreads();
   for (int i = threadIdx.x; i < bins; i += kSortThreads) hist[(int64_t)i * nblk + blockIdx.x] = cnt[i];
 }
 
-// Exclusive scan of m values in place by one block (m is a few hundred thousand at most).
+// One warp per bin: exclusive scan of that bin's per-tile counts in place, bin total to bintot[bin].
+__global__ void __launch_bounds__(256)
+bin_scan_kernel(uint32_t* __restrict__ hist, int bins, int nblk, uint32_t* __restrict__ bintot) {
+  const int bin = blockIdx.x * 8 + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  if (bin >= bins) return;
+  uint32_t* row = hist + (int64_t)bin * nblk;
+  uint32_t carry = 0;
+  for (int b0 = 0; b0 < nblk; b0 += 32) {
+    const int b = b0 + lane;
+    const uint32_t v = (b < nblk) ? row[b] : 0u;
+    uint32_t inc = v;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+      const uint32_t n = __shfl_up_sync(0xffffffffu, inc, off);
+      if (lane >= off) inc += n;
+    }
+    if (b < nblk) row[b] = carry + inc - v;
+    carry += __shfl_sync(0xffffffffu, inc, 31);
+  }
+  if (lane == 0) bintot[bin] = carry;
+}
+
+// Exclusive scan of m values in place by one block (m is a few thousand at most).
 __global__ void __launch_bounds__(kScanThreads)
 scan_exclusive_kernel(uint32_t* __restrict__ data, int64_t m, uint32_t* __restrict__ total_out) {
   __shared__ uint32_t part[kScanThreads];
@@ -237,14 +270,34 @@ scan_exclusive_kernel(uint32_t* __restrict__ data, int64_t m, uint32_t* __restri
 
 // Stable scatter: warp w of the block owns the contiguous items [w*512, (w+1)*512) of the tile and
 // walks them 32 at a time; rank inside a round comes from match_any, across rounds and warps from
-// per-warp running counters that start at the scanned global offset of (digit, tile).
+// per-warp running counters that start at (bins before this digit) + (this digit in earlier tiles).
 __global__ void __launch_bounds__(kSortThreads)
 sort_scatter_kernel(const uint32_t* __restrict__ keys_in, const int32_t* __restrict__ pos_in,
                     uint32_t* __restrict__ keys_out, int32_t* __restrict__ pos_out, int64_t L, int shift,
-                    int bins, int nblk, const uint32_t* __restrict__ hist_scanned) {
-  extern __shared__ uint32_t cnt[];                       // [kSortWarps][bins]
+                    int bins, int nblk, const uint32_t* __restrict__ hist_scanned, const uint32_t* __restrict__ bintot) {
+  extern __shared__ uint32_t cnt[];                       // [kSortWarps][bins], then binbase[bins], wtot[8]
+  uint32_t* binbase = cnt + kSortWarps * bins;
+  uint32_t* wtot = binbase + bins;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   for (int i = threadIdx.x; i < kSortWarps * bins; i += kSortThreads) cnt[i] = 0;
+  // exclusive scan of the bin totals (bins <= 512 = 2 per thread)
+  {
+    const int i0 = 2 * threadIdx.x, i1 = i0 + 1;
+    const uint32_t v0 = (i0 < bins) ? bintot[i0] : 0u, v1 = (i1 < bins) ? bintot[i1] : 0u;
+    uint32_t inc = v0 + v1;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+      const uint32_t n = __shfl_up_sync(0xffffffffu, inc, off);
+      if (lane >= off) inc += n;
+    }
+    if (lane == 31) wtot[warp] = inc;
+    __syncthreads();
+    uint32_t wbase = 0;
+    for (int w = 0; w < warp; ++w) wbase += wtot[w];
+    const uint32_t excl = wbase + inc - (v0 + v1);
+    if (i0 < bins) binbase[i0] = excl;
+    if (i1 < bins) binbase[i1] = excl + v0;
+  }
   __syncthreads();
   const uint32_t mask = (uint32_t)bins - 1u;
   const int64_t wbase = (int64_t)blockIdx.x * kSortTile + (int64_t)warp * (32 * kSortIPT);
@@ -262,7 +315,7 @@ sort_scatter_kernel(const uint32_t* __restrict__ keys_in, const int32_t* __restr
   }
   __syncthreads();
   for (int bin = threadIdx.x; bin < bins; bin += kSortThreads) {
-    uint32_t run = hist_scanned[(int64_t)bin * nblk + blockIdx.x];
+    uint32_t run = binbase[bin] + hist_scanned[(int64_t)bin * nblk + blockIdx.x];
 #pragma unroll
     for (int w = 0; w < kSortWarps; ++w) {
       const uint32_t c = cnt[w * bins + bin];
@@ -303,10 +356,11 @@ unique_count_kernel(const uint32_t* __restrict__ keys, int64_t L, uint32_t senti
   if (threadIdx.x == 0) usum[blockIdx.x] = (uint32_t)c;
 }
 
+// uniq[u], seg[u] at the head of every segment; uidx[i] = segment of sorted position i.
 __global__ void __launch_bounds__(kScanThreads)
 unique_write_kernel(const uint32_t* __restrict__ keys, int64_t L, uint32_t sentinel,
                     const uint32_t* __restrict__ ubase, int32_t* __restrict__ uniq, int32_t* __restrict__ seg,
-                    int32_t* __restrict__ uniq_out, int32_t* __restrict__ seg_out) {
+                    int32_t* __restrict__ uidx, int32_t* __restrict__ uniq_out, int32_t* __restrict__ seg_out) {
   __shared__ uint32_t wsum[32];
   const int64_t i = (int64_t)blockIdx.x * kScanThreads + threadIdx.x;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -333,6 +387,7 @@ unique_write_kernel(const uint32_t* __restrict__ keys, int64_t L, uint32_t senti
     if (uniq_out) uniq_out[before] = (int32_t)k;
     if (seg_out) seg_out[before] = (int32_t)i;
   }
+  if (in) uidx[i] = (int32_t)(before + (h ? 1u : 0u)) - 1;
   // the last valid position closes the last segment: seg[U] = number of valid lookups
   if (in && k < sentinel && (i == L - 1 || keys[i + 1] >= sentinel)) {
     const uint32_t u_end = before + (h ? 1u : 0u);
@@ -350,150 +405,156 @@ __global__ void unique_finish_kernel(const uint32_t* __restrict__ total, int32_t
   scalars[0] = (int32_t)U;
 }
 
-// ---- (4) windowed reduction + row-wise Adagrad -------------------------------------------
-template <int G, int NV>
-struct RowGrad {
-  float4 v[NV];
-  __device__ __forceinline__ void zero() {
-#pragma unroll
-    for (int i = 0; i < NV; ++i) v[i] = make_float4(0.f, 0.f, 0.f, 0.f);
-  }
-};
-
-// s = state + mean_d g^2;  row -= lr * g / (sqrt(s) + eps).  All G lanes of the group call this.
-template <int G, int NV>
-__device__ __forceinline__ void rowwise_adagrad(const RowGrad<G, NV>& g, uint32_t key, int D, int lane,
-                                                unsigned gmask, float* __restrict__ tables,
-                                                float* __restrict__ row_state, float lr, float eps) {
-  const int nvec = D >> 2;
-  float ss = 0.f;
-#pragma unroll
-  for (int i = 0; i < NV; ++i) {
-    if (lane + i * G < nvec) ss += g.v[i].x * g.v[i].x + g.v[i].y * g.v[i].y + g.v[i].z * g.v[i].z + g.v[i].w * g.v[i].w;
-  }
-#pragma unroll
-  for (int off = G / 2; off >= 1; off >>= 1) ss += __shfl_down_sync(gmask, ss, off, G);
-  ss = __shfl_sync(gmask, ss, 0, G);                       // every lane uses lane 0's sum
-  const float s = row_state[key] + ss / (float)D;
-  const float scale = lr / (sqrtf(s) + eps);
-  float4* row = reinterpret_cast<float4*>(tables + (int64_t)key * D);
-#pragma unroll
-  for (int i = 0; i < NV; ++i) {
-    const int c = lane + i * G;
-    if (c < nvec) {
-      float4 r = row[c];
-      r.x -= scale * g.v[i].x; r.y -= scale * g.v[i].y; r.z -= scale * g.v[i].z; r.w -= scale * g.v[i].w;
-      row[c] = r;
-    }
-  }
-  __syncwarp(gmask);
-  if (lane == 0) row_state[key] = s;
-}
-
+// ---- (4) windowed segment reduction ---------------------------------------------------------
+// A lane group owns a window of 32 consecutive sorted positions and adds the gradient rows of each
+// run of equal keys in position order.  A run that lies inside the window is complete: its sum goes
+// to gsum[u].  A run that crosses a window edge leaves a partial sum in the window's slot 0 (run
+// covers the window's first position) or slot 1.
 template <int G, int NV>
 __global__ void __launch_bounds__(256)
 window_reduce_kernel(const uint32_t* __restrict__ keys, const int32_t* __restrict__ perm,
-                     const int32_t* __restrict__ bag_of, int64_t L, uint32_t sentinel, int64_t N, int D, int B,
-                     const float* __restrict__ grad, int64_t ld_grad, int col0,
-                     float* __restrict__ tables, float* __restrict__ row_state, float lr, float eps,
-                     float* __restrict__ partial, int nwin) {
+                     const int32_t* __restrict__ bag_of, const int32_t* __restrict__ uidx, int64_t L,
+                     uint32_t sentinel, int64_t N, int D, int B, const float* __restrict__ grad, int64_t ld_grad,
+                     int col0, float* __restrict__ gsum, float* __restrict__ partial, int nwin) {
   constexpr int kGroups = 256 / G;
   __shared__ uint32_t s_key[kGroups][kWin + 2];            // [0] = key before the window, [kWin+1] = key after
-  __shared__ int32_t s_bag[kGroups][kWin];
+  __shared__ int32_t s_row[kGroups][kWin];                 // float4 index of the lookup's gradient row
+  __shared__ int32_t s_u[kGroups][kWin];
   const int grp = threadIdx.x / G, lane = threadIdx.x % G;
   const int64_t win = (int64_t)blockIdx.x * kGroups + grp;
-  // lanes of a group sit in one warp; mask of this group's lanes
   const unsigned gmask = (G == 32) ? 0xffffffffu : (((1u << G) - 1u) << ((threadIdx.x & 31) / G * G));
   if (win >= nwin) return;
   const int64_t w0 = win * kWin;
+  const int nvec = D >> 2;
+  const int64_t ld4 = ld_grad >> 2;
   for (int i = lane; i < kWin + 2; i += G) {
     const int64_t j = w0 - 1 + i;
     s_key[grp][i] = (j >= 0 && j < L) ? keys[j] : sentinel;
   }
   for (int i = lane; i < kWin; i += G) {
     const int64_t j = w0 + i;
-    s_bag[grp][i] = (j < L) ? bag_of[perm[j]] : 0;
+    int32_t row = -1, u = 0;
+    if (j < L) {
+      const uint32_t key = keys[j];
+      if (key < sentinel) {
+        const int t = (int)(key / (uint64_t)N);
+        const int b = bag_of[perm[j]] - t * B;
+        row = (int32_t)((int64_t)b * ld4 + (int64_t)t * nvec);   // B * ld_grad / 4 < 2^31 is checked on the host
+        u = uidx[j];
+      }
+    }
+    s_row[grp][i] = row;
+    s_u[grp][i] = u;
   }
   __syncwarp(gmask);
-  const int nvec = D >> 2;
-  const float4* grad4 = reinterpret_cast<const float4*>(grad + col0);  // col0 multiple of 4
-  const int64_t ld4 = ld_grad >> 2;
+  const float4* grad4 = reinterpret_cast<const float4*>(grad + col0);  // col0 is a multiple of 4
 
-  RowGrad<G, NV> acc;
-  acc.zero();
-  int run_start = 0;
-  for (int i0 = 0; i0 < kWin; i0 += 4) {
-    float4 gv[4][NV];
+  float4 acc[NV];
 #pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      const uint32_t key = s_key[grp][1 + i0 + u];
-      const bool ok = key < sentinel;
-      const int t = ok ? (int)(key / (uint64_t)N) : 0;
-      const int b = s_bag[grp][i0 + u] - t * B;
+  for (int v = 0; v < NV; ++v) acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
+  int run_start = 0;
+  constexpr int kBatch = NV >= 8 ? 1 : (NV >= 4 ? 2 : (NV >= 2 ? 4 : 8));   // gradient rows in flight per lane
+  for (int i0 = 0; i0 < kWin; i0 += kBatch) {
+    float4 gv[kBatch][NV];
+#pragma unroll
+    for (int u = 0; u < kBatch; ++u) {
+      const int32_t row = s_row[grp][i0 + u];
 #pragma unroll
       for (int v = 0; v < NV; ++v) {
         const int c = lane + v * G;
-        gv[u][v] = (ok && c < nvec) ? __ldg(grad4 + (int64_t)b * ld4 + (int64_t)t * nvec + c)
-                                    : make_float4(0.f, 0.f, 0.f, 0.f);
+        gv[u][v] = (row >= 0 && c < nvec) ? __ldg(grad4 + row + c) : make_float4(0.f, 0.f, 0.f, 0.f);
       }
     }
 #pragma unroll
-    for (int u = 0; u < 4; ++u) {
+    for (int u = 0; u < kBatch; ++u) {
       const int i = i0 + u;
       const uint32_t key = s_key[grp][1 + i];
       if (key >= sentinel) continue;                       // skipped lookups sort last; nothing follows them
 #pragma unroll
-      for (int v = 0; v < NV; ++v) acc.v[v] = add4(acc.v[v], gv[u][v]);
+      for (int v = 0; v < NV; ++v) acc[v] = add4(acc[v], gv[u][v]);
       const uint32_t next = s_key[grp][2 + i];
-      const bool last_in_window = (i == kWin - 1);
-      if (next != key || last_in_window) {
+      if (next != key || i == kWin - 1) {
         const bool head_open = (run_start == 0) && (s_key[grp][0] == key);
         const bool tail_open = (next == key);              // only possible at the window's last position
-        if (!head_open && !tail_open) {
-          rowwise_adagrad<G, NV>(acc, key, D, lane, gmask, tables, row_state, lr, eps);
-        } else {
-          float4* p = reinterpret_cast<float4*>(partial + ((int64_t)win * 2 + (run_start == 0 ? 0 : 1)) * D);
+        float4* dst = (!head_open && !tail_open)
+                          ? reinterpret_cast<float4*>(gsum + (int64_t)s_u[grp][i] * D)
+                          : reinterpret_cast<float4*>(partial + ((int64_t)win * 2 + (run_start == 0 ? 0 : 1)) * D);
 #pragma unroll
-          for (int v = 0; v < NV; ++v) {
-            const int c = lane + v * G;
-            if (c < nvec) p[c] = acc.v[v];
-          }
+        for (int v = 0; v < NV; ++v) {
+          const int c = lane + v * G;
+          if (c < nvec) dst[c] = acc[v];
+          acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
         }
-        acc.zero();
         run_start = i + 1;
       }
     }
   }
 }
 
-// Rows whose run crosses window edges: add the partial sums in window order, then update.
+// ---- (5) row-wise Adagrad, one lane group per distinct row ------------------------------------
+//   g = gsum[u], or the window partials of the row added in window order;
+//   s = state + mean_d g^2;  row -= lr * g / (sqrt(s) + eps)
 template <int G, int NV>
 __global__ void __launch_bounds__(256)
-combine_kernel(const int32_t* __restrict__ uniq, const int32_t* __restrict__ seg, const int32_t* __restrict__ scalars,
-               int D, const float* __restrict__ partial, float* __restrict__ tables, float* __restrict__ row_state,
-               float lr, float eps) {
+apply_rows_kernel(const int32_t* __restrict__ uniq, const int32_t* __restrict__ seg, const int32_t* __restrict__ scalars,
+                  int D, const float* __restrict__ gsum, const float* __restrict__ partial,
+                  float* __restrict__ tables, float* __restrict__ row_state, float lr, float eps) {
   constexpr int kGroups = 256 / G;
   const int grp = threadIdx.x / G, lane = threadIdx.x % G;
   const unsigned gmask = (G == 32) ? 0xffffffffu : (((1u << G) - 1u) << ((threadIdx.x & 31) / G * G));
   const int U = scalars[0];
   const int nvec = D >> 2;
-  for (int64_t u = (int64_t)blockIdx.x * kGroups + grp; u < U; u += (int64_t)gridDim.x * kGroups) {
-    const int s0 = seg[u], s1 = seg[u + 1];
-    const int k0 = s0 / kWin, k1 = (s1 - 1) / kWin;
-    if (k0 == k1) continue;
-    RowGrad<G, NV> acc;
-    acc.zero();
+  const int64_t u = (int64_t)blockIdx.x * kGroups + grp;
+  if (u >= U) return;
+  const int s0 = seg[u], s1 = seg[u + 1];
+  const uint32_t key = (uint32_t)uniq[u];
+  const int k0 = s0 / kWin, k1 = (s1 - 1) / kWin;
+  float4 g[NV];
+  if (k0 == k1) {
+    const float4* p = reinterpret_cast<const float4*>(gsum + u * D);
+#pragma unroll
+    for (int v = 0; v < NV; ++v) {
+      const int c = lane + v * G;
+      g[v] = (c < nvec) ? p[c] : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+  } else {
+#pragma unroll
+    for (int v = 0; v < NV; ++v) g[v] = make_float4(0.f, 0.f, 0.f, 0.f);
     for (int k = k0; k <= k1; ++k) {
       const int slot = (s0 <= k * kWin) ? 0 : 1;           // the run covers the window's first position -> slot 0
       const float4* p = reinterpret_cast<const float4*>(partial + ((int64_t)k * 2 + slot) * D);
 #pragma unroll
       for (int v = 0; v < NV; ++v) {
         const int c = lane + v * G;
-        if (c < nvec) acc.v[v] = add4(acc.v[v], p[c]);
+        if (c < nvec) g[v] = add4(g[v], p[c]);
       }
     }
-    rowwise_adagrad<G, NV>(acc, (uint32_t)uniq[u], D, lane, gmask, tables, row_state, lr, eps);
   }
+  float4* row = reinterpret_cast<float4*>(tables + (int64_t)key * D);
+  float4 r[NV];
+#pragma unroll
+  for (int v = 0; v < NV; ++v) {
+    const int c = lane + v * G;
+    r[v] = (c < nvec) ? row[c] : make_float4(0.f, 0.f, 0.f, 0.f);
+  }
+  const float st = row_state[key];
+  float ss = 0.f;
+#pragma unroll
+  for (int v = 0; v < NV; ++v) ss += g[v].x * g[v].x + g[v].y * g[v].y + g[v].z * g[v].z + g[v].w * g[v].w;
+#pragma unroll
+  for (int off = G / 2; off >= 1; off >>= 1) ss += __shfl_down_sync(gmask, ss, off, G);
+  ss = __shfl_sync(gmask, ss, 0, G);                       // every lane uses lane 0's sum
+  const float s = st + ss / (float)D;
+  const float scale = lr / (sqrtf(s) + eps);
+#pragma unroll
+  for (int v = 0; v < NV; ++v) {
+    const int c = lane + v * G;
+    if (c < nvec) {
+      r[v].x -= scale * g[v].x; r[v].y -= scale * g[v].y; r[v].z -= scale * g[v].z; r[v].w -= scale * g[v].w;
+      row[c] = r[v];
+    }
+  }
+  if (lane == 0) row_state[key] = s;
 }
 
 template <int G, int NV>
@@ -503,15 +564,18 @@ static void launch_reduce(const BwdPlan& p, char* ws, const uint32_t* keys, cons
   constexpr int kGroups = 256 / G;
   const uint32_t sentinel = (uint32_t)((uint64_t)T * (uint64_t)N);
   float* partial = reinterpret_cast<float*>(ws + p.off_partial);
+  float* gsum = reinterpret_cast<float*>(ws + p.off_gsum);
   const unsigned blocks = (unsigned)((p.nwin + kGroups - 1) / kGroups);
-  window_reduce_kernel<G, NV><<<blocks, 256, 0, st>>>(keys, perm, reinterpret_cast<int32_t*>(ws + p.off_bag), p.L,
-                                                      sentinel, N, D, B, grad, ld_grad, col0, tables, row_state,
-                                                      lr, eps, partial, p.nwin);
-  const int sms = num_sms();
-  combine_kernel<G, NV><<<sms * 4, 256, 0, st>>>(reinterpret_cast<int32_t*>(ws + p.off_uniq),
-                                                 reinterpret_cast<int32_t*>(ws + p.off_seg),
-                                                 reinterpret_cast<int32_t*>(ws + p.off_scalars), D, partial, tables,
-                                                 row_state, lr, eps);
+  window_reduce_kernel<G, NV><<<blocks, 256, 0, st>>>(keys, perm, reinterpret_cast<int32_t*>(ws + p.off_bag),
+                                                      reinterpret_cast<int32_t*>(ws + p.off_uidx), p.L, sentinel, N, D,
+                                                      B, grad, ld_grad, col0, gsum, partial, p.nwin);
+  const uint64_t maxkey = (uint64_t)T * (uint64_t)N;
+  const uint64_t umax = (uint64_t)p.L < maxkey ? (uint64_t)p.L : maxkey;
+  const unsigned ublocks = (unsigned)((umax + kGroups - 1) / kGroups);
+  apply_rows_kernel<G, NV><<<ublocks, 256, 0, st>>>(reinterpret_cast<int32_t*>(ws + p.off_uniq),
+                                                    reinterpret_cast<int32_t*>(ws + p.off_seg),
+                                                    reinterpret_cast<int32_t*>(ws + p.off_scalars), D, gsum, partial,
+                                                    tables, row_state, lr, eps);
 }
 
 #define SS_DISPATCH_GNV(D_, CALL)                                                 \
@@ -570,7 +634,7 @@ ss_status ss_embbag_bwd_adagrad(float* tables, float* row_state, int T, int64_t 
   if (T < 0 || B < 0 || N <= 0 || D <= 0 || D > 1024 || (D & 3) || col0 < 0 || L < 0) return SS_ERR_SHAPE;
   if ((uint64_t)T * (uint64_t)N >= (1ull << 31) || L >= (1ll << 31) - kSortTile) return SS_ERR_SHAPE;
   if (!aligned16(tables) || !aligned16(grad) || (ld_grad & 3) || (col0 & 3) || !aligned16(workspace)) return SS_ERR_ALIGN;
-  if (ld_grad < col0 + (int64_t)T * D) return SS_ERR_SHAPE;
+  if (ld_grad < col0 + (int64_t)T * D || (int64_t)B * ld_grad / 4 >= (1ll << 31)) return SS_ERR_SHAPE;
   const BwdPlan p = make_plan(T, N, D, L);
   if (workspace_bytes < p.total) return SS_ERR_WORKSPACE;
   ss_status stt = check_arch();
@@ -583,9 +647,11 @@ ss_status ss_embbag_bwd_adagrad(float* tables, float* row_state, int T, int64_t 
   int32_t* pos_b = reinterpret_cast<int32_t*>(ws + p.off_pos_b);
   int32_t* bag_of = reinterpret_cast<int32_t*>(ws + p.off_bag);
   uint32_t* hist = reinterpret_cast<uint32_t*>(ws + p.off_hist);
+  uint32_t* bintot = reinterpret_cast<uint32_t*>(ws + p.off_bintot);
   uint32_t* usum = reinterpret_cast<uint32_t*>(ws + p.off_usum);
   int32_t* uniq = reinterpret_cast<int32_t*>(ws + p.off_uniq);
   int32_t* seg = reinterpret_cast<int32_t*>(ws + p.off_seg);
+  int32_t* uidx = reinterpret_cast<int32_t*>(ws + p.off_uidx);
   int32_t* scalars = reinterpret_cast<int32_t*>(ws + p.off_scalars);
   const uint32_t sentinel = (uint32_t)((uint64_t)T * (uint64_t)N);
 
@@ -596,8 +662,7 @@ ss_status ss_embbag_bwd_adagrad(float* tables, float* row_state, int T, int64_t 
   }
 
   // (1) keys; positions no bag owns (malformed offsets) keep the sentinel
-  fill_u32_kernel<<<(unsigned)((L + 255) / 256), 256, 0, cs>>>(keys_a, L, sentinel);
-  fill_u32_kernel<<<(unsigned)((L + 255) / 256), 256, 0, cs>>>(reinterpret_cast<uint32_t*>(bag_of), L, 0u);
+  fill_keys_kernel<<<(unsigned)((L + 255) / 256), 256, 0, cs>>>(keys_a, bag_of, L, sentinel);
   build_keys_kernel<<<(unsigned)(((int64_t)T * B + 255) / 256), 256, 0, cs>>>(indices, offsets, T, N, B, L, keys_a,
                                                                                 bag_of, d_status);
   SS_LAUNCH_OK();
@@ -607,12 +672,12 @@ ss_status ss_embbag_bwd_adagrad(float* tables, float* row_state, int T, int64_t 
   int32_t* pin = nullptr;  // first pass: position = index
   int32_t* pout = pos_b;
   int32_t* pnext = pos_a;
-  const size_t smem = (size_t)kSortWarps * p.bins * 4;
+  const size_t smem = ((size_t)kSortWarps * p.bins + p.bins + 8) * 4;
   for (int pass = 0; pass < p.passes; ++pass) {
     const int shift = pass * p.digit_bits;
     sort_hist_kernel<<<p.nblk, kSortThreads, 0, cs>>>(kin, L, shift, p.bins, p.nblk, hist);
-    scan_exclusive_kernel<<<1, kScanThreads, 0, cs>>>(hist, (int64_t)p.nblk * p.bins, nullptr);
-    sort_scatter_kernel<<<p.nblk, kSortThreads, smem, cs>>>(kin, pin, kout, pout, L, shift, p.bins, p.nblk, hist);
+    bin_scan_kernel<<<(p.bins + 7) / 8, 256, 0, cs>>>(hist, p.bins, p.nblk, bintot);
+    sort_scatter_kernel<<<p.nblk, kSortThreads, smem, cs>>>(kin, pin, kout, pout, L, shift, p.bins, p.nblk, hist, bintot);
     SS_LAUNCH_OK();
     uint32_t* tk = kin; kin = kout; kout = tk;
     pin = pout; pout = pnext; pnext = pin;
@@ -624,11 +689,11 @@ ss_status ss_embbag_bwd_adagrad(float* tables, float* row_state, int T, int64_t 
   // (3) unique keys and segment offsets
   unique_count_kernel<<<p.nblk_u, kScanThreads, 0, cs>>>(keys_sorted, L, sentinel, usum);
   scan_exclusive_kernel<<<1, kScanThreads, 0, cs>>>(usum, p.nblk_u, usum + p.nblk_u);
-  unique_write_kernel<<<p.nblk_u, kScanThreads, 0, cs>>>(keys_sorted, L, sentinel, usum, uniq, seg, uniq_keys, seg_off);
+  unique_write_kernel<<<p.nblk_u, kScanThreads, 0, cs>>>(keys_sorted, L, sentinel, usum, uniq, seg, uidx, uniq_keys, seg_off);
   unique_finish_kernel<<<1, 1, 0, cs>>>(usum + p.nblk_u, seg, seg_off, d_num_unique, scalars);
   SS_LAUNCH_OK();
 
-  // (4) windowed segment reduction + row-wise Adagrad
+  // (4) windowed segment reduction, (5) row-wise Adagrad
 #define SS_RED(G_, NV_) \
   launch_reduce<G_, NV_>(p, ws, keys_sorted, perm_sorted, T, N, D, B, grad, ld_grad, col0, tables, row_state, lr, eps, cs)
   SS_DISPATCH_GNV(D, SS_RED);

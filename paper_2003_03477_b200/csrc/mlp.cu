@@ -35,28 +35,114 @@ __global__ void dz_kernel(const float* __restrict__ prob, const float* __restric
   else reinterpret_cast<float*>(dz)[b] = v;
 }
 
-// db[o] = sum_b G[b, o].  Block = 32 columns x 8 row groups; each group adds its rows in ascending
-// order, the 8 partial sums are added in group order.
+// ---------------------------------------------------------------------------------------------
+// Reductions over the batch that are no dense contraction: bias gradients, the gradient of the
+// single-logit layer and of the 13-input layer.  All have the form
+//     out[c * s_cols + j] = sum_b M[b, c] * S[b, j]          (S absent: s_cols = 1, S = 1)
+// One launch takes a list of such jobs.  A block owns 32 columns c and a slice of the batch; its 8
+// row groups add their rows in ascending order, the groups are added in order, and a second kernel
+// adds the slices in order: every sum has a fixed association.
+// ---------------------------------------------------------------------------------------------
+constexpr int kMaxJobs = 2 * kMaxLayers + 2;
+constexpr int kMaxSCols = 16;
+
+struct RedJob {
+  const void* M; const void* S;
+  int64_t ldm, lds;
+  int m_kind, s_kind;      // OperandKind
+  int ncols, s_cols;
+  int tile0;               // first column tile of this job in grid.x
+  int part_off;            // offset of this job's outputs in a partial row
+  int64_t out_off;         // offset into the flat gradient vector
+};
+struct RedJobs {
+  RedJob job[kMaxJobs];
+  int njobs, ntiles, total;   // total = outputs over all jobs
+};
+
+__device__ __forceinline__ float load_kind(const void* p, int kind, int64_t i) {
+  if (kind == OP_BF16) return __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(p)[i]);
+  const float v = reinterpret_cast<const float*>(p)[i];
+  return kind == OP_F32 ? v : __bfloat162float(__float2bfloat16_rn(v));
+}
+
 __global__ void __launch_bounds__(256)
-bias_grad_kernel(const void* __restrict__ G, int g_bf16, int B, int out, float* __restrict__ db) {
-  __shared__ float part[8][33];
+batch_reduce_partial_kernel(const __grid_constant__ RedJobs jobs, int B, int rows_per_split, float* __restrict__ partial) {
+  __shared__ float part[8][32][kMaxSCols + 1];
+  int j = 0;
+  while (j + 1 < jobs.njobs && (int)blockIdx.x >= jobs.job[j + 1].tile0) ++j;
+  const RedJob& J = jobs.job[j];
   const int cx = threadIdx.x & 31, ry = threadIdx.x >> 5;
-  const int o = blockIdx.x * 32 + cx;
-  float s = 0.f;
-  if (o < out) {
-    for (int b = ry; b < B; b += 8) {
-      const int64_t i = (int64_t)b * out + o;
-      s += g_bf16 ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(G)[i]) : reinterpret_cast<const float*>(G)[i];
+  const int c = ((int)blockIdx.x - J.tile0) * 32 + cx;
+  const int sc = J.s_cols;
+  const int r0 = blockIdx.y * rows_per_split;
+  const int r1 = min(B, r0 + rows_per_split);
+  float acc[kMaxSCols];
+#pragma unroll
+  for (int q = 0; q < kMaxSCols; ++q) acc[q] = 0.f;
+  if (c < J.ncols) {
+    for (int b = r0 + ry; b < r1; b += 8) {
+      const float m = load_kind(J.M, J.m_kind, (int64_t)b * J.ldm + c);
+      if (J.S == nullptr) {
+        acc[0] += m;
+      } else {
+#pragma unroll
+        for (int q = 0; q < kMaxSCols; ++q)
+          if (q < sc) acc[q] = fmaf(m, load_kind(J.S, J.s_kind, (int64_t)b * J.lds + q), acc[q]);
+      }
     }
   }
-  part[ry][cx] = s;
-  __syncthreads();
-  if (ry == 0 && o < out) {
-    float t = 0.f;
 #pragma unroll
-    for (int r = 0; r < 8; ++r) t += part[r][cx];
-    db[o] = t;
+  for (int q = 0; q < kMaxSCols; ++q) part[ry][cx][q] = acc[q];
+  __syncthreads();
+  if (ry == 0 && c < J.ncols) {
+    float* dst = partial + (int64_t)blockIdx.y * jobs.total + J.part_off + (int64_t)c * sc;
+    for (int q = 0; q < sc; ++q) {
+      float t = 0.f;
+#pragma unroll
+      for (int r = 0; r < 8; ++r) t += part[r][cx][q];
+      dst[q] = t;
+    }
   }
+}
+
+__global__ void __launch_bounds__(256)
+batch_reduce_final_kernel(const __grid_constant__ RedJobs jobs, int nsplit, const float* __restrict__ partial,
+                          float* __restrict__ g) {
+  const int i = blockIdx.x * 256 + threadIdx.x;
+  if (i >= jobs.total) return;
+  float t = 0.f;
+  for (int s = 0; s < nsplit; ++s) t += partial[(int64_t)s * jobs.total + i];
+  int j = 0;
+  while (j + 1 < jobs.njobs && i >= jobs.job[j + 1].part_off) ++j;
+  g[jobs.job[j].out_off + (i - jobs.job[j].part_off)] = t;
+}
+
+// logit[b] = sum_k X[b, k] * w[k] + bias: one warp per row, lanes stride k, fixed shuffle tree.
+__global__ void __launch_bounds__(256)
+rowdot_kernel(const void* __restrict__ X, int x_kind, int64_t ldx, const void* __restrict__ w, int w_kind, int K,
+              const float* __restrict__ bias, int B, float* __restrict__ logit) {
+  const int b = blockIdx.x * 8 + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  if (b >= B) return;
+  float s = 0.f;
+  for (int k = lane; k < K; k += 32) s = fmaf(load_kind(X, x_kind, (int64_t)b * ldx + k), load_kind(w, w_kind, k), s);
+#pragma unroll
+  for (int off = 16; off >= 1; off >>= 1) s += __shfl_down_sync(0xffffffffu, s, off);
+  if (lane == 0) logit[b] = s + bias[0];
+}
+
+// dX[b, k] = dz[b] * w[k], gated by X[b, k] > 0 (the backward of the single-logit layer).
+__global__ void __launch_bounds__(256)
+outer_mask_kernel(const void* __restrict__ dz, const void* __restrict__ w, const void* __restrict__ X, int kind_dz,
+                  int kind_w, int kind_x, int B, int K, void* __restrict__ dX, int out_bf16) {
+  const int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x;
+  if (i >= (int64_t)B * K) return;
+  const int b = (int)(i / K), k = (int)(i - (int64_t)b * K);
+  float v = load_kind(dz, kind_dz, b) * load_kind(w, kind_w, k);
+  if (!(load_kind(X, kind_x, i) > 0.f)) v = 0.f;
+  if (out_bf16) reinterpret_cast<__nv_bfloat16*>(dX)[i] = __float2bfloat16_rn(v);
+  else reinterpret_cast<float*>(dX)[i] = v;
 }
 
 // Element-wise Adagrad over the flat parameter vector; refreshes the bf16 mirror.  A zero gradient
@@ -148,13 +234,16 @@ ss_status ss_mlp_fwd(const ss_mlp_desc* desc, const float* w, const void* w_bf16
     else A = Operand{ws + p.act[l - 1], act_kind, L.in, 1};
     Bm = p.bf16 ? Operand{reinterpret_cast<const __nv_bfloat16*>(w_bf16) + L.w_off, OP_BF16, L.in, 1}
                 : Operand{w + L.w_off, OP_F32, L.in, 1};
+    if (l == p.nl - 1) {   // one output unit: a dot product per sample
+      rowdot_kernel<<<(B + 7) / 8, 256, 0, cs>>>(A.p, A.kind, A.s_row, Bm.p, Bm.kind, L.in, w + L.b_off, B, logit);
+      SS_LAUNCH_OK();
+      break;
+    }
     Epilogue ep;
     ep.bias = w + L.b_off;
     ep.relu = L.relu;
     ep.lo_cols = L.out;
-    if (l == p.nl - 1) {
-      ep.out_lo = logit; ep.lo_bf16 = 0; ep.ld_lo = 1;
-    } else if (l == p.nb - 1) {
+    if (l == p.nb - 1) {
       ep.out_lo = p.bf16 ? concat_bf16 : (void*)concat_f32; ep.lo_bf16 = p.bf16; ep.ld_lo = p.W;
     } else {
       ep.out_lo = ws + p.act[l]; ep.lo_bf16 = p.bf16; ep.ld_lo = L.out;
@@ -190,10 +279,24 @@ ss_status ss_mlp_bwd(const ss_mlp_desc* desc, float* w, void* w_bf16, float* ada
   float* g = grads ? grads : reinterpret_cast<float*>(ws + p.grads);
   SS_CUDA(cudaMemsetAsync(g, 0, (size_t)p.P * 4, cs));   // pads of the flat layout carry zero gradient
 
-  dz_kernel<<<(B + 255) / 256, 256, 0, cs>>>(prob, labels, B, ws + p.dact[p.nl - 1], p.bf16);
+  const int last = p.nl - 1;
+  const int dz_kind = p.bf16 ? OP_BF16 : OP_F32;
+  dz_kernel<<<(B + 255) / 256, 256, 0, cs>>>(prob, labels, B, ws + p.dact[last], p.bf16);
   SS_LAUNCH_OK();
 
-  for (int l = p.nl - 1; l >= 0; --l) {
+  RedJobs jobs;
+  jobs.njobs = 0; jobs.ntiles = 0; jobs.total = 0;
+  auto add_job = [&](const void* M, int m_kind, int64_t ldm, int ncols, const void* S, int s_kind, int64_t lds,
+                     int s_cols, int64_t out_off) {
+    RedJob& J = jobs.job[jobs.njobs++];
+    J.M = M; J.m_kind = m_kind; J.ldm = ldm; J.ncols = ncols;
+    J.S = S; J.s_kind = s_kind; J.lds = lds; J.s_cols = s_cols;
+    J.tile0 = jobs.ntiles; J.part_off = jobs.total; J.out_off = out_off;
+    jobs.ntiles += (ncols + 31) / 32;
+    jobs.total += ncols * s_cols;
+  };
+
+  for (int l = last; l >= 0; --l) {
     const LayerInfo& L = p.layer[l];
     const void* G = ws + p.dact[l];
     // input of layer l
@@ -201,19 +304,29 @@ ss_status ss_mlp_bwd(const ss_mlp_desc* desc, float* w, void* w_bf16, float* ada
     if (l == 0) X = Operand{dense, p.bf16 ? OP_F32_ROUND_BF16 : OP_F32, 1, p.n_dense};
     else if (l == p.nb) X = Operand{p.bf16 ? concat_bf16 : (const void*)concat_f32, act_kind, 1, p.W};
     else X = Operand{ws + p.act[l - 1], act_kind, 1, L.in};
+    // db[o] = sum_b G[b, o]
+    add_job(G, act_kind, L.out, L.out, nullptr, 0, 0, 1, L.b_off);
     // dW[o, i] = sum_b G[b, o] * X[b, i]
-    {
+    if (l == last) {
+      add_job(X.p, X.kind, X.s_k, L.in, G, dz_kind, 1, 1, L.w_off);          // out = 1: dW[i] = sum_b X[b,i] dz[b]
+    } else if (l == 0 && L.in <= kMaxSCols) {
+      add_job(G, act_kind, L.out, L.out, X.p, X.kind, X.s_k, L.in, L.w_off);  // few inputs: dW[o, :] per column o
+    } else {
       Operand A{G, act_kind, 1, L.out};
       Epilogue ep;
       ep.out_lo = g + L.w_off; ep.lo_bf16 = 0; ep.ld_lo = L.in; ep.lo_cols = L.in;
       st = gemm(L.out, L.in, B, A, X, ep, cs);
       if (st != SS_OK) return st;
     }
-    bias_grad_kernel<<<(L.out + 31) / 32, 256, 0, cs>>>(G, p.bf16, B, L.out, g + L.b_off);
-    SS_LAUNCH_OK();
     if (l == 0) break;
     // dX[b, i] = sum_o G[b, o] * W[o, i], gated by the ReLU of the producing layer
-    {
+    if (l == last && l != p.nb) {
+      const void* wl = p.bf16 ? (const void*)(reinterpret_cast<const __nv_bfloat16*>(w_bf16) + L.w_off) : (const void*)(w + L.w_off);
+      const int64_t cnt = (int64_t)B * L.in;
+      outer_mask_kernel<<<(unsigned)((cnt + 255) / 256), 256, 0, cs>>>(G, wl, ws + p.act[l - 1], dz_kind, act_kind, act_kind,
+                                                                       B, L.in, ws + p.dact[l - 1], p.bf16);
+      SS_LAUNCH_OK();
+    } else {
       Operand A{G, act_kind, L.out, 1};
       Operand Wt = p.bf16 ? Operand{reinterpret_cast<const __nv_bfloat16*>(w_bf16) + L.w_off, OP_BF16, 1, L.in}
                           : Operand{w + L.w_off, OP_F32, 1, L.in};
@@ -231,6 +344,15 @@ ss_status ss_mlp_bwd(const ss_mlp_desc* desc, float* w, void* w_bf16, float* ada
       st = gemm(B, L.in, L.out, A, Wt, ep, cs);
       if (st != SS_OK) return st;
     }
+  }
+  {
+    // all batch reductions of the pass in two launches
+    int rows = ((B + p.red_splits - 1) / p.red_splits + 7) & ~7;
+    const int nsplit = (B + rows - 1) / rows;
+    float* partial = reinterpret_cast<float*>(ws + p.red_partial);
+    batch_reduce_partial_kernel<<<dim3(jobs.ntiles, nsplit), 256, 0, cs>>>(jobs, B, rows, partial);
+    batch_reduce_final_kernel<<<(jobs.total + 255) / 256, 256, 0, cs>>>(jobs, nsplit, partial, g);
+    SS_LAUNCH_OK();
   }
 
   if (apply_update) {

@@ -22,7 +22,8 @@ struct MlpPlan {
   // respect to it after the ReLU mask.  The last bottom layer's output lives in the concat buffer and
   // the last top layer's in logit[], so act[] is unused for those two.
   size_t act[kMaxLayers], dact[kMaxLayers];
-  size_t grads, total;
+  size_t grads, red_partial, total;
+  int red_splits;         // batch slices of the two-stage reductions (bias and skinny weight gradients)
 };
 
 inline int64_t pad32(int64_t x) { return (x + 31) & ~(int64_t)31; }
@@ -62,6 +63,12 @@ inline ss_status make_mlp_plan(const ss_mlp_desc* d, int B, MlpPlan* p) {
     p->dact[l] = take(bytes);
   }
   p->grads = take((size_t)p->P * 4);
+  p->red_splits = B >= 1024 ? 16 : (B >= 256 ? 8 : (B >= 64 ? 2 : 1));
+  size_t red_total = 0;
+  for (int l = 0; l < p->nl; ++l) red_total += (size_t)p->layer[l].out;
+  red_total += (size_t)p->layer[p->nl - 1].in;
+  if (p->layer[0].in <= 16) red_total += (size_t)p->layer[0].in * p->layer[0].out;
+  p->red_partial = take(red_total * 4 * (size_t)p->red_splits);
   p->total = o;
   return SS_OK;
 }
