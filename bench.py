@@ -1,0 +1,440 @@
+#!/usr/bin/env python
+"""Benchmark of the ShadowSync hot path on B200.
+
+    python bench.py --gpus N --steps K --warmup W [--workload medium] [--impl reference]
+
+One "step" is one pass of the whole hot path over one batch per replica: every one of the R replicas
+runs embedding forward, MLP forward, MLP backward + dense Adagrad and embedding backward + row-wise
+Adagrad on its own high-priority stream, while the shadow loop keeps enqueuing the synchronisation
+kernel (S-EASGD / S-MA / S-BMUF as the workload says) on the lowest-priority stream.
+`value` = training examples per second with the shadow sync on, inputs resident in HBM.
+With N > 1 (launched under torchrun) every rank runs the same job on its own GPU: the path does not
+shard across GPUs, so these are independent replicas of the job and the values add (weak scaling).
+
+`--impl reference` times the CPU oracle (oracle/, test infrastructure) on a bounded sample of the same
+workload on the host cores; it is deliberately slow and is a reported baseline, not a target.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "training examples/sec at 1 B200 with shadow sync on; sync HBM GB/s vs peak"
+UNIT = "examples/s"
+RING = 8            # pre-generated batches per replica, cycled through
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return dict(hbm_gbs=p["hbm_gbs"], bf16_tflops=p["bf16_tflops"], bf16_tflops_sustained=p["bf16_tflops_sustained"],
+                    source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
+
+
+class ClockSampler:
+    """nvidia-smi clocks and throttle reasons sampled while the timed region runs."""
+
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu_index, self.proc, self.lines = gpu_index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-lms", "100", "-i", str(self.gpu_index)], stdout=subprocess.PIPE,
+                                         stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+        return self
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ----------------------------------------------------------------------------------------------
+def build_job(cfg, device):
+    """Tables, replicas and a ring of device-resident batches for one GPU."""
+    import torch
+    from paper_2003_03477_b200 import binding as ss, synth, trainer
+    tables = trainer.device_tables(cfg, device)
+    spec = ss.MlpSpec(cfg.bottom, cfg.top, cfg.bf16)
+    w0 = torch.from_numpy(trainer.pack_params(spec, synth.initial_weights(cfg))).to(device)
+    host = [[synth.make_batch(cfg, r, t) for t in range(RING)] for r in range(cfg.R)]
+    max_L = max(b.L for bs in host for b in bs)
+    model = trainer.Model(cfg.T, cfg.N, cfg.D, cfg.B, cfg.bottom, cfg.top, cfg.bf16, cfg.R, w0, tables, cfg.lr, cfg.eps,
+                          max_L=max_L, device=device)
+    dev = [[trainer.DeviceBatch(b.indices, b.offsets, b.dense, b.labels, device) for b in bs] for bs in host]
+    return model, host, dev, max_L
+
+
+def capture_graphs(model, dev):
+    """One CUDA graph per (replica, ring slot): the four calls of a replica step."""
+    import torch
+    graphs = []
+    for r, rep in enumerate(model.replicas):
+        row = []
+        for slot, b in enumerate(dev[r]):
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=rep.stream):
+                model.step(r, b, stream=rep.stream)
+            row.append(g)
+        graphs.append(row)
+    return graphs
+
+
+def run_steps(model, graphs, first_step, n_steps):
+    import torch
+    for t in range(first_step, first_step + n_steps):
+        for r, rep in enumerate(model.replicas):
+            with torch.cuda.stream(rep.stream):
+                graphs[r][t % RING].replay()
+
+
+def timed_region(model, graphs, first_step, n_steps):
+    """Device time of n_steps steps over all replica streams (ms)."""
+    import torch
+    main = torch.cuda.current_stream()
+    torch.cuda.synchronize()
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    start.record(main)
+    for rep in model.replicas:
+        rep.stream.wait_event(start)
+    run_steps(model, graphs, first_step, n_steps)
+    for rep in model.replicas:
+        e = torch.cuda.Event()
+        e.record(rep.stream)
+        main.wait_event(e)
+    stop.record(main)
+    stop.synchronize()
+    return start.elapsed_time(stop)
+
+
+def sync_args(cfg):
+    return dict(rule=cfg.sync, alpha=cfg.alpha, eta=cfg.eta, mu=cfg.mu)
+
+
+def time_kernel_call(fn, stream, reps):
+    """Average device time (ms) of a library call that is exactly one kernel, from CUDA events on its stream."""
+    import torch
+    evs = []
+    for i in range(reps):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        fn(i)
+        b.record(stream)
+        evs.append((a, b))
+    stream.synchronize()
+    return sum(a.elapsed_time(b) for a, b in evs) / reps
+
+
+def bench_gpu(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2003_03477_b200 import binding as ss, synth, trainer
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    device = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=device)
+    cfg = synth.CONFIGS[args.workload]
+    K, W = args.steps, max(args.warmup, 3)
+    peaks = measured_peaks()
+
+    model, host, dev, max_L = build_job(cfg, device)
+    # un-captured warm-up: first-use set-up inside the library (function attributes, symbol addresses)
+    for r in range(cfg.R):
+        model.step(r, dev[r][0])
+    model.sync(**sync_args(cfg))
+    torch.cuda.synchronize()
+    graphs = capture_graphs(model, dev)
+    launches_per_replica_step = None
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    # ---- sync off ------------------------------------------------------------------------
+    run_steps(model, graphs, 0, W)
+    barrier()
+    ms_off = timed_region(model, graphs, W, K)
+
+    # ---- sync on (the headline) -------------------------------------------------------------
+    loop = trainer.ShadowLoop(model, max_in_flight=args.sync_in_flight, pause_s=args.sync_pause, **sync_args(cfg)).start()
+    run_steps(model, graphs, 0, W)
+    barrier()
+    sampler = ClockSampler(local).start()
+    rounds0 = loop.rounds
+    ms_on = timed_region(model, graphs, W, K)
+    rounds = loop.rounds - rounds0
+    clocks = sampler.stop()
+    barrier()
+    loop.stop()
+    torch.cuda.synchronize()
+    if world > 1:
+        t = torch.tensor([ms_on, ms_off], device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_on, ms_off = float(t[0]), float(t[1])
+    examples = cfg.R * cfg.B * K * world
+    value = examples / (ms_on * 1e-3)
+    value_off = examples / (ms_off * 1e-3)
+    status = model.status() | (ss.ss_device_error() << 8)
+
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
+        "ms_per_step": ms_on / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16" if cfg.bf16 else "f32", "data": "synthetic",
+        "config": {"workload": f"{cfg.name}: R={cfg.R} T={cfg.T} N={cfg.N} D={cfg.D} B={cfg.B} "
+                               f"bottom={'-'.join(map(str, cfg.bottom))} top={'-'.join(map(str, cfg.top))} "
+                               f"sync={cfg.sync} alpha={cfg.alpha} background",
+                   "l2": "inputs larger than L2: tables 6.7 GB gathered by Zipf indices, 8 rotating batches per replica",
+                   "multi_gpu": "replicas only (no cross-GPU exchange on this path)"},
+        "clocks": clocks,
+        "status_word": status,
+    }
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    # ---- extra measurements on rank 0 ---------------------------------------------------------
+    out["sync"] = {"rounds_per_s": rounds / (ms_on * 1e-3), "avg_sync_gap_steps": (K / rounds) if rounds else None,
+                   "examples_per_s_sync_off": value_off, "throughput_loss_pct": 100.0 * (1.0 - value / value_off)}
+
+    # dominant-kernel roofline: the embedding-bag forward gather (one kernel per call), timed with events on
+    # its stream; algorithmic bytes = L*(4D+4) + (T*B+1)*4 + T*B*2D (bf16 pooled output)
+    rep = model.replicas[0]
+    s = rep.stream
+    T, N, D, B = cfg.T, cfg.N, cfg.D, cfg.B
+    sp = model.spec
+
+    def fwd(i):
+        b = dev[0][i % RING]
+        ss.ss_embbag_fwd(model.tables, T, N, D, b.indices, b.offsets, B, rep.concat_f32, sp.W, rep.concat_bf16, sp.W,
+                         D, model.d_status, s)
+    with torch.cuda.stream(s):
+        time_kernel_call(fwd, s, 3)
+        ms_fwd = time_kernel_call(fwd, s, 24)
+    Lmean = float(np.mean([b.L for b in host[0]]))
+    out_bytes = T * B * D * (2 if cfg.bf16 else 4)
+    fwd_bytes = Lmean * (4 * D + 4) + (T * B + 1) * 4 + out_bytes
+    achieved = fwd_bytes / (ms_fwd * 1e-3) / 1e9
+    out["roofline"] = {"kernel": "embbag_fwd_kernel", "bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"],
+                       "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"], "traffic": None,
+                       "peak_source": peaks["source"], "bytes_per_launch": fwd_bytes, "us_per_launch": ms_fwd * 1e3}
+
+    # the sync kernel alone at the workload's parameter size (L2-resident) and at 64M elements (HBM-bound)
+    def time_sync(n, R):
+        ws = [torch.randn(n, device=device) * 0.02 for _ in range(R)]
+        c = torch.zeros(n, device=device)
+        d = torch.zeros(n, device=device)
+        fn = {"easgd": lambda i: ss.ss_sync_easgd(ws, c, n, cfg.alpha, 0, None, s),
+              "ma": lambda i: ss.ss_sync_ma(ws, c, n, cfg.alpha, 0, None, s),
+              "bmuf": lambda i: ss.ss_sync_bmuf(ws, c, d, n, cfg.alpha, cfg.eta, cfg.mu, 0, None, s)}[cfg.sync]
+        with torch.cuda.stream(s):
+            time_kernel_call(fn, s, 3)
+            ms = time_kernel_call(fn, s, 20)
+        per = {"easgd": 2 * R + 2, "ma": 2 * R + 1, "bmuf": 2 * R + 4}[cfg.sync]
+        gbs = per * 4 * n / (ms * 1e-3) / 1e9
+        return {"n": n, "R": R, "us": ms * 1e3, "GB/s": gbs, "frac_of_hbm_peak": gbs / peaks["hbm_gbs"]}
+    out["sync"]["kernel_alone_64M"] = time_sync(1 << 26, cfg.R)
+    torch.cuda.synchronize()
+
+    # ---- end to end through the public API with host buffers ------------------------------------
+    out["e2e"] = bench_e2e(model, host, cfg, K, W)
+    out["gpu_launches"] = None
+    out["cpu_baseline"] = cpu_baseline(cfg, budget_s=args.cpu_budget)
+    print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def bench_e2e(model, host, cfg, K, W):
+    """Same metric with the step's inputs in pinned host memory: H2D copy of every batch and a D2H read of the loss
+    inside the timed region, calls made through the binding (no graphs: the input buffers change every step)."""
+    import torch
+    from paper_2003_03477_b200 import trainer
+    pinned = [[tuple(torch.from_numpy(np.ascontiguousarray(a)).pin_memory() for a in
+                     (b.indices, b.offsets, b.dense, b.labels)) for b in bs] for bs in host]
+    Lmax = max(b.L for bs in host for b in bs)
+    stage = []
+    for r in range(cfg.R):
+        stage.append([trainer.DeviceBatch(np.zeros(Lmax, np.int32), host[r][0].offsets, host[r][0].dense, host[r][0].labels,
+                                          model.device) for _ in range(2)])
+    loss_host = [torch.zeros(1).pin_memory() for _ in range(cfg.R)]
+    h2d = d2h = 0
+
+    def step(t):
+        nonlocal h2d, d2h
+        for r, rep in enumerate(model.replicas):
+            src, dst = pinned[r][t % RING], stage[r][t % 2]
+            with torch.cuda.stream(rep.stream):
+                L = src[0].numel()
+                dst.indices[:L].copy_(src[0], non_blocking=True)
+                dst.offsets.copy_(src[1], non_blocking=True)
+                dst.dense.copy_(src[2], non_blocking=True)
+                dst.labels.copy_(src[3], non_blocking=True)
+                dst.L = L
+                model.step(r, dst)
+                loss_host[r].copy_(rep.loss, non_blocking=True)
+            h2d += sum(x.numel() * x.element_size() for x in src)
+            d2h += 4
+
+    loop = trainer.ShadowLoop(model, cfg.sync, cfg.alpha, cfg.eta, cfg.mu).start()
+    for t in range(W):
+        step(t)
+    torch.cuda.synchronize()
+    h2d = d2h = 0
+    t0 = time.perf_counter()
+    for t in range(W, W + K):
+        step(t)
+    for rep in model.replicas:
+        rep.stream.synchronize()
+    dt = time.perf_counter() - t0
+    loop.stop()
+    torch.cuda.synchronize()
+    return {"value": cfg.R * cfg.B * K / dt, "unit": UNIT, "h2d_bytes_per_step": h2d // K, "d2h_bytes_per_step": d2h // K,
+            "timing": "host wall clock around K steps incl. stream sync (copies and launches inside)"}
+
+
+# ----------------------------------------------------------------------------------------------
+def oracle_sample(cfg, budget_s):
+    """Times the oracle on replica steps of the workload's shape with a reduced batch (same bag mix, index
+    skew, layer widths); returns (examples, seconds, description)."""
+    from oracle import shadowsync_oracle as O
+    from paper_2003_03477_b200 import synth
+    Bs = min(cfg.B, 64)
+    small = synth.scaled(cfg, B=Bs, R=1)
+    batch = synth.make_batch(small, 0, 0)
+    # compact table: only the rows this sample touches (the full table does not need to exist on the host)
+    lens = np.diff(batch.offsets.astype(np.int64))
+    tbl = np.repeat(np.arange(cfg.T * Bs) // Bs, lens)
+    keys = tbl.astype(np.int64) * cfg.N + batch.indices
+    uniq, inv = np.unique(keys, return_inverse=True)
+    rows_per_t = [uniq[(uniq // cfg.N) == t] % cfg.N for t in range(cfg.T)]
+    nmax = max(len(r) for r in rows_per_t)
+    tables = np.zeros((cfg.T, nmax, cfg.D), np.float32)
+    remap = np.zeros(len(uniq), np.int64)
+    for t in range(cfg.T):
+        tables[t, :len(rows_per_t[t])] = synth.table_rows(cfg, t, rows_per_t[t])
+        remap[(uniq // cfg.N) == t] = np.arange(len(rows_per_t[t]))
+    batch.indices = remap[inv].astype(np.int32)
+    layers = synth.initial_weights(cfg)
+    accs = [(np.zeros_like(W), np.zeros_like(b)) for W, b in layers]
+    state = np.zeros((cfg.T, nmax), np.float32)
+    n, t0 = 0, time.perf_counter()
+    while True:
+        O.replica_step(tables, state, layers, accs, len(cfg.bottom) - 1, batch, cfg.lr, cfg.eps, cfg.bf16)
+        n += Bs
+        dt = time.perf_counter() - t0
+        if dt > budget_s:
+            break
+    return n, dt, f"{n // Bs} replica steps of batch {Bs} (full model widths, same bag/index recipe, touched rows only)"
+
+
+def cpu_baseline(cfg, budget_s):
+    n, dt, what = oracle_sample(cfg, budget_s)
+    return {"value": n / dt, "unit": UNIT, "cores": threads_used(), "kind": "oracle", "sample": what}
+
+
+def threads_used():
+    try:
+        from threadpoolctl import threadpool_info
+        return max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def bench_reference(args):
+    """The oracle as it stands on the host cores, on the same workload's shapes (bounded sample per step)."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from paper_2003_03477_b200 import synth
+    cfg = synth.CONFIGS[args.workload]
+    K, W = args.steps, args.warmup
+    per_step = max(1.0, min(10.0, 120.0 / max(1, K + W)))
+    for _ in range(min(W, 1)):
+        oracle_sample(cfg, 0.0)
+    n = dt = 0.0
+    what = ""
+    for _ in range(K):
+        a, b, what = oracle_sample(cfg, per_step)
+        n += a
+        dt += b
+    v = n / dt
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": int(os.environ.get("WORLD_SIZE", "1")),
+        "steps": K, "warmup": W, "ms_per_step": 1e3 * dt / K, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": f"{cfg.name} (CPU oracle on a bounded sample)"},
+        "cpu_baseline": {"value": v, "unit": UNIT, "cores": threads_used(), "kind": "oracle", "sample": what + " per step"},
+        "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0}))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="medium", choices=["tiny", "medium", "medium_bmuf", "large"])
+    ap.add_argument("--sync-in-flight", type=int, default=2)
+    ap.add_argument("--sync-pause", type=float, default=0.0)
+    ap.add_argument("--cpu-budget", type=float, default=15.0)
+    args = ap.parse_args()
+    if args.impl == "reference":
+        bench_reference(args)
+    else:
+        bench_gpu(args)
+
+
+if __name__ == "__main__":
+    main()

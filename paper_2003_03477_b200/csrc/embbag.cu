@@ -207,13 +207,17 @@ sort_hist_kernel(const uint32_t* __restrict__ keys, int64_t L, int shift, int bi
   const int lane = threadIdx.x & 31;
   const int64_t base = (int64_t)blockIdx.x * kSortTile;
   const uint32_t mask = (uint32_t)bins - 1u;
-#pragma unroll 4
-  for (int k = 0; k < kSortIPT; ++k) {
+  uint32_t digit[kSortIPT];
+#pragma unroll
+  for (int k = 0; k < kSortIPT; ++k) {                      // all loads first, then the counting
     const int64_t i = base + (int64_t)k * kSortThreads + threadIdx.x;
-    const bool valid = i < L;
-    const uint32_t digit = valid ? ((keys[i] >> shift) & mask) : (uint32_t)bins;
-    const uint32_t peers = __match_any_sync(0xffffffffu, digit);
-    if (valid && lane == (__ffs(peers) - 1)) atomicAdd(&cnt[digit], (uint32_t)__popc(peers));  // integer: order-free
+    digit[k] = (i < L) ? ((keys[i] >> shift) & mask) : (uint32_t)bins;
+  }
+#pragma unroll
+  for (int k = 0; k < kSortIPT; ++k) {
+    const uint32_t peers = __match_any_sync(0xffffffffu, digit[k]);
+    if (digit[k] < (uint32_t)bins && lane == (__ffs(peers) - 1))
+      atomicAdd(&cnt[digit[k]], (uint32_t)__popc(peers));   // integer counts: order-free
   }
   __syncthreads();
   for (int i = threadIdx.x; i < bins; i += kSortThreads) hist[(int64_t)i * nblk + blockIdx.x] = cnt[i];
@@ -494,67 +498,84 @@ window_reduce_kernel(const uint32_t* __restrict__ keys, const int32_t* __restric
 // ---- (5) row-wise Adagrad, one lane group per distinct row ------------------------------------
 //   g = gsum[u], or the window partials of the row added in window order;
 //   s = state + mean_d g^2;  row -= lr * g / (sqrt(s) + eps)
+template <int NV> struct RowsPerGroup { static constexpr int value = NV == 1 ? 4 : (NV == 2 ? 2 : 1); };
+
 template <int G, int NV>
 __global__ void __launch_bounds__(256)
 apply_rows_kernel(const int32_t* __restrict__ uniq, const int32_t* __restrict__ seg, const int32_t* __restrict__ scalars,
                   int D, const float* __restrict__ gsum, const float* __restrict__ partial,
                   float* __restrict__ tables, float* __restrict__ row_state, float lr, float eps) {
   constexpr int kGroups = 256 / G;
+  constexpr int RB = RowsPerGroup<NV>::value;              // rows per group, their loads issued together
   const int grp = threadIdx.x / G, lane = threadIdx.x % G;
   const unsigned gmask = (G == 32) ? 0xffffffffu : (((1u << G) - 1u) << ((threadIdx.x & 31) / G * G));
   const int U = scalars[0];
   const int nvec = D >> 2;
-  const int64_t u = (int64_t)blockIdx.x * kGroups + grp;
-  if (u >= U) return;
-  const int s0 = seg[u], s1 = seg[u + 1];
-  const uint32_t key = (uint32_t)uniq[u];
-  const int k0 = s0 / kWin, k1 = (s1 - 1) / kWin;
-  float4 g[NV];
-  if (k0 == k1) {
-    const float4* p = reinterpret_cast<const float4*>(gsum + u * D);
+  const int64_t u0 = ((int64_t)blockIdx.x * kGroups + grp) * RB;
+  if (u0 >= U) return;
+  int sg[RB + 1];
+  uint32_t key[RB];
+  bool valid[RB];
+#pragma unroll
+  for (int r = 0; r <= RB; ++r) sg[r] = seg[min((int64_t)U, u0 + r)];
+#pragma unroll
+  for (int r = 0; r < RB; ++r) {
+    valid[r] = u0 + r < U;
+    key[r] = valid[r] ? (uint32_t)uniq[u0 + r] : 0u;
+  }
+  float4 g[RB][NV], rw[RB][NV];
+  float st[RB];
+#pragma unroll
+  for (int r = 0; r < RB; ++r) {
+    const bool single = valid[r] && (sg[r] / kWin == (sg[r + 1] - 1) / kWin);
+    const float4* p = reinterpret_cast<const float4*>(gsum + (u0 + r) * D);
+    const float4* row = reinterpret_cast<const float4*>(tables + (int64_t)key[r] * D);
 #pragma unroll
     for (int v = 0; v < NV; ++v) {
       const int c = lane + v * G;
-      g[v] = (c < nvec) ? p[c] : make_float4(0.f, 0.f, 0.f, 0.f);
+      g[r][v] = (single && c < nvec) ? p[c] : make_float4(0.f, 0.f, 0.f, 0.f);
+      rw[r][v] = (valid[r] && c < nvec) ? row[c] : make_float4(0.f, 0.f, 0.f, 0.f);
     }
-  } else {
+    st[r] = valid[r] ? row_state[key[r]] : 0.f;
+  }
 #pragma unroll
-    for (int v = 0; v < NV; ++v) g[v] = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int k = k0; k <= k1; ++k) {
-      const int slot = (s0 <= k * kWin) ? 0 : 1;           // the run covers the window's first position -> slot 0
+  for (int r = 0; r < RB; ++r) {
+    if (!valid[r]) continue;
+    const int k0 = sg[r] / kWin, k1 = (sg[r + 1] - 1) / kWin;
+    for (int k = k0; k <= k1 && k0 != k1; ++k) {           // a row whose run crosses window edges
+      const int slot = (sg[r] <= k * kWin) ? 0 : 1;        // the run covers the window's first position -> slot 0
       const float4* p = reinterpret_cast<const float4*>(partial + ((int64_t)k * 2 + slot) * D);
 #pragma unroll
       for (int v = 0; v < NV; ++v) {
         const int c = lane + v * G;
-        if (c < nvec) g[v] = add4(g[v], p[c]);
+        if (c < nvec) g[r][v] = add4(g[r][v], p[c]);
       }
     }
   }
-  float4* row = reinterpret_cast<float4*>(tables + (int64_t)key * D);
-  float4 r[NV];
 #pragma unroll
-  for (int v = 0; v < NV; ++v) {
-    const int c = lane + v * G;
-    r[v] = (c < nvec) ? row[c] : make_float4(0.f, 0.f, 0.f, 0.f);
-  }
-  const float st = row_state[key];
-  float ss = 0.f;
+  for (int r = 0; r < RB; ++r) {
+    float ss = 0.f;
 #pragma unroll
-  for (int v = 0; v < NV; ++v) ss += g[v].x * g[v].x + g[v].y * g[v].y + g[v].z * g[v].z + g[v].w * g[v].w;
+    for (int v = 0; v < NV; ++v)
+      ss += g[r][v].x * g[r][v].x + g[r][v].y * g[r][v].y + g[r][v].z * g[r][v].z + g[r][v].w * g[r][v].w;
 #pragma unroll
-  for (int off = G / 2; off >= 1; off >>= 1) ss += __shfl_down_sync(gmask, ss, off, G);
-  ss = __shfl_sync(gmask, ss, 0, G);                       // every lane uses lane 0's sum
-  const float s = st + ss / (float)D;
-  const float scale = lr / (sqrtf(s) + eps);
+    for (int off = G / 2; off >= 1; off >>= 1) ss += __shfl_down_sync(gmask, ss, off, G);
+    ss = __shfl_sync(gmask, ss, 0, G);                     // every lane uses lane 0's sum
+    if (!valid[r]) continue;
+    const float s = st[r] + ss / (float)D;
+    const float scale = lr / (sqrtf(s) + eps);
+    float4* row = reinterpret_cast<float4*>(tables + (int64_t)key[r] * D);
 #pragma unroll
-  for (int v = 0; v < NV; ++v) {
-    const int c = lane + v * G;
-    if (c < nvec) {
-      r[v].x -= scale * g[v].x; r[v].y -= scale * g[v].y; r[v].z -= scale * g[v].z; r[v].w -= scale * g[v].w;
-      row[c] = r[v];
+    for (int v = 0; v < NV; ++v) {
+      const int c = lane + v * G;
+      if (c < nvec) {
+        float4 o = rw[r][v];
+        o.x -= scale * g[r][v].x; o.y -= scale * g[r][v].y; o.z -= scale * g[r][v].z; o.w -= scale * g[r][v].w;
+        row[c] = o;
+      }
     }
+    if (lane == 0) row_state[key[r]] = s;
   }
-  if (lane == 0) row_state[key] = s;
 }
 
 template <int G, int NV>
@@ -571,7 +592,8 @@ static void launch_reduce(const BwdPlan& p, char* ws, const uint32_t* keys, cons
                                                       B, grad, ld_grad, col0, gsum, partial, p.nwin);
   const uint64_t maxkey = (uint64_t)T * (uint64_t)N;
   const uint64_t umax = (uint64_t)p.L < maxkey ? (uint64_t)p.L : maxkey;
-  const unsigned ublocks = (unsigned)((umax + kGroups - 1) / kGroups);
+  const uint64_t per_block = (uint64_t)kGroups * RowsPerGroup<NV>::value;
+  const unsigned ublocks = (unsigned)((umax + per_block - 1) / per_block);
   apply_rows_kernel<G, NV><<<ublocks, 256, 0, st>>>(reinterpret_cast<int32_t*>(ws + p.off_uniq),
                                                     reinterpret_cast<int32_t*>(ws + p.off_seg),
                                                     reinterpret_cast<int32_t*>(ws + p.off_scalars), D, gsum, partial,
