@@ -182,6 +182,8 @@ def bench_gpu(args):
     if world > 1:
         dist.init_process_group("nccl", device_id=device)
     cfg = synth.CONFIGS[args.workload]
+    if args.replicas:
+        cfg = synth.scaled(cfg, R=args.replicas)
     K, W = args.steps, max(args.warmup, 3)
     peaks = measured_peaks()
 
@@ -287,9 +289,10 @@ def bench_gpu(args):
     torch.cuda.synchronize()
 
     # ---- end to end through the public API with host buffers ------------------------------------
-    out["e2e"] = bench_e2e(model, host, cfg, K, W)
+    if not args.quick:
+        out["e2e"] = bench_e2e(model, host, cfg, K, W)
+        out["cpu_baseline"] = cpu_baseline(cfg, budget_s=args.cpu_budget)
     out["gpu_launches"] = None
-    out["cpu_baseline"] = cpu_baseline(cfg, budget_s=args.cpu_budget)
     print(json.dumps(out))
     if world > 1:
         dist.destroy_process_group()
@@ -429,6 +432,8 @@ def main():
     ap.add_argument("--sync-in-flight", type=int, default=2)
     ap.add_argument("--sync-pause", type=float, default=0.0)
     ap.add_argument("--cpu-budget", type=float, default=15.0)
+    ap.add_argument("--replicas", type=int, default=0, help="override the workload's replica count (experiments)")
+    ap.add_argument("--quick", action="store_true", help="skip the e2e and CPU-baseline legs (experiments)")
     args = ap.parse_args()
     if args.impl == "reference":
         bench_reference(args)

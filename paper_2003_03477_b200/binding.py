@@ -25,7 +25,7 @@ SS_SYNC_EASGD_LITERAL = 1
 EXPORTS = ["ss_status_str", "ss_last_cuda_error", "ss_num_sms", "ss_embbag_fwd", "ss_embbag_bwd_workspace_bytes",
            "ss_embbag_bwd_adagrad", "ss_mlp_param_count", "ss_mlp_param_offsets", "ss_mlp_workspace_bytes",
            "ss_mlp_fwd", "ss_mlp_bwd", "ss_sync_easgd", "ss_sync_ma", "ss_sync_bmuf", "ss_to_bf16",
-           "ss_gemm_bf16", "ss_device_error", "ssh_fill_uniform"]
+           "ss_gemm_bf16", "ss_device_error", "ssh_fill_uniform", "ss_profile", "ss_profile_collect"]
 
 
 class SsError(RuntimeError):
@@ -78,6 +78,8 @@ def lib() -> C.CDLL:
         L.ss_to_bf16.argtypes = [vp, vp, i64, vp]
         L.ss_gemm_bf16.argtypes = [vp, i32, i64, vp, i32, i64, vp, i64, i32, i32, i32, i32, vp]
         L.ss_device_error.argtypes = [i32]
+        L.ss_profile.argtypes = [i32]
+        L.ss_profile_collect.argtypes = [C.c_char_p, sz, C.POINTER(f32), i32]
         L.ssh_fill_uniform.argtypes = [vp, i64, C.c_uint64, C.c_uint64, f32, f32, vp]
         for name in EXPORTS:
             if name not in ("ss_status_str", "ss_last_cuda_error", "ss_num_sms", "ss_embbag_bwd_workspace_bytes",
@@ -228,3 +230,18 @@ def ss_to_bf16(src, dst_bf16, n, stream=None) -> None:
 def ssh_fill_uniform(dst, count, key, counter0, scale, mid, stream=None) -> None:
     _check("ssh_fill_uniform", lib().ssh_fill_uniform(_ptr(dst), count, int(key), int(counter0), scale, mid,
                                                        _stream(stream)))
+
+
+def ss_profile(on: bool) -> bool:
+    """Switch the library's per-kernel timers on or off (off while capturing CUDA graphs)."""
+    return bool(lib().ss_profile(1 if on else 0))
+
+
+def ss_profile_collect(max_records: int = 1 << 16):
+    """[(kernel name, milliseconds)] of every launch timed since the last collect, in launch order."""
+    names = C.create_string_buffer(max_records * 32)
+    ms = (C.c_float * max_records)()
+    n = lib().ss_profile_collect(names, len(names), ms, max_records)
+    if n < 0:
+        raise SsError("ss_profile_collect", -7, lib().ss_last_cuda_error())
+    return list(zip(names.value.decode().split("\n")[:n], list(ms[:n])))

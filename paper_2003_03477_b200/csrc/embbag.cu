@@ -7,13 +7,14 @@
 //
 // Backward: (1) keys t*N+row, (2) stable LSD radix sort of (key, position) with a hand-written
 // histogram / scan / ranked-scatter pass per digit, (3) head flags + scan -> unique keys and segment
-// offsets, (4) the sorted lookups are cut into windows of 32 consecutive positions; a lane group
+// offsets, (4) the sorted lookups are cut into windows of 16 consecutive positions; a lane group
 // sums the gradients of each run of equal keys inside its window in position order.  A run that
 // lies inside one window is final and is updated at once; a run that crosses a window edge leaves a
 // partial sum, and a second kernel adds the partials of such a row in window order and updates it.
 // Work per group is the same whatever the skew of the row distribution, and every sum has a fixed
 // association, so results do not depend on scheduling.
 #include "common.cuh"
+#include "profile.cuh"
 
 namespace ss {
 
@@ -98,8 +99,10 @@ static void launch_fwd(const float* tables, int T, int64_t N, int D, const int32
   const int64_t bags = (int64_t)T * B;
   const int per_block = 256 / G;
   const unsigned blocks = (unsigned)((bags + per_block - 1) / per_block);
+  { SS_TIMED("embbag_fwd_kernel", st);
   embbag_fwd_kernel<G, NV><<<blocks, 256, 0, st>>>(tables, T, N, D, indices, offsets, B, out_f32, ld_f32,
                                                     out_bf16, ld_bf16, col0, d_status);
+  }
 }
 
 // ======================================================================================
@@ -110,7 +113,7 @@ constexpr int kSortWarps = kSortThreads / 32;
 constexpr int kSortIPT = 16;                              // items per thread
 constexpr int kSortTile = kSortThreads * kSortIPT;        // 4096 items per block
 constexpr int kMaxBins = 512;
-constexpr int kWin = 32;                                  // sorted positions per reduction window
+constexpr int kWin = 16;                                  // sorted positions per reduction window
 constexpr int kScanThreads = 1024;
 
 struct BwdPlan {
@@ -120,7 +123,7 @@ struct BwdPlan {
   int nwin;
   int nblk_u;        // blocks of the unique pass (1024 items each)
   size_t off_keys_a, off_keys_b, off_pos_a, off_pos_b, off_bag, off_hist, off_bintot, off_usum, off_uniq, off_seg,
-      off_uidx, off_partial, off_gsum, off_scalars, total;
+      off_uidx, off_partial, off_long, off_gsum, off_scalars, total;
 };
 
 static inline size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
@@ -154,6 +157,7 @@ static BwdPlan make_plan(int T, int64_t N, int D, int64_t L) {
   p.off_seg = o; o += align256((size_t)(L + 1) * 4);
   p.off_uidx = o; o += l4;
   p.off_partial = o; o += align256((size_t)p.nwin * 2 * (size_t)D * 4);
+  p.off_long = o; o += align256((size_t)p.nwin * 4);
   const uint64_t umax = (uint64_t)L < maxkey ? (uint64_t)L : maxkey;   // distinct rows cannot exceed either
   p.off_gsum = o; o += align256((size_t)(umax > 0 ? umax : 1) * (size_t)D * 4);
   p.off_scalars = o; o += 256;
@@ -407,6 +411,7 @@ __global__ void unique_finish_kernel(const uint32_t* __restrict__ total, int32_t
   if (U == 0) { seg[0] = 0; if (seg_out) seg_out[0] = 0; }
   if (d_num_unique) *d_num_unique = (int32_t)U;
   scalars[0] = (int32_t)U;
+  scalars[1] = 0;                                          // rows whose run crosses a window edge (filled by the window kernel)
 }
 
 // ---- (4) windowed segment reduction ---------------------------------------------------------
@@ -419,7 +424,8 @@ __global__ void __launch_bounds__(256)
 window_reduce_kernel(const uint32_t* __restrict__ keys, const int32_t* __restrict__ perm,
                      const int32_t* __restrict__ bag_of, const int32_t* __restrict__ uidx, int64_t L,
                      uint32_t sentinel, int64_t N, int D, int B, const float* __restrict__ grad, int64_t ld_grad,
-                     int col0, float* __restrict__ gsum, float* __restrict__ partial, int nwin) {
+                     int col0, float* __restrict__ gsum, float* __restrict__ partial, int32_t* __restrict__ long_list,
+                     int32_t* __restrict__ scalars, int nwin) {
   constexpr int kGroups = 256 / G;
   __shared__ uint32_t s_key[kGroups][kWin + 2];            // [0] = key before the window, [kWin+1] = key after
   __shared__ int32_t s_row[kGroups][kWin];                 // float4 index of the lookup's gradient row
@@ -489,22 +495,108 @@ window_reduce_kernel(const uint32_t* __restrict__ keys, const int32_t* __restric
           if (c < nvec) dst[c] = acc[v];
           acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
         }
+        // the window in which a multi-window run starts enters the row in the list of rows to combine
+        if (!head_open && tail_open && lane == 0) long_list[atomicAdd(&scalars[1], 1)] = s_u[grp][i];
         run_start = i + 1;
       }
     }
   }
 }
 
-// ---- (5) row-wise Adagrad, one lane group per distinct row ------------------------------------
-//   g = gsum[u], or the window partials of the row added in window order;
-//   s = state + mean_d g^2;  row -= lr * g / (sqrt(s) + eps)
-template <int NV> struct RowsPerGroup { static constexpr int value = NV == 1 ? 4 : (NV == 2 ? 2 : 1); };
+// ---- (5) rows whose run crosses window edges: add their window partials ---------------------------
+// Rows spanning up to four windows: one lane group adds the partials in window order.  Longer rows: one
+// block per row, lane group j adds the partials of windows k0+j, k0+j+groups, ... in ascending order and
+// the group sums are then added in group order.  The association is fixed by the
+// segment's position alone (the order of the list does not matter).
+template <int G, int NV>
+__global__ void __launch_bounds__(256)
+combine_rows_kernel(const int32_t* __restrict__ seg, const int32_t* __restrict__ scalars,
+                    const int32_t* __restrict__ long_list, int D, const float* __restrict__ partial,
+                    float* __restrict__ gsum) {
+  constexpr int kGroups = 256 / G;
+  extern __shared__ float4 s_part[];                       // [kGroups][D/4]
+  const int grp = threadIdx.x / G, lane = threadIdx.x % G;
+  const int nvec = D >> 2;
+  const int n = scalars[1];
+  constexpr int kShort = 4;                                // spans up to this many windows: one group per row
+  // phase A: short spans, one lane group per listed row, all partial loads issued together
+  for (int i = blockIdx.x * kGroups + grp; i < n; i += gridDim.x * kGroups) {
+    const int u = long_list[i];
+    const int s0 = seg[u], s1 = seg[u + 1];
+    const int k0 = s0 / kWin, k1 = (s1 - 1) / kWin;
+    if (k1 - k0 + 1 > kShort) continue;
+    float4 pv[kShort][NV];
+#pragma unroll
+    for (int j = 0; j < kShort; ++j) {
+      const int k = k0 + j;
+      const int slot = (s0 <= k * kWin) ? 0 : 1;           // the run covers the window's first position -> slot 0
+      const float4* p = reinterpret_cast<const float4*>(partial + ((int64_t)k * 2 + slot) * D);
+#pragma unroll
+      for (int v = 0; v < NV; ++v) {
+        const int c = lane + v * G;
+        pv[j][v] = (k <= k1 && c < nvec) ? p[c] : make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+    }
+    float4* dst = reinterpret_cast<float4*>(gsum + (int64_t)u * D);
+#pragma unroll
+    for (int v = 0; v < NV; ++v) {
+      const int c = lane + v * G;
+      float4 t = pv[0][v];
+#pragma unroll
+      for (int j = 1; j < kShort; ++j) t = add4(t, pv[j][v]);   // adding zeros for absent windows changes nothing
+      if (c < nvec) dst[c] = t;
+    }
+  }
+  // phase B: long spans, the whole block per row
+  for (int i = blockIdx.x; i < n; i += gridDim.x) {
+    const int u = long_list[i];
+    const int s0 = seg[u], s1 = seg[u + 1];
+    const int k0 = s0 / kWin, k1 = (s1 - 1) / kWin;
+    if (k1 - k0 + 1 <= kShort) continue;                   // uniform over the block
+    float4 acc[NV];
+#pragma unroll
+    for (int v = 0; v < NV; ++v) acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int k = k0 + grp; k <= k1; k += kGroups) {
+      const int slot = (s0 <= k * kWin) ? 0 : 1;
+      const float4* p = reinterpret_cast<const float4*>(partial + ((int64_t)k * 2 + slot) * D);
+#pragma unroll
+      for (int v = 0; v < NV; ++v) {
+        const int c = lane + v * G;
+        if (c < nvec) acc[v] = add4(acc[v], p[c]);
+      }
+    }
+#pragma unroll
+    for (int v = 0; v < NV; ++v) {
+      const int c = lane + v * G;
+      if (c < nvec) s_part[grp * nvec + c] = acc[v];
+    }
+    __syncthreads();
+    if (grp == 0) {
+      const int used = min(kGroups, k1 - k0 + 1);
+      float4* dst = reinterpret_cast<float4*>(gsum + (int64_t)u * D);
+#pragma unroll
+      for (int v = 0; v < NV; ++v) {
+        const int c = lane + v * G;
+        if (c < nvec) {
+          float4 t = s_part[c];
+          for (int j = 1; j < used; ++j) t = add4(t, s_part[j * nvec + c]);
+          dst[c] = t;
+        }
+      }
+    }
+    __syncthreads();
+  }
+}
+
+// ---- (6) row-wise Adagrad, one lane group per two distinct rows ----------------------------------
+//   g = gsum[u];  s = state + mean_d g^2;  row -= lr * g / (sqrt(s) + eps)
+template <int NV> struct RowsPerGroup { static constexpr int value = NV == 1 ? 2 : 1; };
 
 template <int G, int NV>
 __global__ void __launch_bounds__(256)
-apply_rows_kernel(const int32_t* __restrict__ uniq, const int32_t* __restrict__ seg, const int32_t* __restrict__ scalars,
-                  int D, const float* __restrict__ gsum, const float* __restrict__ partial,
-                  float* __restrict__ tables, float* __restrict__ row_state, float lr, float eps) {
+apply_rows_kernel(const int32_t* __restrict__ uniq, const int32_t* __restrict__ scalars, int D,
+                  const float* __restrict__ gsum, float* __restrict__ tables, float* __restrict__ row_state,
+                  float lr, float eps) {
   constexpr int kGroups = 256 / G;
   constexpr int RB = RowsPerGroup<NV>::value;              // rows per group, their loads issued together
   const int grp = threadIdx.x / G, lane = threadIdx.x % G;
@@ -513,11 +605,8 @@ apply_rows_kernel(const int32_t* __restrict__ uniq, const int32_t* __restrict__ 
   const int nvec = D >> 2;
   const int64_t u0 = ((int64_t)blockIdx.x * kGroups + grp) * RB;
   if (u0 >= U) return;
-  int sg[RB + 1];
   uint32_t key[RB];
   bool valid[RB];
-#pragma unroll
-  for (int r = 0; r <= RB; ++r) sg[r] = seg[min((int64_t)U, u0 + r)];
 #pragma unroll
   for (int r = 0; r < RB; ++r) {
     valid[r] = u0 + r < U;
@@ -527,30 +616,15 @@ apply_rows_kernel(const int32_t* __restrict__ uniq, const int32_t* __restrict__ 
   float st[RB];
 #pragma unroll
   for (int r = 0; r < RB; ++r) {
-    const bool single = valid[r] && (sg[r] / kWin == (sg[r + 1] - 1) / kWin);
     const float4* p = reinterpret_cast<const float4*>(gsum + (u0 + r) * D);
     const float4* row = reinterpret_cast<const float4*>(tables + (int64_t)key[r] * D);
 #pragma unroll
     for (int v = 0; v < NV; ++v) {
       const int c = lane + v * G;
-      g[r][v] = (single && c < nvec) ? p[c] : make_float4(0.f, 0.f, 0.f, 0.f);
+      g[r][v] = (valid[r] && c < nvec) ? p[c] : make_float4(0.f, 0.f, 0.f, 0.f);
       rw[r][v] = (valid[r] && c < nvec) ? row[c] : make_float4(0.f, 0.f, 0.f, 0.f);
     }
     st[r] = valid[r] ? row_state[key[r]] : 0.f;
-  }
-#pragma unroll
-  for (int r = 0; r < RB; ++r) {
-    if (!valid[r]) continue;
-    const int k0 = sg[r] / kWin, k1 = (sg[r + 1] - 1) / kWin;
-    for (int k = k0; k <= k1 && k0 != k1; ++k) {           // a row whose run crosses window edges
-      const int slot = (sg[r] <= k * kWin) ? 0 : 1;        // the run covers the window's first position -> slot 0
-      const float4* p = reinterpret_cast<const float4*>(partial + ((int64_t)k * 2 + slot) * D);
-#pragma unroll
-      for (int v = 0; v < NV; ++v) {
-        const int c = lane + v * G;
-        if (c < nvec) g[r][v] = add4(g[r][v], p[c]);
-      }
-    }
   }
 #pragma unroll
   for (int r = 0; r < RB; ++r) {
@@ -587,17 +661,29 @@ static void launch_reduce(const BwdPlan& p, char* ws, const uint32_t* keys, cons
   float* partial = reinterpret_cast<float*>(ws + p.off_partial);
   float* gsum = reinterpret_cast<float*>(ws + p.off_gsum);
   const unsigned blocks = (unsigned)((p.nwin + kGroups - 1) / kGroups);
-  window_reduce_kernel<G, NV><<<blocks, 256, 0, st>>>(keys, perm, reinterpret_cast<int32_t*>(ws + p.off_bag),
-                                                      reinterpret_cast<int32_t*>(ws + p.off_uidx), p.L, sentinel, N, D,
-                                                      B, grad, ld_grad, col0, gsum, partial, p.nwin);
+  int32_t* scalars = reinterpret_cast<int32_t*>(ws + p.off_scalars);
+  int32_t* long_list = reinterpret_cast<int32_t*>(ws + p.off_long);
+  int32_t* seg = reinterpret_cast<int32_t*>(ws + p.off_seg);
+  {
+    SS_TIMED("window_reduce_kernel", st);
+    window_reduce_kernel<G, NV><<<blocks, 256, 0, st>>>(keys, perm, reinterpret_cast<int32_t*>(ws + p.off_bag),
+                                                        reinterpret_cast<int32_t*>(ws + p.off_uidx), p.L, sentinel, N, D,
+                                                        B, grad, ld_grad, col0, gsum, partial, long_list, scalars, p.nwin);
+  }
+  {
+    SS_TIMED("combine_rows_kernel", st);
+    const int cblocks = p.nwin < num_sms() * 8 ? p.nwin : num_sms() * 8;
+    combine_rows_kernel<G, NV><<<cblocks, 256, (size_t)kGroups * D * 4, st>>>(seg, scalars, long_list, D, partial, gsum);
+  }
   const uint64_t maxkey = (uint64_t)T * (uint64_t)N;
   const uint64_t umax = (uint64_t)p.L < maxkey ? (uint64_t)p.L : maxkey;
   const uint64_t per_block = (uint64_t)kGroups * RowsPerGroup<NV>::value;
   const unsigned ublocks = (unsigned)((umax + per_block - 1) / per_block);
-  apply_rows_kernel<G, NV><<<ublocks, 256, 0, st>>>(reinterpret_cast<int32_t*>(ws + p.off_uniq),
-                                                    reinterpret_cast<int32_t*>(ws + p.off_seg),
-                                                    reinterpret_cast<int32_t*>(ws + p.off_scalars), D, gsum, partial,
-                                                    tables, row_state, lr, eps);
+  {
+    SS_TIMED("apply_rows_kernel", st);
+    apply_rows_kernel<G, NV><<<ublocks, 256, 0, st>>>(reinterpret_cast<int32_t*>(ws + p.off_uniq), scalars, D, gsum,
+                                                      tables, row_state, lr, eps);
+  }
 }
 
 #define SS_DISPATCH_GNV(D_, CALL)                                                 \
@@ -678,15 +764,21 @@ ss_status ss_embbag_bwd_adagrad(float* tables, float* row_state, int T, int64_t 
   const uint32_t sentinel = (uint32_t)((uint64_t)T * (uint64_t)N);
 
   if (L == 0 || (int64_t)T * B == 0) {
+    { SS_TIMED("unique_finish_kernel", cs);
     unique_finish_kernel<<<1, 1, 0, cs>>>(nullptr, seg, seg_off, d_num_unique, scalars);
+    }
     SS_LAUNCH_OK();
     return SS_OK;
   }
 
   // (1) keys; positions no bag owns (malformed offsets) keep the sentinel
+  { SS_TIMED("fill_keys_kernel", cs);
   fill_keys_kernel<<<(unsigned)((L + 255) / 256), 256, 0, cs>>>(keys_a, bag_of, L, sentinel);
+  }
+  { SS_TIMED("build_keys_kernel", cs);
   build_keys_kernel<<<(unsigned)(((int64_t)T * B + 255) / 256), 256, 0, cs>>>(indices, offsets, T, N, B, L, keys_a,
                                                                                 bag_of, d_status);
+  }
   SS_LAUNCH_OK();
 
   // (2) LSD radix sort, `passes` digits of `digit_bits` bits
@@ -697,9 +789,15 @@ ss_status ss_embbag_bwd_adagrad(float* tables, float* row_state, int T, int64_t 
   const size_t smem = ((size_t)kSortWarps * p.bins + p.bins + 8) * 4;
   for (int pass = 0; pass < p.passes; ++pass) {
     const int shift = pass * p.digit_bits;
+    { SS_TIMED("sort_hist_kernel", cs);
     sort_hist_kernel<<<p.nblk, kSortThreads, 0, cs>>>(kin, L, shift, p.bins, p.nblk, hist);
+    }
+    { SS_TIMED("bin_scan_kernel", cs);
     bin_scan_kernel<<<(p.bins + 7) / 8, 256, 0, cs>>>(hist, p.bins, p.nblk, bintot);
+    }
+    { SS_TIMED("sort_scatter_kernel", cs);
     sort_scatter_kernel<<<p.nblk, kSortThreads, smem, cs>>>(kin, pin, kout, pout, L, shift, p.bins, p.nblk, hist, bintot);
+    }
     SS_LAUNCH_OK();
     uint32_t* tk = kin; kin = kout; kout = tk;
     pin = pout; pout = pnext; pnext = pin;
@@ -709,10 +807,18 @@ ss_status ss_embbag_bwd_adagrad(float* tables, float* row_state, int T, int64_t 
   if (perm) SS_CUDA(cudaMemcpyAsync(perm, perm_sorted, (size_t)L * 4, cudaMemcpyDeviceToDevice, cs));
 
   // (3) unique keys and segment offsets
+  { SS_TIMED("unique_count_kernel", cs);
   unique_count_kernel<<<p.nblk_u, kScanThreads, 0, cs>>>(keys_sorted, L, sentinel, usum);
+  }
+  { SS_TIMED("scan_exclusive_kernel", cs);
   scan_exclusive_kernel<<<1, kScanThreads, 0, cs>>>(usum, p.nblk_u, usum + p.nblk_u);
+  }
+  { SS_TIMED("unique_write_kernel", cs);
   unique_write_kernel<<<p.nblk_u, kScanThreads, 0, cs>>>(keys_sorted, L, sentinel, usum, uniq, seg, uidx, uniq_keys, seg_off);
+  }
+  { SS_TIMED("unique_finish_kernel", cs);
   unique_finish_kernel<<<1, 1, 0, cs>>>(usum + p.nblk_u, seg, seg_off, d_num_unique, scalars);
+  }
   SS_LAUNCH_OK();
 
   // (4) windowed segment reduction, (5) row-wise Adagrad

@@ -1,6 +1,7 @@
 // SIMT GEMM with arbitrary operand strides: the float path of the small configuration and the
 // layers that are no dense contraction (13 input features, a single output logit).
 #include "gemm.cuh"
+#include "profile.cuh"
 
 namespace ss {
 
@@ -78,6 +79,7 @@ ss_status gemm_simt(int M, int N, int K, const Operand& A, const Operand& B, con
 #define SS_GO(KA, KB)                                                                                         \
   gemm_simt_kernel<KA, KB><<<grid, 256, 0, st>>>(M, N, K, A.p, A.s_row, A.s_k, B.p, B.s_row, B.s_k, ep)
   const int key = A.kind * 3 + B.kind;
+  SS_TIMED("gemm_simt_kernel", st);
   switch (key) {
     case OP_F32 * 3 + OP_F32: SS_GO(OP_F32, OP_F32); break;
     case OP_BF16 * 3 + OP_BF16: SS_GO(OP_BF16, OP_BF16); break;

@@ -19,6 +19,7 @@
 #include <cuda.h>
 #include <cudaTypedefs.h>
 #include "gemm.cuh"
+#include "profile.cuh"
 
 namespace ss {
 
@@ -350,7 +351,9 @@ ss_status gemm_tc(int M, int N, int K, const Operand& A, const Operand& B, const
   const bool okb = p.b_mn ? make_map(&mb, B.p, N, K, B.s_k, 64, 64) : make_map(&mb, B.p, K, N, B.s_row, 64, kBN);
   if (!oka || !okb) return SS_ERR_CUDA;
   dim3 grid((N + kBN - 1) / kBN, (M + kBM - 1) / kBM);
+  { SS_TIMED("gemm_tc_kernel", st);
   gemm_tc_kernel<<<grid, kTcThreads, kTcSmem, st>>>(ma, mb, p);
+  }
   SS_LAUNCH_OK();
   return SS_OK;
 }

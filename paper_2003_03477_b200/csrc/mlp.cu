@@ -1,5 +1,6 @@
 // Bottom MLP -> concat -> top MLP -> sigmoid/BCE, its backward pass and the dense Adagrad update.
 #include "gemm.cuh"
+#include "profile.cuh"
 #include "mlp_plan.cuh"
 
 namespace ss {
@@ -69,9 +70,14 @@ __device__ __forceinline__ float load_kind(const void* p, int kind, int64_t i) {
 __global__ void __launch_bounds__(256)
 batch_reduce_partial_kernel(const __grid_constant__ RedJobs jobs, int B, int rows_per_split, float* __restrict__ partial) {
   __shared__ float part[8][32][kMaxSCols + 1];
-  int j = 0;
-  while (j + 1 < jobs.njobs && (int)blockIdx.x >= jobs.job[j + 1].tile0) ++j;
-  const RedJob& J = jobs.job[j];
+  __shared__ RedJob s_job;
+  if (threadIdx.x == 0) {
+    int j = 0;
+    while (j + 1 < jobs.njobs && (int)blockIdx.x >= jobs.job[j + 1].tile0) ++j;
+    s_job = jobs.job[j];
+  }
+  __syncthreads();
+  const RedJob J = s_job;                                    // the job's fields in registers
   const int cx = threadIdx.x & 31, ry = threadIdx.x >> 5;
   const int c = ((int)blockIdx.x - J.tile0) * 32 + cx;
   const int sc = J.s_cols;
@@ -81,11 +87,46 @@ batch_reduce_partial_kernel(const __grid_constant__ RedJobs jobs, int B, int row
 #pragma unroll
   for (int q = 0; q < kMaxSCols; ++q) acc[q] = 0.f;
   if (c < J.ncols) {
-    for (int b = r0 + ry; b < r1; b += 8) {
-      const float m = load_kind(J.M, J.m_kind, (int64_t)b * J.ldm + c);
-      if (J.S == nullptr) {
-        acc[0] += m;
-      } else {
+    if (J.S == nullptr) {
+      // column sums: four rows in flight per thread
+      int b = r0 + ry;
+      for (; b + 24 < r1; b += 32) {
+        const float m0 = load_kind(J.M, J.m_kind, (int64_t)b * J.ldm + c);
+        const float m1 = load_kind(J.M, J.m_kind, (int64_t)(b + 8) * J.ldm + c);
+        const float m2 = load_kind(J.M, J.m_kind, (int64_t)(b + 16) * J.ldm + c);
+        const float m3 = load_kind(J.M, J.m_kind, (int64_t)(b + 24) * J.ldm + c);
+        acc[0] = ((acc[0] + m0) + m1) + m2 + m3;
+      }
+      for (; b < r1; b += 8) acc[0] += load_kind(J.M, J.m_kind, (int64_t)b * J.ldm + c);
+    } else if (sc == 1) {
+      int b = r0 + ry;
+      for (; b + 24 < r1; b += 32) {
+        float m[4], s4[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          m[u] = load_kind(J.M, J.m_kind, (int64_t)(b + 8 * u) * J.ldm + c);
+          s4[u] = load_kind(J.S, J.s_kind, (int64_t)(b + 8 * u) * J.lds);
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) acc[0] = fmaf(m[u], s4[u], acc[0]);
+      }
+      for (; b < r1; b += 8)
+        acc[0] = fmaf(load_kind(J.M, J.m_kind, (int64_t)b * J.ldm + c), load_kind(J.S, J.s_kind, (int64_t)b * J.lds), acc[0]);
+    } else {
+      int b = r0 + ry;
+      for (; b + 8 < r1; b += 16) {
+        const float m0 = load_kind(J.M, J.m_kind, (int64_t)b * J.ldm + c);
+        const float m1 = load_kind(J.M, J.m_kind, (int64_t)(b + 8) * J.ldm + c);
+#pragma unroll
+        for (int q = 0; q < kMaxSCols; ++q)
+          if (q < sc) {
+            const float s0 = load_kind(J.S, J.s_kind, (int64_t)b * J.lds + q);
+            const float s1 = load_kind(J.S, J.s_kind, (int64_t)(b + 8) * J.lds + q);
+            acc[q] = fmaf(m1, s1, fmaf(m0, s0, acc[q]));
+          }
+      }
+      for (; b < r1; b += 8) {
+        const float m = load_kind(J.M, J.m_kind, (int64_t)b * J.ldm + c);
 #pragma unroll
         for (int q = 0; q < kMaxSCols; ++q)
           if (q < sc) acc[q] = fmaf(m, load_kind(J.S, J.s_kind, (int64_t)b * J.lds + q), acc[q]);
@@ -235,7 +276,9 @@ ss_status ss_mlp_fwd(const ss_mlp_desc* desc, const float* w, const void* w_bf16
     Bm = p.bf16 ? Operand{reinterpret_cast<const __nv_bfloat16*>(w_bf16) + L.w_off, OP_BF16, L.in, 1}
                 : Operand{w + L.w_off, OP_F32, L.in, 1};
     if (l == p.nl - 1) {   // one output unit: a dot product per sample
+      { SS_TIMED("rowdot_kernel", cs);
       rowdot_kernel<<<(B + 7) / 8, 256, 0, cs>>>(A.p, A.kind, A.s_row, Bm.p, Bm.kind, L.in, w + L.b_off, B, logit);
+      }
       SS_LAUNCH_OK();
       break;
     }
@@ -251,7 +294,9 @@ ss_status ss_mlp_fwd(const ss_mlp_desc* desc, const float* w, const void* w_bf16
     st = gemm(B, L.out, L.in, A, Bm, ep, cs);
     if (st != SS_OK) return st;
   }
+  { SS_TIMED("bce_loss_kernel", cs);
   bce_loss_kernel<<<1, 1024, 0, cs>>>(logit, labels, B, prob, loss);
+  }
   SS_LAUNCH_OK();
   return SS_OK;
 }
@@ -281,7 +326,9 @@ ss_status ss_mlp_bwd(const ss_mlp_desc* desc, float* w, void* w_bf16, float* ada
 
   const int last = p.nl - 1;
   const int dz_kind = p.bf16 ? OP_BF16 : OP_F32;
+  { SS_TIMED("dz_kernel", cs);
   dz_kernel<<<(B + 255) / 256, 256, 0, cs>>>(prob, labels, B, ws + p.dact[last], p.bf16);
+  }
   SS_LAUNCH_OK();
 
   RedJobs jobs;
@@ -323,8 +370,10 @@ ss_status ss_mlp_bwd(const ss_mlp_desc* desc, float* w, void* w_bf16, float* ada
     if (l == last && l != p.nb) {
       const void* wl = p.bf16 ? (const void*)(reinterpret_cast<const __nv_bfloat16*>(w_bf16) + L.w_off) : (const void*)(w + L.w_off);
       const int64_t cnt = (int64_t)B * L.in;
+      { SS_TIMED("outer_mask_kernel", cs);
       outer_mask_kernel<<<(unsigned)((cnt + 255) / 256), 256, 0, cs>>>(G, wl, ws + p.act[l - 1], dz_kind, act_kind, act_kind,
                                                                        B, L.in, ws + p.dact[l - 1], p.bf16);
+      }
       SS_LAUNCH_OK();
     } else {
       Operand A{G, act_kind, L.out, 1};
@@ -350,15 +399,21 @@ ss_status ss_mlp_bwd(const ss_mlp_desc* desc, float* w, void* w_bf16, float* ada
     int rows = ((B + p.red_splits - 1) / p.red_splits + 7) & ~7;
     const int nsplit = (B + rows - 1) / rows;
     float* partial = reinterpret_cast<float*>(ws + p.red_partial);
+    { SS_TIMED("batch_reduce_partial_kernel", cs);
     batch_reduce_partial_kernel<<<dim3(jobs.ntiles, nsplit), 256, 0, cs>>>(jobs, B, rows, partial);
+    }
+    { SS_TIMED("batch_reduce_final_kernel", cs);
     batch_reduce_final_kernel<<<(jobs.total + 255) / 256, 256, 0, cs>>>(jobs, nsplit, partial, g);
+    }
     SS_LAUNCH_OK();
   }
 
   if (apply_update) {
     const int64_t n4 = p.P / 4;
+    { SS_TIMED("adagrad_kernel", cs);
     adagrad_kernel<<<(unsigned)((n4 + 255) / 256), 256, 0, cs>>>(w, adagrad_acc, g,
                                                                  reinterpret_cast<__nv_bfloat16*>(w_bf16), n4, lr, eps);
+    }
     SS_LAUNCH_OK();
   }
   return SS_OK;

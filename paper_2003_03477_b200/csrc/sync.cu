@@ -6,6 +6,7 @@
 // every vector, which is what bounds the kernel (HBM for vectors beyond L2).  The replica pointers
 // travel in the kernel parameter block, so there is no pointer table in device memory.
 #include "common.cuh"
+#include "profile.cuh"
 
 namespace ss {
 
@@ -120,9 +121,13 @@ static ss_status launch_r(const SyncPtrs& p, bool mirror, float* c, float* delta
   if (blocks == 0) blocks = 1;
   if (blocks > 0x7fffffffLL) return SS_ERR_SHAPE;
   if (mirror)
+    { SS_TIMED("sync_kernel", st);
     sync_kernel<RULE, R, true><<<(unsigned)blocks, 256, 0, st>>>(p, c, delta, n4, n, s);
+    }
   else
+    { SS_TIMED("sync_kernel", st);
     sync_kernel<RULE, R, false><<<(unsigned)blocks, 256, 0, st>>>(p, c, delta, n4, n, s);
+    }
   SS_LAUNCH_OK();
   return SS_OK;
 }

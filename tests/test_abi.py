@@ -20,7 +20,7 @@ def lib():
 
 def _declared():
     names = set()
-    for h in ("shadowsync.h", "shadowsync_harness.h"):
+    for h in ("shadowsync.h", "shadowsync_harness.h", "shadowsync_profile.h"):
         src = open(os.path.join(ROOT, "include", h)).read()
         src = re.sub(r"/\*.*?\*/", "", src, flags=re.S)
         names |= set(re.findall(r"\b(ssh?_[a-z0-9_]+)\s*\(", src))
