@@ -200,8 +200,20 @@ __global__ void fill_keys_kernel(uint32_t* __restrict__ keys, int32_t* __restric
 }
 
 // ---- (2) radix sort pass ----------------------------------------------------------------
+// Lanes of the warp that hold the same digit, from one ballot per digit bit (cost independent of how many
+// distinct digits the warp holds).  `digit` is below 2^nbits, or exactly 2^nbits for a lane past the end.
+__device__ __forceinline__ uint32_t same_digit_lanes(uint32_t digit, int nbits) {
+  uint32_t peers = 0xffffffffu;
+  for (int b = 0; b <= nbits; ++b) {
+    const bool bit = (digit >> b) & 1u;
+    const uint32_t m = __ballot_sync(0xffffffffu, bit);
+    peers &= bit ? m : ~m;
+  }
+  return peers;
+}
+
 // hist[bin * nblk + blk] = number of keys of tile blk whose digit is bin.  Lanes holding the same
-// digit are counted together (match_any), so a hot row does not serialise on one counter.
+// digit are counted together, so a hot row does not serialise on one counter.
 __global__ void __launch_bounds__(kSortThreads)
 sort_hist_kernel(const uint32_t* __restrict__ keys, int64_t L, int shift, int bins, int nblk,
                  uint32_t* __restrict__ hist) {
@@ -211,6 +223,7 @@ sort_hist_kernel(const uint32_t* __restrict__ keys, int64_t L, int shift, int bi
   const int lane = threadIdx.x & 31;
   const int64_t base = (int64_t)blockIdx.x * kSortTile;
   const uint32_t mask = (uint32_t)bins - 1u;
+  const int nbits = 31 - __clz(bins);
   uint32_t digit[kSortIPT];
 #pragma unroll
   for (int k = 0; k < kSortIPT; ++k) {                      // all loads first, then the counting
@@ -219,7 +232,7 @@ sort_hist_kernel(const uint32_t* __restrict__ keys, int64_t L, int shift, int bi
   }
 #pragma unroll
   for (int k = 0; k < kSortIPT; ++k) {
-    const uint32_t peers = __match_any_sync(0xffffffffu, digit[k]);
+    const uint32_t peers = same_digit_lanes(digit[k], nbits);
     if (digit[k] < (uint32_t)bins && lane == (__ffs(peers) - 1))
       atomicAdd(&cnt[digit[k]], (uint32_t)__popc(peers));   // integer counts: order-free
   }
@@ -277,7 +290,7 @@ scan_exclusive_kernel(uint32_t* __restrict__ data, int64_t m, uint32_t* __restri
 }
 
 // Stable scatter: warp w of the block owns the contiguous items [w*512, (w+1)*512) of the tile and
-// walks them 32 at a time; rank inside a round comes from match_any, across rounds and warps from
+// walks them 32 at a time; rank inside a round comes from the lanes holding the same digit, across rounds and warps from
 // per-warp running counters that start at (bins before this digit) + (this digit in earlier tiles).
 __global__ void __launch_bounds__(kSortThreads)
 sort_scatter_kernel(const uint32_t* __restrict__ keys_in, const int32_t* __restrict__ pos_in,
@@ -308,6 +321,7 @@ sort_scatter_kernel(const uint32_t* __restrict__ keys_in, const int32_t* __restr
   }
   __syncthreads();
   const uint32_t mask = (uint32_t)bins - 1u;
+  const int nbits = 31 - __clz(bins);
   const int64_t wbase = (int64_t)blockIdx.x * kSortTile + (int64_t)warp * (32 * kSortIPT);
   uint32_t key[kSortIPT];
   uint32_t* mycnt = cnt + warp * bins;
@@ -317,7 +331,7 @@ sort_scatter_kernel(const uint32_t* __restrict__ keys_in, const int32_t* __restr
     const bool valid = i < L;
     key[k] = valid ? keys_in[i] : 0u;
     const uint32_t digit = valid ? ((key[k] >> shift) & mask) : (uint32_t)bins;   // invalid lanes pair up apart
-    const uint32_t peers = __match_any_sync(0xffffffffu, digit);
+    const uint32_t peers = same_digit_lanes(digit, nbits);
     if (valid && lane == (__ffs(peers) - 1)) mycnt[digit] += __popc(peers);
     __syncwarp();
   }
@@ -337,7 +351,7 @@ sort_scatter_kernel(const uint32_t* __restrict__ keys_in, const int32_t* __restr
     const int64_t i = wbase + k * 32 + lane;
     const bool valid = i < L;
     const uint32_t digit = valid ? ((key[k] >> shift) & mask) : (uint32_t)bins;
-    const uint32_t peers = __match_any_sync(0xffffffffu, digit);
+    const uint32_t peers = same_digit_lanes(digit, nbits);
     uint32_t dst = 0;
     if (valid) dst = mycnt[digit] + __popc(peers & ((1u << lane) - 1u));
     __syncwarp();

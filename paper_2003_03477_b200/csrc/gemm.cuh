@@ -37,7 +37,10 @@ struct Operand {
 ss_status gemm_simt(int M, int N, int K, const Operand& A, const Operand& B, const Epilogue& ep, cudaStream_t st);
 // bf16 operands on the tensor cores (tcgen05); see gemm_tc_eligible for what it accepts.
 bool gemm_tc_eligible(int M, int N, int K, const Operand& A, const Operand& B, const Epilogue& ep);
-ss_status gemm_tc(int M, int N, int K, const Operand& A, const Operand& B, const Epilogue& ep, cudaStream_t st);
+// k_splits > 1 cuts K into slices computed by different CTAs; slice z stores its fp32 partial product at
+// out_lo + z * split_stride (plain stores only: no bias, ReLU, mask or bf16 output); the caller adds the slices.
+ss_status gemm_tc(int M, int N, int K, const Operand& A, const Operand& B, const Epilogue& ep, cudaStream_t st,
+                  int k_splits, int64_t split_stride);
 // Tensor cores when eligible, SIMT otherwise.
 ss_status gemm(int M, int N, int K, const Operand& A, const Operand& B, const Epilogue& ep, cudaStream_t st);
 // The device error flag raised by a bounded wait that ran out (0 = none); synchronises the device.

@@ -38,6 +38,8 @@ __device__ int g_device_error = 0;   // 0 ok; otherwise the code of the first wa
 struct TcParams {
   int M, N, K;
   int a_mn, b_mn;          // 1 = MN-major operand
+  int k_splits;            // the K range is cut into this many slices (grid.z); slice z writes out_lo + z*split_stride
+  int64_t split_stride;    // in floats
   Epilogue ep;
   int* err;
 };
@@ -137,7 +139,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int m0 = blockIdx.y * kBM, n0 = blockIdx.x * kBN;
-  const int nk = (p.K + kBK - 1) / kBK;
+  const int nk_all = (p.K + kBK - 1) / kBK;
+  const int kb_begin = (int)((int64_t)nk_all * blockIdx.z / p.k_splits);
+  const int nk = (int)((int64_t)nk_all * (blockIdx.z + 1) / p.k_splits) - kb_begin;   // >= 1: k_splits <= nk_all
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) { mbar_init(full(s), 1); mbar_init(empty(s), 1); }
@@ -163,7 +167,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         mbar_wait(empty(s), ph ^ 1u, aborted, p.err, 1);
         mbar_expect_tx(full(s), kStageBytes);
         const uint32_t sa = tiles + s * kStageBytes, sb = sa + kTileBytes;
-        const int k0 = kb * kBK;
+        const int k0 = (kb_begin + kb) * kBK;
         if (p.a_mn) {                       // A stored [K, M]: two boxes of 64 k-rows x 64 m
           tma_load_2d(sa, &map_a, full(s), m0, k0);
           tma_load_2d(sa + kTileBytes / 2, &map_a, full(s), m0 + 64, k0);
@@ -252,7 +256,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             o.x = pack2(x[0], x[1]); o.y = pack2(x[2], x[3]); o.z = pack2(x[4], x[5]); o.w = pack2(x[6], x[7]);
             *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(ep.out_lo) + m * ep.ld_lo + n) = o;
           } else {
-            float4* o = reinterpret_cast<float4*>(reinterpret_cast<float*>(ep.out_lo) + m * ep.ld_lo + n);
+            float4* o = reinterpret_cast<float4*>(reinterpret_cast<float*>(ep.out_lo) + (int64_t)blockIdx.z * p.split_stride + m * ep.ld_lo + n);
             o[0] = make_float4(x[0], x[1], x[2], x[3]);
             o[1] = make_float4(x[4], x[5], x[6], x[7]);
           }
@@ -331,7 +335,8 @@ bool gemm_tc_eligible(int M, int N, int K, const Operand& A, const Operand& B, c
   return true;
 }
 
-ss_status gemm_tc(int M, int N, int K, const Operand& A, const Operand& B, const Epilogue& ep, cudaStream_t st) {
+ss_status gemm_tc(int M, int N, int K, const Operand& A, const Operand& B, const Epilogue& ep, cudaStream_t st,
+                  int k_splits, int64_t split_stride) {
   static bool attr_set[64];
   int dev = 0;
   SS_CUDA(cudaGetDevice(&dev));
@@ -343,6 +348,12 @@ ss_status gemm_tc(int M, int N, int K, const Operand& A, const Operand& B, const
   p.M = M; p.N = N; p.K = K;
   p.a_mn = (A.s_k != 1);
   p.b_mn = (B.s_k != 1);
+  const int nk_all = (K + kBK - 1) / kBK;
+  if (k_splits < 1) k_splits = 1;
+  if (k_splits > nk_all) k_splits = nk_all;
+  if (k_splits > 1 && (ep.lo_bf16 || ep.lo_cols < N || ep.bias || ep.relu || ep.mask)) return SS_ERR_SHAPE;   // slices are plain fp32 sums
+  p.k_splits = k_splits;
+  p.split_stride = split_stride;
   p.ep = ep;
   p.err = device_error_ptr();
   if (!p.err) return SS_ERR_CUDA;
@@ -350,7 +361,7 @@ ss_status gemm_tc(int M, int N, int K, const Operand& A, const Operand& B, const
   const bool oka = p.a_mn ? make_map(&ma, A.p, M, K, A.s_k, 64, 64) : make_map(&ma, A.p, K, M, A.s_row, 64, kBM);
   const bool okb = p.b_mn ? make_map(&mb, B.p, N, K, B.s_k, 64, 64) : make_map(&mb, B.p, K, N, B.s_row, 64, kBN);
   if (!oka || !okb) return SS_ERR_CUDA;
-  dim3 grid((N + kBN - 1) / kBN, (M + kBM - 1) / kBM);
+  dim3 grid((N + kBN - 1) / kBN, (M + kBM - 1) / kBM, k_splits);
   { SS_TIMED("gemm_tc_kernel", st);
   gemm_tc_kernel<<<grid, kTcThreads, kTcSmem, st>>>(ma, mb, p);
   }
@@ -371,7 +382,7 @@ int read_device_error(bool clear) {
 }
 
 ss_status gemm(int M, int N, int K, const Operand& A, const Operand& B, const Epilogue& ep, cudaStream_t st) {
-  if (gemm_tc_eligible(M, N, K, A, B, ep)) return gemm_tc(M, N, K, A, B, ep, st);
+  if (gemm_tc_eligible(M, N, K, A, B, ep)) return gemm_tc(M, N, K, A, B, ep, st, 1, 0);
   return gemm_simt(M, N, K, A, B, ep, st);
 }
 
@@ -394,7 +405,7 @@ ss_status ss_gemm_bf16(const void* a, int a_mn_major, int64_t lda, const void* b
   ep.out_lo = c; ep.lo_bf16 = 0; ep.ld_lo = ldc; ep.lo_cols = N;
   if (force_simt) return gemm_simt(M, N, K, A, B, ep, as_stream(stream));
   if (!gemm_tc_eligible(M, N, K, A, B, ep)) return SS_ERR_ALIGN;
-  return gemm_tc(M, N, K, A, B, ep, as_stream(stream));
+  return gemm_tc(M, N, K, A, B, ep, as_stream(stream), 1, 0);
 }
 
 }  // extern "C"

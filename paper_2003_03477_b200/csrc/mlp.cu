@@ -67,9 +67,12 @@ __device__ __forceinline__ float load_kind(const void* p, int kind, int64_t i) {
   return kind == OP_F32 ? v : __bfloat162float(__float2bfloat16_rn(v));
 }
 
+constexpr int kRedRows = 256;     // most rows of the batch a block takes (bounds the staged S tile)
+
 __global__ void __launch_bounds__(256)
 batch_reduce_partial_kernel(const __grid_constant__ RedJobs jobs, int B, int rows_per_split, float* __restrict__ partial) {
   __shared__ float part[8][32][kMaxSCols + 1];
+  __shared__ float s_tile[kRedRows * kMaxSCols];           // S rows of this block's batch slice, as float
   __shared__ RedJob s_job;
   if (threadIdx.x == 0) {
     int j = 0;
@@ -83,53 +86,37 @@ batch_reduce_partial_kernel(const __grid_constant__ RedJobs jobs, int B, int row
   const int sc = J.s_cols;
   const int r0 = blockIdx.y * rows_per_split;
   const int r1 = min(B, r0 + rows_per_split);
+  const int nrows = r1 - r0;
+  if (J.S != nullptr) {
+    for (int i = threadIdx.x; i < nrows * sc; i += 256) {
+      const int rr = i / sc, q = i - rr * sc;
+      s_tile[rr * kMaxSCols + q] = load_kind(J.S, J.s_kind, (int64_t)(r0 + rr) * J.lds + q);
+    }
+    __syncthreads();
+  }
   float acc[kMaxSCols];
 #pragma unroll
   for (int q = 0; q < kMaxSCols; ++q) acc[q] = 0.f;
   if (c < J.ncols) {
-    if (J.S == nullptr) {
-      // column sums: four rows in flight per thread
-      int b = r0 + ry;
-      for (; b + 24 < r1; b += 32) {
-        const float m0 = load_kind(J.M, J.m_kind, (int64_t)b * J.ldm + c);
-        const float m1 = load_kind(J.M, J.m_kind, (int64_t)(b + 8) * J.ldm + c);
-        const float m2 = load_kind(J.M, J.m_kind, (int64_t)(b + 16) * J.ldm + c);
-        const float m3 = load_kind(J.M, J.m_kind, (int64_t)(b + 24) * J.ldm + c);
-        acc[0] = ((acc[0] + m0) + m1) + m2 + m3;
-      }
-      for (; b < r1; b += 8) acc[0] += load_kind(J.M, J.m_kind, (int64_t)b * J.ldm + c);
-    } else if (sc == 1) {
-      int b = r0 + ry;
-      for (; b + 24 < r1; b += 32) {
-        float m[4], s4[4];
+    // four rows of M in flight per thread; rows are added in ascending order
+    for (int rr = ry; rr < nrows; rr += 32) {
+      float m[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u)
+        m[u] = (rr + 8 * u < nrows) ? load_kind(J.M, J.m_kind, (int64_t)(r0 + rr + 8 * u) * J.ldm + c) : 0.f;
+      if (J.S == nullptr) {
+#pragma unroll
+        for (int u = 0; u < 4; ++u) acc[0] += m[u];
+      } else {
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
-          m[u] = load_kind(J.M, J.m_kind, (int64_t)(b + 8 * u) * J.ldm + c);
-          s4[u] = load_kind(J.S, J.s_kind, (int64_t)(b + 8 * u) * J.lds);
-        }
+          if (rr + 8 * u < nrows) {
+            const float* srow = s_tile + (rr + 8 * u) * kMaxSCols;
 #pragma unroll
-        for (int u = 0; u < 4; ++u) acc[0] = fmaf(m[u], s4[u], acc[0]);
-      }
-      for (; b < r1; b += 8)
-        acc[0] = fmaf(load_kind(J.M, J.m_kind, (int64_t)b * J.ldm + c), load_kind(J.S, J.s_kind, (int64_t)b * J.lds), acc[0]);
-    } else {
-      int b = r0 + ry;
-      for (; b + 8 < r1; b += 16) {
-        const float m0 = load_kind(J.M, J.m_kind, (int64_t)b * J.ldm + c);
-        const float m1 = load_kind(J.M, J.m_kind, (int64_t)(b + 8) * J.ldm + c);
-#pragma unroll
-        for (int q = 0; q < kMaxSCols; ++q)
-          if (q < sc) {
-            const float s0 = load_kind(J.S, J.s_kind, (int64_t)b * J.lds + q);
-            const float s1 = load_kind(J.S, J.s_kind, (int64_t)(b + 8) * J.lds + q);
-            acc[q] = fmaf(m1, s1, fmaf(m0, s0, acc[q]));
+            for (int q = 0; q < kMaxSCols; ++q)
+              if (q < sc) acc[q] = fmaf(m[u], srow[q], acc[q]);
           }
-      }
-      for (; b < r1; b += 8) {
-        const float m = load_kind(J.M, J.m_kind, (int64_t)b * J.ldm + c);
-#pragma unroll
-        for (int q = 0; q < kMaxSCols; ++q)
-          if (q < sc) acc[q] = fmaf(m, load_kind(J.S, J.s_kind, (int64_t)b * J.lds + q), acc[q]);
+        }
       }
     }
   }
@@ -186,14 +173,38 @@ outer_mask_kernel(const void* __restrict__ dz, const void* __restrict__ w, const
   else reinterpret_cast<float*>(dX)[i] = v;
 }
 
-// Element-wise Adagrad over the flat parameter vector; refreshes the bf16 mirror.  A zero gradient
-// (pads, dead units) leaves the element untouched.
+// Weight gradients that were computed in K slices: slice z of layer t lies at gpart[off + z*size ...].
+struct SplitTable {
+  int n;
+  int64_t begin[kMaxLayers], end[kMaxLayers], off[kMaxLayers];
+  int nsplit[kMaxLayers];
+};
+
+// Element-wise Adagrad over the flat parameter vector; refreshes the bf16 mirror.  The gradient of an
+// element is the flat vector's value, or the sum of its K slices in slice order.  A zero gradient
+// (pads, dead units) leaves the element untouched.  g_out (nullable, may alias g) receives the gradient.
 __global__ void __launch_bounds__(256)
-adagrad_kernel(float* __restrict__ w, float* __restrict__ acc, const float* __restrict__ g,
-               __nv_bfloat16* __restrict__ mirror, int64_t n4, float lr, float eps) {
+adagrad_kernel(float* __restrict__ w, float* __restrict__ acc, const float* g, const float* __restrict__ gpart,
+               const __grid_constant__ SplitTable tab, __nv_bfloat16* __restrict__ mirror, int64_t n4, float lr,
+               float eps, float* g_out, int apply) {
   const int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x;
   if (i >= n4) return;
-  const float4 gv = reinterpret_cast<const float4*>(g)[i];
+  const int64_t e = i * 4;
+  float4 gv = reinterpret_cast<const float4*>(g)[i];
+  for (int t = 0; t < tab.n; ++t) {
+    if (e >= tab.begin[t] && e < tab.end[t]) {
+      const int64_t size = tab.end[t] - tab.begin[t];
+      const float4* p = reinterpret_cast<const float4*>(gpart + tab.off[t] + (e - tab.begin[t]));
+      gv = p[0];
+      for (int z = 1; z < tab.nsplit[t]; ++z) {
+        const float4 q = p[(int64_t)z * (size >> 2)];
+        gv.x += q.x; gv.y += q.y; gv.z += q.z; gv.w += q.w;
+      }
+      break;
+    }
+  }
+  if (g_out) reinterpret_cast<float4*>(g_out)[i] = gv;
+  if (!apply) return;
   float4 wv = reinterpret_cast<float4*>(w)[i];
   float4 av = reinterpret_cast<float4*>(acc)[i];
 #define SS_UPD(F)                                  \
@@ -331,6 +342,9 @@ ss_status ss_mlp_bwd(const ss_mlp_desc* desc, float* w, void* w_bf16, float* ada
   }
   SS_LAUNCH_OK();
 
+  float* gpart = reinterpret_cast<float*>(ws + p.gpart);
+  SplitTable tab;
+  tab.n = 0;
   RedJobs jobs;
   jobs.njobs = 0; jobs.ntiles = 0; jobs.total = 0;
   auto add_job = [&](const void* M, int m_kind, int64_t ldm, int ncols, const void* S, int s_kind, int64_t lds,
@@ -362,7 +376,16 @@ ss_status ss_mlp_bwd(const ss_mlp_desc* desc, float* w, void* w_bf16, float* ada
       Operand A{G, act_kind, 1, L.out};
       Epilogue ep;
       ep.out_lo = g + L.w_off; ep.lo_bf16 = 0; ep.ld_lo = L.in; ep.lo_cols = L.in;
-      st = gemm(L.out, L.in, B, A, X, ep, cs);
+      if (p.k_splits[l] > 1 && gemm_tc_eligible(L.out, L.in, B, A, X, ep)) {
+        // K = batch cut into slices; the update kernel adds them in slice order
+        const int64_t size = (int64_t)L.in * L.out;
+        ep.out_lo = gpart + p.gpart_off[l];
+        st = gemm_tc(L.out, L.in, B, A, X, ep, cs, p.k_splits[l], size);
+        const int t = tab.n++;
+        tab.begin[t] = L.w_off; tab.end[t] = L.w_off + size; tab.off[t] = p.gpart_off[l]; tab.nsplit[t] = p.k_splits[l];
+      } else {
+        st = gemm(L.out, L.in, B, A, X, ep, cs);
+      }
       if (st != SS_OK) return st;
     }
     if (l == 0) break;
@@ -396,7 +419,7 @@ ss_status ss_mlp_bwd(const ss_mlp_desc* desc, float* w, void* w_bf16, float* ada
   }
   {
     // all batch reductions of the pass in two launches
-    int rows = ((B + p.red_splits - 1) / p.red_splits + 7) & ~7;
+    int rows = ((B + p.red_splits - 1) / p.red_splits + 7) & ~7;   // <= kRedRows by the choice of red_splits
     const int nsplit = (B + rows - 1) / rows;
     float* partial = reinterpret_cast<float*>(ws + p.red_partial);
     { SS_TIMED("batch_reduce_partial_kernel", cs);
@@ -408,12 +431,12 @@ ss_status ss_mlp_bwd(const ss_mlp_desc* desc, float* w, void* w_bf16, float* ada
     SS_LAUNCH_OK();
   }
 
-  if (apply_update) {
+  if (apply_update || tab.n > 0) {
     const int64_t n4 = p.P / 4;
-    { SS_TIMED("adagrad_kernel", cs);
-    adagrad_kernel<<<(unsigned)((n4 + 255) / 256), 256, 0, cs>>>(w, adagrad_acc, g,
-                                                                 reinterpret_cast<__nv_bfloat16*>(w_bf16), n4, lr, eps);
-    }
+    SS_TIMED("adagrad_kernel", cs);
+    adagrad_kernel<<<(unsigned)((n4 + 255) / 256), 256, 0, cs>>>(w, adagrad_acc, g, gpart, tab,
+                                                                 reinterpret_cast<__nv_bfloat16*>(w_bf16), n4, lr, eps,
+                                                                 (grads || !apply_update) ? g : nullptr, apply_update);
     SS_LAUNCH_OK();
   }
   return SS_OK;

@@ -22,7 +22,9 @@ struct MlpPlan {
   // respect to it after the ReLU mask.  The last bottom layer's output lives in the concat buffer and
   // the last top layer's in logit[], so act[] is unused for those two.
   size_t act[kMaxLayers], dact[kMaxLayers];
-  size_t grads, red_partial, total;
+  size_t grads, red_partial, gpart, total;
+  int k_splits[kMaxLayers];      // K slices of the weight-gradient GEMM of each layer (1 = none)
+  int64_t gpart_off[kMaxLayers]; // float offset of the layer's slice buffer inside the gpart region
   int red_splits;         // batch slices of the two-stage reductions (bias and skinny weight gradients)
 };
 
@@ -63,12 +65,31 @@ inline ss_status make_mlp_plan(const ss_mlp_desc* d, int B, MlpPlan* p) {
     p->dact[l] = take(bytes);
   }
   p->grads = take((size_t)p->P * 4);
-  p->red_splits = B >= 1024 ? 16 : (B >= 256 ? 8 : (B >= 64 ? 2 : 1));
+  p->red_splits = B >= 1024 ? (B + 127) / 128 : (B >= 256 ? 8 : (B >= 64 ? 2 : 1));   // at most 128-row slices
   size_t red_total = 0;
   for (int l = 0; l < p->nl; ++l) red_total += (size_t)p->layer[l].out;
   red_total += (size_t)p->layer[p->nl - 1].in;
   if (p->layer[0].in <= 16) red_total += (size_t)p->layer[0].in * p->layer[0].out;
   p->red_partial = take(red_total * 4 * (size_t)p->red_splits);
+  // weight-gradient GEMMs contract over the batch and have small outputs: cut K so that about one
+  // wave of CTAs works on each of them; the slices are added in order by the update kernel
+  int64_t gp = 0;
+  const int nk = (B + 63) / 64;
+  for (int l = 0; l < p->nl; ++l) {
+    const LayerInfo& L = p->layer[l];
+    int s = 1;
+    if (p->bf16 && l != p->nl - 1 && !(l == 0 && L.in <= 16) && B >= 16) {
+      const int tiles = ((L.out + 127) / 128) * ((L.in + 127) / 128);
+      s = (148 + tiles - 1) / tiles;
+      if (s > 16) s = 16;
+      if (s > nk) s = nk;
+      if (s < 1) s = 1;
+    }
+    p->k_splits[l] = s;
+    p->gpart_off[l] = gp;
+    if (s > 1) gp += (int64_t)s * L.in * L.out;
+  }
+  p->gpart = take((size_t)gp * 4);
   p->total = o;
   return SS_OK;
 }
