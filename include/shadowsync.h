@@ -102,6 +102,19 @@ ss_status ss_embbag_bwd_adagrad(float* tables, float* row_state, int T, int64_t 
                                 int32_t* uniq_keys, int32_t* seg_off, int32_t* perm,
                                 int32_t* d_num_unique, int32_t* d_status, ss_stream stream);
 
+/* The same operation in two calls, so that its first half can be enqueued early on another stream:
+ * steps 1-2 depend only on the batch's indices, steps 3-4 also on the gradient.
+ *   ss_embbag_bwd_sort   steps 1-2 into the workspace (and the optional uniq_keys / seg_off / perm outputs)
+ *   ss_embbag_bwd_apply  steps 3-4 from a workspace that ss_embbag_bwd_sort filled for the same batch
+ * Arguments as in ss_embbag_bwd_adagrad; the caller orders the two calls (same stream, or an event). */
+ss_status ss_embbag_bwd_sort(int T, int64_t N, int D, const int32_t* indices, const int32_t* offsets, int B,
+                             int64_t L, void* workspace, size_t workspace_bytes,
+                             int32_t* uniq_keys, int32_t* seg_off, int32_t* perm,
+                             int32_t* d_num_unique, int32_t* d_status, ss_stream stream);
+ss_status ss_embbag_bwd_apply(float* tables, float* row_state, int T, int64_t N, int D, int B, int64_t L,
+                              const float* grad, int64_t ld_grad, int col0, float lr, float eps,
+                              void* workspace, size_t workspace_bytes, ss_stream stream);
+
 /* ------------------------------------------------------------------------------------------
  * Bottom MLP, concat interaction, top MLP, sigmoid + binary cross-entropy (Section 3.1, Fig. 1;
  * "Trainer": forward pass, then gradients for all parameters, local parameters updated directly).

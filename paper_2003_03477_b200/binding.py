@@ -23,7 +23,7 @@ SS_DEV_BAD_INDEX, SS_DEV_BAD_OFFSET = 1, 2
 SS_SYNC_EASGD_LITERAL = 1
 
 EXPORTS = ["ss_status_str", "ss_last_cuda_error", "ss_num_sms", "ss_embbag_fwd", "ss_embbag_bwd_workspace_bytes",
-           "ss_embbag_bwd_adagrad", "ss_mlp_param_count", "ss_mlp_param_offsets", "ss_mlp_workspace_bytes",
+           "ss_embbag_bwd_adagrad", "ss_embbag_bwd_sort", "ss_embbag_bwd_apply", "ss_mlp_param_count", "ss_mlp_param_offsets", "ss_mlp_workspace_bytes",
            "ss_mlp_fwd", "ss_mlp_bwd", "ss_sync_easgd", "ss_sync_ma", "ss_sync_bmuf", "ss_to_bf16",
            "ss_gemm_bf16", "ss_device_error", "ssh_fill_uniform", "ss_profile", "ss_profile_collect"]
 
@@ -64,6 +64,8 @@ def lib() -> C.CDLL:
         L.ss_embbag_bwd_workspace_bytes.argtypes = [i32, i64, i32, i32, i64]
         L.ss_embbag_bwd_adagrad.argtypes = [vp, vp, i32, i64, i32, vp, vp, i32, i64, vp, i64, i32, f32, f32,
                                             vp, sz, vp, vp, vp, vp, vp, vp]
+        L.ss_embbag_bwd_sort.argtypes = [i32, i64, i32, vp, vp, i32, i64, vp, sz, vp, vp, vp, vp, vp, vp]
+        L.ss_embbag_bwd_apply.argtypes = [vp, vp, i32, i64, i32, i32, i64, vp, i64, i32, f32, f32, vp, sz, vp]
         L.ss_mlp_param_count.restype = i64
         L.ss_mlp_param_count.argtypes = [C.POINTER(MlpDesc)]
         L.ss_mlp_param_offsets.argtypes = [C.POINTER(MlpDesc), C.POINTER(i64), C.POINTER(i64)]
@@ -180,6 +182,20 @@ def ss_embbag_bwd_adagrad(tables, row_state, T, N, D, indices, offsets, B, L, gr
                                        _ptr(grad), ld_grad, col0, lr, eps, _ptr(workspace),
                                        workspace.numel() * workspace.element_size(), _ptr(uniq_keys), _ptr(seg_off),
                                        _ptr(perm), _ptr(d_num_unique), _ptr(d_status), _stream(stream)))
+
+
+def ss_embbag_bwd_sort(T, N, D, indices, offsets, B, L, workspace, uniq_keys, seg_off, perm, d_num_unique, d_status,
+                       stream=None) -> None:
+    _check("ss_embbag_bwd_sort",
+           lib().ss_embbag_bwd_sort(T, N, D, _ptr(indices), _ptr(offsets), B, L, _ptr(workspace),
+                                    workspace.numel() * workspace.element_size(), _ptr(uniq_keys), _ptr(seg_off),
+                                    _ptr(perm), _ptr(d_num_unique), _ptr(d_status), _stream(stream)))
+
+
+def ss_embbag_bwd_apply(tables, row_state, T, N, D, B, L, grad, ld_grad, col0, lr, eps, workspace, stream=None) -> None:
+    _check("ss_embbag_bwd_apply",
+           lib().ss_embbag_bwd_apply(_ptr(tables), _ptr(row_state), T, N, D, B, L, _ptr(grad), ld_grad, col0, lr, eps,
+                                     _ptr(workspace), workspace.numel() * workspace.element_size(), _stream(stream)))
 
 
 def ss_mlp_fwd(spec: MlpSpec, w, w_bf16, dense, concat_f32, concat_bf16, B, labels, logit, prob, loss, workspace,

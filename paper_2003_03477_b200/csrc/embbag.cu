@@ -57,25 +57,25 @@ embbag_fwd_kernel(const float* __restrict__ tables, int T, int64_t N, int D,
 #pragma unroll
   for (int v = 0; v < NV; ++v) acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
 
-  for (int j = lo; j < hi; j += 4) {
-    int idx[4];
-    bool ok[4];
+  // kRows lookups per round: their indices are loaded first, then their rows
+  constexpr int kRows = 4;
+  for (int j = lo; j < hi; j += kRows) {
+    int idx[kRows];
 #pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      idx[u] = (j + u < hi) ? indices[j + u] : -1;
-      ok[u] = (idx[u] >= 0) && (idx[u] < N);
-      if (j + u < hi && !ok[u]) bad |= SS_DEV_BAD_INDEX;
-    }
-    float4 rowv[4][NV];
+    for (int u = 0; u < kRows; ++u) idx[u] = (j + u < hi) ? indices[j + u] : 0;
+    float4 rowv[kRows][NV];
 #pragma unroll
-    for (int u = 0; u < 4; ++u)
+    for (int u = 0; u < kRows; ++u) {
+      const bool ok = (j + u < hi) && (idx[u] >= 0) && (idx[u] < N);
+      if (j + u < hi && !ok) bad |= SS_DEV_BAD_INDEX;
 #pragma unroll
       for (int v = 0; v < NV; ++v) {
         const int c = lane + v * G;
-        rowv[u][v] = (ok[u] && c < nvec) ? tab[(int64_t)idx[u] * nvec + c] : make_float4(0.f, 0.f, 0.f, 0.f);
+        rowv[u][v] = (ok && c < nvec) ? tab[(int64_t)idx[u] * nvec + c] : make_float4(0.f, 0.f, 0.f, 0.f);
       }
+    }
 #pragma unroll
-    for (int u = 0; u < 4; ++u)          // lookups are added in bag order
+    for (int u = 0; u < kRows; ++u)      // lookups are added in bag order
 #pragma unroll
       for (int v = 0; v < NV; ++v) acc[v] = add4(acc[v], rowv[u][v]);
   }
@@ -477,7 +477,7 @@ window_reduce_kernel(const uint32_t* __restrict__ keys, const int32_t* __restric
 #pragma unroll
   for (int v = 0; v < NV; ++v) acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
   int run_start = 0;
-  constexpr int kBatch = NV >= 8 ? 1 : (NV >= 4 ? 2 : (NV >= 2 ? 4 : 8));   // gradient rows in flight per lane
+  constexpr int kBatch = NV >= 8 ? 2 : (NV >= 4 ? 4 : (NV >= 2 ? 8 : 16));  // gradient rows in flight per lane
   for (int i0 = 0; i0 < kWin; i0 += kBatch) {
     float4 gv[kBatch][NV];
 #pragma unroll
@@ -510,7 +510,10 @@ window_reduce_kernel(const uint32_t* __restrict__ keys, const int32_t* __restric
           acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
         }
         // the window in which a multi-window run starts enters the row in the list of rows to combine
-        if (!head_open && tail_open && lane == 0) long_list[atomicAdd(&scalars[1], 1)] = s_u[grp][i];
+        if (!head_open && tail_open && lane == 0) {
+          const int slot = atomicAdd(&scalars[1], 1);
+          if (slot < nwin) long_list[slot] = s_u[grp][i];   // at most one such run per window
+        }
         run_start = i + 1;
       }
     }
@@ -525,13 +528,13 @@ window_reduce_kernel(const uint32_t* __restrict__ keys, const int32_t* __restric
 template <int G, int NV>
 __global__ void __launch_bounds__(256)
 combine_rows_kernel(const int32_t* __restrict__ seg, const int32_t* __restrict__ scalars,
-                    const int32_t* __restrict__ long_list, int D, const float* __restrict__ partial,
+                    const int32_t* __restrict__ long_list, int nwin, int D, const float* __restrict__ partial,
                     float* __restrict__ gsum) {
   constexpr int kGroups = 256 / G;
   extern __shared__ float4 s_part[];                       // [kGroups][D/4]
   const int grp = threadIdx.x / G, lane = threadIdx.x % G;
   const int nvec = D >> 2;
-  const int n = scalars[1];
+  const int n = min(scalars[1], nwin);
   constexpr int kShort = 4;                                // spans up to this many windows: one group per row
   // phase A: short spans, one lane group per listed row, all partial loads issued together
   for (int i = blockIdx.x * kGroups + grp; i < n; i += gridDim.x * kGroups) {
@@ -602,13 +605,13 @@ combine_rows_kernel(const int32_t* __restrict__ seg, const int32_t* __restrict__
   }
 }
 
-// ---- (6) row-wise Adagrad, one lane group per two distinct rows ----------------------------------
+// ---- (6) row-wise Adagrad, one lane group per four distinct rows ----------------------------------
 //   g = gsum[u];  s = state + mean_d g^2;  row -= lr * g / (sqrt(s) + eps)
-template <int NV> struct RowsPerGroup { static constexpr int value = NV == 1 ? 2 : 1; };
+template <int NV> struct RowsPerGroup { static constexpr int value = NV == 1 ? 4 : (NV == 2 ? 2 : 1); };
 
 template <int G, int NV>
 __global__ void __launch_bounds__(256)
-apply_rows_kernel(const int32_t* __restrict__ uniq, const int32_t* __restrict__ scalars, int D,
+apply_rows_kernel(const int32_t* __restrict__ uniq, int32_t* __restrict__ scalars, int D,
                   const float* __restrict__ gsum, float* __restrict__ tables, float* __restrict__ row_state,
                   float lr, float eps) {
   constexpr int kGroups = 256 / G;
@@ -616,6 +619,8 @@ apply_rows_kernel(const int32_t* __restrict__ uniq, const int32_t* __restrict__ 
   const int grp = threadIdx.x / G, lane = threadIdx.x % G;
   const unsigned gmask = (G == 32) ? 0xffffffffu : (((1u << G) - 1u) << ((threadIdx.x & 31) / G * G));
   const int U = scalars[0];
+  // the list of multi-window rows has been consumed by the previous kernel: empty it for the next reduction
+  if (blockIdx.x == 0 && threadIdx.x == 0) scalars[1] = 0;
   const int nvec = D >> 2;
   const int64_t u0 = ((int64_t)blockIdx.x * kGroups + grp) * RB;
   if (u0 >= U) return;
@@ -687,7 +692,7 @@ static void launch_reduce(const BwdPlan& p, char* ws, const uint32_t* keys, cons
   {
     SS_TIMED("combine_rows_kernel", st);
     const int cblocks = p.nwin < num_sms() * 8 ? p.nwin : num_sms() * 8;
-    combine_rows_kernel<G, NV><<<cblocks, 256, (size_t)kGroups * D * 4, st>>>(seg, scalars, long_list, D, partial, gsum);
+    combine_rows_kernel<G, NV><<<cblocks, 256, (size_t)kGroups * D * 4, st>>>(seg, scalars, long_list, p.nwin, D, partial, gsum);
   }
   const uint64_t maxkey = (uint64_t)T * (uint64_t)N;
   const uint64_t umax = (uint64_t)p.L < maxkey ? (uint64_t)p.L : maxkey;
@@ -746,17 +751,22 @@ size_t ss_embbag_bwd_workspace_bytes(int T, int64_t N, int D, int B, int64_t L) 
   return ss::make_plan(T, N, D, L).total;
 }
 
-ss_status ss_embbag_bwd_adagrad(float* tables, float* row_state, int T, int64_t N, int D, const int32_t* indices,
-                                const int32_t* offsets, int B, int64_t L, const float* grad, int64_t ld_grad,
-                                int col0, float lr, float eps, void* workspace, size_t workspace_bytes,
-                                int32_t* uniq_keys, int32_t* seg_off, int32_t* perm, int32_t* d_num_unique,
-                                int32_t* d_status, ss_stream stream) {
+static ss_status bwd_impl(bool do_sort, bool do_apply, float* tables, float* row_state, int T, int64_t N, int D,
+                          const int32_t* indices, const int32_t* offsets, int B, int64_t L, const float* grad,
+                          int64_t ld_grad, int col0, float lr, float eps, void* workspace, size_t workspace_bytes,
+                          int32_t* uniq_keys, int32_t* seg_off, int32_t* perm, int32_t* d_num_unique,
+                          int32_t* d_status, ss_stream stream) {
   using namespace ss;
-  if (!tables || !row_state || (!indices && L > 0) || !offsets || !grad || !workspace) return SS_ERR_NULL;
+  if (!workspace) return SS_ERR_NULL;
+  if (do_sort && ((!indices && L > 0) || !offsets)) return SS_ERR_NULL;
+  if (do_apply && (!tables || !row_state || !grad)) return SS_ERR_NULL;
   if (T < 0 || B < 0 || N <= 0 || D <= 0 || D > 1024 || (D & 3) || col0 < 0 || L < 0) return SS_ERR_SHAPE;
   if ((uint64_t)T * (uint64_t)N >= (1ull << 31) || L >= (1ll << 31) - kSortTile) return SS_ERR_SHAPE;
-  if (!aligned16(tables) || !aligned16(grad) || (ld_grad & 3) || (col0 & 3) || !aligned16(workspace)) return SS_ERR_ALIGN;
-  if (ld_grad < col0 + (int64_t)T * D || (int64_t)B * ld_grad / 4 >= (1ll << 31)) return SS_ERR_SHAPE;
+  if (!aligned16(workspace)) return SS_ERR_ALIGN;
+  if (do_apply) {
+    if (!aligned16(tables) || !aligned16(grad) || (ld_grad & 3) || (col0 & 3)) return SS_ERR_ALIGN;
+    if (ld_grad < col0 + (int64_t)T * D || (int64_t)B * ld_grad / 4 >= (1ll << 31)) return SS_ERR_SHAPE;
+  }
   const BwdPlan p = make_plan(T, N, D, L);
   if (workspace_bytes < p.total) return SS_ERR_WORKSPACE;
   ss_status stt = check_arch();
@@ -778,12 +788,17 @@ ss_status ss_embbag_bwd_adagrad(float* tables, float* row_state, int T, int64_t 
   const uint32_t sentinel = (uint32_t)((uint64_t)T * (uint64_t)N);
 
   if (L == 0 || (int64_t)T * B == 0) {
-    { SS_TIMED("unique_finish_kernel", cs);
-    unique_finish_kernel<<<1, 1, 0, cs>>>(nullptr, seg, seg_off, d_num_unique, scalars);
+    if (do_sort) {
+      SS_TIMED("unique_finish_kernel", cs);
+      unique_finish_kernel<<<1, 1, 0, cs>>>(nullptr, seg, seg_off, d_num_unique, scalars);
+      SS_LAUNCH_OK();
     }
-    SS_LAUNCH_OK();
     return SS_OK;
   }
+  // the sorted arrays end up in the buffers the last pass wrote
+  const uint32_t* keys_sorted = (p.passes & 1) ? keys_b : keys_a;
+  const int32_t* perm_sorted = (p.passes & 1) ? pos_b : pos_a;
+  if (do_sort) {
 
   // (1) keys; positions no bag owns (malformed offsets) keep the sentinel
   { SS_TIMED("fill_keys_kernel", cs);
@@ -816,8 +831,6 @@ ss_status ss_embbag_bwd_adagrad(float* tables, float* row_state, int T, int64_t 
     uint32_t* tk = kin; kin = kout; kout = tk;
     pin = pout; pout = pnext; pnext = pin;
   }
-  const uint32_t* keys_sorted = kin;
-  const int32_t* perm_sorted = pin;
   if (perm) SS_CUDA(cudaMemcpyAsync(perm, perm_sorted, (size_t)L * 4, cudaMemcpyDeviceToDevice, cs));
 
   // (3) unique keys and segment offsets
@@ -835,13 +848,40 @@ ss_status ss_embbag_bwd_adagrad(float* tables, float* row_state, int T, int64_t 
   }
   SS_LAUNCH_OK();
 
-  // (4) windowed segment reduction, (5) row-wise Adagrad
+  }  // do_sort
+
+  // (4) windowed segment reduction, (5) combine, (6) row-wise Adagrad
+  if (do_apply) {
 #define SS_RED(G_, NV_) \
   launch_reduce<G_, NV_>(p, ws, keys_sorted, perm_sorted, T, N, D, B, grad, ld_grad, col0, tables, row_state, lr, eps, cs)
-  SS_DISPATCH_GNV(D, SS_RED);
+    SS_DISPATCH_GNV(D, SS_RED);
 #undef SS_RED
-  SS_LAUNCH_OK();
+    SS_LAUNCH_OK();
+  }
   return SS_OK;
+}
+
+ss_status ss_embbag_bwd_adagrad(float* tables, float* row_state, int T, int64_t N, int D, const int32_t* indices,
+                                const int32_t* offsets, int B, int64_t L, const float* grad, int64_t ld_grad,
+                                int col0, float lr, float eps, void* workspace, size_t workspace_bytes,
+                                int32_t* uniq_keys, int32_t* seg_off, int32_t* perm, int32_t* d_num_unique,
+                                int32_t* d_status, ss_stream stream) {
+  return bwd_impl(true, true, tables, row_state, T, N, D, indices, offsets, B, L, grad, ld_grad, col0, lr, eps, workspace,
+                  workspace_bytes, uniq_keys, seg_off, perm, d_num_unique, d_status, stream);
+}
+
+ss_status ss_embbag_bwd_sort(int T, int64_t N, int D, const int32_t* indices, const int32_t* offsets, int B, int64_t L,
+                             void* workspace, size_t workspace_bytes, int32_t* uniq_keys, int32_t* seg_off,
+                             int32_t* perm, int32_t* d_num_unique, int32_t* d_status, ss_stream stream) {
+  return bwd_impl(true, false, nullptr, nullptr, T, N, D, indices, offsets, B, L, nullptr, 0, 0, 0.f, 0.f, workspace,
+                  workspace_bytes, uniq_keys, seg_off, perm, d_num_unique, d_status, stream);
+}
+
+ss_status ss_embbag_bwd_apply(float* tables, float* row_state, int T, int64_t N, int D, int B, int64_t L,
+                              const float* grad, int64_t ld_grad, int col0, float lr, float eps, void* workspace,
+                              size_t workspace_bytes, ss_stream stream) {
+  return bwd_impl(false, true, tables, row_state, T, N, D, nullptr, nullptr, B, L, grad, ld_grad, col0, lr, eps, workspace,
+                  workspace_bytes, nullptr, nullptr, nullptr, nullptr, nullptr, stream);
 }
 
 }  // extern "C"

@@ -61,6 +61,7 @@ class Replica:
             self.seg_off = torch.empty(max_L + 1, dtype=torch.int32, device=dev)
             self.perm = torch.empty(max_L, dtype=torch.int32, device=dev)
         self.stream = torch.cuda.Stream(device=dev, priority=priority)
+        self.side = torch.cuda.Stream(device=dev, priority=priority)   # the index sort of the backward runs here
         self.steps_done = 0
 
 
@@ -89,20 +90,39 @@ class Model:
         torch.cuda.synchronize()
 
     # ---------------------------------------------------------------- training step of one replica
-    def step(self, r: int, batch: DeviceBatch, stream: Optional[torch.cuda.Stream] = None) -> None:
-        """Enqueue one worker iteration of Algorithm 1 for replica r on its stream (no synchronisation)."""
+    def step(self, r: int, batch: DeviceBatch, stream: Optional[torch.cuda.Stream] = None,
+             overlap_sort: bool = True) -> None:
+        """Enqueue one worker iteration of Algorithm 1 for replica r on its stream (no synchronisation).
+
+        With overlap_sort the sort / unique half of the embedding backward, which needs only the batch's
+        indices, is forked onto the replica's side stream at the start of the step and joined before the
+        gradient reduction, so it runs under the forward and backward passes of the MLP.
+        """
         rep, sp = self.replicas[r], self.spec
         s = stream or rep.stream
         T, N, D, B = self.T, self.N, self.D, self.B
+        if overlap_sort:
+            fork = torch.cuda.Event()
+            fork.record(s)
+            rep.side.wait_event(fork)
+            ss.ss_embbag_bwd_sort(T, N, D, batch.indices, batch.offsets, B, batch.L, rep.emb_ws, rep.uniq_keys,
+                                  rep.seg_off, rep.perm, rep.num_unique, self.d_status, rep.side)
+            join = torch.cuda.Event()
+            join.record(rep.side)
         ss.ss_embbag_fwd(self.tables, T, N, D, batch.indices, batch.offsets, B, rep.concat_f32, sp.W,
                          rep.concat_bf16, sp.W, D, self.d_status, s)
         ss.ss_mlp_fwd(sp, rep.w, rep.w_bf16, batch.dense, rep.concat_f32, rep.concat_bf16, B, batch.labels,
                       rep.logit, rep.prob, rep.loss, rep.mlp_ws, s)
         ss.ss_mlp_bwd(sp, rep.w, rep.w_bf16, rep.acc, None, batch.dense, rep.concat_f32, rep.concat_bf16,
                       batch.labels, rep.prob, B, self.lr, self.eps, 1, rep.grad_pooled, T * D, rep.mlp_ws, s)
-        ss.ss_embbag_bwd_adagrad(self.tables, self.row_state, T, N, D, batch.indices, batch.offsets, B, batch.L,
-                                 rep.grad_pooled, T * D, 0, self.lr, self.eps, rep.emb_ws, rep.uniq_keys,
-                                 rep.seg_off, rep.perm, rep.num_unique, self.d_status, s)
+        if overlap_sort:
+            s.wait_event(join)
+            ss.ss_embbag_bwd_apply(self.tables, self.row_state, T, N, D, B, batch.L, rep.grad_pooled, T * D, 0,
+                                   self.lr, self.eps, rep.emb_ws, s)
+        else:
+            ss.ss_embbag_bwd_adagrad(self.tables, self.row_state, T, N, D, batch.indices, batch.offsets, B, batch.L,
+                                     rep.grad_pooled, T * D, 0, self.lr, self.eps, rep.emb_ws, rep.uniq_keys,
+                                     rep.seg_off, rep.perm, rep.num_unique, self.d_status, s)
         rep.steps_done += 1
 
     # ---------------------------------------------------------------- one synchronisation pass

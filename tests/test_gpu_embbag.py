@@ -169,3 +169,30 @@ def test_device_table_fill_matches_host_generator():
     cfg = synth.scaled(synth.CONFIGS["tiny"], T=3, N=1000, D=16)
     dev = trainer.device_tables(cfg).cpu().numpy()
     assert np.array_equal(dev, synth.tables_dense(cfg))
+
+
+def test_sort_once_apply_twice_matches_two_oracle_updates():
+    # the two-call form: the sort half fills the workspace, the apply half may be repeated on it
+    cfg = synth.scaled(synth.CONFIGS["medium"], T=3, N=4000, D=64, B=256, bottom=(13, 64, 64), top=(256, 64, 1))
+    b = synth.make_batch(cfg, 0, 1)
+    tables = synth.tables_dense(cfg)
+    state = np.zeros((cfg.T, cfg.N), np.float32)
+    rng = np.random.default_rng(3)
+    gp = (rng.normal(size=(cfg.B, cfg.T * cfg.D)) * 1e-3).astype(np.float32)
+    t_o, s_o = tables.copy(), state.copy()
+    for _ in range(3):
+        uniq, seg, perm = O.embbag_bwd_adagrad(t_o, s_o, b.indices, b.offsets, cfg.B, gp, cfg.lr, cfg.eps)
+    T, N, D, B, L = cfg.T, cfg.N, cfg.D, cfg.B, b.L
+    dt, ds = _cuda(tables), _cuda(state.reshape(-1))
+    ws = torch.empty(ss.ss_embbag_bwd_workspace_bytes(T, N, D, B, L), dtype=torch.uint8, device="cuda")
+    nu = torch.zeros(1, dtype=torch.int32, device="cuda")
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    perm_d = torch.empty(L, dtype=torch.int32, device="cuda")
+    ss.ss_embbag_bwd_sort(T, N, D, _cuda(b.indices), _cuda(b.offsets), B, L, ws, None, None, perm_d, nu, st)
+    dg = _cuda(gp)
+    for _ in range(3):
+        ss.ss_embbag_bwd_apply(dt, ds, T, N, D, B, L, dg, T * D, 0, cfg.lr, cfg.eps, ws)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0 and int(nu.item()) == len(uniq) and np.array_equal(perm_d.cpu().numpy(), perm)
+    assert_close(dt.cpu().numpy() - tables, t_o.astype(np.float64) - tables, 2e-5, "tables after three updates")
+    assert_close(ds.cpu().numpy().reshape(T, N), s_o, RTOL_F32, "row state")
