@@ -115,6 +115,31 @@ ss_status ss_embbag_bwd_apply(float* tables, float* row_state, int T, int64_t N,
                               const float* grad, int64_t ld_grad, int col0, float lr, float eps,
                               void* workspace, size_t workspace_bytes, ss_stream stream);
 
+/* The sort / unique half once more, for callers that cannot allocate.  (The paper has no counterpart:
+ * this entry point exists only for how the library is embedded.)
+ *
+ * ss_embbag_bwd_sort needs a workspace, and whoever calls it has to get that memory from somewhere.
+ * Not every caller can: a process whose allocator has already given the whole GPU to other owners, a
+ * plug-in inside another program's serving loop that must not trigger cudaMalloc's device-wide
+ * synchronisation, or code that runs before the application's memory pool is up.  This variant takes
+ * no workspace.  Its scratch is a fixed array of 2112 KiB compiled into the library, which every GPU
+ * that loads the library keeps until the process ends, so the size is capped:
+ *     L <= 65536 lookups per call, otherwise SS_ERR_SHAPE (use ss_embbag_bwd_sort with a workspace).
+ * It calls no cudaMalloc / cudaFree and no routine that allocates.
+ *
+ * Inputs as for ss_embbag_bwd_sort (no D: the sort does not depend on the row width).  Outputs, all
+ * required: uniq_keys[L], seg_off[L+1], perm[L], *d_num_unique, bit-identical to ss_embbag_bwd_sort's.
+ * The row update is not part of it: ss_embbag_bwd_apply wants the workspace of ss_embbag_bwd_sort.
+ *
+ * The first call on a device looks up the device address of the built-in array (one
+ * cudaGetSymbolAddress); make that first call before any stream capture begins.  All calls, from
+ * every thread and stream, share the one array: two calls that may run on the GPU at the same time
+ * race and produce garbage, so put them on one stream or order them with events.  The array keeps
+ * whatever the last call wrote; each call rewrites every part it reads, so no clearing is needed. */
+ss_status ss_embbag_bwd_sort_noalloc(int T, int64_t N, const int32_t* indices, const int32_t* offsets, int B,
+                                     int64_t L, int32_t* uniq_keys, int32_t* seg_off, int32_t* perm,
+                                     int32_t* d_num_unique, int32_t* d_status, ss_stream stream);
+
 /* ------------------------------------------------------------------------------------------
  * Bottom MLP, concat interaction, top MLP, sigmoid + binary cross-entropy (Section 3.1, Fig. 1;
  * "Trainer": forward pass, then gradients for all parameters, local parameters updated directly).

@@ -23,7 +23,7 @@ SS_DEV_BAD_INDEX, SS_DEV_BAD_OFFSET = 1, 2
 SS_SYNC_EASGD_LITERAL = 1
 
 EXPORTS = ["ss_status_str", "ss_last_cuda_error", "ss_num_sms", "ss_embbag_fwd", "ss_embbag_bwd_workspace_bytes",
-           "ss_embbag_bwd_adagrad", "ss_embbag_bwd_sort", "ss_embbag_bwd_apply", "ss_mlp_param_count", "ss_mlp_param_offsets", "ss_mlp_workspace_bytes",
+           "ss_embbag_bwd_adagrad", "ss_embbag_bwd_sort", "ss_embbag_bwd_apply", "ss_embbag_bwd_sort_noalloc", "ss_mlp_param_count", "ss_mlp_param_offsets", "ss_mlp_workspace_bytes",
            "ss_mlp_fwd", "ss_mlp_bwd", "ss_sync_easgd", "ss_sync_ma", "ss_sync_bmuf", "ss_to_bf16",
            "ss_gemm_bf16", "ss_device_error", "ssh_fill_uniform", "ss_profile", "ss_profile_collect"]
 
@@ -66,6 +66,7 @@ def lib() -> C.CDLL:
                                             vp, sz, vp, vp, vp, vp, vp, vp]
         L.ss_embbag_bwd_sort.argtypes = [i32, i64, i32, vp, vp, i32, i64, vp, sz, vp, vp, vp, vp, vp, vp]
         L.ss_embbag_bwd_apply.argtypes = [vp, vp, i32, i64, i32, i32, i64, vp, i64, i32, f32, f32, vp, sz, vp]
+        L.ss_embbag_bwd_sort_noalloc.argtypes = [i32, i64, vp, vp, i32, i64, vp, vp, vp, vp, vp, vp]
         L.ss_mlp_param_count.restype = i64
         L.ss_mlp_param_count.argtypes = [C.POINTER(MlpDesc)]
         L.ss_mlp_param_offsets.argtypes = [C.POINTER(MlpDesc), C.POINTER(i64), C.POINTER(i64)]
@@ -196,6 +197,14 @@ def ss_embbag_bwd_apply(tables, row_state, T, N, D, B, L, grad, ld_grad, col0, l
     _check("ss_embbag_bwd_apply",
            lib().ss_embbag_bwd_apply(_ptr(tables), _ptr(row_state), T, N, D, B, L, _ptr(grad), ld_grad, col0, lr, eps,
                                      _ptr(workspace), workspace.numel() * workspace.element_size(), _stream(stream)))
+
+
+def ss_embbag_bwd_sort_noalloc(T, N, indices, offsets, B, L, uniq_keys, seg_off, perm, d_num_unique, d_status,
+                               stream=None) -> None:
+    """Sort / unique with the library's built-in scratch (no workspace, nothing allocated); L <= 65536."""
+    _check("ss_embbag_bwd_sort_noalloc",
+           lib().ss_embbag_bwd_sort_noalloc(T, N, _ptr(indices), _ptr(offsets), B, L, _ptr(uniq_keys), _ptr(seg_off),
+                                            _ptr(perm), _ptr(d_num_unique), _ptr(d_status), _stream(stream)))
 
 
 def ss_mlp_fwd(spec: MlpSpec, w, w_bf16, dense, concat_f32, concat_bf16, B, labels, logit, prob, loss, workspace,

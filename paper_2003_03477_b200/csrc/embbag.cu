@@ -884,4 +884,111 @@ ss_status ss_embbag_bwd_apply(float* tables, float* row_state, int T, int64_t N,
                   workspace_bytes, nullptr, nullptr, nullptr, nullptr, nullptr, stream);
 }
 
+// ------------------------------------------------------------------------------------------------
+// Sort / unique without any caller-provided or allocated scratch.
+//
+// Some callers of this library may not allocate device memory at the moment they need the sort: a
+// host process whose memory pool has already handed every byte of the GPU to other owners, a plug-in
+// that runs inside somebody else's serving loop where cudaMalloc's implicit device-wide
+// synchronisation would stall unrelated streams, or start-up code that runs before the application's
+// allocator exists.  For them the scratch of the sort lives in the array below, which is part of the
+// library image: every GPU that loads the library holds these bytes until the process exits.
+// ------------------------------------------------------------------------------------------------
+constexpr int64_t kNoAllocMaxL = 65536;                       // most lookups one call may sort
+constexpr size_t kNoAllocScratchBytes = 2162688;              // 2112 KiB, enough for kNoAllocMaxL lookups
+static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoAllocScratchBytes];
+
+// Device address of the array for the current device.  The array's name is only a handle on the
+// host: the address a kernel can use comes from cudaGetSymbolAddress, asked once per device.
+static ss_status noalloc_scratch_ptr(unsigned char** out) {
+  static unsigned char* ptr[64];
+  int dev = 0;
+  SS_CUDA(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= 64) return SS_ERR_SHAPE;
+  if (!ptr[dev]) {
+    void* p = nullptr;
+    SS_CUDA(cudaGetSymbolAddress(&p, g_noalloc_scratch));
+    ptr[dev] = reinterpret_cast<unsigned char*>(p);
+  }
+  *out = ptr[dev];
+  return SS_OK;
+}
+
+ss_status ss_embbag_bwd_sort_noalloc(int T, int64_t N, const int32_t* indices, const int32_t* offsets, int B,
+                                     int64_t L, int32_t* uniq_keys, int32_t* seg_off, int32_t* perm,
+                                     int32_t* d_num_unique, int32_t* d_status, ss_stream stream) {
+  using namespace ss;
+  if (!offsets || (!indices && L > 0) || !uniq_keys || !seg_off || !perm || !d_num_unique) return SS_ERR_NULL;
+  if (T < 0 || B < 0 || N <= 0 || L < 0) return SS_ERR_SHAPE;
+  if (L > kNoAllocMaxL) return SS_ERR_SHAPE;                   // beyond the built-in scratch: use ss_embbag_bwd_sort
+  if ((uint64_t)T * (uint64_t)N >= (1ull << 31)) return SS_ERR_SHAPE;
+  ss_status stt = check_arch();
+  if (stt != SS_OK) return stt;
+  unsigned char* ws = nullptr;
+  stt = noalloc_scratch_ptr(&ws);
+  if (stt != SS_OK) return stt;
+  cudaStream_t cs = as_stream(stream);
+
+  // digit plan of the radix sort (same rule as the workspace variant)
+  const uint64_t maxkey = (uint64_t)T * (uint64_t)N;
+  int bits = 1;
+  while ((maxkey >> bits) != 0) ++bits;
+  const int passes = (bits + 8) / 9;
+  const int digit_bits = (bits + passes - 1) / passes;
+  const int bins = 1 << digit_bits;
+  const int nblk = L > 0 ? (int)((L + kSortTile - 1) / kSortTile) : 1;
+  const int nblk_u = L > 0 ? (int)((L + kScanThreads - 1) / kScanThreads) : 1;
+
+  // carve the array; every piece is rewritten in full by each call before it is read, so nothing
+  // depends on what an earlier call left behind
+  size_t o = 0;
+  auto take = [&](size_t bytes) { size_t r = o; o += align256(bytes); return r; };
+  const size_t l4 = (size_t)kNoAllocMaxL * 4;
+  uint32_t* keys_a = reinterpret_cast<uint32_t*>(ws + take(l4));
+  uint32_t* keys_b = reinterpret_cast<uint32_t*>(ws + take(l4));
+  int32_t* pos_a = reinterpret_cast<int32_t*>(ws + take(l4));
+  int32_t* pos_b = reinterpret_cast<int32_t*>(ws + take(l4));
+  int32_t* bag_of = reinterpret_cast<int32_t*>(ws + take(l4));
+  int32_t* uniq = reinterpret_cast<int32_t*>(ws + take(l4));
+  int32_t* uidx = reinterpret_cast<int32_t*>(ws + take(l4));
+  int32_t* seg = reinterpret_cast<int32_t*>(ws + take(l4 + 4));
+  uint32_t* hist = reinterpret_cast<uint32_t*>(ws + take((size_t)(kNoAllocMaxL / kSortTile) * kMaxBins * 4));
+  uint32_t* bintot = reinterpret_cast<uint32_t*>(ws + take((size_t)kMaxBins * 4));
+  uint32_t* usum = reinterpret_cast<uint32_t*>(ws + take((size_t)(kNoAllocMaxL / kScanThreads + 1) * 4));
+  int32_t* scalars = reinterpret_cast<int32_t*>(ws + take(256));
+  if (o > kNoAllocScratchBytes) return SS_ERR_WORKSPACE;
+  const uint32_t sentinel = (uint32_t)maxkey;
+
+  if (L == 0 || (int64_t)T * B == 0) {
+    unique_finish_kernel<<<1, 1, 0, cs>>>(nullptr, seg, seg_off, d_num_unique, scalars);
+    SS_LAUNCH_OK();
+    return SS_OK;
+  }
+  fill_keys_kernel<<<(unsigned)((L + 255) / 256), 256, 0, cs>>>(keys_a, bag_of, L, sentinel);
+  build_keys_kernel<<<(unsigned)(((int64_t)T * B + 255) / 256), 256, 0, cs>>>(indices, offsets, T, N, B, L, keys_a,
+                                                                                bag_of, d_status);
+  SS_LAUNCH_OK();
+  uint32_t* kin = keys_a; uint32_t* kout = keys_b;
+  int32_t* pin = nullptr;
+  int32_t* pout = pos_b;
+  int32_t* pnext = pos_a;
+  const size_t smem = ((size_t)kSortWarps * bins + bins + 8) * 4;
+  for (int pass = 0; pass < passes; ++pass) {
+    const int shift = pass * digit_bits;
+    sort_hist_kernel<<<nblk, kSortThreads, 0, cs>>>(kin, L, shift, bins, nblk, hist);
+    bin_scan_kernel<<<(bins + 7) / 8, 256, 0, cs>>>(hist, bins, nblk, bintot);
+    sort_scatter_kernel<<<nblk, kSortThreads, smem, cs>>>(kin, pin, kout, pout, L, shift, bins, nblk, hist, bintot);
+    SS_LAUNCH_OK();
+    uint32_t* tk = kin; kin = kout; kout = tk;
+    pin = pout; pout = pnext; pnext = pin;
+  }
+  SS_CUDA(cudaMemcpyAsync(perm, pin, (size_t)L * 4, cudaMemcpyDeviceToDevice, cs));
+  unique_count_kernel<<<nblk_u, kScanThreads, 0, cs>>>(kin, L, sentinel, usum);
+  scan_exclusive_kernel<<<1, kScanThreads, 0, cs>>>(usum, nblk_u, usum + nblk_u);
+  unique_write_kernel<<<nblk_u, kScanThreads, 0, cs>>>(kin, L, sentinel, usum, uniq, seg, uidx, uniq_keys, seg_off);
+  unique_finish_kernel<<<1, 1, 0, cs>>>(usum + nblk_u, seg, seg_off, d_num_unique, scalars);
+  SS_LAUNCH_OK();
+  return SS_OK;
+}
+
 }  // extern "C"
