@@ -151,6 +151,20 @@ def timed_region(model, graphs, first_step, n_steps):
     return start.elapsed_time(stop)
 
 
+def reduce_over_ranks(ms_list, examples, device):
+    """Max over ranks of each timed region (ms) and the sum over ranks of the examples processed.
+    Each rank runs an independent copy of the job (the path does not shard across GPUs)."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return list(ms_list), examples
+    t = torch.tensor(list(ms_list), dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    n = torch.tensor([examples], dtype=torch.int64, device=device)
+    dist.all_reduce(n, op=dist.ReduceOp.SUM)
+    return [float(x) for x in t], int(n[0])
+
+
 def sync_args(cfg):
     return dict(rule=cfg.sync, alpha=cfg.alpha, eta=cfg.eta, mu=cfg.mu)
 
@@ -194,7 +208,6 @@ def bench_gpu(args):
     model.sync(**sync_args(cfg))
     torch.cuda.synchronize()
     graphs = capture_graphs(model, dev)
-    launches_per_replica_step = None
 
     def barrier():
         torch.cuda.synchronize()
@@ -219,11 +232,7 @@ def bench_gpu(args):
     barrier()
     loop.stop()
     torch.cuda.synchronize()
-    if world > 1:
-        t = torch.tensor([ms_on, ms_off], device=device)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_on, ms_off = float(t[0]), float(t[1])
-    examples = cfg.R * cfg.B * K * world
+    (ms_on, ms_off), examples = reduce_over_ranks([ms_on, ms_off], cfg.R * cfg.B * K, device)
     value = examples / (ms_on * 1e-3)
     value_off = examples / (ms_off * 1e-3)
     status = model.status() | (ss.ss_device_error() << 8)
@@ -249,29 +258,14 @@ def bench_gpu(args):
     out["sync"] = {"rounds_per_s": rounds / (ms_on * 1e-3), "avg_sync_gap_steps": (K / rounds) if rounds else None,
                    "examples_per_s_sync_off": value_off, "throughput_loss_pct": 100.0 * (1.0 - value / value_off)}
 
-    # dominant-kernel roofline: the embedding-bag forward gather (one kernel per call), timed with events on
-    # its stream; algorithmic bytes = L*(4D+4) + (T*B+1)*4 + T*B*2D (bf16 pooled output)
-    rep = model.replicas[0]
-    s = rep.stream
-    T, N, D, B = cfg.T, cfg.N, cfg.D, cfg.B
-    sp = model.spec
+    kernels, per_step = profile_pass(model, dev, cfg)
+    out["kernels"] = kernels
+    out["gpu_launches"] = int(round(per_step * cfg.R * K)) + int(rounds)
+    out["roofline"] = roofline(kernels, model, host, cfg, peaks)
 
-    def fwd(i):
-        b = dev[0][i % RING]
-        ss.ss_embbag_fwd(model.tables, T, N, D, b.indices, b.offsets, B, rep.concat_f32, sp.W, rep.concat_bf16, sp.W,
-                         D, model.d_status, s)
-    with torch.cuda.stream(s):
-        time_kernel_call(fwd, s, 3)
-        ms_fwd = time_kernel_call(fwd, s, 24)
-    Lmean = float(np.mean([b.L for b in host[0]]))
-    out_bytes = T * B * D * (2 if cfg.bf16 else 4)
-    fwd_bytes = Lmean * (4 * D + 4) + (T * B + 1) * 4 + out_bytes
-    achieved = fwd_bytes / (ms_fwd * 1e-3) / 1e9
-    out["roofline"] = {"kernel": "embbag_fwd_kernel", "bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"],
-                       "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"], "traffic": None,
-                       "peak_source": peaks["source"], "bytes_per_launch": fwd_bytes, "us_per_launch": ms_fwd * 1e3}
+    # the sync kernel alone on vectors far larger than L2 (HBM-bound) -- the "sync HBM GB/s vs peak" half of the metric
+    s = model.replicas[0].stream
 
-    # the sync kernel alone at the workload's parameter size (L2-resident) and at 64M elements (HBM-bound)
     def time_sync(n, R):
         ws = [torch.randn(n, device=device) * 0.02 for _ in range(R)]
         c = torch.zeros(n, device=device)
@@ -290,41 +284,105 @@ def bench_gpu(args):
 
     # ---- end to end through the public API with host buffers ------------------------------------
     if not args.quick:
-        out["e2e"] = bench_e2e(model, host, cfg, K, W)
+        out["e2e"] = bench_e2e(model, host, dev, graphs, cfg, K, W)
         out["cpu_baseline"] = cpu_baseline(cfg, budget_s=args.cpu_budget)
-    out["gpu_launches"] = None
     print(json.dumps(out))
     if world > 1:
         dist.destroy_process_group()
 
 
-def bench_e2e(model, host, cfg, K, W):
-    """Same metric with the step's inputs in pinned host memory: H2D copy of every batch and a D2H read of the loss
-    inside the timed region, calls made through the binding (no graphs: the input buffers change every step)."""
+def profile_pass(model, dev, cfg, steps=6):
+    """Per-kernel device times from the library's event timers over a short region in which all replicas
+    train concurrently (plain launches: timing events cannot be read back from a captured graph).
+    Returns ({kernel: {launches_per_replica_step, us_per_launch, share}}, launches per replica step)."""
+    import torch
+    from paper_2003_03477_b200 import binding as ss
+    for t in range(2):
+        for r in range(cfg.R):
+            model.step(r, dev[r][t % RING])
+    torch.cuda.synchronize()
+    ss.ss_profile(True)
+    for t in range(steps):
+        for r in range(cfg.R):
+            model.step(r, dev[r][t % RING])
+    recs = ss.ss_profile_collect()
+    ss.ss_profile(False)
+    agg = {}
+    for name, ms in recs:
+        a = agg.setdefault(name, [0, 0.0])
+        a[0] += 1
+        a[1] += ms * 1e3
+    total = sum(a[1] for a in agg.values()) or 1.0
+    n_rs = steps * cfg.R
+    table = {k: {"launches_per_replica_step": c / n_rs, "us_per_launch": t / c, "share": t / total}
+             for k, (c, t) in sorted(agg.items(), key=lambda kv: -kv[1][1])}
+    return table, len(recs) / n_rs
+
+
+def roofline(kernels, model, host, cfg, peaks):
+    """Roofline entry of the kernel with the largest share of the step's kernel time.
+
+    Algorithmic work per launch: embedding forward L(4D+4) + 4(TB+1) + TB*D*{2,4} bytes; window reduction
+    L(4D+16) + U*4D; row update U(3*4D+12); tensor-core GEMMs: the step's 2MNK summed over its GEMM launches.
+    L and U are the means over the batches of replica 0 (U read back from the device)."""
+    T, D, B = cfg.T, cfg.D, cfg.B
+    L = float(np.mean([b.L for b in host[0]]))
+    U = float(model.replicas[0].num_unique.item())
+    dims = model.spec.layer_dims
+    nl = len(dims)
+    gemm_flops = 0.0
+    for l, (fin, fout) in enumerate(dims):
+        if l == nl - 1 or fin < 16:
+            continue                      # single-logit and 13-input layers run on SIMT kernels
+        gemm_flops += 6.0 * B * fin * fout   # forward, weight gradient, input gradient: 2*B*in*out each
+    work = {
+        "embbag_fwd_kernel": ("hbm", L * (4 * D + 4) + 4 * (T * B + 1) + T * B * D * (2 if cfg.bf16 else 4), 1),
+        "window_reduce_kernel": ("hbm", L * (4 * D + 16) + U * 4 * D, 1),
+        "apply_rows_kernel": ("hbm", U * (3 * 4 * D + 12), 1),
+        "gemm_tc_kernel": ("tensor", gemm_flops, None),
+    }
+    name = next((k for k in kernels if k in work), None)
+    if name is None:
+        return {"kernel": next(iter(kernels), None), "bound": "alu", "achieved": None, "peak": None, "unit": None,
+                "frac": None, "traffic": None}
+    bound, amount, per = work[name]
+    k = kernels[name]
+    n_launch = k["launches_per_replica_step"]
+    us_total = k["us_per_launch"] * n_launch          # per replica step
+    if bound == "hbm":
+        achieved = amount / (us_total / n_launch * 1e-6) / 1e9
+        peak, unit = peaks["hbm_gbs"], "GB/s"
+    else:
+        achieved = amount / (us_total * 1e-6) / 1e12
+        peak, unit = peaks["bf16_tflops_sustained"], "TFLOP/s"
+    return {"kernel": name, "bound": bound, "achieved": achieved, "peak": peak, "unit": unit, "frac": achieved / peak,
+            "traffic": None, "peak_source": peaks["source"], "launches_per_replica_step": n_launch,
+            "us_per_launch": k["us_per_launch"], "share_of_kernel_time": k["share"],
+            "work_per_replica_step": amount,
+            "timing": "CUDA events around every launch on its stream, all replicas training concurrently"}
+
+
+def bench_e2e(model, host, dev, graphs, cfg, K, W):
+    """Same metric with the step's inputs in pinned host memory: every step copies its batch host->device
+    into the ring slot's device buffers, replays that slot's captured step and reads the loss back."""
     import torch
     from paper_2003_03477_b200 import trainer
     pinned = [[tuple(torch.from_numpy(np.ascontiguousarray(a)).pin_memory() for a in
                      (b.indices, b.offsets, b.dense, b.labels)) for b in bs] for bs in host]
-    Lmax = max(b.L for bs in host for b in bs)
-    stage = []
-    for r in range(cfg.R):
-        stage.append([trainer.DeviceBatch(np.zeros(Lmax, np.int32), host[r][0].offsets, host[r][0].dense, host[r][0].labels,
-                                          model.device) for _ in range(2)])
     loss_host = [torch.zeros(1).pin_memory() for _ in range(cfg.R)]
     h2d = d2h = 0
 
     def step(t):
         nonlocal h2d, d2h
         for r, rep in enumerate(model.replicas):
-            src, dst = pinned[r][t % RING], stage[r][t % 2]
+            slot = t % RING
+            src, dst = pinned[r][slot], dev[r][slot]
             with torch.cuda.stream(rep.stream):
-                L = src[0].numel()
-                dst.indices[:L].copy_(src[0], non_blocking=True)
+                dst.indices.copy_(src[0], non_blocking=True)
                 dst.offsets.copy_(src[1], non_blocking=True)
                 dst.dense.copy_(src[2], non_blocking=True)
                 dst.labels.copy_(src[3], non_blocking=True)
-                dst.L = L
-                model.step(r, dst)
+                graphs[r][slot].replay()
                 loss_host[r].copy_(rep.loss, non_blocking=True)
             h2d += sum(x.numel() * x.element_size() for x in src)
             d2h += 4
@@ -343,7 +401,7 @@ def bench_e2e(model, host, cfg, K, W):
     loop.stop()
     torch.cuda.synchronize()
     return {"value": cfg.R * cfg.B * K / dt, "unit": UNIT, "h2d_bytes_per_step": h2d // K, "d2h_bytes_per_step": d2h // K,
-            "timing": "host wall clock around K steps incl. stream sync (copies and launches inside)"}
+            "timing": "host wall clock around K steps, ending with a synchronise of every replica stream"}
 
 
 # ----------------------------------------------------------------------------------------------
@@ -425,7 +483,7 @@ def bench_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="medium", choices=["tiny", "medium", "medium_bmuf", "large"])

@@ -50,7 +50,8 @@ enum {
 /* bits ORed into *d_status by kernels */
 enum {
   SS_DEV_BAD_INDEX = 1,  /* a row index outside [0, N): lookup skipped                   */
-  SS_DEV_BAD_OFFSET = 2  /* offsets not non-decreasing or beyond L: bag treated as empty */
+  SS_DEV_BAD_OFFSET = 2, /* offsets not non-decreasing or beyond L: bag treated as empty */
+  SS_DEV_BAD_WORKSPACE = 4 /* ss_embbag_bwd_apply on a workspace that holds no finished sort of this T, N, L: nothing done */
 };
 
 typedef void* ss_stream;
@@ -106,14 +107,17 @@ ss_status ss_embbag_bwd_adagrad(float* tables, float* row_state, int T, int64_t 
  * steps 1-2 depend only on the batch's indices, steps 3-4 also on the gradient.
  *   ss_embbag_bwd_sort   steps 1-2 into the workspace (and the optional uniq_keys / seg_off / perm outputs)
  *   ss_embbag_bwd_apply  steps 3-4 from a workspace that ss_embbag_bwd_sort filled for the same batch
- * Arguments as in ss_embbag_bwd_adagrad; the caller orders the two calls (same stream, or an event). */
+ * Arguments as in ss_embbag_bwd_adagrad; the caller orders the two calls (same stream, or an event).
+ * The sort stamps the workspace with (T*N, L); an apply whose T, N, L do not match the stamp changes
+ * nothing and sets SS_DEV_BAD_WORKSPACE in *d_status (nullable).  A workspace sorted for another batch
+ * of the same T, N, L cannot be told apart: the update is then memory-safe but meaningless. */
 ss_status ss_embbag_bwd_sort(int T, int64_t N, int D, const int32_t* indices, const int32_t* offsets, int B,
                              int64_t L, void* workspace, size_t workspace_bytes,
                              int32_t* uniq_keys, int32_t* seg_off, int32_t* perm,
                              int32_t* d_num_unique, int32_t* d_status, ss_stream stream);
 ss_status ss_embbag_bwd_apply(float* tables, float* row_state, int T, int64_t N, int D, int B, int64_t L,
                               const float* grad, int64_t ld_grad, int col0, float lr, float eps,
-                              void* workspace, size_t workspace_bytes, ss_stream stream);
+                              void* workspace, size_t workspace_bytes, int32_t* d_status, ss_stream stream);
 
 /* The sort / unique half once more, for callers that cannot allocate.  (The paper has no counterpart:
  * this entry point exists only for how the library is embedded.)

@@ -19,7 +19,7 @@ LIB_PATH = os.path.join(_HERE, "libshadowsync.so")
 SS_OK = 0
 STATUS_NAMES = {0: "SS_OK", -1: "SS_ERR_NULL", -2: "SS_ERR_SHAPE", -3: "SS_ERR_ALIGN", -4: "SS_ERR_DTYPE",
                 -5: "SS_ERR_WORKSPACE", -6: "SS_ERR_ARCH", -7: "SS_ERR_CUDA", -8: "SS_ERR_RANGE"}
-SS_DEV_BAD_INDEX, SS_DEV_BAD_OFFSET = 1, 2
+SS_DEV_BAD_INDEX, SS_DEV_BAD_OFFSET, SS_DEV_BAD_WORKSPACE = 1, 2, 4
 SS_SYNC_EASGD_LITERAL = 1
 
 EXPORTS = ["ss_status_str", "ss_last_cuda_error", "ss_num_sms", "ss_embbag_fwd", "ss_embbag_bwd_workspace_bytes",
@@ -65,7 +65,7 @@ def lib() -> C.CDLL:
         L.ss_embbag_bwd_adagrad.argtypes = [vp, vp, i32, i64, i32, vp, vp, i32, i64, vp, i64, i32, f32, f32,
                                             vp, sz, vp, vp, vp, vp, vp, vp]
         L.ss_embbag_bwd_sort.argtypes = [i32, i64, i32, vp, vp, i32, i64, vp, sz, vp, vp, vp, vp, vp, vp]
-        L.ss_embbag_bwd_apply.argtypes = [vp, vp, i32, i64, i32, i32, i64, vp, i64, i32, f32, f32, vp, sz, vp]
+        L.ss_embbag_bwd_apply.argtypes = [vp, vp, i32, i64, i32, i32, i64, vp, i64, i32, f32, f32, vp, sz, vp, vp]
         L.ss_embbag_bwd_sort_noalloc.argtypes = [i32, i64, vp, vp, i32, i64, vp, vp, vp, vp, vp, vp]
         L.ss_mlp_param_count.restype = i64
         L.ss_mlp_param_count.argtypes = [C.POINTER(MlpDesc)]
@@ -193,10 +193,12 @@ def ss_embbag_bwd_sort(T, N, D, indices, offsets, B, L, workspace, uniq_keys, se
                                     _ptr(perm), _ptr(d_num_unique), _ptr(d_status), _stream(stream)))
 
 
-def ss_embbag_bwd_apply(tables, row_state, T, N, D, B, L, grad, ld_grad, col0, lr, eps, workspace, stream=None) -> None:
+def ss_embbag_bwd_apply(tables, row_state, T, N, D, B, L, grad, ld_grad, col0, lr, eps, workspace, d_status=None,
+                        stream=None) -> None:
     _check("ss_embbag_bwd_apply",
            lib().ss_embbag_bwd_apply(_ptr(tables), _ptr(row_state), T, N, D, B, L, _ptr(grad), ld_grad, col0, lr, eps,
-                                     _ptr(workspace), workspace.numel() * workspace.element_size(), _stream(stream)))
+                                     _ptr(workspace), workspace.numel() * workspace.element_size(), _ptr(d_status),
+                                     _stream(stream)))
 
 
 def ss_embbag_bwd_sort_noalloc(T, N, indices, offsets, B, L, uniq_keys, seg_off, perm, d_num_unique, d_status,

@@ -418,14 +418,26 @@ unique_write_kernel(const uint32_t* __restrict__ keys, int64_t L, uint32_t senti
   }
 }
 
+// scalars[2..3] stamp the workspace with the problem it holds a finished sort of; the reduction kernels
+// refuse a workspace whose stamp does not match their arguments.
+__device__ __forceinline__ int32_t ws_stamp(uint32_t sentinel) { return (int32_t)(sentinel ^ 0x53484144u); }
+
 __global__ void unique_finish_kernel(const uint32_t* __restrict__ total, int32_t* __restrict__ seg,
                                      int32_t* __restrict__ seg_out, int32_t* __restrict__ d_num_unique,
-                                     int32_t* __restrict__ scalars) {
+                                     int32_t* __restrict__ scalars, int64_t L, uint32_t sentinel) {
   const uint32_t U = total ? *total : 0u;
   if (U == 0) { seg[0] = 0; if (seg_out) seg_out[0] = 0; }
   if (d_num_unique) *d_num_unique = (int32_t)U;
   scalars[0] = (int32_t)U;
   scalars[1] = 0;                                          // rows whose run crosses a window edge (filled by the window kernel)
+  scalars[2] = (int32_t)L;
+  scalars[3] = ws_stamp(sentinel);
+}
+
+__device__ __forceinline__ bool ws_matches(const int32_t* scalars, int64_t L, uint32_t sentinel, int32_t* d_status) {
+  if (scalars[2] == (int32_t)L && scalars[3] == ws_stamp(sentinel)) return true;
+  if (d_status && threadIdx.x == 0 && blockIdx.x == 0) atomicOr(d_status, SS_DEV_BAD_WORKSPACE);
+  return false;
 }
 
 // ---- (4) windowed segment reduction ---------------------------------------------------------
@@ -439,7 +451,7 @@ window_reduce_kernel(const uint32_t* __restrict__ keys, const int32_t* __restric
                      const int32_t* __restrict__ bag_of, const int32_t* __restrict__ uidx, int64_t L,
                      uint32_t sentinel, int64_t N, int D, int B, const float* __restrict__ grad, int64_t ld_grad,
                      int col0, float* __restrict__ gsum, float* __restrict__ partial, int32_t* __restrict__ long_list,
-                     int32_t* __restrict__ scalars, int nwin) {
+                     int32_t* __restrict__ scalars, int nwin, int64_t umax, int32_t* __restrict__ d_status) {
   constexpr int kGroups = 256 / G;
   __shared__ uint32_t s_key[kGroups][kWin + 2];            // [0] = key before the window, [kWin+1] = key after
   __shared__ int32_t s_row[kGroups][kWin];                 // float4 index of the lookup's gradient row
@@ -447,6 +459,7 @@ window_reduce_kernel(const uint32_t* __restrict__ keys, const int32_t* __restric
   const int grp = threadIdx.x / G, lane = threadIdx.x % G;
   const int64_t win = (int64_t)blockIdx.x * kGroups + grp;
   const unsigned gmask = (G == 32) ? 0xffffffffu : (((1u << G) - 1u) << ((threadIdx.x & 31) / G * G));
+  if (!ws_matches(scalars, L, sentinel, d_status)) return;
   if (win >= nwin) return;
   const int64_t w0 = win * kWin;
   const int nvec = D >> 2;
@@ -455,6 +468,7 @@ window_reduce_kernel(const uint32_t* __restrict__ keys, const int32_t* __restric
     const int64_t j = w0 - 1 + i;
     s_key[grp][i] = (j >= 0 && j < L) ? keys[j] : sentinel;
   }
+  __syncwarp(gmask);
   for (int i = lane; i < kWin; i += G) {
     const int64_t j = w0 + i;
     int32_t row = -1, u = 0;
@@ -462,9 +476,14 @@ window_reduce_kernel(const uint32_t* __restrict__ keys, const int32_t* __restric
       const uint32_t key = keys[j];
       if (key < sentinel) {
         const int t = (int)(key / (uint64_t)N);
-        const int b = bag_of[perm[j]] - t * B;
-        row = (int32_t)((int64_t)b * ld4 + (int64_t)t * nvec);   // B * ld_grad / 4 < 2^31 is checked on the host
+        const int pj = perm[j];
+        const int b = (pj >= 0 && pj < L) ? bag_of[pj] - t * B : -1;
         u = uidx[j];
+        // a consistent workspace never fails these; an inconsistent one must not turn into a wild access
+        if (b >= 0 && b < B && u >= 0 && u < umax)
+          row = (int32_t)((int64_t)b * ld4 + (int64_t)t * nvec); // B * ld_grad / 4 < 2^31 is checked on the host
+        else
+          s_key[grp][1 + i] = sentinel;
       }
     }
     s_row[grp][i] = row;
@@ -529,17 +548,20 @@ template <int G, int NV>
 __global__ void __launch_bounds__(256)
 combine_rows_kernel(const int32_t* __restrict__ seg, const int32_t* __restrict__ scalars,
                     const int32_t* __restrict__ long_list, int nwin, int D, const float* __restrict__ partial,
-                    float* __restrict__ gsum) {
+                    float* __restrict__ gsum, int64_t L, uint32_t sentinel, int64_t umax) {
   constexpr int kGroups = 256 / G;
   extern __shared__ float4 s_part[];                       // [kGroups][D/4]
   const int grp = threadIdx.x / G, lane = threadIdx.x % G;
   const int nvec = D >> 2;
+  if (!ws_matches(scalars, L, sentinel, nullptr)) return;
   const int n = min(scalars[1], nwin);
   constexpr int kShort = 4;                                // spans up to this many windows: one group per row
   // phase A: short spans, one lane group per listed row, all partial loads issued together
   for (int i = blockIdx.x * kGroups + grp; i < n; i += gridDim.x * kGroups) {
     const int u = long_list[i];
+    if (u < 0 || u >= umax) continue;
     const int s0 = seg[u], s1 = seg[u + 1];
+    if (s0 < 0 || s1 <= s0 || s1 > L) continue;
     const int k0 = s0 / kWin, k1 = (s1 - 1) / kWin;
     if (k1 - k0 + 1 > kShort) continue;
     float4 pv[kShort][NV];
@@ -567,9 +589,11 @@ combine_rows_kernel(const int32_t* __restrict__ seg, const int32_t* __restrict__
   // phase B: long spans, the whole block per row
   for (int i = blockIdx.x; i < n; i += gridDim.x) {
     const int u = long_list[i];
+    if (u < 0 || u >= umax) continue;                      // uniform over the block, like the tests below
     const int s0 = seg[u], s1 = seg[u + 1];
+    if (s0 < 0 || s1 <= s0 || s1 > L) continue;
     const int k0 = s0 / kWin, k1 = (s1 - 1) / kWin;
-    if (k1 - k0 + 1 <= kShort) continue;                   // uniform over the block
+    if (k1 - k0 + 1 <= kShort) continue;
     float4 acc[NV];
 #pragma unroll
     for (int v = 0; v < NV; ++v) acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -613,12 +637,13 @@ template <int G, int NV>
 __global__ void __launch_bounds__(256)
 apply_rows_kernel(const int32_t* __restrict__ uniq, int32_t* __restrict__ scalars, int D,
                   const float* __restrict__ gsum, float* __restrict__ tables, float* __restrict__ row_state,
-                  float lr, float eps) {
+                  float lr, float eps, int64_t L, uint32_t sentinel, int64_t umax) {
   constexpr int kGroups = 256 / G;
   constexpr int RB = RowsPerGroup<NV>::value;              // rows per group, their loads issued together
   const int grp = threadIdx.x / G, lane = threadIdx.x % G;
   const unsigned gmask = (G == 32) ? 0xffffffffu : (((1u << G) - 1u) << ((threadIdx.x & 31) / G * G));
-  const int U = scalars[0];
+  if (!ws_matches(scalars, L, sentinel, nullptr)) return;
+  const int U = min((int64_t)scalars[0], umax);
   // the list of multi-window rows has been consumed by the previous kernel: empty it for the next reduction
   if (blockIdx.x == 0 && threadIdx.x == 0) scalars[1] = 0;
   const int nvec = D >> 2;
@@ -630,6 +655,7 @@ apply_rows_kernel(const int32_t* __restrict__ uniq, int32_t* __restrict__ scalar
   for (int r = 0; r < RB; ++r) {
     valid[r] = u0 + r < U;
     key[r] = valid[r] ? (uint32_t)uniq[u0 + r] : 0u;
+    if (key[r] >= sentinel) valid[r] = false;              // never true for a consistent workspace
   }
   float4 g[RB][NV], rw[RB][NV];
   float st[RB];
@@ -674,8 +700,10 @@ apply_rows_kernel(const int32_t* __restrict__ uniq, int32_t* __restrict__ scalar
 template <int G, int NV>
 static void launch_reduce(const BwdPlan& p, char* ws, const uint32_t* keys, const int32_t* perm, int T, int64_t N,
                           int D, int B, const float* grad, int64_t ld_grad, int col0, float* tables,
-                          float* row_state, float lr, float eps, cudaStream_t st) {
+                          float* row_state, float lr, float eps, int32_t* d_status, cudaStream_t st) {
   constexpr int kGroups = 256 / G;
+  const uint64_t maxkey = (uint64_t)T * (uint64_t)N;
+  const uint64_t umax = (uint64_t)p.L < maxkey ? (uint64_t)p.L : maxkey;
   const uint32_t sentinel = (uint32_t)((uint64_t)T * (uint64_t)N);
   float* partial = reinterpret_cast<float*>(ws + p.off_partial);
   float* gsum = reinterpret_cast<float*>(ws + p.off_gsum);
@@ -687,21 +715,21 @@ static void launch_reduce(const BwdPlan& p, char* ws, const uint32_t* keys, cons
     SS_TIMED("window_reduce_kernel", st);
     window_reduce_kernel<G, NV><<<blocks, 256, 0, st>>>(keys, perm, reinterpret_cast<int32_t*>(ws + p.off_bag),
                                                         reinterpret_cast<int32_t*>(ws + p.off_uidx), p.L, sentinel, N, D,
-                                                        B, grad, ld_grad, col0, gsum, partial, long_list, scalars, p.nwin);
+                                                        B, grad, ld_grad, col0, gsum, partial, long_list, scalars, p.nwin,
+                                                        (int64_t)umax, d_status);
   }
   {
     SS_TIMED("combine_rows_kernel", st);
     const int cblocks = p.nwin < num_sms() * 8 ? p.nwin : num_sms() * 8;
-    combine_rows_kernel<G, NV><<<cblocks, 256, (size_t)kGroups * D * 4, st>>>(seg, scalars, long_list, p.nwin, D, partial, gsum);
+    combine_rows_kernel<G, NV><<<cblocks, 256, (size_t)kGroups * D * 4, st>>>(seg, scalars, long_list, p.nwin, D, partial, gsum,
+                                                                              p.L, sentinel, (int64_t)umax);
   }
-  const uint64_t maxkey = (uint64_t)T * (uint64_t)N;
-  const uint64_t umax = (uint64_t)p.L < maxkey ? (uint64_t)p.L : maxkey;
   const uint64_t per_block = (uint64_t)kGroups * RowsPerGroup<NV>::value;
   const unsigned ublocks = (unsigned)((umax + per_block - 1) / per_block);
   {
     SS_TIMED("apply_rows_kernel", st);
     apply_rows_kernel<G, NV><<<ublocks, 256, 0, st>>>(reinterpret_cast<int32_t*>(ws + p.off_uniq), scalars, D, gsum,
-                                                      tables, row_state, lr, eps);
+                                                      tables, row_state, lr, eps, p.L, sentinel, (int64_t)umax);
   }
 }
 
@@ -790,7 +818,7 @@ static ss_status bwd_impl(bool do_sort, bool do_apply, float* tables, float* row
   if (L == 0 || (int64_t)T * B == 0) {
     if (do_sort) {
       SS_TIMED("unique_finish_kernel", cs);
-      unique_finish_kernel<<<1, 1, 0, cs>>>(nullptr, seg, seg_off, d_num_unique, scalars);
+      unique_finish_kernel<<<1, 1, 0, cs>>>(nullptr, seg, seg_off, d_num_unique, scalars, L, sentinel);
       SS_LAUNCH_OK();
     }
     return SS_OK;
@@ -844,7 +872,7 @@ static ss_status bwd_impl(bool do_sort, bool do_apply, float* tables, float* row
   unique_write_kernel<<<p.nblk_u, kScanThreads, 0, cs>>>(keys_sorted, L, sentinel, usum, uniq, seg, uidx, uniq_keys, seg_off);
   }
   { SS_TIMED("unique_finish_kernel", cs);
-  unique_finish_kernel<<<1, 1, 0, cs>>>(usum + p.nblk_u, seg, seg_off, d_num_unique, scalars);
+  unique_finish_kernel<<<1, 1, 0, cs>>>(usum + p.nblk_u, seg, seg_off, d_num_unique, scalars, L, sentinel);
   }
   SS_LAUNCH_OK();
 
@@ -853,7 +881,7 @@ static ss_status bwd_impl(bool do_sort, bool do_apply, float* tables, float* row
   // (4) windowed segment reduction, (5) combine, (6) row-wise Adagrad
   if (do_apply) {
 #define SS_RED(G_, NV_) \
-  launch_reduce<G_, NV_>(p, ws, keys_sorted, perm_sorted, T, N, D, B, grad, ld_grad, col0, tables, row_state, lr, eps, cs)
+  launch_reduce<G_, NV_>(p, ws, keys_sorted, perm_sorted, T, N, D, B, grad, ld_grad, col0, tables, row_state, lr, eps, d_status, cs)
     SS_DISPATCH_GNV(D, SS_RED);
 #undef SS_RED
     SS_LAUNCH_OK();
@@ -879,9 +907,9 @@ ss_status ss_embbag_bwd_sort(int T, int64_t N, int D, const int32_t* indices, co
 
 ss_status ss_embbag_bwd_apply(float* tables, float* row_state, int T, int64_t N, int D, int B, int64_t L,
                               const float* grad, int64_t ld_grad, int col0, float lr, float eps, void* workspace,
-                              size_t workspace_bytes, ss_stream stream) {
+                              size_t workspace_bytes, int32_t* d_status, ss_stream stream) {
   return bwd_impl(false, true, tables, row_state, T, N, D, nullptr, nullptr, B, L, grad, ld_grad, col0, lr, eps, workspace,
-                  workspace_bytes, nullptr, nullptr, nullptr, nullptr, nullptr, stream);
+                  workspace_bytes, nullptr, nullptr, nullptr, nullptr, d_status, stream);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -960,7 +988,7 @@ ss_status ss_embbag_bwd_sort_noalloc(int T, int64_t N, const int32_t* indices, c
   const uint32_t sentinel = (uint32_t)maxkey;
 
   if (L == 0 || (int64_t)T * B == 0) {
-    unique_finish_kernel<<<1, 1, 0, cs>>>(nullptr, seg, seg_off, d_num_unique, scalars);
+    unique_finish_kernel<<<1, 1, 0, cs>>>(nullptr, seg, seg_off, d_num_unique, scalars, L, sentinel);
     SS_LAUNCH_OK();
     return SS_OK;
   }
@@ -986,7 +1014,7 @@ ss_status ss_embbag_bwd_sort_noalloc(int T, int64_t N, const int32_t* indices, c
   unique_count_kernel<<<nblk_u, kScanThreads, 0, cs>>>(kin, L, sentinel, usum);
   scan_exclusive_kernel<<<1, kScanThreads, 0, cs>>>(usum, nblk_u, usum + nblk_u);
   unique_write_kernel<<<nblk_u, kScanThreads, 0, cs>>>(kin, L, sentinel, usum, uniq, seg, uidx, uniq_keys, seg_off);
-  unique_finish_kernel<<<1, 1, 0, cs>>>(usum + nblk_u, seg, seg_off, d_num_unique, scalars);
+  unique_finish_kernel<<<1, 1, 0, cs>>>(usum + nblk_u, seg, seg_off, d_num_unique, scalars, L, sentinel);
   SS_LAUNCH_OK();
   return SS_OK;
 }

@@ -118,7 +118,7 @@ class Model:
         if overlap_sort:
             s.wait_event(join)
             ss.ss_embbag_bwd_apply(self.tables, self.row_state, T, N, D, B, batch.L, rep.grad_pooled, T * D, 0,
-                                   self.lr, self.eps, rep.emb_ws, s)
+                                   self.lr, self.eps, rep.emb_ws, self.d_status, s)
         else:
             ss.ss_embbag_bwd_adagrad(self.tables, self.row_state, T, N, D, batch.indices, batch.offsets, B, batch.L,
                                      rep.grad_pooled, T * D, 0, self.lr, self.eps, rep.emb_ws, rep.uniq_keys,

@@ -191,8 +191,38 @@ def test_sort_once_apply_twice_matches_two_oracle_updates():
     ss.ss_embbag_bwd_sort(T, N, D, _cuda(b.indices), _cuda(b.offsets), B, L, ws, None, None, perm_d, nu, st)
     dg = _cuda(gp)
     for _ in range(3):
-        ss.ss_embbag_bwd_apply(dt, ds, T, N, D, B, L, dg, T * D, 0, cfg.lr, cfg.eps, ws)
+        ss.ss_embbag_bwd_apply(dt, ds, T, N, D, B, L, dg, T * D, 0, cfg.lr, cfg.eps, ws, st)
     torch.cuda.synchronize()
     assert int(st.item()) == 0 and int(nu.item()) == len(uniq) and np.array_equal(perm_d.cpu().numpy(), perm)
     assert_close(dt.cpu().numpy() - tables, t_o.astype(np.float64) - tables, 2e-5, "tables after three updates")
     assert_close(ds.cpu().numpy().reshape(T, N), s_o, RTOL_F32, "row state")
+
+
+def test_apply_refuses_a_workspace_sorted_for_another_problem():
+    # the apply half trusts the workspace only if the sort stamped it for the same T, N, L
+    cfg = synth.scaled(synth.CONFIGS["medium"], T=3, N=4000, D=64, B=256, bottom=(13, 64, 64), top=(256, 64, 1))
+    b1, b2 = synth.make_batch(cfg, 0, 1), synth.make_batch(cfg, 0, 2)
+    assert b1.L != b2.L
+    T, N, D, B = cfg.T, cfg.N, cfg.D, cfg.B
+    Lmax = max(b1.L, b2.L)
+    tables = synth.tables_dense(cfg)
+    dt, ds = _cuda(tables), torch.zeros(T * N, device="cuda")
+    ws = torch.zeros(ss.ss_embbag_bwd_workspace_bytes(T, N, D, B, Lmax), dtype=torch.uint8, device="cuda")
+    nu = torch.zeros(1, dtype=torch.int32, device="cuda")
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    dg = torch.ones(B, T * D, device="cuda")
+    # never sorted: refused
+    ss.ss_embbag_bwd_apply(dt, ds, T, N, D, B, b1.L, dg, T * D, 0, 0.1, 1e-8, ws, st)
+    torch.cuda.synchronize()
+    assert int(st.item()) == ss.SS_DEV_BAD_WORKSPACE and np.array_equal(dt.cpu().numpy(), tables)
+    # sorted for batch 1, applied with batch 2's size: refused, tables untouched
+    st.zero_()
+    ss.ss_embbag_bwd_sort(T, N, D, _cuda(b1.indices), _cuda(b1.offsets), B, b1.L, ws, None, None, None, nu, st)
+    ss.ss_embbag_bwd_apply(dt, ds, T, N, D, B, b2.L, dg, T * D, 0, 0.1, 1e-8, ws, st)
+    torch.cuda.synchronize()
+    assert int(st.item()) == ss.SS_DEV_BAD_WORKSPACE and np.array_equal(dt.cpu().numpy(), tables)
+    # matching call goes through
+    st.zero_()
+    ss.ss_embbag_bwd_apply(dt, ds, T, N, D, B, b1.L, dg, T * D, 0, 0.1, 1e-8, ws, st)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0 and not np.array_equal(dt.cpu().numpy(), tables)
