@@ -1,0 +1,132 @@
+"""Parity at the benchmark's full sizes, in the launch configuration the benchmark times (one captured CUDA
+graph per replica step, sort forked onto the side stream): the medium workload's whole first step against the
+oracle, and the sync kernels on HBM-sized vectors.
+
+The oracle cannot hold 26 tables of a million rows, and does not need to: table rows are a pure function of
+(table, row, column), so the batch is remapped onto a compact table of exactly the rows it touches (the remap is
+monotone per table, so sort order, permutation and segment structure are unchanged) and the oracle runs the
+complete step on that."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import shadowsync_oracle as O
+from paper_2003_03477_b200 import binding as ss
+from paper_2003_03477_b200 import synth, trainer
+from parity import RTOL_BF16, RTOL_F32, RTOL_SYNC, assert_close
+
+pytestmark = pytest.mark.gpu
+
+
+def _compact(cfg, batch):
+    lens = np.diff(batch.offsets.astype(np.int64))
+    tbl = np.repeat(np.arange(cfg.T * cfg.B) // cfg.B, lens)
+    keys = tbl * cfg.N + batch.indices
+    uniq, inv = np.unique(keys, return_inverse=True)
+    t_of = uniq // cfg.N
+    counts = np.bincount(t_of, minlength=cfg.T)
+    nmax = int(counts.max())
+    starts = np.concatenate([[0], np.cumsum(counts)[:-1]])
+    local = np.arange(len(uniq)) - starts[t_of]                  # rank of the row inside its table
+    tables = np.zeros((cfg.T, nmax, cfg.D), np.float32)
+    for t in range(cfg.T):
+        rows = (uniq[t_of == t] % cfg.N)
+        tables[t, :len(rows)] = synth.table_rows(cfg, t, rows)
+    small = synth.Batch(local[inv].astype(np.int32), batch.offsets, batch.dense, batch.labels)
+    return tables, small, uniq, t_of, local, nmax
+
+
+def test_medium_workload_first_step_full_size_as_benchmarked():
+    cfg = synth.scaled(synth.CONFIGS["medium"], R=1)
+    batch = synth.make_batch(cfg, 0, 0)
+    layers = synth.initial_weights(cfg)
+    spec = ss.MlpSpec(cfg.bottom, cfg.top, cfg.bf16)
+    w0 = torch.from_numpy(trainer.pack_params(spec, layers)).cuda()
+    model = trainer.Model(cfg.T, cfg.N, cfg.D, cfg.B, cfg.bottom, cfg.top, cfg.bf16, 1, w0, trainer.device_tables(cfg),
+                          cfg.lr, cfg.eps, max_L=batch.L, keep_sort_outputs=True, keep_f32_concat=True)
+    dev = trainer.DeviceBatch(batch.indices, batch.offsets, batch.dense, batch.labels)
+    rep = model.replicas[0]
+    # first-use set-up happens outside capture, on a scratch copy of the state that is restored afterwards
+    w_keep, acc_keep = rep.w.clone(), rep.acc.clone()
+    model.step(0, dev)
+    torch.cuda.synchronize()
+    model.tables.copy_(trainer.device_tables(cfg))
+    model.row_state.zero_()
+    rep.w.copy_(w_keep); rep.acc.copy_(acc_keep)
+    ss.ss_to_bf16(rep.w, rep.w_bf16, spec.param_count)
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=rep.stream):
+        model.step(0, dev, stream=rep.stream)
+    with torch.cuda.stream(rep.stream):
+        g.replay()
+    torch.cuda.synchronize()
+    assert model.status() == 0 and ss.ss_device_error() == 0
+
+    # ---- oracle on the compact problem
+    tables_c, small, uniq, t_of, local, nmax = _compact(cfg, batch)
+    t_before = tables_c.copy()
+    state = np.zeros((cfg.T, nmax), np.float32)
+    accs = [(np.zeros_like(W), np.zeros_like(b)) for W, b in layers]
+    w_before = [(W.copy(), b.copy()) for W, b in layers]
+    out = O.replica_step(tables_c, state, layers, accs, len(cfg.bottom) - 1, small, cfg.lr, cfg.eps, cfg.bf16)
+
+    # integer outputs, bit-exact at full size (560k lookups, 3 radix passes, 137 sort tiles)
+    U = int(rep.num_unique.item())
+    assert U == len(uniq) == len(out["uniq_keys"])
+    assert np.array_equal(rep.uniq_keys.cpu().numpy()[:U], uniq)
+    assert np.array_equal(rep.seg_off.cpu().numpy()[:U + 1], out["seg_off"])
+    assert np.array_equal(rep.perm.cpu().numpy()[:batch.L], out["perm"])
+    # pooled embeddings (float32 copy of the concat buffer), every bag
+    assert_close(rep.concat_f32.cpu().numpy()[:, cfg.D:], out["pooled"].reshape(cfg.B, -1), RTOL_F32, "pooled")
+    # MLP outputs through the tensor-core path
+    assert_close(rep.logit.cpu().numpy(), out["logit"], RTOL_BF16, "logit")
+    assert abs(float(rep.loss.item()) - out["loss"]) <= RTOL_BF16 * abs(out["loss"])
+    # gradients sit behind ReLU gates: see assert_close on outlier_frac
+    assert_close(rep.grad_pooled.cpu().numpy(), out["grad_pooled"], RTOL_BF16, "grad_pooled", outlier_frac=5e-3)
+    new = trainer.unpack_params(spec, rep.w.cpu().numpy())
+    for l in range(len(layers)):
+        assert_close(new[l][0] - w_before[l][0], layers[l][0].astype(np.float64) - w_before[l][0], RTOL_BF16, f"dW[{l}]", outlier_frac=5e-3)
+        assert_close(new[l][1] - w_before[l][1], layers[l][1].astype(np.float64) - w_before[l][1], RTOL_BF16, f"db[{l}]", outlier_frac=5e-3)
+    # every touched row of the 6.7 GB tables, and its optimizer state
+    rows_dev = model.tables.view(-1, cfg.D)[torch.from_numpy(uniq).cuda()].cpu().numpy()
+    want = tables_c[t_of, local]
+    assert_close(rows_dev - t_before[t_of, local], want.astype(np.float64) - t_before[t_of, local], RTOL_BF16, "row updates", outlier_frac=5e-3)
+    assert_close(model.row_state[torch.from_numpy(uniq).cuda()].cpu().numpy(), state[t_of, local], RTOL_BF16, "row state", outlier_frac=5e-3)
+    # rows the batch did not touch are unchanged (a sample)
+    rng = np.random.default_rng(0)
+    for t in (0, 13, 25):
+        rows = np.setdiff1d(rng.integers(0, cfg.N, 400), uniq[t_of == t] % cfg.N)
+        got = model.tables[t][torch.from_numpy(rows).cuda()].cpu().numpy()
+        assert np.array_equal(got, synth.table_rows(cfg, t, rows))
+
+
+@pytest.mark.parametrize("rule", ["easgd", "ma", "bmuf"])
+def test_sync_rules_on_hbm_sized_vectors(rule):
+    # 4 replicas of 64M floats (1.3 GB moved per pass); the rules are element-wise, so slices are checked exactly
+    n, R = 1 << 26, 4
+    g = torch.Generator(device="cuda").manual_seed(5)
+    ws = [torch.randn(n, device="cuda", generator=g) * 0.02 for _ in range(R)]
+    c = torch.randn(n, device="cuda", generator=g) * 0.02
+    d = torch.randn(n, device="cuda", generator=g) * 0.002
+    idx = [slice(0, 4096), slice(n // 2 - 1111, n // 2 + 3001), slice(n - 5000, n)]
+    before = [([w[s].cpu().numpy().copy() for w in ws], c[s].cpu().numpy().copy(), d[s].cpu().numpy().copy()) for s in idx]
+    if rule == "easgd":
+        ss.ss_sync_easgd(ws, c, n, 0.1)
+    elif rule == "ma":
+        ss.ss_sync_ma(ws, c, n, 0.1)
+    else:
+        ss.ss_sync_bmuf(ws, c, d, n, 0.1, 1.0, 0.9)
+    torch.cuda.synchronize()
+    for s, (w0, c0, d0) in zip(idx, before):
+        if rule == "easgd":
+            O.sync_easgd(w0, c0, 0.1)
+        elif rule == "ma":
+            O.sync_ma(w0, 0.1, c0)
+        else:
+            O.sync_bmuf(w0, c0, d0, 0.1, 1.0, 0.9)
+        for r in range(R):
+            assert_close(ws[r][s].cpu().numpy(), w0[r], RTOL_SYNC, f"{rule} replica {r}")
+        assert_close(c[s].cpu().numpy(), c0, RTOL_SYNC, f"{rule} centre")
+        if rule == "bmuf":
+            assert_close(d[s].cpu().numpy(), d0, RTOL_SYNC, "delta")
