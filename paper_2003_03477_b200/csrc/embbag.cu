@@ -123,7 +123,7 @@ struct BwdPlan {
   int nwin;
   int nblk_u;        // blocks of the unique pass (1024 items each)
   size_t off_keys_a, off_keys_b, off_pos_a, off_pos_b, off_bag, off_hist, off_bintot, off_usum, off_uniq, off_seg,
-      off_uidx, off_partial, off_long, off_gsum, off_scalars, total;
+      off_uidx, off_sbag, off_partial, off_long, off_gsum, off_scalars, total;
 };
 
 static inline size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
@@ -156,6 +156,7 @@ static BwdPlan make_plan(int T, int64_t N, int D, int64_t L) {
   p.off_uniq = o; o += l4;
   p.off_seg = o; o += align256((size_t)(L + 1) * 4);
   p.off_uidx = o; o += l4;
+  p.off_sbag = o; o += l4;
   p.off_partial = o; o += align256((size_t)p.nwin * 2 * (size_t)D * 4);
   p.off_long = o; o += align256((size_t)p.nwin * 4);
   const uint64_t umax = (uint64_t)L < maxkey ? (uint64_t)L : maxkey;   // distinct rows cannot exceed either
@@ -378,11 +379,12 @@ unique_count_kernel(const uint32_t* __restrict__ keys, int64_t L, uint32_t senti
   if (threadIdx.x == 0) usum[blockIdx.x] = (uint32_t)c;
 }
 
-// uniq[u], seg[u] at the head of every segment; uidx[i] = segment of sorted position i.
+// uniq[u], seg[u] at the head of every segment; uidx[i] = segment of sorted position i; sbag[i] = its bag.
 __global__ void __launch_bounds__(kScanThreads)
 unique_write_kernel(const uint32_t* __restrict__ keys, int64_t L, uint32_t sentinel,
                     const uint32_t* __restrict__ ubase, int32_t* __restrict__ uniq, int32_t* __restrict__ seg,
-                    int32_t* __restrict__ uidx, int32_t* __restrict__ uniq_out, int32_t* __restrict__ seg_out) {
+                    int32_t* __restrict__ uidx, int32_t* __restrict__ uniq_out, int32_t* __restrict__ seg_out,
+                    const int32_t* __restrict__ perm, const int32_t* __restrict__ bag_of, int32_t* __restrict__ sbag) {
   __shared__ uint32_t wsum[32];
   const int64_t i = (int64_t)blockIdx.x * kScanThreads + threadIdx.x;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -410,6 +412,11 @@ unique_write_kernel(const uint32_t* __restrict__ keys, int64_t L, uint32_t senti
     if (seg_out) seg_out[before] = (int32_t)i;
   }
   if (in) uidx[i] = (int32_t)(before + (h ? 1u : 0u)) - 1;
+  // bag of every sorted position, so that the reduction reads it with one coalesced load
+  if (in && sbag) {
+    const int pj = perm[i];
+    sbag[i] = (pj >= 0 && pj < L) ? bag_of[pj] : -1;
+  }
   // the last valid position closes the last segment: seg[U] = number of valid lookups
   if (in && k < sentinel && (i == L - 1 || keys[i + 1] >= sentinel)) {
     const uint32_t u_end = before + (h ? 1u : 0u);
@@ -447,8 +454,8 @@ __device__ __forceinline__ bool ws_matches(const int32_t* scalars, int64_t L, ui
 // covers the window's first position) or slot 1.
 template <int G, int NV>
 __global__ void __launch_bounds__(256)
-window_reduce_kernel(const uint32_t* __restrict__ keys, const int32_t* __restrict__ perm,
-                     const int32_t* __restrict__ bag_of, const int32_t* __restrict__ uidx, int64_t L,
+window_reduce_kernel(const uint32_t* __restrict__ keys, const int32_t* __restrict__ sbag,
+                     const int32_t* __restrict__ uidx, int64_t L,
                      uint32_t sentinel, int64_t N, int D, int B, const float* __restrict__ grad, int64_t ld_grad,
                      int col0, float* __restrict__ gsum, float* __restrict__ partial, int32_t* __restrict__ long_list,
                      int32_t* __restrict__ scalars, int nwin, int64_t umax, int32_t* __restrict__ d_status) {
@@ -476,8 +483,7 @@ window_reduce_kernel(const uint32_t* __restrict__ keys, const int32_t* __restric
       const uint32_t key = keys[j];
       if (key < sentinel) {
         const int t = (int)(key / (uint64_t)N);
-        const int pj = perm[j];
-        const int b = (pj >= 0 && pj < L) ? bag_of[pj] - t * B : -1;
+        const int b = sbag[j] - t * B;
         u = uidx[j];
         // a consistent workspace never fails these; an inconsistent one must not turn into a wild access
         if (b >= 0 && b < B && u >= 0 && u < umax)
@@ -496,7 +502,7 @@ window_reduce_kernel(const uint32_t* __restrict__ keys, const int32_t* __restric
 #pragma unroll
   for (int v = 0; v < NV; ++v) acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
   int run_start = 0;
-  constexpr int kBatch = NV >= 8 ? 2 : (NV >= 4 ? 4 : (NV >= 2 ? 8 : 16));  // gradient rows in flight per lane
+  constexpr int kBatch = NV >= 8 ? 1 : (NV >= 4 ? 2 : (NV >= 2 ? 4 : 8));   // gradient rows in flight per lane
   for (int i0 = 0; i0 < kWin; i0 += kBatch) {
     float4 gv[kBatch][NV];
 #pragma unroll
@@ -713,7 +719,7 @@ static void launch_reduce(const BwdPlan& p, char* ws, const uint32_t* keys, cons
   int32_t* seg = reinterpret_cast<int32_t*>(ws + p.off_seg);
   {
     SS_TIMED("window_reduce_kernel", st);
-    window_reduce_kernel<G, NV><<<blocks, 256, 0, st>>>(keys, perm, reinterpret_cast<int32_t*>(ws + p.off_bag),
+    window_reduce_kernel<G, NV><<<blocks, 256, 0, st>>>(keys, reinterpret_cast<int32_t*>(ws + p.off_sbag),
                                                         reinterpret_cast<int32_t*>(ws + p.off_uidx), p.L, sentinel, N, D,
                                                         B, grad, ld_grad, col0, gsum, partial, long_list, scalars, p.nwin,
                                                         (int64_t)umax, d_status);
@@ -869,7 +875,8 @@ static ss_status bwd_impl(bool do_sort, bool do_apply, float* tables, float* row
   scan_exclusive_kernel<<<1, kScanThreads, 0, cs>>>(usum, p.nblk_u, usum + p.nblk_u);
   }
   { SS_TIMED("unique_write_kernel", cs);
-  unique_write_kernel<<<p.nblk_u, kScanThreads, 0, cs>>>(keys_sorted, L, sentinel, usum, uniq, seg, uidx, uniq_keys, seg_off);
+  unique_write_kernel<<<p.nblk_u, kScanThreads, 0, cs>>>(keys_sorted, L, sentinel, usum, uniq, seg, uidx, uniq_keys, seg_off,
+                                                         perm_sorted, bag_of, reinterpret_cast<int32_t*>(ws + p.off_sbag));
   }
   { SS_TIMED("unique_finish_kernel", cs);
   unique_finish_kernel<<<1, 1, 0, cs>>>(usum + p.nblk_u, seg, seg_off, d_num_unique, scalars, L, sentinel);
@@ -1013,7 +1020,8 @@ ss_status ss_embbag_bwd_sort_noalloc(int T, int64_t N, const int32_t* indices, c
   SS_CUDA(cudaMemcpyAsync(perm, pin, (size_t)L * 4, cudaMemcpyDeviceToDevice, cs));
   unique_count_kernel<<<nblk_u, kScanThreads, 0, cs>>>(kin, L, sentinel, usum);
   scan_exclusive_kernel<<<1, kScanThreads, 0, cs>>>(usum, nblk_u, usum + nblk_u);
-  unique_write_kernel<<<nblk_u, kScanThreads, 0, cs>>>(kin, L, sentinel, usum, uniq, seg, uidx, uniq_keys, seg_off);
+  unique_write_kernel<<<nblk_u, kScanThreads, 0, cs>>>(kin, L, sentinel, usum, uniq, seg, uidx, uniq_keys, seg_off,
+                                                       nullptr, nullptr, nullptr);
   unique_finish_kernel<<<1, 1, 0, cs>>>(usum + nblk_u, seg, seg_off, d_num_unique, scalars, L, sentinel);
   SS_LAUNCH_OK();
   return SS_OK;

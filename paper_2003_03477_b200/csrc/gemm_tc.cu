@@ -3,7 +3,7 @@
 //   C[m, n] = sum_k A(m, k) * B(n, k)
 //
 // One CTA computes a 128 x 128 tile.  Warp 0 (one lane) streams 128 x 64 / 64 x 128 operand tiles
-// into a ring of shared-memory stages with TMA (128-byte swizzle); warp 1 (one lane) issues
+// into a ring of shared-memory stages (3 or 6 deep) with TMA (128-byte swizzle); warp 1 (one lane) issues
 // tcgen05.mma (M = 128, N = 128, K = 16, accumulators in tensor memory) and releases stages with
 // tcgen05.commit; warps 2-5 wait for the accumulator, read it with tcgen05.ld (one row per thread)
 // and apply the epilogue (bias, ReLU, ReLU-gradient mask, bf16 / fp32 stores).
@@ -24,12 +24,15 @@
 namespace ss {
 
 constexpr int kBM = 128, kBN = 128, kBK = 64;
-constexpr int kStages = 5;
+// Ring depth: 3 stages (97 KiB, two CTAs per SM) for the small GEMMs of a training step, where several
+// replicas' kernels share the SMs and a second resident CTA hides more latency than a deeper ring does;
+// 6 stages (193 KiB, one CTA per SM) for large products that fill the machine on their own.
+constexpr int kStagesSmall = 3, kStagesLarge = 6;
 constexpr int kTileBytes = kBM * kBK * 2;                 // 16 KiB per operand tile
 constexpr int kStageBytes = 2 * kTileBytes;
 constexpr int kTcThreads = 192;
 constexpr int kTmemCols = 128;
-constexpr size_t kTcSmem = (size_t)kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr size_t tc_smem_bytes(int stages) { return (size_t)stages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/; }
 constexpr long long kWaitCycles = 400ll * 1000 * 1000;    // ~0.2 s: far beyond any legitimate wait
 constexpr long long kWaitCyclesAborted = 2ll * 1000 * 1000;
 
@@ -122,6 +125,7 @@ __device__ __forceinline__ uint32_t pack2(float a, float b) {
 }
 
 // ---------------------------------------------------------------------------------------- kernel
+template <int kStages>
 __global__ void __launch_bounds__(kTcThreads, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, TcParams p) {
   extern __shared__ uint8_t smem_raw[];
@@ -341,7 +345,10 @@ ss_status gemm_tc(int M, int N, int K, const Operand& A, const Operand& B, const
   int dev = 0;
   SS_CUDA(cudaGetDevice(&dev));
   if (dev >= 0 && dev < 64 && !attr_set[dev]) {
-    SS_CUDA(cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTcSmem));
+    SS_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<kStagesSmall>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)tc_smem_bytes(kStagesSmall)));
+    SS_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<kStagesLarge>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)tc_smem_bytes(kStagesLarge)));
     attr_set[dev] = true;
   }
   TcParams p;
@@ -363,7 +370,12 @@ ss_status gemm_tc(int M, int N, int K, const Operand& A, const Operand& B, const
   if (!oka || !okb) return SS_ERR_CUDA;
   dim3 grid((N + kBN - 1) / kBN, (M + kBM - 1) / kBM, k_splits);
   { SS_TIMED("gemm_tc_kernel", st);
-  gemm_tc_kernel<<<grid, kTcThreads, kTcSmem, st>>>(ma, mb, p);
+  const long long ctas = (long long)grid.x * grid.y * grid.z;
+  const int nk_slice = (nk_all + k_splits - 1) / k_splits;
+  if (ctas >= 2ll * num_sms() && nk_slice >= 2 * kStagesLarge)
+    gemm_tc_kernel<kStagesLarge><<<grid, kTcThreads, tc_smem_bytes(kStagesLarge), st>>>(ma, mb, p);
+  else
+    gemm_tc_kernel<kStagesSmall><<<grid, kTcThreads, tc_smem_bytes(kStagesSmall), st>>>(ma, mb, p);
   }
   SS_LAUNCH_OK();
   return SS_OK;
