@@ -452,14 +452,21 @@ __device__ __forceinline__ bool ws_matches(const int32_t* scalars, int64_t L, ui
 // run of equal keys in position order.  A run that lies inside the window is complete: its sum goes
 // to gsum[u].  A run that crosses a window edge leaves a partial sum in the window's slot 0 (run
 // covers the window's first position) or slot 1.
-template <int G, int NV>
+// FUSE (rows of at most 128 floats): the sums of the complete runs stay in shared memory and the group applies
+// row-wise Adagrad to those rows itself, four rows' loads in flight, so their sums never travel through global
+// memory; only rows crossing window edges go through gsum and the kernels that follow.
+template <int G, int NV, bool FUSE>
 __global__ void __launch_bounds__(256)
 window_reduce_kernel(const uint32_t* __restrict__ keys, const int32_t* __restrict__ sbag,
                      const int32_t* __restrict__ uidx, int64_t L,
                      uint32_t sentinel, int64_t N, int D, int B, const float* __restrict__ grad, int64_t ld_grad,
                      int col0, float* __restrict__ gsum, float* __restrict__ partial, int32_t* __restrict__ long_list,
-                     int32_t* __restrict__ scalars, int nwin, int64_t umax, int32_t* __restrict__ d_status) {
+                     int32_t* __restrict__ scalars, int nwin, int64_t umax, int32_t* __restrict__ d_status,
+                     float* __restrict__ tables, float* __restrict__ row_state, float lr, float eps) {
   constexpr int kGroups = 256 / G;
+  extern __shared__ float4 s_sum[];                        // FUSE: [kGroups][kWin][D/4] sums of complete runs
+  __shared__ uint32_t s_runkey[FUSE ? kGroups : 1][kWin];
+  int nr = 0;
   __shared__ uint32_t s_key[kGroups][kWin + 2];            // [0] = key before the window, [kWin+1] = key after
   __shared__ int32_t s_row[kGroups][kWin];                 // float4 index of the lookup's gradient row
   __shared__ int32_t s_u[kGroups][kWin];
@@ -525,14 +532,21 @@ window_reduce_kernel(const uint32_t* __restrict__ keys, const int32_t* __restric
       if (next != key || i == kWin - 1) {
         const bool head_open = (run_start == 0) && (s_key[grp][0] == key);
         const bool tail_open = (next == key);              // only possible at the window's last position
-        float4* dst = (!head_open && !tail_open)
-                          ? reinterpret_cast<float4*>(gsum + (int64_t)s_u[grp][i] * D)
-                          : reinterpret_cast<float4*>(partial + ((int64_t)win * 2 + (run_start == 0 ? 0 : 1)) * D);
+        const bool complete = !head_open && !tail_open;
+        if (FUSE && complete) {
+          if (lane < nvec) s_sum[((size_t)grp * kWin + nr) * nvec + lane] = acc[0];
+          if (lane == 0) s_runkey[grp][nr] = key;
+          ++nr;
+          acc[0] = make_float4(0.f, 0.f, 0.f, 0.f);
+        } else {
+          float4* dst = complete ? reinterpret_cast<float4*>(gsum + (int64_t)s_u[grp][i] * D)
+                                 : reinterpret_cast<float4*>(partial + ((int64_t)win * 2 + (run_start == 0 ? 0 : 1)) * D);
 #pragma unroll
-        for (int v = 0; v < NV; ++v) {
-          const int c = lane + v * G;
-          if (c < nvec) dst[c] = acc[v];
-          acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
+          for (int v = 0; v < NV; ++v) {
+            const int c = lane + v * G;
+            if (c < nvec) dst[c] = acc[v];
+            acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
+          }
         }
         // the window in which a multi-window run starts enters the row in the list of rows to combine
         if (!head_open && tail_open && lane == 0) {
@@ -540,6 +554,40 @@ window_reduce_kernel(const uint32_t* __restrict__ keys, const int32_t* __restric
           if (slot < nwin) long_list[slot] = s_u[grp][i];   // at most one such run per window
         }
         run_start = i + 1;
+      }
+    }
+  }
+  if (FUSE) {
+    // row-wise Adagrad on the rows whose whole run lay in this window
+    __syncwarp(gmask);
+    for (int r0 = 0; r0 < nr; r0 += 4) {
+      uint32_t rk[4];
+      float4 rw[4], g[4];
+      float st[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const bool ok = r0 + j < nr;
+        rk[j] = ok ? s_runkey[grp][r0 + j] : 0u;
+        const float4* row = reinterpret_cast<const float4*>(tables + (int64_t)rk[j] * D);
+        rw[j] = (ok && lane < nvec) ? row[lane] : make_float4(0.f, 0.f, 0.f, 0.f);
+        g[j] = (ok && lane < nvec) ? s_sum[((size_t)grp * kWin + r0 + j) * nvec + lane] : make_float4(0.f, 0.f, 0.f, 0.f);
+        st[j] = ok ? row_state[rk[j]] : 0.f;
+      }
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        float ss = g[j].x * g[j].x + g[j].y * g[j].y + g[j].z * g[j].z + g[j].w * g[j].w;
+#pragma unroll
+        for (int off = G / 2; off >= 1; off >>= 1) ss += __shfl_down_sync(gmask, ss, off, G);
+        ss = __shfl_sync(gmask, ss, 0, G);                 // every lane uses lane 0's sum
+        if (r0 + j >= nr) continue;
+        const float sn = st[j] + ss / (float)D;
+        const float scale = lr / (sqrtf(sn) + eps);
+        if (lane < nvec) {
+          float4 o = rw[j];
+          o.x -= scale * g[j].x; o.y -= scale * g[j].y; o.z -= scale * g[j].z; o.w -= scale * g[j].w;
+          reinterpret_cast<float4*>(tables + (int64_t)rk[j] * D)[lane] = o;
+        }
+        if (lane == 0) row_state[rk[j]] = sn;
       }
     }
   }
@@ -641,33 +689,36 @@ template <int NV> struct RowsPerGroup { static constexpr int value = NV == 1 ? 4
 
 template <int G, int NV>
 __global__ void __launch_bounds__(256)
-apply_rows_kernel(const int32_t* __restrict__ uniq, int32_t* __restrict__ scalars, int D,
+apply_rows_kernel(const int32_t* __restrict__ uniq, const int32_t* __restrict__ scalars, int D,
                   const float* __restrict__ gsum, float* __restrict__ tables, float* __restrict__ row_state,
-                  float lr, float eps, int64_t L, uint32_t sentinel, int64_t umax) {
+                  float lr, float eps, int64_t L, uint32_t sentinel, int64_t umax,
+                  const int32_t* __restrict__ list, int list_cap) {
   constexpr int kGroups = 256 / G;
   constexpr int RB = RowsPerGroup<NV>::value;              // rows per group, their loads issued together
   const int grp = threadIdx.x / G, lane = threadIdx.x % G;
   const unsigned gmask = (G == 32) ? 0xffffffffu : (((1u << G) - 1u) << ((threadIdx.x & 31) / G * G));
   if (!ws_matches(scalars, L, sentinel, nullptr)) return;
-  const int U = min((int64_t)scalars[0], umax);
-  // the list of multi-window rows has been consumed by the previous kernel: empty it for the next reduction
-  if (blockIdx.x == 0 && threadIdx.x == 0) scalars[1] = 0;
+  // all distinct rows, or (list given) only the listed ones: the rows whose run crossed window edges
+  const int U = list ? min(scalars[1], list_cap) : (int)min((int64_t)scalars[0], umax);
   const int nvec = D >> 2;
   const int64_t u0 = ((int64_t)blockIdx.x * kGroups + grp) * RB;
   if (u0 >= U) return;
   uint32_t key[RB];
+  int64_t urow[RB];
   bool valid[RB];
 #pragma unroll
   for (int r = 0; r < RB; ++r) {
     valid[r] = u0 + r < U;
-    key[r] = valid[r] ? (uint32_t)uniq[u0 + r] : 0u;
+    urow[r] = valid[r] ? (list ? (int64_t)list[u0 + r] : u0 + r) : 0;
+    if (urow[r] < 0 || urow[r] >= umax) { valid[r] = false; urow[r] = 0; }
+    key[r] = valid[r] ? (uint32_t)uniq[urow[r]] : 0u;
     if (key[r] >= sentinel) valid[r] = false;              // never true for a consistent workspace
   }
   float4 g[RB][NV], rw[RB][NV];
   float st[RB];
 #pragma unroll
   for (int r = 0; r < RB; ++r) {
-    const float4* p = reinterpret_cast<const float4*>(gsum + (u0 + r) * D);
+    const float4* p = reinterpret_cast<const float4*>(gsum + urow[r] * D);
     const float4* row = reinterpret_cast<const float4*>(tables + (int64_t)key[r] * D);
 #pragma unroll
     for (int v = 0; v < NV; ++v) {
@@ -717,12 +768,26 @@ static void launch_reduce(const BwdPlan& p, char* ws, const uint32_t* keys, cons
   int32_t* scalars = reinterpret_cast<int32_t*>(ws + p.off_scalars);
   int32_t* long_list = reinterpret_cast<int32_t*>(ws + p.off_long);
   int32_t* seg = reinterpret_cast<int32_t*>(ws + p.off_seg);
+  int32_t* uniq = reinterpret_cast<int32_t*>(ws + p.off_uniq);
+  constexpr bool kFuse = (NV == 1);
+  // the list of rows crossing window edges starts empty (the apply half may be repeated on one sort)
+  cudaMemsetAsync(scalars + 1, 0, sizeof(int32_t), st);
   {
     SS_TIMED("window_reduce_kernel", st);
-    window_reduce_kernel<G, NV><<<blocks, 256, 0, st>>>(keys, reinterpret_cast<int32_t*>(ws + p.off_sbag),
-                                                        reinterpret_cast<int32_t*>(ws + p.off_uidx), p.L, sentinel, N, D,
-                                                        B, grad, ld_grad, col0, gsum, partial, long_list, scalars, p.nwin,
-                                                        (int64_t)umax, d_status);
+    const size_t smem = kFuse ? (size_t)kGroups * kWin * D * 4 : 0;
+    if (kFuse) {
+      static bool attr_set[64];
+      int dev = 0;
+      if (cudaGetDevice(&dev) == cudaSuccess && dev >= 0 && dev < 64 && !attr_set[dev]) {
+        cudaFuncSetAttribute(window_reduce_kernel<G, NV, kFuse>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             65536);   // kGroups * kWin * (4G floats) * 4 bytes for every G
+        attr_set[dev] = true;
+      }
+    }
+    window_reduce_kernel<G, NV, kFuse><<<blocks, 256, smem, st>>>(
+        keys, reinterpret_cast<int32_t*>(ws + p.off_sbag), reinterpret_cast<int32_t*>(ws + p.off_uidx), p.L, sentinel, N, D,
+        B, grad, ld_grad, col0, gsum, partial, long_list, scalars, p.nwin, (int64_t)umax, d_status, tables, row_state, lr,
+        eps);
   }
   {
     SS_TIMED("combine_rows_kernel", st);
@@ -730,12 +795,14 @@ static void launch_reduce(const BwdPlan& p, char* ws, const uint32_t* keys, cons
     combine_rows_kernel<G, NV><<<cblocks, 256, (size_t)kGroups * D * 4, st>>>(seg, scalars, long_list, p.nwin, D, partial, gsum,
                                                                               p.L, sentinel, (int64_t)umax);
   }
+  // row update: every distinct row, or with the fused window kernel only the rows that crossed window edges
   const uint64_t per_block = (uint64_t)kGroups * RowsPerGroup<NV>::value;
-  const unsigned ublocks = (unsigned)((umax + per_block - 1) / per_block);
+  const uint64_t nrows = kFuse ? (uint64_t)p.nwin : umax;
+  const unsigned ublocks = (unsigned)((nrows + per_block - 1) / per_block);
   {
     SS_TIMED("apply_rows_kernel", st);
-    apply_rows_kernel<G, NV><<<ublocks, 256, 0, st>>>(reinterpret_cast<int32_t*>(ws + p.off_uniq), scalars, D, gsum,
-                                                      tables, row_state, lr, eps, p.L, sentinel, (int64_t)umax);
+    apply_rows_kernel<G, NV><<<ublocks, 256, 0, st>>>(uniq, scalars, D, gsum, tables, row_state, lr, eps, p.L, sentinel,
+                                                      (int64_t)umax, kFuse ? long_list : nullptr, p.nwin);
   }
 }
 
