@@ -221,6 +221,25 @@ ss_status ss_sync_bmuf(float* const* w, int R, float* global, float* delta, int6
                        void* const* w_bf16, ss_stream stream);
 
 /* ------------------------------------------------------------------------------------------
+ * The shadow thread (Section 3.2; "shadow thread do" of Algorithms 1-4): ss_shadow_start spawns a host
+ * thread that loops  { one synchronisation pass on `stream` }  until ss_shadow_stop, the rule's
+ * arguments as in ss_sync_easgd (rule 0), ss_sync_ma (rule 1, center = global_out) or ss_sync_bmuf
+ * (rule 2).  It waits on nothing but its own earlier passes: at most max_in_flight (1..8) passes are
+ * queued ahead of the device; pause_us > 0 sleeps between passes; it ends by itself after max_rounds
+ * passes.  Give it a stream of the lowest priority and the training streams a higher one, and the
+ * device runs the passes in whatever room training leaves.  The pointer arrays are copied; the
+ * buffers they point to must outlive ss_shadow_stop, which joins the thread, waits for the queued
+ * passes, stores the number of passes in *rounds_out (nullable), frees the handle and returns the
+ * first error the thread met (SS_OK if none).  ss_shadow_rounds reads the running count.
+ * ---------------------------------------------------------------------------------------- */
+typedef struct ss_shadow ss_shadow;
+ss_status ss_shadow_start(ss_shadow** out, int rule, float* const* w, int R, float* center, float* delta, int64_t n,
+                          float alpha, float eta, float mu, int flags, void* const* w_bf16, ss_stream stream,
+                          int max_in_flight, int pause_us, int64_t max_rounds);
+int64_t ss_shadow_rounds(const ss_shadow* h);
+ss_status ss_shadow_stop(ss_shadow* h, int64_t* rounds_out);
+
+/* ------------------------------------------------------------------------------------------
  * The tensor-core building block of ss_mlp_fwd / ss_mlp_bwd, exposed for testing and timing:
  *   C[m, n] = sum_k A(m, k) * B(n, k),  bf16 operands, float accumulation, float C [M, ldc].
  * a_mn_major = 0: A is stored [M, lda] with k contiguous (activations, weights in the forward pass).

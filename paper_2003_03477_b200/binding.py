@@ -24,7 +24,7 @@ SS_SYNC_EASGD_LITERAL = 1
 
 EXPORTS = ["ss_status_str", "ss_last_cuda_error", "ss_num_sms", "ss_embbag_fwd", "ss_embbag_bwd_workspace_bytes",
            "ss_embbag_bwd_adagrad", "ss_embbag_bwd_sort", "ss_embbag_bwd_apply", "ss_embbag_bwd_sort_noalloc", "ss_mlp_param_count", "ss_mlp_param_offsets", "ss_mlp_workspace_bytes",
-           "ss_mlp_fwd", "ss_mlp_bwd", "ss_sync_easgd", "ss_sync_ma", "ss_sync_bmuf", "ss_to_bf16",
+           "ss_mlp_fwd", "ss_mlp_bwd", "ss_sync_easgd", "ss_sync_ma", "ss_sync_bmuf", "ss_shadow_start", "ss_shadow_rounds", "ss_shadow_stop", "ss_to_bf16",
            "ss_gemm_bf16", "ss_device_error", "ssh_fill_uniform", "ss_profile", "ss_profile_collect"]
 
 
@@ -78,6 +78,11 @@ def lib() -> C.CDLL:
         L.ss_sync_easgd.argtypes = [C.POINTER(vp), i32, vp, i64, f32, i32, C.POINTER(vp), vp]
         L.ss_sync_ma.argtypes = [C.POINTER(vp), i32, vp, i64, f32, i32, C.POINTER(vp), vp]
         L.ss_sync_bmuf.argtypes = [C.POINTER(vp), i32, vp, vp, i64, f32, f32, f32, i32, C.POINTER(vp), vp]
+        L.ss_shadow_start.argtypes = [C.POINTER(vp), i32, C.POINTER(vp), i32, vp, vp, i64, f32, f32, f32, i32, C.POINTER(vp), vp,
+                                      i32, i32, i64]
+        L.ss_shadow_rounds.argtypes = [vp]
+        L.ss_shadow_rounds.restype = i64
+        L.ss_shadow_stop.argtypes = [vp, C.POINTER(i64)]
         L.ss_to_bf16.argtypes = [vp, vp, i64, vp]
         L.ss_gemm_bf16.argtypes = [vp, i32, i64, vp, i32, i64, vp, i64, i32, i32, i32, i32, vp]
         L.ss_device_error.argtypes = [i32]
@@ -86,7 +91,7 @@ def lib() -> C.CDLL:
         L.ssh_fill_uniform.argtypes = [vp, i64, C.c_uint64, C.c_uint64, f32, f32, vp]
         for name in EXPORTS:
             if name not in ("ss_status_str", "ss_last_cuda_error", "ss_num_sms", "ss_embbag_bwd_workspace_bytes",
-                            "ss_mlp_param_count", "ss_mlp_workspace_bytes"):
+                            "ss_mlp_param_count", "ss_mlp_workspace_bytes", "ss_shadow_rounds"):
                 getattr(L, name).restype = i32
         _lib = L
     return _lib
@@ -248,6 +253,30 @@ def ss_gemm_bf16(a, a_mn_major, lda, b, b_mn_major, ldb, c, ldc, M, N, K, force_
 
 def ss_device_error(clear: bool = True) -> int:
     return lib().ss_device_error(1 if clear else 0)
+
+
+RULES = {"easgd": 0, "ma": 1, "bmuf": 2}
+
+
+def ss_shadow_start(rule, w, center, delta, n, alpha, eta=1.0, mu=0.0, flags=0, w_bf16=None, stream=None,
+                    max_in_flight=2, pause_us=0, max_rounds=1 << 40):
+    """Start the native shadow thread; returns its handle (pass it to ss_shadow_rounds / ss_shadow_stop)."""
+    h = C.c_void_p()
+    _check("ss_shadow_start", lib().ss_shadow_start(C.byref(h), RULES[rule], _ptr_array(w), len(w), _ptr(center),
+                                                     _ptr(delta), n, alpha, eta, mu, flags, _ptr_array(w_bf16),
+                                                     _stream(stream), max_in_flight, pause_us, max_rounds))
+    return h
+
+
+def ss_shadow_rounds(handle) -> int:
+    return int(lib().ss_shadow_rounds(handle))
+
+
+def ss_shadow_stop(handle) -> int:
+    """Stop and join the shadow thread; returns the number of synchronisation passes it enqueued."""
+    rounds = C.c_int64(0)
+    _check("ss_shadow_stop", lib().ss_shadow_stop(handle, C.byref(rounds)))
+    return int(rounds.value)
 
 
 def ss_to_bf16(src, dst_bf16, n, stream=None) -> None:

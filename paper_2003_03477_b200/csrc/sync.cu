@@ -206,4 +206,92 @@ ss_status ss_sync_bmuf(float* const* w, int R, float* global, float* delta, int6
   return ss::launch<ss::RULE_BMUF>(R, p, w_bf16 != nullptr, global, delta, n, s, ss::as_stream(stream));
 }
 
+// ------------------------------------------------------------------------------------------------
+// The shadow thread (Section 3.2, Algorithm 1): a host thread that does nothing but enqueue one
+// synchronisation pass after another on the stream it was given, with a bounded number of passes in
+// flight.  It shares no event with any training stream and knows nothing about training.
+// ------------------------------------------------------------------------------------------------
+}  // extern "C"
+
+#include <atomic>
+#include <chrono>
+#include <thread>
+
+struct ss_shadow {
+  int rule, R, flags, device, max_in_flight, pause_us;
+  float* w[ss::kMaxR];
+  void* m[ss::kMaxR];
+  bool mirror;
+  float *center, *delta;
+  int64_t n, max_rounds;
+  float alpha, eta, mu;
+  cudaStream_t stream;
+  std::atomic<int64_t> rounds{0};
+  std::atomic<int> stop{0};
+  std::atomic<int> status{SS_OK};
+  std::thread thread;
+};
+
+static void shadow_main(ss_shadow* h) {
+  if (cudaSetDevice(h->device) != cudaSuccess) { h->status = SS_ERR_CUDA; return; }
+  const int depth = h->max_in_flight < 1 ? 1 : (h->max_in_flight > 8 ? 8 : h->max_in_flight);
+  cudaEvent_t ev[8];
+  for (int i = 0; i < depth; ++i)
+    if (cudaEventCreateWithFlags(&ev[i], cudaEventDisableTiming) != cudaSuccess) { h->status = SS_ERR_CUDA; return; }
+  int64_t k = 0;
+  while (!h->stop.load(std::memory_order_relaxed) && k < h->max_rounds) {
+    const int slot = (int)(k % depth);
+    if (k >= depth && cudaEventSynchronize(ev[slot]) != cudaSuccess) { h->status = SS_ERR_CUDA; break; }
+    ss_status st;
+    void* const* mir = h->mirror ? h->m : nullptr;
+    if (h->rule == 0) st = ss_sync_easgd(h->w, h->R, h->center, h->n, h->alpha, h->flags, mir, h->stream);
+    else if (h->rule == 1) st = ss_sync_ma(h->w, h->R, h->center, h->n, h->alpha, h->flags, mir, h->stream);
+    else st = ss_sync_bmuf(h->w, h->R, h->center, h->delta, h->n, h->alpha, h->eta, h->mu, h->flags, mir, h->stream);
+    if (st != SS_OK) { h->status = st; break; }
+    cudaEventRecord(ev[slot], h->stream);
+    h->rounds.store(++k, std::memory_order_relaxed);
+    if (h->pause_us > 0) std::this_thread::sleep_for(std::chrono::microseconds(h->pause_us));
+  }
+  for (int i = 0; i < depth; ++i) {
+    cudaEventSynchronize(ev[i]);
+    cudaEventDestroy(ev[i]);
+  }
+}
+
+extern "C" {
+
+ss_status ss_shadow_start(ss_shadow** out, int rule, float* const* w, int R, float* center, float* delta, int64_t n,
+                          float alpha, float eta, float mu, int flags, void* const* w_bf16, ss_stream stream,
+                          int max_in_flight, int pause_us, int64_t max_rounds) {
+  if (!out || !w || !center) return SS_ERR_NULL;
+  if (rule < 0 || rule > 2 || R < 1 || R > ss::kMaxR || n < 0 || max_rounds < 0) return SS_ERR_SHAPE;
+  if (rule == 2 && !delta) return SS_ERR_NULL;
+  if (!(alpha >= 0.f && alpha <= 1.f)) return SS_ERR_RANGE;
+  ss_status st = ss::check_arch();
+  if (st != SS_OK) return st;
+  ss_shadow* h = new ss_shadow();
+  h->rule = rule; h->R = R; h->flags = flags; h->max_in_flight = max_in_flight; h->pause_us = pause_us;
+  h->mirror = w_bf16 != nullptr;
+  for (int r = 0; r < ss::kMaxR; ++r) { h->w[r] = r < R ? w[r] : nullptr; h->m[r] = (w_bf16 && r < R) ? w_bf16[r] : nullptr; }
+  h->center = center; h->delta = delta; h->n = n; h->max_rounds = max_rounds;
+  h->alpha = alpha; h->eta = eta; h->mu = mu;
+  h->stream = ss::as_stream(stream);
+  if (cudaGetDevice(&h->device) != cudaSuccess) { delete h; return SS_ERR_CUDA; }
+  h->thread = std::thread(shadow_main, h);
+  *out = h;
+  return SS_OK;
+}
+
+int64_t ss_shadow_rounds(const ss_shadow* h) { return h ? h->rounds.load(std::memory_order_relaxed) : -1; }
+
+ss_status ss_shadow_stop(ss_shadow* h, int64_t* rounds_out) {
+  if (!h) return SS_ERR_NULL;
+  h->stop.store(1);
+  if (h->thread.joinable()) h->thread.join();
+  if (rounds_out) *rounds_out = h->rounds.load();
+  const ss_status st = (ss_status)h->status.load();
+  delete h;
+  return st;
+}
+
 }  // extern "C"

@@ -10,8 +10,6 @@ This module allocates torch tensors and calls the binding; it computes nothing i
 """
 from __future__ import annotations
 
-import threading
-import time
 from typing import List, Optional, Sequence
 
 import numpy as np
@@ -148,49 +146,36 @@ class Model:
 class ShadowLoop:
     """The shadow thread: loops the synchronisation on the low-priority stream, unaware of training.
 
-    At most `max_in_flight` sync kernels are queued ahead of the device; `pause_s` > 0 paces the loop.
+    The loop itself is a native host thread inside the library (ss_shadow_start), so it neither holds nor
+    waits for the Python interpreter lock.  At most `max_in_flight` sync kernels are queued ahead of the
+    device; `pause_s` > 0 paces the loop.
     """
 
     def __init__(self, model: Model, rule: str, alpha: float, eta: float = 1.0, mu: float = 0.0,
-                 max_in_flight: int = 2, pause_s: float = 0.0, max_rounds: int = 1 << 30):
+                 max_in_flight: int = 2, pause_s: float = 0.0, max_rounds: int = 1 << 40):
         self.model, self.rule, self.alpha, self.eta, self.mu = model, rule, alpha, eta, mu
         self.max_in_flight, self.pause_s, self.max_rounds = max_in_flight, pause_s, max_rounds
-        self.rounds = 0
-        self._stop = threading.Event()
-        self._thread: Optional[threading.Thread] = None
-        self.error: Optional[BaseException] = None
+        self._handle = None
+        self._final = 0
 
-    def _run(self) -> None:
-        try:
-            torch.cuda.set_device(self.model.tables.device)
-            pending: List[torch.cuda.Event] = []
-            while not self._stop.is_set() and self.rounds < self.max_rounds:
-                if len(pending) >= self.max_in_flight:
-                    pending.pop(0).synchronize()
-                self.model.sync(self.rule, self.alpha, self.eta, self.mu)
-                ev = torch.cuda.Event()
-                ev.record(self.model.sync_stream)
-                pending.append(ev)
-                self.rounds += 1
-                if self.pause_s > 0:
-                    time.sleep(self.pause_s)
-            for ev in pending:
-                ev.synchronize()
-        except BaseException as e:  # surfaced by stop()
-            self.error = e
+    @property
+    def rounds(self) -> int:
+        return ss.ss_shadow_rounds(self._handle) if self._handle is not None else self._final
 
     def start(self) -> "ShadowLoop":
-        self._thread = threading.Thread(target=self._run, name="shadow", daemon=True)
-        self._thread.start()
+        m = self.model
+        ws = [rep.w for rep in m.replicas]
+        mirrors = [rep.w_bf16 for rep in m.replicas] if m.spec.bf16 else None
+        self._handle = ss.ss_shadow_start(self.rule, ws, m.center, m.delta, m.spec.param_count, self.alpha, self.eta,
+                                          self.mu, 0, mirrors, m.sync_stream, self.max_in_flight,
+                                          int(self.pause_s * 1e6), self.max_rounds)
         return self
 
     def stop(self) -> int:
-        self._stop.set()
-        if self._thread is not None:
-            self._thread.join()
-        if self.error is not None:
-            raise self.error
-        return self.rounds
+        if self._handle is not None:
+            self._final = ss.ss_shadow_stop(self._handle)
+            self._handle = None
+        return self._final
 
 
 # ------------------------------------------------------------------------------------------
