@@ -281,6 +281,8 @@ def bench_gpu(args):
         return {"n": n, "R": R, "us": ms * 1e3, "GB/s": gbs, "frac_of_hbm_peak": gbs / peaks["hbm_gbs"]}
     out["sync"]["kernel_alone_64M"] = time_sync(1 << 26, cfg.R)
     torch.cuda.synchronize()
+    if cfg.bf16:
+        out["gemm_alone"] = gemm_alone(s, peaks)
 
     # ---- end to end through the public API with host buffers ------------------------------------
     if not args.quick:
@@ -289,6 +291,36 @@ def bench_gpu(args):
     print(json.dumps(out))
     if world > 1:
         dist.destroy_process_group()
+
+
+def gemm_alone(stream, peaks):
+    """The tensor-core GEMM kernel on its own (ss_gemm_bf16, bf16 in, fp32 out), timed with events around a
+    captured graph of back-to-back launches: a product large enough to fill the machine, and the largest
+    product of the medium model's step, against the measured burst bf16 peak."""
+    import torch
+    from paper_2003_03477_b200 import binding as ss
+    res = []
+    for M, N, K, reps in ((4096, 4096, 4096, 10), (2048, 1728, 512, 20)):
+        a = torch.randn(M, K, device="cuda").to(torch.bfloat16)
+        b = torch.randn(N, K, device="cuda").to(torch.bfloat16)
+        c = torch.empty(M, N, device="cuda")
+        ss.ss_gemm_bf16(a, 0, K, b, 0, K, c, N, M, N, K, 0, stream)
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=stream):
+            for _ in range(reps):
+                ss.ss_gemm_bf16(a, 0, K, b, 0, K, c, N, M, N, K, 0, stream)
+        with torch.cuda.stream(stream):
+            g.replay()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            g.replay()
+            e1.record(stream)
+        torch.cuda.synchronize()
+        us = e0.elapsed_time(e1) * 1e3 / reps
+        tf = 2.0 * M * N * K / us / 1e6
+        res.append({"M": M, "N": N, "K": K, "us": us, "TFLOP/s": tf, "frac_of_bf16_peak": tf / peaks["bf16_tflops"]})
+    return res
 
 
 def profile_pass(model, dev, cfg, steps=6):
@@ -480,6 +512,36 @@ def bench_reference(args):
         "gpu_launches": 0}))
 
 
+def bench_sweep(args):
+    """Isolated sync-kernel sweep: n in {1M, 8M, 64M, 256M} floats per replica, R in {2, 4, 8, 16}, all three
+    rules (S-EASGD alpha 0.1, S-MA alpha 0.1, S-BMUF mu 0.9 eta 1); one JSON line with GB/s against the HBM peak."""
+    import torch
+    from paper_2003_03477_b200 import binding as ss
+    torch.cuda.set_device(0)
+    peaks = measured_peaks()
+    s = torch.cuda.current_stream()
+    rows = []
+    for n in (1 << 20, 1 << 23, 1 << 26, 1 << 28):
+        for R in (2, 4, 8, 16):
+            if (R + 2) * n * 4 > 60e9:
+                continue
+            ws = [torch.randn(n, device="cuda") * 0.02 for _ in range(R)]
+            c = torch.randn(n, device="cuda") * 0.02
+            d = torch.zeros(n, device="cuda")
+            for rule, fn, per in (("easgd", lambda i: ss.ss_sync_easgd(ws, c, n, 0.1, 0, None, s), 2 * R + 2),
+                                  ("ma", lambda i: ss.ss_sync_ma(ws, c, n, 0.1, 0, None, s), 2 * R + 1),
+                                  ("bmuf", lambda i: ss.ss_sync_bmuf(ws, c, d, n, 0.1, 1.0, 0.9, 0, None, s), 2 * R + 4)):
+                time_kernel_call(fn, s, 3)
+                reps = 50 if n <= (1 << 23) else 10
+                ms = time_kernel_call(fn, s, reps)
+                gbs = per * 4 * n / (ms * 1e-3) / 1e9
+                rows.append({"rule": rule, "R": R, "n": n, "us": round(ms * 1e3, 2), "GB/s": round(gbs, 1),
+                             "frac_of_hbm_peak": round(gbs / peaks["hbm_gbs"], 3),
+                             "l2_resident": bool(per * 4 * n < 100e6)})
+            del ws, c, d
+    print(json.dumps({"sweep": "sync kernels alone", "peak_gbs": peaks["hbm_gbs"], "peak_source": peaks["source"], "rows": rows}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -492,8 +554,11 @@ def main():
     ap.add_argument("--cpu-budget", type=float, default=15.0)
     ap.add_argument("--replicas", type=int, default=0, help="override the workload's replica count (experiments)")
     ap.add_argument("--quick", action="store_true", help="skip the e2e and CPU-baseline legs (experiments)")
+    ap.add_argument("--sweep", action="store_true", help="isolated sync-kernel sweep instead of the training benchmark")
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.sweep:
+        bench_sweep(args)
+    elif args.impl == "reference":
         bench_reference(args)
     else:
         bench_gpu(args)

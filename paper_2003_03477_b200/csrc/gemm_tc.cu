@@ -2,9 +2,9 @@
 //
 //   C[m, n] = sum_k A(m, k) * B(n, k)
 //
-// One CTA computes a 128 x 128 tile.  Warp 0 (one lane) streams 128 x 64 / 64 x 128 operand tiles
+// One CTA computes a 128 x 128 (or, for large products, 128 x 256) tile.  Warp 0 (one lane) streams 128 x 64 / 64 x 128 operand tiles
 // into a ring of shared-memory stages (3 or 6 deep) with TMA (128-byte swizzle); warp 1 (one lane) issues
-// tcgen05.mma (M = 128, N = 128, K = 16, accumulators in tensor memory) and releases stages with
+// tcgen05.mma (M = 128, N = 128 or 256, K = 16, accumulators in tensor memory) and releases stages with
 // tcgen05.commit; warps 2-5 wait for the accumulator, read it with tcgen05.ld (one row per thread)
 // and apply the epilogue (bias, ReLU, ReLU-gradient mask, bf16 / fp32 stores).
 //
@@ -23,16 +23,18 @@
 
 namespace ss {
 
-constexpr int kBM = 128, kBN = 128, kBK = 64;
+constexpr int kBM = 128, kBK = 64;   // tile rows and k depth; the tile width kBN (128 or 256) is a template parameter
 // Ring depth: 3 stages (97 KiB, two CTAs per SM) for the small GEMMs of a training step, where several
 // replicas' kernels share the SMs and a second resident CTA hides more latency than a deeper ring does;
 // 6 stages (193 KiB, one CTA per SM) for large products that fill the machine on their own.
 constexpr int kStagesSmall = 3, kStagesLarge = 6;
-constexpr int kTileBytes = kBM * kBK * 2;                 // 16 KiB per operand tile
-constexpr int kStageBytes = 2 * kTileBytes;
+// 128 x 256 tiles (4 stages of 48 KiB) for products large enough to fill the machine with them: a quarter less
+// shared-memory traffic per flop than 128 x 128, which is what bounds the 128-wide tile.
+constexpr int kStagesWide = 4;
+constexpr int kTileBytes = kBM * kBK * 2;                 // 16 KiB: the A tile, and every 128 columns of the B tile
+__host__ __device__ constexpr int stage_bytes(int bn) { return kTileBytes + bn * kBK * 2; }
 constexpr int kTcThreads = 192;
-constexpr int kTmemCols = 128;
-constexpr size_t tc_smem_bytes(int stages) { return (size_t)stages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/; }
+constexpr size_t tc_smem_bytes(int stages, int bn) { return (size_t)stages * stage_bytes(bn) + 1024 /*alignment slack*/ + 256 /*barriers*/; }
 constexpr long long kWaitCycles = 400ll * 1000 * 1000;    // ~0.2 s: far beyond any legitimate wait
 constexpr long long kWaitCyclesAborted = 2ll * 1000 * 1000;
 
@@ -125,10 +127,12 @@ __device__ __forceinline__ uint32_t pack2(float a, float b) {
 }
 
 // ---------------------------------------------------------------------------------------- kernel
-template <int kStages>
+template <int kStages, int kBN>
 __global__ void __launch_bounds__(kTcThreads, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, TcParams p) {
   extern __shared__ uint8_t smem_raw[];
+  constexpr int kStageBytes = stage_bytes(kBN);
+  constexpr int kTmemCols = kBN;                           // one fp32 accumulator column per tile column
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t tiles = (raw + 1023u) & ~1023u;                 // 1024-byte aligned swizzle atoms
   uint8_t* gen = smem_raw + (tiles - raw);
@@ -179,8 +183,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           tma_load_2d(sa, &map_a, full(s), k0, m0);
         }
         if (p.b_mn) {
-          tma_load_2d(sb, &map_b, full(s), n0, k0);
-          tma_load_2d(sb + kTileBytes / 2, &map_b, full(s), n0 + 64, k0);
+#pragma unroll
+          for (int a = 0; a < kBN / 64; ++a) tma_load_2d(sb + a * (kTileBytes / 2), &map_b, full(s), n0 + 64 * a, k0);
         } else {
           tma_load_2d(sb, &map_b, full(s), k0, n0);
         }
@@ -345,10 +349,12 @@ ss_status gemm_tc(int M, int N, int K, const Operand& A, const Operand& B, const
   int dev = 0;
   SS_CUDA(cudaGetDevice(&dev));
   if (dev >= 0 && dev < 64 && !attr_set[dev]) {
-    SS_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<kStagesSmall>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)tc_smem_bytes(kStagesSmall)));
-    SS_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<kStagesLarge>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)tc_smem_bytes(kStagesLarge)));
+    SS_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<kStagesSmall, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)tc_smem_bytes(kStagesSmall, 128)));
+    SS_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<kStagesLarge, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)tc_smem_bytes(kStagesLarge, 128)));
+    SS_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<kStagesWide, 256>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)tc_smem_bytes(kStagesWide, 256)));
     attr_set[dev] = true;
   }
   TcParams p;
@@ -366,16 +372,22 @@ ss_status gemm_tc(int M, int N, int K, const Operand& A, const Operand& B, const
   if (!p.err) return SS_ERR_CUDA;
   alignas(64) CUtensorMap ma, mb;
   const bool oka = p.a_mn ? make_map(&ma, A.p, M, K, A.s_k, 64, 64) : make_map(&ma, A.p, K, M, A.s_row, 64, kBM);
-  const bool okb = p.b_mn ? make_map(&mb, B.p, N, K, B.s_k, 64, 64) : make_map(&mb, B.p, K, N, B.s_row, 64, kBN);
+  const int nk_all2 = (K + kBK - 1) / kBK;
+  const int nk_slice = (nk_all2 + k_splits - 1) / k_splits;
+  const long long ctas128 = (long long)((N + 127) / 128) * ((M + kBM - 1) / kBM) * k_splits;
+  const long long ctas256 = (long long)((N + 255) / 256) * ((M + kBM - 1) / kBM) * k_splits;
+  const bool wide = N >= 256 && ctas256 >= 2ll * num_sms() && nk_slice >= 2 * kStagesWide;
+  const int bn = wide ? 256 : 128;
+  const bool okb = p.b_mn ? make_map(&mb, B.p, N, K, B.s_k, 64, 64) : make_map(&mb, B.p, K, N, B.s_row, 64, bn);
   if (!oka || !okb) return SS_ERR_CUDA;
-  dim3 grid((N + kBN - 1) / kBN, (M + kBM - 1) / kBM, k_splits);
+  dim3 grid((N + bn - 1) / bn, (M + kBM - 1) / kBM, k_splits);
   { SS_TIMED("gemm_tc_kernel", st);
-  const long long ctas = (long long)grid.x * grid.y * grid.z;
-  const int nk_slice = (nk_all + k_splits - 1) / k_splits;
-  if (ctas >= 2ll * num_sms() && nk_slice >= 2 * kStagesLarge)
-    gemm_tc_kernel<kStagesLarge><<<grid, kTcThreads, tc_smem_bytes(kStagesLarge), st>>>(ma, mb, p);
+  if (wide)
+    gemm_tc_kernel<kStagesWide, 256><<<grid, kTcThreads, tc_smem_bytes(kStagesWide, 256), st>>>(ma, mb, p);
+  else if (ctas128 >= 2ll * num_sms() && nk_slice >= 2 * kStagesLarge)
+    gemm_tc_kernel<kStagesLarge, 128><<<grid, kTcThreads, tc_smem_bytes(kStagesLarge, 128), st>>>(ma, mb, p);
   else
-    gemm_tc_kernel<kStagesSmall><<<grid, kTcThreads, tc_smem_bytes(kStagesSmall), st>>>(ma, mb, p);
+    gemm_tc_kernel<kStagesSmall, 128><<<grid, kTcThreads, tc_smem_bytes(kStagesSmall, 128), st>>>(ma, mb, p);
   }
   SS_LAUNCH_OK();
   return SS_OK;

@@ -25,7 +25,9 @@ def _operand(rng, rows, k, mn_major, ld_pad):
 
 
 SHAPES = [(128, 128, 64), (256, 256, 320), (200, 72, 104), (328, 512, 1728), (512, 1728, 2048), (64, 64, 16),
-          (1000, 8, 24)]
+          (1000, 8, 24),
+          (2400, 4000, 520),     # enough tiles for the 128 x 256 variant: ragged last tile in M, N and K
+          (19 * 128, 2048, 1024)]  # enough 128 x 128 tiles for the deep (6-stage) ring
 
 
 @pytest.mark.parametrize("a_mn,b_mn", [(0, 0), (0, 1), (1, 0), (1, 1)])
