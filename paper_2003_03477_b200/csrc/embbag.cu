@@ -455,8 +455,50 @@ __device__ __forceinline__ bool ws_matches(const int32_t* scalars, int64_t L, ui
 // FUSE (rows of at most 128 floats): the sums of the complete runs stay in shared memory and the group applies
 // row-wise Adagrad to those rows itself, four rows' loads in flight, so their sums never travel through global
 // memory; only rows crossing window edges go through gsum and the kernels that follow.
+// Row-wise Adagrad on the nr rows a lane group has stashed in shared memory (sums in s_sum, keys in s_runkey),
+// the loads of four rows in flight at a time.  All lanes of the group call it together.
+template <int G>
+__device__ __forceinline__ void update_stashed_rows(int nr, const float4* __restrict__ s_sum, const uint32_t* __restrict__ s_runkey,
+                                                    int lane, int nvec, int D, unsigned gmask, float* __restrict__ tables,
+                                                    float* __restrict__ row_state, float lr, float eps) {
+  __syncwarp(gmask);
+  for (int r0 = 0; r0 < nr; r0 += 4) {
+    uint32_t rk[4];
+    float4 rw[4], g[4];
+    float st[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const bool ok = r0 + j < nr;
+      rk[j] = ok ? s_runkey[r0 + j] : 0u;
+      const float4* row = reinterpret_cast<const float4*>(tables + (int64_t)rk[j] * D);
+      rw[j] = (ok && lane < nvec) ? row[lane] : make_float4(0.f, 0.f, 0.f, 0.f);
+      g[j] = (ok && lane < nvec) ? s_sum[(size_t)(r0 + j) * nvec + lane] : make_float4(0.f, 0.f, 0.f, 0.f);
+      st[j] = ok ? row_state[rk[j]] : 0.f;
+    }
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      float ss = g[j].x * g[j].x + g[j].y * g[j].y + g[j].z * g[j].z + g[j].w * g[j].w;
+#pragma unroll
+      for (int off = G / 2; off >= 1; off >>= 1) ss += __shfl_down_sync(gmask, ss, off, G);
+      ss = __shfl_sync(gmask, ss, 0, G);                   // every lane uses lane 0's sum
+      if (r0 + j >= nr) continue;
+      const float sn = st[j] + ss / (float)D;
+      const float scale = lr / (sqrtf(sn) + eps);
+      if (lane < nvec) {
+        float4 o = rw[j];
+        o.x -= scale * g[j].x; o.y -= scale * g[j].y; o.z -= scale * g[j].z; o.w -= scale * g[j].w;
+        reinterpret_cast<float4*>(tables + (int64_t)rk[j] * D)[lane] = o;
+      }
+      if (lane == 0) row_state[rk[j]] = sn;
+    }
+  }
+  __syncwarp(gmask);
+}
+
+constexpr int kStash = kWin; // complete runs a group can keep in shared memory (a window holds at most kWin)
+
 template <int G, int NV, bool FUSE>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(256, FUSE ? 3 : 1)
 window_reduce_kernel(const uint32_t* __restrict__ keys, const int32_t* __restrict__ sbag,
                      const int32_t* __restrict__ uidx, int64_t L,
                      uint32_t sentinel, int64_t N, int D, int B, const float* __restrict__ grad, int64_t ld_grad,
@@ -464,8 +506,8 @@ window_reduce_kernel(const uint32_t* __restrict__ keys, const int32_t* __restric
                      int32_t* __restrict__ scalars, int nwin, int64_t umax, int32_t* __restrict__ d_status,
                      float* __restrict__ tables, float* __restrict__ row_state, float lr, float eps) {
   constexpr int kGroups = 256 / G;
-  extern __shared__ float4 s_sum[];                        // FUSE: [kGroups][kWin][D/4] sums of complete runs
-  __shared__ uint32_t s_runkey[FUSE ? kGroups : 1][kWin];
+  extern __shared__ float4 s_sum[];                        // FUSE: [kGroups][kStash][D/4] sums of complete runs
+  __shared__ uint32_t s_runkey[FUSE ? kGroups : 1][kStash];
   int nr = 0;
   __shared__ uint32_t s_key[kGroups][kWin + 2];            // [0] = key before the window, [kWin+1] = key after
   __shared__ int32_t s_row[kGroups][kWin];                 // float4 index of the lookup's gradient row
@@ -478,29 +520,26 @@ window_reduce_kernel(const uint32_t* __restrict__ keys, const int32_t* __restric
   const int64_t w0 = win * kWin;
   const int nvec = D >> 2;
   const int64_t ld4 = ld_grad >> 2;
+  // keys (one before and one after the window included), bag and segment of every position: one round of loads
   for (int i = lane; i < kWin + 2; i += G) {
     const int64_t j = w0 - 1 + i;
-    s_key[grp][i] = (j >= 0 && j < L) ? keys[j] : sentinel;
-  }
-  __syncwarp(gmask);
-  for (int i = lane; i < kWin; i += G) {
-    const int64_t j = w0 + i;
-    int32_t row = -1, u = 0;
-    if (j < L) {
-      const uint32_t key = keys[j];
-      if (key < sentinel) {
-        const int t = (int)(key / (uint64_t)N);
-        const int b = sbag[j] - t * B;
-        u = uidx[j];
-        // a consistent workspace never fails these; an inconsistent one must not turn into a wild access
-        if (b >= 0 && b < B && u >= 0 && u < umax)
-          row = (int32_t)((int64_t)b * ld4 + (int64_t)t * nvec); // B * ld_grad / 4 < 2^31 is checked on the host
-        else
-          s_key[grp][1 + i] = sentinel;
-      }
+    const bool in_range = j >= 0 && j < L;
+    const bool body = i >= 1 && i <= kWin;
+    uint32_t key = in_range ? keys[j] : sentinel;
+    const int sb = (body && in_range) ? sbag[j] : 0;
+    const int u = (body && in_range) ? uidx[j] : 0;
+    int32_t row = -1;
+    if (body && key < sentinel) {
+      const int t = (int)(key / (uint64_t)N);
+      const int b = sb - t * B;
+      // a consistent workspace never fails these; an inconsistent one must not turn into a wild access
+      if (b >= 0 && b < B && u >= 0 && u < umax)
+        row = (int32_t)((int64_t)b * ld4 + (int64_t)t * nvec);   // B * ld_grad / 4 < 2^31 is checked on the host
+      else
+        key = sentinel;
     }
-    s_row[grp][i] = row;
-    s_u[grp][i] = u;
+    s_key[grp][i] = key;
+    if (body) { s_row[grp][i - 1] = row; s_u[grp][i - 1] = u; }
   }
   __syncwarp(gmask);
   const float4* grad4 = reinterpret_cast<const float4*>(grad + col0);  // col0 is a multiple of 4
@@ -534,7 +573,7 @@ window_reduce_kernel(const uint32_t* __restrict__ keys, const int32_t* __restric
         const bool tail_open = (next == key);              // only possible at the window's last position
         const bool complete = !head_open && !tail_open;
         if (FUSE && complete) {
-          if (lane < nvec) s_sum[((size_t)grp * kWin + nr) * nvec + lane] = acc[0];
+          if (lane < nvec) s_sum[((size_t)grp * kStash + nr) * nvec + lane] = acc[0];
           if (lane == 0) s_runkey[grp][nr] = key;
           ++nr;
           acc[0] = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -557,40 +596,8 @@ window_reduce_kernel(const uint32_t* __restrict__ keys, const int32_t* __restric
       }
     }
   }
-  if (FUSE) {
-    // row-wise Adagrad on the rows whose whole run lay in this window
-    __syncwarp(gmask);
-    for (int r0 = 0; r0 < nr; r0 += 4) {
-      uint32_t rk[4];
-      float4 rw[4], g[4];
-      float st[4];
-#pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        const bool ok = r0 + j < nr;
-        rk[j] = ok ? s_runkey[grp][r0 + j] : 0u;
-        const float4* row = reinterpret_cast<const float4*>(tables + (int64_t)rk[j] * D);
-        rw[j] = (ok && lane < nvec) ? row[lane] : make_float4(0.f, 0.f, 0.f, 0.f);
-        g[j] = (ok && lane < nvec) ? s_sum[((size_t)grp * kWin + r0 + j) * nvec + lane] : make_float4(0.f, 0.f, 0.f, 0.f);
-        st[j] = ok ? row_state[rk[j]] : 0.f;
-      }
-#pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        float ss = g[j].x * g[j].x + g[j].y * g[j].y + g[j].z * g[j].z + g[j].w * g[j].w;
-#pragma unroll
-        for (int off = G / 2; off >= 1; off >>= 1) ss += __shfl_down_sync(gmask, ss, off, G);
-        ss = __shfl_sync(gmask, ss, 0, G);                 // every lane uses lane 0's sum
-        if (r0 + j >= nr) continue;
-        const float sn = st[j] + ss / (float)D;
-        const float scale = lr / (sqrtf(sn) + eps);
-        if (lane < nvec) {
-          float4 o = rw[j];
-          o.x -= scale * g[j].x; o.y -= scale * g[j].y; o.z -= scale * g[j].z; o.w -= scale * g[j].w;
-          reinterpret_cast<float4*>(tables + (int64_t)rk[j] * D)[lane] = o;
-        }
-        if (lane == 0) row_state[rk[j]] = sn;
-      }
-    }
-  }
+  if (FUSE && nr > 0)
+    update_stashed_rows<G>(nr, s_sum + (size_t)grp * kStash * nvec, s_runkey[grp], lane, nvec, D, gmask, tables, row_state, lr, eps);
 }
 
 // ---- (5) rows whose run crosses window edges: add their window partials ---------------------------
@@ -774,13 +781,13 @@ static void launch_reduce(const BwdPlan& p, char* ws, const uint32_t* keys, cons
   cudaMemsetAsync(scalars + 1, 0, sizeof(int32_t), st);
   {
     SS_TIMED("window_reduce_kernel", st);
-    const size_t smem = kFuse ? (size_t)kGroups * kWin * D * 4 : 0;
+    const size_t smem = kFuse ? (size_t)kGroups * kStash * D * 4 : 0;
     if (kFuse) {
       static bool attr_set[64];
       int dev = 0;
       if (cudaGetDevice(&dev) == cudaSuccess && dev >= 0 && dev < 64 && !attr_set[dev]) {
         cudaFuncSetAttribute(window_reduce_kernel<G, NV, kFuse>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             65536);   // kGroups * kWin * (4G floats) * 4 bytes for every G
+                             65536);   // kGroups * kStash * (4G floats) * 4 bytes for every G
         attr_set[dev] = true;
       }
     }
