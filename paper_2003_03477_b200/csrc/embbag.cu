@@ -168,36 +168,42 @@ static BwdPlan make_plan(int T, int64_t N, int D, int64_t L) {
 
 // ---- (1) keys ---------------------------------------------------------------------------
 // One thread per bag: key = t*N + row for each of its lookups, and the bag id of each position.
+// Every position in [0, L) is written by somebody: a bag owns [lo, hi) with both ends clamped to
+// [0, L] (consecutive bags share an end, so the clamped ranges tile [clamp(off[0]), clamp(off[T*B])) even
+// when the offsets are not monotone), the first and the last bag also take what lies before and after.
+// Positions of a malformed bag, and lookups with a row index outside the table, get the sentinel key.
 __global__ void __launch_bounds__(256)
 build_keys_kernel(const int32_t* __restrict__ indices, const int32_t* __restrict__ offsets, int T, int64_t N,
                   int B, int64_t L, uint32_t* __restrict__ keys, int32_t* __restrict__ bag_of,
                   int32_t* __restrict__ d_status) {
   const int64_t bag = (int64_t)blockIdx.x * 256 + threadIdx.x;
-  if (bag >= (int64_t)T * B) return;
+  const int64_t nbags = (int64_t)T * B;
+  if (bag >= nbags) return;
   const uint32_t sentinel = (uint32_t)((uint64_t)T * (uint64_t)N);
   const int t = (int)(bag / B);
-  int lo = offsets[bag], hi = offsets[bag + 1];
-  int bad = 0;
-  if (lo < 0 || hi < lo || hi > L) {
-    // a malformed bag owns no positions; positions nobody owns keep the sentinel written by the fill
-    bad = SS_DEV_BAD_OFFSET;
-    hi = lo = 0;
-  }
-  for (int j = lo; j < hi; ++j) {
-    const int idx = indices[j];
+  const int lo = offsets[bag], hi = offsets[bag + 1];
+  const int64_t clo = lo < 0 ? 0 : (lo > L ? L : lo), chi = hi < 0 ? 0 : (hi > L ? L : hi);
+  const bool well_formed = (lo == clo) && (hi == chi) && (lo <= hi);
+  int bad = well_formed ? 0 : SS_DEV_BAD_OFFSET;
+  for (int64_t j = clo; j < chi; ++j) {
     uint32_t key = sentinel;
-    if (idx >= 0 && idx < N) key = (uint32_t)((uint64_t)t * (uint64_t)N + (uint64_t)idx);
-    else bad |= SS_DEV_BAD_INDEX;
+    if (well_formed) {
+      const int idx = indices[j];
+      if (idx >= 0 && idx < N) key = (uint32_t)((uint64_t)t * (uint64_t)N + (uint64_t)idx);
+      else bad |= SS_DEV_BAD_INDEX;
+    }
     keys[j] = key;
     bag_of[j] = (int32_t)bag;
   }
+  if (bag == 0) {
+    if (lo != 0) bad |= SS_DEV_BAD_OFFSET;
+    for (int64_t j = 0; j < clo; ++j) { keys[j] = sentinel; bag_of[j] = 0; }
+  }
+  if (bag == nbags - 1) {
+    if (hi != L) bad |= SS_DEV_BAD_OFFSET;
+    for (int64_t j = chi; j < L; ++j) { keys[j] = sentinel; bag_of[j] = 0; }
+  }
   if (bad && d_status) atomicOr(d_status, bad);
-}
-
-// keys <- sentinel, bag_of <- 0 for all positions (those no well-formed bag owns stay that way)
-__global__ void fill_keys_kernel(uint32_t* __restrict__ keys, int32_t* __restrict__ bag_of, int64_t n, uint32_t v) {
-  int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (i < n) { keys[i] = v; bag_of[i] = 0; }
 }
 
 // ---- (2) radix sort pass ----------------------------------------------------------------
@@ -265,8 +271,27 @@ bin_scan_kernel(uint32_t* __restrict__ hist, int bins, int nblk, uint32_t* __res
 }
 
 // Exclusive scan of m values in place by one block (m is a few thousand at most).
+// scalars[2..3] stamp the workspace with the problem it holds a finished sort of; the reduction kernels
+// refuse a workspace whose stamp does not match their arguments.
+__device__ __forceinline__ int32_t ws_stamp(uint32_t sentinel) { return (int32_t)(sentinel ^ 0x53484144u); }
+
+struct UniqueFinish {      // what the scan of the per-block head counts also writes when it closes the unique pass
+  int32_t* seg; int32_t* seg_out; int32_t* d_num_unique; int32_t* scalars;
+  int64_t L; uint32_t sentinel;
+};
+
+// U distinct keys: close the segment list when there is none, publish U, stamp the workspace.
+__device__ __forceinline__ void finish_unique(uint32_t U, const UniqueFinish& f) {
+  if (U == 0) { f.seg[0] = 0; if (f.seg_out) f.seg_out[0] = 0; }
+  if (f.d_num_unique) *f.d_num_unique = (int32_t)U;
+  f.scalars[0] = (int32_t)U;
+  f.scalars[1] = 0;                                        // rows whose run crosses a window edge (filled by the window kernel)
+  f.scalars[2] = (int32_t)f.L;
+  f.scalars[3] = ws_stamp(f.sentinel);
+}
+
 __global__ void __launch_bounds__(kScanThreads)
-scan_exclusive_kernel(uint32_t* __restrict__ data, int64_t m, uint32_t* __restrict__ total_out) {
+scan_exclusive_kernel(uint32_t* __restrict__ data, int64_t m, uint32_t* __restrict__ total_out, UniqueFinish fin) {
   __shared__ uint32_t part[kScanThreads];
   const int64_t chunk = (m + kScanThreads - 1) / kScanThreads;
   const int64_t lo = (int64_t)threadIdx.x * chunk;
@@ -288,6 +313,7 @@ scan_exclusive_kernel(uint32_t* __restrict__ data, int64_t m, uint32_t* __restri
     run += v;
   }
   if (total_out && threadIdx.x == kScanThreads - 1) *total_out = part[kScanThreads - 1];
+  if (fin.scalars && threadIdx.x == kScanThreads - 1) finish_unique(part[kScanThreads - 1], fin);
 }
 
 // Stable scatter: warp w of the block owns the contiguous items [w*512, (w+1)*512) of the tile and
@@ -424,10 +450,6 @@ unique_write_kernel(const uint32_t* __restrict__ keys, int64_t L, uint32_t senti
     if (seg_out) seg_out[u_end] = (int32_t)(i + 1);
   }
 }
-
-// scalars[2..3] stamp the workspace with the problem it holds a finished sort of; the reduction kernels
-// refuse a workspace whose stamp does not match their arguments.
-__device__ __forceinline__ int32_t ws_stamp(uint32_t sentinel) { return (int32_t)(sentinel ^ 0x53484144u); }
 
 __global__ void unique_finish_kernel(const uint32_t* __restrict__ total, int32_t* __restrict__ seg,
                                      int32_t* __restrict__ seg_out, int32_t* __restrict__ d_num_unique,
@@ -908,10 +930,7 @@ static ss_status bwd_impl(bool do_sort, bool do_apply, float* tables, float* row
   const int32_t* perm_sorted = (p.passes & 1) ? pos_b : pos_a;
   if (do_sort) {
 
-  // (1) keys; positions no bag owns (malformed offsets) keep the sentinel
-  { SS_TIMED("fill_keys_kernel", cs);
-  fill_keys_kernel<<<(unsigned)((L + 255) / 256), 256, 0, cs>>>(keys_a, bag_of, L, sentinel);
-  }
+  // (1) keys
   { SS_TIMED("build_keys_kernel", cs);
   build_keys_kernel<<<(unsigned)(((int64_t)T * B + 255) / 256), 256, 0, cs>>>(indices, offsets, T, N, B, L, keys_a,
                                                                                 bag_of, d_status);
@@ -946,14 +965,12 @@ static ss_status bwd_impl(bool do_sort, bool do_apply, float* tables, float* row
   unique_count_kernel<<<p.nblk_u, kScanThreads, 0, cs>>>(keys_sorted, L, sentinel, usum);
   }
   { SS_TIMED("scan_exclusive_kernel", cs);
-  scan_exclusive_kernel<<<1, kScanThreads, 0, cs>>>(usum, p.nblk_u, usum + p.nblk_u);
+  scan_exclusive_kernel<<<1, kScanThreads, 0, cs>>>(usum, p.nblk_u, usum + p.nblk_u,
+                                                    UniqueFinish{seg, seg_off, d_num_unique, scalars, L, sentinel});
   }
   { SS_TIMED("unique_write_kernel", cs);
   unique_write_kernel<<<p.nblk_u, kScanThreads, 0, cs>>>(keys_sorted, L, sentinel, usum, uniq, seg, uidx, uniq_keys, seg_off,
                                                          perm_sorted, bag_of, reinterpret_cast<int32_t*>(ws + p.off_sbag));
-  }
-  { SS_TIMED("unique_finish_kernel", cs);
-  unique_finish_kernel<<<1, 1, 0, cs>>>(usum + p.nblk_u, seg, seg_off, d_num_unique, scalars, L, sentinel);
   }
   SS_LAUNCH_OK();
 
@@ -1073,7 +1090,6 @@ ss_status ss_embbag_bwd_sort_noalloc(int T, int64_t N, const int32_t* indices, c
     SS_LAUNCH_OK();
     return SS_OK;
   }
-  fill_keys_kernel<<<(unsigned)((L + 255) / 256), 256, 0, cs>>>(keys_a, bag_of, L, sentinel);
   build_keys_kernel<<<(unsigned)(((int64_t)T * B + 255) / 256), 256, 0, cs>>>(indices, offsets, T, N, B, L, keys_a,
                                                                                 bag_of, d_status);
   SS_LAUNCH_OK();
@@ -1093,10 +1109,10 @@ ss_status ss_embbag_bwd_sort_noalloc(int T, int64_t N, const int32_t* indices, c
   }
   SS_CUDA(cudaMemcpyAsync(perm, pin, (size_t)L * 4, cudaMemcpyDeviceToDevice, cs));
   unique_count_kernel<<<nblk_u, kScanThreads, 0, cs>>>(kin, L, sentinel, usum);
-  scan_exclusive_kernel<<<1, kScanThreads, 0, cs>>>(usum, nblk_u, usum + nblk_u);
+  scan_exclusive_kernel<<<1, kScanThreads, 0, cs>>>(usum, nblk_u, usum + nblk_u,
+                                                    UniqueFinish{seg, seg_off, d_num_unique, scalars, L, sentinel});
   unique_write_kernel<<<nblk_u, kScanThreads, 0, cs>>>(kin, L, sentinel, usum, uniq, seg, uidx, uniq_keys, seg_off,
                                                        nullptr, nullptr, nullptr);
-  unique_finish_kernel<<<1, 1, 0, cs>>>(usum + nblk_u, seg, seg_off, d_num_unique, scalars, L, sentinel);
   SS_LAUNCH_OK();
   return SS_OK;
 }

@@ -134,18 +134,6 @@ batch_reduce_partial_kernel(const __grid_constant__ RedJobs jobs, int B, int row
   }
 }
 
-__global__ void __launch_bounds__(256)
-batch_reduce_final_kernel(const __grid_constant__ RedJobs jobs, int nsplit, const float* __restrict__ partial,
-                          float* __restrict__ g) {
-  const int i = blockIdx.x * 256 + threadIdx.x;
-  if (i >= jobs.total) return;
-  float t = 0.f;
-  for (int s = 0; s < nsplit; ++s) t += partial[(int64_t)s * jobs.total + i];
-  int j = 0;
-  while (j + 1 < jobs.njobs && i >= jobs.job[j + 1].part_off) ++j;
-  g[jobs.job[j].out_off + (i - jobs.job[j].part_off)] = t;
-}
-
 // logit[b] = sum_k X[b, k] * w[k] + bias: one warp per row, lanes stride k, fixed shuffle tree.
 __global__ void __launch_bounds__(256)
 rowdot_kernel(const void* __restrict__ X, int x_kind, int64_t ldx, const void* __restrict__ w, int w_kind, int K,
@@ -173,32 +161,52 @@ outer_mask_kernel(const void* __restrict__ dz, const void* __restrict__ w, const
   else reinterpret_cast<float*>(dX)[i] = v;
 }
 
-// Weight gradients that were computed in K slices: slice z of layer t lies at gpart[off + z*size ...].
-struct SplitTable {
+// Where the gradient of each parameter tensor is found when the update kernel runs.
+//   GRAD_FLAT    in the flat gradient vector itself (a GEMM wrote it there)
+//   GRAD_SLICES  nsplit K slices of a weight-gradient GEMM: src[off + z*stride + i]
+//   GRAD_BATCH   nsplit batch slices of the batched reduction (bias, skinny weights): src[off + z*stride + i]
+// Elements that belong to no tensor (pads of the layout) have gradient zero.
+enum { GRAD_FLAT = 0, GRAD_SLICES = 1, GRAD_BATCH = 2 };
+constexpr int kMaxGradRanges = 2 * kMaxLayers;
+struct GradTable {
   int n;
-  int64_t begin[kMaxLayers], end[kMaxLayers], off[kMaxLayers];
-  int nsplit[kMaxLayers];
+  int64_t begin[kMaxGradRanges], end[kMaxGradRanges], off[kMaxGradRanges], stride[kMaxGradRanges];
+  int kind[kMaxGradRanges], nsplit[kMaxGradRanges];
 };
 
-// Element-wise Adagrad over the flat parameter vector; refreshes the bf16 mirror.  The gradient of an
-// element is the flat vector's value, or the sum of its K slices in slice order.  A zero gradient
-// (pads, dead units) leaves the element untouched.  g_out (nullable, may alias g) receives the gradient.
+// Element-wise Adagrad over the flat parameter vector; refreshes the bf16 mirror.  The slices of a
+// gradient are added in slice order.  A zero gradient (pads, dead units) leaves the element
+// untouched.  g_out (nullable, may alias g) receives the assembled gradient.
 __global__ void __launch_bounds__(256)
 adagrad_kernel(float* __restrict__ w, float* __restrict__ acc, const float* g, const float* __restrict__ gpart,
-               const __grid_constant__ SplitTable tab, __nv_bfloat16* __restrict__ mirror, int64_t n4, float lr,
-               float eps, float* g_out, int apply) {
+               const float* __restrict__ bpart, const __grid_constant__ GradTable tab,
+               __nv_bfloat16* __restrict__ mirror, int64_t n4, float lr, float eps, float* g_out, int apply) {
   const int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x;
   if (i >= n4) return;
   const int64_t e = i * 4;
-  float4 gv = reinterpret_cast<const float4*>(g)[i];
+  float4 gv = make_float4(0.f, 0.f, 0.f, 0.f);
   for (int t = 0; t < tab.n; ++t) {
-    if (e >= tab.begin[t] && e < tab.end[t]) {
-      const int64_t size = tab.end[t] - tab.begin[t];
-      const float4* p = reinterpret_cast<const float4*>(gpart + tab.off[t] + (e - tab.begin[t]));
-      gv = p[0];
-      for (int z = 1; z < tab.nsplit[t]; ++z) {
-        const float4 q = p[(int64_t)z * (size >> 2)];
-        gv.x += q.x; gv.y += q.y; gv.z += q.z; gv.w += q.w;
+    if (e >= tab.begin[t] && e < tab.end[t]) {               // tensors start on multiples of 32: no float4 straddles a start
+      const int64_t rel = e - tab.begin[t];
+      if (tab.kind[t] == GRAD_FLAT) {
+        gv = reinterpret_cast<const float4*>(g)[i];
+      } else if (tab.kind[t] == GRAD_SLICES) {               // sizes are multiples of 8: aligned float4 loads
+        const float4* p = reinterpret_cast<const float4*>(gpart + tab.off[t] + rel);
+        gv = p[0];
+        for (int z = 1; z < tab.nsplit[t]; ++z) {
+          const float4 q = p[(int64_t)z * (tab.stride[t] >> 2)];
+          gv.x += q.x; gv.y += q.y; gv.z += q.z; gv.w += q.w;
+        }
+      } else {                                               // any size: scalar loads, elements past the end stay zero
+        const int64_t left = tab.end[t] - e;
+        const float* p = bpart + tab.off[t] + rel;
+        float v[4] = {0.f, 0.f, 0.f, 0.f};
+        for (int z = 0; z < tab.nsplit[t]; ++z) {
+          const float* q = p + (int64_t)z * tab.stride[t];
+#pragma unroll
+          for (int k = 0; k < 4; ++k) if (k < left) v[k] += q[k];
+        }
+        gv = make_float4(v[0], v[1], v[2], v[3]);
       }
       break;
     }
@@ -333,7 +341,6 @@ ss_status ss_mlp_bwd(const ss_mlp_desc* desc, float* w, void* w_bf16, float* ada
   char* ws = reinterpret_cast<char*>(workspace);
   const int act_kind = p.bf16 ? OP_BF16 : OP_F32;
   float* g = grads ? grads : reinterpret_cast<float*>(ws + p.grads);
-  SS_CUDA(cudaMemsetAsync(g, 0, (size_t)p.P * 4, cs));   // pads of the flat layout carry zero gradient
 
   const int last = p.nl - 1;
   const int dz_kind = p.bf16 ? OP_BF16 : OP_F32;
@@ -343,8 +350,13 @@ ss_status ss_mlp_bwd(const ss_mlp_desc* desc, float* w, void* w_bf16, float* ada
   SS_LAUNCH_OK();
 
   float* gpart = reinterpret_cast<float*>(ws + p.gpart);
-  SplitTable tab;
+  GradTable tab;
   tab.n = 0;
+  auto add_range = [&](int64_t begin, int64_t count, int kind, int64_t off, int64_t stride, int nsplit) {
+    const int t = tab.n++;
+    tab.begin[t] = begin; tab.end[t] = begin + count; tab.kind[t] = kind; tab.off[t] = off; tab.stride[t] = stride;
+    tab.nsplit[t] = nsplit;
+  };
   RedJobs jobs;
   jobs.njobs = 0; jobs.ntiles = 0; jobs.total = 0;
   auto add_job = [&](const void* M, int m_kind, int64_t ldm, int ncols, const void* S, int s_kind, int64_t lds,
@@ -381,10 +393,10 @@ ss_status ss_mlp_bwd(const ss_mlp_desc* desc, float* w, void* w_bf16, float* ada
         const int64_t size = (int64_t)L.in * L.out;
         ep.out_lo = gpart + p.gpart_off[l];
         st = gemm_tc(L.out, L.in, B, A, X, ep, cs, p.k_splits[l], size);
-        const int t = tab.n++;
-        tab.begin[t] = L.w_off; tab.end[t] = L.w_off + size; tab.off[t] = p.gpart_off[l]; tab.nsplit[t] = p.k_splits[l];
+        add_range(L.w_off, size, GRAD_SLICES, p.gpart_off[l], size, p.k_splits[l]);
       } else {
         st = gemm(L.out, L.in, B, A, X, ep, cs);
+        add_range(L.w_off, (int64_t)L.in * L.out, GRAD_FLAT, 0, 0, 1);
       }
       if (st != SS_OK) return st;
     }
@@ -418,23 +430,20 @@ ss_status ss_mlp_bwd(const ss_mlp_desc* desc, float* w, void* w_bf16, float* ada
     }
   }
   {
-    // all batch reductions of the pass in two launches
+    // all batch reductions of the pass in one launch; the update kernel adds the batch slices
     int rows = ((B + p.red_splits - 1) / p.red_splits + 7) & ~7;   // <= kRedRows by the choice of red_splits
     const int nsplit = (B + rows - 1) / rows;
     float* partial = reinterpret_cast<float*>(ws + p.red_partial);
     { SS_TIMED("batch_reduce_partial_kernel", cs);
     batch_reduce_partial_kernel<<<dim3(jobs.ntiles, nsplit), 256, 0, cs>>>(jobs, B, rows, partial);
     }
-    { SS_TIMED("batch_reduce_final_kernel", cs);
-    batch_reduce_final_kernel<<<(jobs.total + 255) / 256, 256, 0, cs>>>(jobs, nsplit, partial, g);
-    }
     SS_LAUNCH_OK();
-  }
-
-  if (apply_update || tab.n > 0) {
+    for (int j = 0; j < jobs.njobs; ++j)
+      add_range(jobs.job[j].out_off, (int64_t)jobs.job[j].ncols * jobs.job[j].s_cols, GRAD_BATCH, jobs.job[j].part_off,
+                jobs.total, nsplit);
     const int64_t n4 = p.P / 4;
     SS_TIMED("adagrad_kernel", cs);
-    adagrad_kernel<<<(unsigned)((n4 + 255) / 256), 256, 0, cs>>>(w, adagrad_acc, g, gpart, tab,
+    adagrad_kernel<<<(unsigned)((n4 + 255) / 256), 256, 0, cs>>>(w, adagrad_acc, g, gpart, partial, tab,
                                                                  reinterpret_cast<__nv_bfloat16*>(w_bf16), n4, lr, eps,
                                                                  (grads || !apply_update) ? g : nullptr, apply_update);
     SS_LAUNCH_OK();
