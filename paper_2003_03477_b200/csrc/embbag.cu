@@ -622,17 +622,44 @@ window_reduce_kernel(const uint32_t* __restrict__ keys, const int32_t* __restric
     update_stashed_rows<G>(nr, s_sum + (size_t)grp * kStash * nvec, s_runkey[grp], lane, nvec, D, gmask, tables, row_state, lr, eps);
 }
 
+// Row-wise Adagrad on one row whose gradient slice is in the lanes' registers (rows of at most 4G floats).
+template <int G>
+__device__ __forceinline__ void adagrad_one_row(float4 g, uint32_t key, int lane, int nvec, int D, unsigned gmask,
+                                                float* __restrict__ tables, float* __restrict__ row_state, float lr,
+                                                float eps) {
+  float4* row = reinterpret_cast<float4*>(tables + (int64_t)key * D);
+  const float4 r = lane < nvec ? row[lane] : make_float4(0.f, 0.f, 0.f, 0.f);
+  const float st = row_state[key];
+  float ss = g.x * g.x + g.y * g.y + g.z * g.z + g.w * g.w;
+#pragma unroll
+  for (int off = G / 2; off >= 1; off >>= 1) ss += __shfl_down_sync(gmask, ss, off, G);
+  ss = __shfl_sync(gmask, ss, 0, G);                       // every lane uses lane 0's sum
+  const float sn = st + ss / (float)D;
+  const float scale = lr / (sqrtf(sn) + eps);
+  if (lane < nvec) {
+    float4 o = r;
+    o.x -= scale * g.x; o.y -= scale * g.y; o.z -= scale * g.z; o.w -= scale * g.w;
+    row[lane] = o;
+  }
+  __syncwarp(gmask);
+  if (lane == 0) row_state[key] = sn;
+}
+
 // ---- (5) rows whose run crosses window edges: add their window partials ---------------------------
 // Rows spanning up to four windows: one lane group adds the partials in window order.  Longer rows: one
 // block per row, lane group j adds the partials of windows k0+j, k0+j+groups, ... in ascending order and
 // the group sums are then added in group order.  The association is fixed by the
 // segment's position alone (the order of the list does not matter).
-template <int G, int NV>
+// FUSE (rows of at most 128 floats): the combined sum is not stored; the row is updated here.
+template <int G, int NV, bool FUSE>
 __global__ void __launch_bounds__(256)
 combine_rows_kernel(const int32_t* __restrict__ seg, const int32_t* __restrict__ scalars,
                     const int32_t* __restrict__ long_list, int nwin, int D, const float* __restrict__ partial,
-                    float* __restrict__ gsum, int64_t L, uint32_t sentinel, int64_t umax) {
+                    float* __restrict__ gsum, int64_t L, uint32_t sentinel, int64_t umax,
+                    const int32_t* __restrict__ uniq, float* __restrict__ tables, float* __restrict__ row_state,
+                    float lr, float eps) {
   constexpr int kGroups = 256 / G;
+  const unsigned gmask = (G == 32) ? 0xffffffffu : (((1u << G) - 1u) << ((threadIdx.x & 31) / G * G));
   extern __shared__ float4 s_part[];                       // [kGroups][D/4]
   const int grp = threadIdx.x / G, lane = threadIdx.x % G;
   const int nvec = D >> 2;
@@ -660,13 +687,19 @@ combine_rows_kernel(const int32_t* __restrict__ seg, const int32_t* __restrict__
       }
     }
     float4* dst = reinterpret_cast<float4*>(gsum + (int64_t)u * D);
+    float4 t0 = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
     for (int v = 0; v < NV; ++v) {
       const int c = lane + v * G;
       float4 t = pv[0][v];
 #pragma unroll
       for (int j = 1; j < kShort; ++j) t = add4(t, pv[j][v]);   // adding zeros for absent windows changes nothing
-      if (c < nvec) dst[c] = t;
+      if (!FUSE && c < nvec) dst[c] = t;
+      if (v == 0) t0 = t;
+    }
+    if (FUSE) {
+      const uint32_t key = (uint32_t)uniq[u];
+      if (key < sentinel) adagrad_one_row<G>(t0, key, lane, nvec, D, gmask, tables, row_state, lr, eps);
     }
   }
   // phase B: long spans, the whole block per row
@@ -698,14 +731,20 @@ combine_rows_kernel(const int32_t* __restrict__ seg, const int32_t* __restrict__
     if (grp == 0) {
       const int used = min(kGroups, k1 - k0 + 1);
       float4* dst = reinterpret_cast<float4*>(gsum + (int64_t)u * D);
+      float4 t0 = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
       for (int v = 0; v < NV; ++v) {
         const int c = lane + v * G;
         if (c < nvec) {
           float4 t = s_part[c];
           for (int j = 1; j < used; ++j) t = add4(t, s_part[j * nvec + c]);
-          dst[c] = t;
+          if (!FUSE) dst[c] = t;
+          if (v == 0) t0 = t;
         }
+      }
+      if (FUSE) {
+        const uint32_t key = (uint32_t)uniq[u];
+        if (key < sentinel) adagrad_one_row<G>(t0, key, lane, nvec, D, gmask, tables, row_state, lr, eps);
       }
     }
     __syncthreads();
@@ -821,17 +860,16 @@ static void launch_reduce(const BwdPlan& p, char* ws, const uint32_t* keys, cons
   {
     SS_TIMED("combine_rows_kernel", st);
     const int cblocks = p.nwin < num_sms() * 8 ? p.nwin : num_sms() * 8;
-    combine_rows_kernel<G, NV><<<cblocks, 256, (size_t)kGroups * D * 4, st>>>(seg, scalars, long_list, p.nwin, D, partial, gsum,
-                                                                              p.L, sentinel, (int64_t)umax);
+    combine_rows_kernel<G, NV, kFuse><<<cblocks, 256, (size_t)kGroups * D * 4, st>>>(
+        seg, scalars, long_list, p.nwin, D, partial, gsum, p.L, sentinel, (int64_t)umax, uniq, tables, row_state, lr, eps);
   }
-  // row update: every distinct row, or with the fused window kernel only the rows that crossed window edges
-  const uint64_t per_block = (uint64_t)kGroups * RowsPerGroup<NV>::value;
-  const uint64_t nrows = kFuse ? (uint64_t)p.nwin : umax;
-  const unsigned ublocks = (unsigned)((nrows + per_block - 1) / per_block);
-  {
+  if (!kFuse) {
+    // rows wider than 128 floats: every distinct row is updated from its sum in gsum
+    const uint64_t per_block = (uint64_t)kGroups * RowsPerGroup<NV>::value;
+    const unsigned ublocks = (unsigned)((umax + per_block - 1) / per_block);
     SS_TIMED("apply_rows_kernel", st);
     apply_rows_kernel<G, NV><<<ublocks, 256, 0, st>>>(uniq, scalars, D, gsum, tables, row_state, lr, eps, p.L, sentinel,
-                                                      (int64_t)umax, kFuse ? long_list : nullptr, p.nwin);
+                                                      (int64_t)umax, nullptr, 0);
   }
 }
 
