@@ -262,6 +262,12 @@ def bench_gpu(args):
     out["kernels"] = kernels
     out["gpu_launches"] = int(round(per_step * cfg.R * K)) + int(rounds)
     out["roofline"] = roofline(kernels, model, host, cfg, peaks)
+    # the same kernel with one replica training alone (no other replica's kernels competing for the SMs)
+    k1, _ = profile_pass(model, dev, cfg, replicas=[0])
+    alone = roofline({out["roofline"]["kernel"]: k1[out["roofline"]["kernel"]]}, model, host, cfg, peaks) \
+        if out["roofline"]["kernel"] in k1 else None
+    if alone:
+        out["roofline"]["one_replica_alone"] = {k: alone[k] for k in ("achieved", "frac", "us_per_launch")}
 
     # the sync kernel alone on vectors far larger than L2 (HBM-bound) -- the "sync HBM GB/s vs peak" half of the metric
     s = model.replicas[0].stream
@@ -323,19 +329,20 @@ def gemm_alone(stream, peaks):
     return res
 
 
-def profile_pass(model, dev, cfg, steps=6):
+def profile_pass(model, dev, cfg, steps=6, replicas=None):
     """Per-kernel device times from the library's event timers over a short region in which all replicas
     train concurrently (plain launches: timing events cannot be read back from a captured graph).
     Returns ({kernel: {launches_per_replica_step, us_per_launch, share}}, launches per replica step)."""
     import torch
     from paper_2003_03477_b200 import binding as ss
+    reps = list(range(cfg.R)) if replicas is None else list(replicas)
     for t in range(2):
-        for r in range(cfg.R):
+        for r in reps:
             model.step(r, dev[r][t % RING])
     torch.cuda.synchronize()
     ss.ss_profile(True)
     for t in range(steps):
-        for r in range(cfg.R):
+        for r in reps:
             model.step(r, dev[r][t % RING])
     recs = ss.ss_profile_collect()
     ss.ss_profile(False)
@@ -345,7 +352,7 @@ def profile_pass(model, dev, cfg, steps=6):
         a[0] += 1
         a[1] += ms * 1e3
     total = sum(a[1] for a in agg.values()) or 1.0
-    n_rs = steps * cfg.R
+    n_rs = steps * len(reps)
     table = {k: {"launches_per_replica_step": c / n_rs, "us_per_launch": t / c, "share": t / total}
              for k, (c, t) in sorted(agg.items(), key=lambda kv: -kv[1][1])}
     return table, len(recs) / n_rs
