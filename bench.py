@@ -232,6 +232,28 @@ def bench_gpu(args):
     barrier()
     loop.stop()
     torch.cuda.synchronize()
+    # ---- foreground variant (the paper's FR-* baselines): the sync pass inside the training loop every k steps
+    ms_fg = None
+    if args.foreground > 0:
+        def fg_region(n_steps):
+            for t0 in range(0, n_steps, args.foreground):
+                run_steps(model, graphs, W + t0, min(args.foreground, n_steps - t0))
+                model.foreground_sync(**sync_args(cfg))
+        fg_region(W)
+        barrier()
+        main = torch.cuda.current_stream()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(main)
+        for rep in model.replicas:
+            rep.stream.wait_event(e0)
+        fg_region(K)
+        for rep in model.replicas:
+            e = torch.cuda.Event()
+            e.record(rep.stream)
+            main.wait_event(e)
+        e1.record(main)
+        e1.synchronize()
+        ms_fg = e0.elapsed_time(e1)
     (ms_on, ms_off), examples = reduce_over_ranks([ms_on, ms_off], cfg.R * cfg.B * K, device)
     value = examples / (ms_on * 1e-3)
     value_off = examples / (ms_off * 1e-3)
@@ -258,6 +280,9 @@ def bench_gpu(args):
     out["sync"] = {"rounds_per_s": rounds / (ms_on * 1e-3), "avg_sync_gap_steps": (K / rounds) if rounds else None,
                    "examples_per_s_sync_off": value_off, "throughput_loss_pct": 100.0 * (1.0 - value / value_off)}
 
+    if ms_fg is not None:
+        out["sync"]["foreground"] = {"every_k_steps": args.foreground, "examples_per_s": cfg.R * cfg.B * K / (ms_fg * 1e-3),
+                                     "note": "same kernels enqueued on the training streams (FR-* of the paper)"}
     kernels, per_step = profile_pass(model, dev, cfg)
     out["kernels"] = kernels
     out["gpu_launches"] = int(round(per_step * cfg.R * K)) + int(rounds)
@@ -561,6 +586,8 @@ def main():
     ap.add_argument("--cpu-budget", type=float, default=15.0)
     ap.add_argument("--replicas", type=int, default=0, help="override the workload's replica count (experiments)")
     ap.add_argument("--quick", action="store_true", help="skip the e2e and CPU-baseline legs (experiments)")
+    ap.add_argument("--foreground", type=int, default=0,
+                    help="also time the foreground variant: one sync pass on the training streams every k steps")
     ap.add_argument("--sweep", action="store_true", help="isolated sync-kernel sweep instead of the training benchmark")
     args = ap.parse_args()
     if args.sweep:

@@ -194,6 +194,18 @@ ss_status ss_mlp_bwd(const ss_mlp_desc* desc, float* w, void* w_bf16, float* ada
                      void* workspace, size_t workspace_bytes, ss_stream stream);
 
 /* ------------------------------------------------------------------------------------------
+ * Normalised entropy (Section 4, "Evaluation Metrics"): the mean cross-entropy of the predictions divided
+ * by the entropy of the empirical click rate.  ss_ne_accumulate adds one batch to acc (device double[3]:
+ * sum of cross-entropies computed from the logits, sum of labels, count; the caller zeroes it before the
+ * first batch); ss_ne_value writes NE of everything accumulated so far to out (device double[1]).
+ * Fed with the logits ss_mlp_fwd returns -- predictions made before the step's update -- it gives the
+ * paper's Train NE; fed with logits of held-out batches, its Eval NE.  Calls on one acc must be ordered
+ * (same stream): the accumulation is a plain read-modify-write.
+ * ---------------------------------------------------------------------------------------- */
+ss_status ss_ne_accumulate(const float* logit, const float* labels, int B, double* acc, ss_stream stream);
+ss_status ss_ne_value(const double* acc, double* out, ss_stream stream);
+
+/* ------------------------------------------------------------------------------------------
  * Background synchronisation of the replicated dense parameters (Algorithms 2, 3, 4).  Each call
  * is ONE kernel that reads all R replica vectors and the centre/global copy once and writes them
  * back.  w: HOST array of R device pointers to float[n]; w_bf16: NULL or HOST array of R device
@@ -202,7 +214,8 @@ ss_status ss_mlp_bwd(const ss_mlp_desc* desc, float* w, void* w_bf16, float* ada
  * as the paper's shadow thread does with its worker threads (Section 3.2).
  * ---------------------------------------------------------------------------------------- */
 enum {
-  SS_SYNC_EASGD_LITERAL = 1  /* Algorithm 2 line by line: the replica interpolates toward the updated centre */
+  SS_SYNC_EASGD_LITERAL = 1, /* Algorithm 2 line by line: the replica interpolates toward the updated centre */
+  SS_SYNC_BMUF_NESTEROV = 2  /* Algorithm 4 with the Nesterov variant its comment allows: pull toward g + mu*delta */
 };
 
 /* Shadow EASGD (Algorithm 2), the R trainers visiting the centre in turn, r = 0..R-1:
@@ -215,7 +228,8 @@ ss_status ss_sync_ma(float* const* w, int R, float* global_out, int64_t n, float
                      void* const* w_bf16, ss_stream stream);
 
 /* Shadow BMUF (Algorithm 4) with block momentum: m = mean_r w_r;  delta = mu*delta + eta*(m - g);
- *   g += delta;  w_r = (1-alpha) w_r + alpha g.   mu = 0 is the algorithm as printed. */
+ *   g += delta;  w_r = (1-alpha) w_r + alpha g.   mu = 0 is the algorithm as printed.
+ * flags & SS_SYNC_BMUF_NESTEROV: the replicas are pulled toward the look-ahead point g + mu*delta instead of g. */
 ss_status ss_sync_bmuf(float* const* w, int R, float* global, float* delta, int64_t n,
                        float alpha, float eta, float mu, int flags,
                        void* const* w_bf16, ss_stream stream);

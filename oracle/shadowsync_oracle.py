@@ -230,19 +230,22 @@ def sync_ma(ws, alpha, global_out=None):
         w[...] = ((1.0 - alpha) * w.astype(F64) + alpha * m).astype(F32)
 
 
-def sync_bmuf(ws, g, delta, alpha, eta, mu=0.0):
+def sync_bmuf(ws, g, delta, alpha, eta, mu=0.0, nesterov=False):
     """Shadow BMUF (Algorithm 4) with classical block momentum, in place.
 
     m = mean_r w_r;  desc = m - g;  delta <- mu*delta + eta*desc;  g <- g + delta;
     w_r <- (1-alpha) w_r + alpha g.   mu = 0 is Algorithm 4 as printed.
+    nesterov=True (the acceleration Algorithm 4's comment mentions): the replicas interpolate toward
+    the look-ahead point g + mu*delta instead of g.
     """
     m = np.mean(np.stack([w.astype(F64) for w in ws]), axis=0)
     d = mu * delta.astype(F64) + eta * (m - g.astype(F64))
     delta[...] = d.astype(F32)
     g_new = (g.astype(F64) + delta.astype(F64)).astype(F32)
     g[...] = g_new
+    target = g_new.astype(F64) + (mu * delta.astype(F64) if nesterov else 0.0)
     for w in ws:
-        w[...] = ((1.0 - alpha) * w.astype(F64) + alpha * g_new.astype(F64)).astype(F32)
+        w[...] = ((1.0 - alpha) * w.astype(F64) + alpha * target).astype(F32)
 
 
 # --------------------------------------------------------------------------------------

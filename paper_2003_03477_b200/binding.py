@@ -21,10 +21,11 @@ STATUS_NAMES = {0: "SS_OK", -1: "SS_ERR_NULL", -2: "SS_ERR_SHAPE", -3: "SS_ERR_A
                 -5: "SS_ERR_WORKSPACE", -6: "SS_ERR_ARCH", -7: "SS_ERR_CUDA", -8: "SS_ERR_RANGE"}
 SS_DEV_BAD_INDEX, SS_DEV_BAD_OFFSET, SS_DEV_BAD_WORKSPACE = 1, 2, 4
 SS_SYNC_EASGD_LITERAL = 1
+SS_SYNC_BMUF_NESTEROV = 2
 
 EXPORTS = ["ss_status_str", "ss_last_cuda_error", "ss_num_sms", "ss_embbag_fwd", "ss_embbag_bwd_workspace_bytes",
            "ss_embbag_bwd_adagrad", "ss_embbag_bwd_sort", "ss_embbag_bwd_apply", "ss_embbag_bwd_sort_noalloc", "ss_mlp_param_count", "ss_mlp_param_offsets", "ss_mlp_workspace_bytes",
-           "ss_mlp_fwd", "ss_mlp_bwd", "ss_sync_easgd", "ss_sync_ma", "ss_sync_bmuf", "ss_shadow_start", "ss_shadow_rounds", "ss_shadow_stop", "ss_to_bf16",
+           "ss_mlp_fwd", "ss_mlp_bwd", "ss_ne_accumulate", "ss_ne_value", "ss_sync_easgd", "ss_sync_ma", "ss_sync_bmuf", "ss_shadow_start", "ss_shadow_rounds", "ss_shadow_stop", "ss_to_bf16",
            "ss_gemm_bf16", "ss_device_error", "ssh_fill_uniform", "ss_profile", "ss_profile_collect"]
 
 
@@ -75,6 +76,8 @@ def lib() -> C.CDLL:
         L.ss_mlp_fwd.argtypes = [C.POINTER(MlpDesc), vp, vp, vp, vp, vp, i32, vp, vp, vp, vp, vp, sz, vp]
         L.ss_mlp_bwd.argtypes = [C.POINTER(MlpDesc), vp, vp, vp, vp, vp, vp, vp, vp, vp, i32, f32, f32, i32,
                                  vp, i64, vp, sz, vp]
+        L.ss_ne_accumulate.argtypes = [vp, vp, i32, vp, vp]
+        L.ss_ne_value.argtypes = [vp, vp, vp]
         L.ss_sync_easgd.argtypes = [C.POINTER(vp), i32, vp, i64, f32, i32, C.POINTER(vp), vp]
         L.ss_sync_ma.argtypes = [C.POINTER(vp), i32, vp, i64, f32, i32, C.POINTER(vp), vp]
         L.ss_sync_bmuf.argtypes = [C.POINTER(vp), i32, vp, vp, i64, f32, f32, f32, i32, C.POINTER(vp), vp]
@@ -228,6 +231,14 @@ def ss_mlp_bwd(spec: MlpSpec, w, w_bf16, adagrad_acc, grads, dense, concat_f32, 
                                            _ptr(dense), _ptr(concat_f32), _ptr(concat_bf16), _ptr(labels), _ptr(prob),
                                            B, lr, eps, int(apply_update), _ptr(grad_pooled), ld_grad, _ptr(workspace),
                                            workspace.numel() * workspace.element_size(), _stream(stream)))
+
+
+def ss_ne_accumulate(logit, labels, B, acc, stream=None) -> None:
+    _check("ss_ne_accumulate", lib().ss_ne_accumulate(_ptr(logit), _ptr(labels), B, _ptr(acc), _stream(stream)))
+
+
+def ss_ne_value(acc, out, stream=None) -> None:
+    _check("ss_ne_value", lib().ss_ne_value(_ptr(acc), _ptr(out), _stream(stream)))
 
 
 def ss_sync_easgd(w: Sequence[torch.Tensor], center, n, alpha, flags=0, w_bf16=None, stream=None) -> None:

@@ -451,4 +451,62 @@ ss_status ss_mlp_bwd(const ss_mlp_desc* desc, float* w, void* w_bf16, float* ada
   return SS_OK;
 }
 
+// ---- normalised entropy (Section 4, "Evaluation Metrics") --------------------------------------
+}  // extern "C"
+
+namespace ss {
+// acc[0] += sum_b cross-entropy(z_b, y_b), acc[1] += sum_b y_b, acc[2] += B; one block, fixed tree, double.
+__global__ void __launch_bounds__(1024)
+ne_accumulate_kernel(const float* __restrict__ logit, const float* __restrict__ labels, int B, double* __restrict__ acc) {
+  __shared__ double red[2][1024];
+  double ce = 0.0, pos = 0.0;
+  for (int b = threadIdx.x; b < B; b += 1024) {
+    const double z = logit[b], y = labels[b];
+    ce += fmax(z, 0.0) - z * y + log1p(exp(-fabs(z)));
+    pos += y;
+  }
+  red[0][threadIdx.x] = ce;
+  red[1][threadIdx.x] = pos;
+  __syncthreads();
+  for (int off = 512; off >= 1; off >>= 1) {
+    if (threadIdx.x < off) {
+      red[0][threadIdx.x] += red[0][threadIdx.x + off];
+      red[1][threadIdx.x] += red[1][threadIdx.x + off];
+    }
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) { acc[0] += red[0][0]; acc[1] += red[1][0]; acc[2] += (double)B; }
+}
+
+// NE = (mean cross-entropy) / (entropy of the empirical click rate p = acc[1]/acc[2])
+__global__ void ne_value_kernel(const double* __restrict__ acc, double* __restrict__ out) {
+  const double n = acc[2], p = acc[1] / n;
+  out[0] = (acc[0] / n) / -(p * log(p) + (1.0 - p) * log(1.0 - p));
+}
+}  // namespace ss
+
+extern "C" {
+
+ss_status ss_ne_accumulate(const float* logit, const float* labels, int B, double* acc, ss_stream stream) {
+  if (!logit || !labels || !acc) return SS_ERR_NULL;
+  if (B < 1) return SS_ERR_SHAPE;
+  if (reinterpret_cast<uintptr_t>(acc) & 7u) return SS_ERR_ALIGN;
+  ss_status st = ss::check_arch();
+  if (st != SS_OK) return st;
+  SS_TIMED("ne_accumulate_kernel", ss::as_stream(stream));
+  ss::ne_accumulate_kernel<<<1, 1024, 0, ss::as_stream(stream)>>>(logit, labels, B, acc);
+  SS_LAUNCH_OK();
+  return SS_OK;
+}
+
+ss_status ss_ne_value(const double* acc, double* out, ss_stream stream) {
+  if (!acc || !out) return SS_ERR_NULL;
+  if ((reinterpret_cast<uintptr_t>(acc) | reinterpret_cast<uintptr_t>(out)) & 7u) return SS_ERR_ALIGN;
+  ss_status st = ss::check_arch();
+  if (st != SS_OK) return st;
+  ss::ne_value_kernel<<<1, 1, 0, ss::as_stream(stream)>>>(acc, out);
+  SS_LAUNCH_OK();
+  return SS_OK;
+}
+
 }  // extern "C"

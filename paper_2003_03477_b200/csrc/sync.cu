@@ -26,7 +26,9 @@ __device__ __forceinline__ uint2 pack_bf16x4(float4 v) {
   return r;
 }
 
-enum { RULE_EASGD = 0, RULE_EASGD_LITERAL = 1, RULE_MA = 2, RULE_BMUF = 3 };
+enum { RULE_EASGD = 0, RULE_EASGD_LITERAL = 1, RULE_MA = 2, RULE_BMUF = 3, RULE_BMUF_NESTEROV = 4 };
+
+template <int RULE> struct IsBmuf { static constexpr bool value = (RULE == 3 || RULE == 4); };
 
 struct SyncScalars {
   float alpha, eta, mu, inv_r;
@@ -59,8 +61,10 @@ __device__ __forceinline__ void apply_rule(float (&w)[R], float& c, float& dl, c
       dl = s.mu * dl + s.eta * (m - c);
       c = c + dl;
     }
+    // Nesterov look-ahead: the replicas are pulled toward where the global model is heading
+    const float target = (RULE == RULE_BMUF_NESTEROV) ? c + s.mu * dl : c;
 #pragma unroll
-    for (int r = 0; r < R; ++r) w[r] = w[r] + s.alpha * (c - w[r]);
+    for (int r = 0; r < R; ++r) w[r] = w[r] + s.alpha * (target - w[r]);
   }
 }
 
@@ -75,7 +79,7 @@ sync_kernel(SyncPtrs p, float* __restrict__ c, float* __restrict__ delta, int64_
     for (int r = 0; r < R; ++r) wv[r] = reinterpret_cast<const float4*>(p.w[r])[i];
     float4 cv = make_float4(0.f, 0.f, 0.f, 0.f), dv = cv;
     if (kReadC) cv = reinterpret_cast<const float4*>(c)[i];
-    if (RULE == RULE_BMUF) dv = reinterpret_cast<const float4*>(delta)[i];
+    if (IsBmuf<RULE>::value) dv = reinterpret_cast<const float4*>(delta)[i];
 
     float a[R];
 #define SS_LANE(F)                                         \
@@ -93,7 +97,7 @@ sync_kernel(SyncPtrs p, float* __restrict__ c, float* __restrict__ delta, int64_
       if (MIRROR) reinterpret_cast<uint2*>(p.m[r])[i] = pack_bf16x4(wv[r]);
     }
     if (c != nullptr) reinterpret_cast<float4*>(c)[i] = cv;
-    if (RULE == RULE_BMUF) reinterpret_cast<float4*>(delta)[i] = dv;
+    if (IsBmuf<RULE>::value) reinterpret_cast<float4*>(delta)[i] = dv;
   }
   // ragged tail (n not a multiple of 4): the first threads of block 0 take one scalar each
   if (blockIdx.x == 0 && threadIdx.x < (int)(n - n4 * 4)) {
@@ -101,7 +105,7 @@ sync_kernel(SyncPtrs p, float* __restrict__ c, float* __restrict__ delta, int64_
     float a[R];
 #pragma unroll
     for (int r = 0; r < R; ++r) a[r] = p.w[r][k];
-    float cs = (kReadC ? c[k] : 0.f), ds = (RULE == RULE_BMUF ? delta[k] : 0.f);
+    float cs = (kReadC ? c[k] : 0.f), ds = (IsBmuf<RULE>::value ? delta[k] : 0.f);
     apply_rule<RULE, R>(a, cs, ds, s);
 #pragma unroll
     for (int r = 0; r < R; ++r) {
@@ -109,7 +113,7 @@ sync_kernel(SyncPtrs p, float* __restrict__ c, float* __restrict__ delta, int64_
       if (MIRROR) p.m[r][k] = __float2bfloat16_rn(a[r]);
     }
     if (c != nullptr) c[k] = cs;
-    if (RULE == RULE_BMUF) delta[k] = ds;
+    if (IsBmuf<RULE>::value) delta[k] = ds;
   }
 }
 
@@ -194,7 +198,6 @@ ss_status ss_sync_ma(float* const* w, int R, float* global_out, int64_t n, float
 
 ss_status ss_sync_bmuf(float* const* w, int R, float* global, float* delta, int64_t n,
                        float alpha, float eta, float mu, int flags, void* const* w_bf16, ss_stream stream) {
-  (void)flags;
   ss::SyncPtrs p;
   if (!global || !delta) return SS_ERR_NULL;
   ss_status st = ss::collect(w, R, n, w_bf16, alpha, &p);
@@ -203,6 +206,8 @@ ss_status ss_sync_bmuf(float* const* w, int R, float* global, float* delta, int6
   if (!(mu >= 0.f && mu < 1.f) || !(eta >= 0.f)) return SS_ERR_RANGE;
   if (n == 0) return SS_OK;
   ss::SyncScalars s{alpha, eta, mu, 1.f / (float)R};
+  if (flags & SS_SYNC_BMUF_NESTEROV)
+    return ss::launch<ss::RULE_BMUF_NESTEROV>(R, p, w_bf16 != nullptr, global, delta, n, s, ss::as_stream(stream));
   return ss::launch<ss::RULE_BMUF>(R, p, w_bf16 != nullptr, global, delta, n, s, ss::as_stream(stream));
 }
 

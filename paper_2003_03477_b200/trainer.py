@@ -139,6 +139,31 @@ class Model:
         else:
             raise ValueError(rule)
 
+    def foreground_sync(self, rule: str, alpha: float, eta: float = 1.0, mu: float = 0.0, flags: int = 0) -> None:
+        """The foreground variants the paper compares against (FR-EASGD, FR-MA, FR-BMUF; Section 4): the
+        same kernels, but enqueued on the training streams, so training waits for them.
+
+        EASGD is centralised: every replica interpolates with the centre on its own, on its own stream, as
+        a worker would with the sync PS (replicas' passes may interleave; the centre is shared lock-free).
+        MA and BMUF need all replicas: every training stream joins, one pass runs, every stream waits for it.
+        """
+        n = self.spec.param_count
+        if rule == "easgd":
+            for rep in self.replicas:
+                ss.ss_sync_easgd([rep.w], self.center, n, alpha, flags, [rep.w_bf16] if self.spec.bf16 else None,
+                                 rep.stream)
+            return
+        lead = self.replicas[0].stream
+        for rep in self.replicas[1:]:
+            e = torch.cuda.Event()
+            e.record(rep.stream)
+            lead.wait_event(e)
+        self.sync(rule, alpha, eta, mu, stream=lead, flags=flags)
+        done = torch.cuda.Event()
+        done.record(lead)
+        for rep in self.replicas[1:]:
+            rep.stream.wait_event(done)
+
     def status(self) -> int:
         return int(self.d_status.item())
 

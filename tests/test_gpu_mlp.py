@@ -136,3 +136,30 @@ def test_mlp_rejects_bad_arguments():
     with pytest.raises(ss.SsError) as e:
         ss.ss_mlp_fwd(spec_h, w, None, dense, concat, None, B, z, z, z, z, ws)   # bf16 mode without bf16 buffers
     assert e.value.status == -4
+
+
+def test_normalized_entropy_accumulates_over_batches():
+    rng = np.random.default_rng(11)
+    acc = torch.zeros(3, dtype=torch.float64, device="cuda")
+    out = torch.zeros(1, dtype=torch.float64, device="cuda")
+    zs, ys = [], []
+    for B in (2048, 777, 1):
+        z = (rng.normal(size=B) * 2 - 3).astype(np.float32)
+        y = (rng.random(B) < 0.05).astype(np.float32)
+        if B == 2048:
+            y[:3] = 1.0
+        ss.ss_ne_accumulate(torch.from_numpy(z).cuda(), torch.from_numpy(y).cuda(), B, acc)
+        zs.append(z); ys.append(y)
+    ss.ss_ne_value(acc, out)
+    torch.cuda.synchronize()
+    z, y = np.concatenate(zs).astype(np.float64), np.concatenate(ys)
+    want = O.normalized_entropy(1.0 / (1.0 + np.exp(-z)), y)
+    assert abs(float(out.item()) - want) <= 1e-9 * want
+    # the constant predictor at the empirical rate has NE = 1
+    p = float(y.mean())
+    acc.zero_()
+    const = torch.full((len(y),), float(np.log(p / (1 - p))), device="cuda")
+    ss.ss_ne_accumulate(const, torch.from_numpy(y).cuda(), len(y), acc)
+    ss.ss_ne_value(acc, out)
+    torch.cuda.synchronize()
+    assert abs(float(out.item()) - 1.0) < 1e-6

@@ -29,8 +29,8 @@ def _run(rule, R, n, alpha, eta=1.0, mu=0.0, flags=0, mirror=False, seed=1, floo
         ss.ss_sync_ma(dw, dc, n, alpha, 0, mir)
         O.sync_ma(ws, alpha, c)
     else:
-        ss.ss_sync_bmuf(dw, dc, dd, n, alpha, eta, mu, 0, mir)
-        O.sync_bmuf(ws, c, d, alpha, eta, mu)
+        ss.ss_sync_bmuf(dw, dc, dd, n, alpha, eta, mu, flags, mir)
+        O.sync_bmuf(ws, c, d, alpha, eta, mu, nesterov=bool(flags & ss.SS_SYNC_BMUF_NESTEROV))
     torch.cuda.synchronize()
     for r in range(R):
         assert_close(dw[r].cpu().numpy(), ws[r], RTOL_SYNC, f"{rule} w[{r}]", floor)
@@ -63,6 +63,10 @@ def test_sync_tiny_and_empty():
             # a handful of elements: the operands' scale (std 0.02) is the reference, not a cancelled result
             _run("easgd", 2, n, 0.3, floor=0.02)
             _run("bmuf", 2, n, 0.3, 0.5, 0.9, floor=0.02)
+
+
+def test_bmuf_nesterov_flag():
+    _run("bmuf", 4, 6 * 1024 + 1, 0.1, eta=1.0, mu=0.9, flags=ss.SS_SYNC_BMUF_NESTEROV, mirror=True)
 
 
 def test_easgd_literal_flag():

@@ -145,3 +145,43 @@ def test_shadow_loop_free_running_keeps_invariants():
     assert torch.isfinite(m.center).all() and torch.isfinite(m.tables).all()
     # elastic averaging keeps the replicas within a small distance of the centre
     assert float((m.replicas[0].w - m.center).abs().max()) < 0.5
+
+
+def test_foreground_sync_variants_match_the_oracle_rules():
+    # FR-EASGD: each replica interpolates with the centre on its own stream; FR-MA / FR-BMUF: one joint pass
+    cfg = synth.scaled(synth.CONFIGS["tiny"], R=3)
+    tables = synth.tables_dense(cfg)
+    layers = synth.initial_weights(cfg)
+    m = _model(cfg, tables, layers, 16, keep=False)
+    rng = np.random.default_rng(2)
+    n = m.spec.param_count
+    for rep in m.replicas:
+        rep.w.copy_(torch.from_numpy((rng.normal(size=n) * 0.02).astype(np.float32)))
+    m.center.copy_(torch.from_numpy((rng.normal(size=n) * 0.02).astype(np.float32)))
+    torch.cuda.synchronize()
+    for rule in ("ma", "bmuf", "easgd"):
+        ws = [rep.w.cpu().numpy().copy() for rep in m.replicas]
+        c, d = m.center.cpu().numpy().copy(), m.delta.cpu().numpy().copy()
+        m.foreground_sync(rule, 0.2, eta=0.8, mu=0.5)
+        torch.cuda.synchronize()
+        if rule == "ma":
+            O.sync_ma(ws, 0.2, c)
+        elif rule == "bmuf":
+            O.sync_bmuf(ws, c, d, 0.2, 0.8, 0.5)
+        else:
+            # replicas' passes run on different streams: any visiting order is legal; each order is an oracle run
+            import itertools
+            got = [rep.w.cpu().numpy() for rep in m.replicas] + [m.center.cpu().numpy()]
+            ok = False
+            for order in itertools.permutations(range(cfg.R)):
+                w2, c2 = [w.copy() for w in ws], c.copy()
+                for r in order:
+                    O.sync_easgd([w2[r]], c2, 0.2)
+                if all(np.allclose(a, b, rtol=1e-6, atol=1e-9) for a, b in zip(got, w2 + [c2])):
+                    ok = True
+                    break
+            assert ok, "FR-EASGD result matches no visiting order of the replicas"
+            continue
+        for rep, w in zip(m.replicas, ws):
+            assert_close(rep.w.cpu().numpy(), w, RTOL_SYNC, f"FR-{rule} replica")
+        assert_close(m.center.cpu().numpy(), c, RTOL_SYNC, f"FR-{rule} global")

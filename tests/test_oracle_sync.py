@@ -164,6 +164,29 @@ def test_bmuf_golden():
         assert (g[0], d[0], ws[0][0], ws[1][0]) == (g1, d1, w1, w2)
 
 
+def test_bmuf_nesterov_golden_and_limits():
+    for mu, d0, g1, d1, w1, w2 in _rows("bmuf_nesterov_scalar.txt"):
+        ws = [np.array([1.0], np.float32), np.array([3.0], np.float32)]
+        g, d = np.array([0.0], np.float32), np.array([d0], np.float32)
+        O.sync_bmuf(ws, g, d, alpha=0.25, eta=0.5, mu=mu, nesterov=True)
+        assert (g[0], d[0], ws[0][0], ws[1][0]) == (g1, d1, w1, w2)
+    # without momentum the look-ahead point is the global model itself
+    a, b = _vecs(3, 500), _vecs(3, 500)
+    ga, gb = _vecs(1, 500, 4)[0], _vecs(1, 500, 4)[0]
+    da, db = np.zeros(500, np.float32), np.zeros(500, np.float32)
+    O.sync_bmuf(a, ga, da, 0.1, 0.7, 0.0, nesterov=True)
+    O.sync_bmuf(b, gb, db, 0.1, 0.7, 0.0, nesterov=False)
+    assert all(np.array_equal(x, y) for x, y in zip(a, b)) and np.array_equal(ga, gb)
+    # the global model and the momentum do not depend on the variant; replicas differ by alpha*mu*delta
+    a, b = _vecs(3, 500), _vecs(3, 500)
+    ga, gb = _vecs(1, 500, 4)[0], _vecs(1, 500, 4)[0]
+    da, db = _vecs(1, 500, 6)[0], _vecs(1, 500, 6)[0]
+    O.sync_bmuf(a, ga, da, 0.2, 1.0, 0.9, nesterov=True)
+    O.sync_bmuf(b, gb, db, 0.2, 1.0, 0.9, nesterov=False)
+    assert np.array_equal(ga, gb) and np.array_equal(da, db)
+    np.testing.assert_allclose(a[1].astype(np.float64) - b[1], 0.2 * 0.9 * da.astype(np.float64), atol=1e-8)
+
+
 def test_bmuf_mu0_eta1_equals_ma():
     ws_a = _vecs(8, 3000)
     ws_b = [w.copy() for w in ws_a]
