@@ -94,7 +94,7 @@ class ClockSampler:
 
 
 # ----------------------------------------------------------------------------------------------
-def build_job(cfg, device):
+def build_job(cfg, device, workers=1):
     """Tables, replicas and a ring of device-resident batches for one GPU."""
     import torch
     from paper_2003_03477_b200 import binding as ss, synth, trainer
@@ -104,7 +104,7 @@ def build_job(cfg, device):
     host = [[synth.make_batch(cfg, r, t) for t in range(RING)] for r in range(cfg.R)]
     max_L = max(b.L for bs in host for b in bs)
     model = trainer.Model(cfg.T, cfg.N, cfg.D, cfg.B, cfg.bottom, cfg.top, cfg.bf16, cfg.R, w0, tables, cfg.lr, cfg.eps,
-                          max_L=max_L, device=device)
+                          max_L=max_L, device=device, workers=workers)
     dev = [[trainer.DeviceBatch(b.indices, b.offsets, b.dense, b.labels, device) for b in bs] for bs in host]
     return model, host, dev, max_L
 
@@ -201,7 +201,7 @@ def bench_gpu(args):
     K, W = args.steps, max(args.warmup, 3)
     peaks = measured_peaks()
 
-    model, host, dev, max_L = build_job(cfg, device)
+    model, host, dev, max_L = build_job(cfg, device, workers=max(1, args.workers))
     # un-captured warm-up: first-use set-up inside the library (function attributes, symbol addresses)
     for r in range(cfg.R):
         model.step(r, dev[r][0])
@@ -254,6 +254,50 @@ def bench_gpu(args):
         e1.record(main)
         e1.synchronize()
         ms_fg = e0.elapsed_time(e1)
+    # ---- intra-trainer Hogwild: m workers per replica, each on its own batches, sharing the replica's parameters
+    ms_hw = None
+    if args.workers > 1:
+        m = args.workers
+        for r in range(cfg.R):
+            for k in range(1, m):
+                model.step(r, dev[r][k % RING], worker=k)
+        torch.cuda.synchronize()
+        wg = []
+        for r in range(cfg.R):
+            per_worker = []
+            for k in range(m):
+                wk, row = model.workers[r][k], []
+                for slot in range(RING):
+                    g = torch.cuda.CUDAGraph()
+                    with torch.cuda.graph(g, stream=wk.stream):
+                        model.step(r, dev[r][(slot + 3 * k) % RING], stream=wk.stream, worker=k)
+                    row.append(g)
+                per_worker.append(row)
+            wg.append(per_worker)
+
+        def hw_steps(first, n):
+            for t in range(first, first + n):
+                for r in range(cfg.R):
+                    for k in range(m):
+                        with torch.cuda.stream(model.workers[r][k].stream):
+                            wg[r][k][t % RING].replay()
+        hw_steps(0, W)
+        barrier()
+        main = torch.cuda.current_stream()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(main)
+        for ws_ in model.workers:
+            for wk in ws_:
+                wk.stream.wait_event(e0)
+        hw_steps(W, K)
+        for ws_ in model.workers:
+            for wk in ws_:
+                e = torch.cuda.Event()
+                e.record(wk.stream)
+                main.wait_event(e)
+        e1.record(main)
+        e1.synchronize()
+        ms_hw = e0.elapsed_time(e1)
     (ms_on, ms_off), examples = reduce_over_ranks([ms_on, ms_off], cfg.R * cfg.B * K, device)
     value = examples / (ms_on * 1e-3)
     value_off = examples / (ms_off * 1e-3)
@@ -283,6 +327,9 @@ def bench_gpu(args):
     if ms_fg is not None:
         out["sync"]["foreground"] = {"every_k_steps": args.foreground, "examples_per_s": cfg.R * cfg.B * K / (ms_fg * 1e-3),
                                      "note": "same kernels enqueued on the training streams (FR-* of the paper)"}
+    if ms_hw is not None:
+        out["hogwild"] = {"workers_per_replica": args.workers, "sync": "off",
+                          "examples_per_s": cfg.R * args.workers * cfg.B * K / (ms_hw * 1e-3)}
     kernels, per_step = profile_pass(model, dev, cfg)
     out["kernels"] = kernels
     out["gpu_launches"] = int(round(per_step * cfg.R * K)) + int(rounds)
@@ -588,6 +635,8 @@ def main():
     ap.add_argument("--quick", action="store_true", help="skip the e2e and CPU-baseline legs (experiments)")
     ap.add_argument("--foreground", type=int, default=0,
                     help="also time the foreground variant: one sync pass on the training streams every k steps")
+    ap.add_argument("--workers", type=int, default=1,
+                    help="also time m lock-free workers per replica sharing its parameters (intra-trainer Hogwild)")
     ap.add_argument("--sweep", action="store_true", help="isolated sync-kernel sweep instead of the training benchmark")
     args = ap.parse_args()
     if args.sweep:

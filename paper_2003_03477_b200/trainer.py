@@ -36,14 +36,20 @@ class DeviceBatch:
 class Replica:
     """Buffers of one trainer replica: w^(i), its Adagrad accumulator, bf16 mirror, activations, stream."""
 
-    def __init__(self, model: "Model", w0_flat: torch.Tensor, priority: int, max_L: int, keep_sort_outputs: bool):
+    def __init__(self, model: "Model", w0_flat: torch.Tensor, priority: int, max_L: int, keep_sort_outputs: bool,
+                 share: Optional["Replica"] = None):
         m, dev = model, model.device
         B, spec = m.B, m.spec
-        self.w = w0_flat.clone()
-        self.acc = torch.zeros_like(self.w)
-        self.w_bf16 = torch.empty(spec.param_count, dtype=torch.bfloat16, device=dev) if spec.bf16 else None
-        if spec.bf16:
-            ss.ss_to_bf16(self.w, self.w_bf16, spec.param_count)
+        if share is not None:
+            # a further worker of the same trainer: its own activations and streams, but the trainer's single
+            # copy of the parameters and of the optimizer state, updated lock-free (Section 3.2)
+            self.w, self.acc, self.w_bf16 = share.w, share.acc, share.w_bf16
+        else:
+            self.w = w0_flat.clone()
+            self.acc = torch.zeros_like(self.w)
+            self.w_bf16 = torch.empty(spec.param_count, dtype=torch.bfloat16, device=dev) if spec.bf16 else None
+            if spec.bf16:
+                ss.ss_to_bf16(self.w, self.w_bf16, spec.param_count)
         self.concat_f32 = torch.zeros(B, spec.W, dtype=torch.float32, device=dev) if (not spec.bf16 or m.keep_f32_concat) else None
         self.concat_bf16 = torch.zeros(B, spec.W, dtype=torch.bfloat16, device=dev) if spec.bf16 else None
         self.logit = torch.empty(B, dtype=torch.float32, device=dev)
@@ -68,7 +74,8 @@ class Model:
 
     def __init__(self, T: int, N: int, D: int, B: int, bottom: Sequence[int], top: Sequence[int], bf16: bool,
                  R: int, w0_flat: torch.Tensor, tables: torch.Tensor, lr: float = 0.01, eps: float = 1e-8,
-                 max_L: int = 0, keep_sort_outputs: bool = False, keep_f32_concat: bool = False, device="cuda"):
+                 max_L: int = 0, keep_sort_outputs: bool = False, keep_f32_concat: bool = False, device="cuda",
+                 workers: int = 1):
         self.T, self.N, self.D, self.B, self.R = T, N, D, B, R
         self.lr, self.eps = lr, eps
         self.device = device
@@ -82,6 +89,11 @@ class Model:
         lo, hi = torch.cuda.Stream.priority_range()   # (lowest priority value, highest), e.g. (0, -5)
         self.prio_low, self.prio_high = lo, hi
         self.replicas: List[Replica] = [Replica(self, w0_flat, hi, max_L, keep_sort_outputs) for _ in range(R)]
+        # workers[r][k]: worker k of trainer r; worker 0 is the replica itself, further workers share its parameters
+        # (the paper's intra-trainer Hogwild: m threads, each on its own batch, updating one local copy)
+        self.workers: List[List[Replica]] = [
+            [rep] + [Replica(self, w0_flat, hi, max_L, keep_sort_outputs, share=rep) for _ in range(workers - 1)]
+            for rep in self.replicas]
         self.center = w0_flat.clone()              # w^PS (EASGD) / w^global (MA, BMUF), initialised to w0
         self.delta = torch.zeros_like(self.center)  # BMUF block momentum
         self.sync_stream = torch.cuda.Stream(device=device, priority=lo)
@@ -89,14 +101,14 @@ class Model:
 
     # ---------------------------------------------------------------- training step of one replica
     def step(self, r: int, batch: DeviceBatch, stream: Optional[torch.cuda.Stream] = None,
-             overlap_sort: bool = True) -> None:
+             overlap_sort: bool = True, worker: int = 0) -> None:
         """Enqueue one worker iteration of Algorithm 1 for replica r on its stream (no synchronisation).
 
         With overlap_sort the sort / unique half of the embedding backward, which needs only the batch's
         indices, is forked onto the replica's side stream at the start of the step and joined before the
         gradient reduction, so it runs under the forward and backward passes of the MLP.
         """
-        rep, sp = self.replicas[r], self.spec
+        rep, sp = self.workers[r][worker], self.spec
         s = stream or rep.stream
         T, N, D, B = self.T, self.N, self.D, self.B
         if overlap_sort:

@@ -185,3 +185,35 @@ def test_foreground_sync_variants_match_the_oracle_rules():
         for rep, w in zip(m.replicas, ws):
             assert_close(rep.w.cpu().numpy(), w, RTOL_SYNC, f"FR-{rule} replica")
         assert_close(m.center.cpu().numpy(), c, RTOL_SYNC, f"FR-{rule} global")
+
+
+def test_intra_replica_hogwild_workers_share_one_parameter_copy():
+    # two workers per trainer, each on its own batches and streams, updating the trainer's single copy of the
+    # parameters and optimizer state lock-free: any interleaving is legal, so invariants only
+    cfg = synth.scaled(synth.CONFIGS["tiny"], steps=24)
+    tables = synth.tables_dense(cfg)
+    layers = synth.initial_weights(cfg)
+    spec = ss.MlpSpec(cfg.bottom, cfg.top, cfg.bf16)
+    w0 = torch.from_numpy(trainer.pack_params(spec, layers)).cuda()
+    host = [[[synth.make_batch(cfg, 2 * r + k, t) for t in range(6)] for k in range(2)] for r in range(cfg.R)]
+    m = trainer.Model(cfg.T, cfg.N, cfg.D, cfg.B, cfg.bottom, cfg.top, cfg.bf16, cfg.R, w0,
+                      torch.from_numpy(tables.copy()).cuda(), cfg.lr, cfg.eps,
+                      max_L=max(b.L for a in host for bs in a for b in bs), workers=2)
+    dev = [[[_dev_batch(b) for b in bs] for bs in a] for a in host]
+    assert m.workers[0][1].w.data_ptr() == m.replicas[0].w.data_ptr()          # shared parameters
+    assert m.workers[0][1].logit.data_ptr() != m.replicas[0].logit.data_ptr()  # own activations
+    first = None
+    for t in range(cfg.steps):
+        for r in range(cfg.R):
+            for k in range(2):
+                m.step(r, dev[r][k][t % 6], worker=k)
+        if t == 0:
+            torch.cuda.synchronize()
+            first = float(m.replicas[0].loss.item())
+    torch.cuda.synchronize()
+    assert m.status() == 0
+    for r in range(cfg.R):
+        assert torch.isfinite(m.replicas[r].w).all() and torch.isfinite(m.replicas[r].acc).all()
+        for k in range(2):
+            assert float(m.workers[r][k].loss.item()) < first      # both workers' losses fell from ln 2
+    assert first > 0.5 and torch.isfinite(m.tables).all()
