@@ -72,7 +72,7 @@ constexpr int kRedRows = 256;     // most rows of the batch a block takes (bound
 __global__ void __launch_bounds__(256)
 batch_reduce_partial_kernel(const __grid_constant__ RedJobs jobs, int B, int rows_per_split, float* __restrict__ partial) {
   __shared__ float part[8][32][kMaxSCols + 1];
-  __shared__ float s_tile[kRedRows * kMaxSCols];           // S rows of this block's batch slice, as float
+  __shared__ __align__(16) float s_tile[kRedRows * kMaxSCols];   // S rows of this block's batch slice, as float
   __shared__ RedJob s_job;
   if (threadIdx.x == 0) {
     int j = 0;
@@ -88,9 +88,10 @@ batch_reduce_partial_kernel(const __grid_constant__ RedJobs jobs, int B, int row
   const int r1 = min(B, r0 + rows_per_split);
   const int nrows = r1 - r0;
   if (J.S != nullptr) {
-    for (int i = threadIdx.x; i < nrows * sc; i += 256) {
-      const int rr = i / sc, q = i - rr * sc;
-      s_tile[rr * kMaxSCols + q] = load_kind(J.S, J.s_kind, (int64_t)(r0 + rr) * J.lds + q);
+    // S rows as float, padded with zeros to kMaxSCols columns so that the inner product needs no column test
+    for (int i = threadIdx.x; i < nrows * kMaxSCols; i += 256) {
+      const int rr = i / kMaxSCols, q = i % kMaxSCols;
+      s_tile[i] = q < sc ? load_kind(J.S, J.s_kind, (int64_t)(r0 + rr) * J.lds + q) : 0.f;
     }
     __syncthreads();
   }
@@ -107,14 +108,23 @@ batch_reduce_partial_kernel(const __grid_constant__ RedJobs jobs, int B, int row
       if (J.S == nullptr) {
 #pragma unroll
         for (int u = 0; u < 4; ++u) acc[0] += m[u];
+      } else if (sc == 1) {
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+          if (rr + 8 * u < nrows) acc[0] = fmaf(m[u], s_tile[(rr + 8 * u) * kMaxSCols], acc[0]);
       } else {
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
           if (rr + 8 * u < nrows) {
-            const float* srow = s_tile + (rr + 8 * u) * kMaxSCols;
+            const float4* srow = reinterpret_cast<const float4*>(s_tile + (rr + 8 * u) * kMaxSCols);
 #pragma unroll
-            for (int q = 0; q < kMaxSCols; ++q)
-              if (q < sc) acc[q] = fmaf(m[u], srow[q], acc[q]);
+            for (int q4 = 0; q4 < kMaxSCols / 4; ++q4) {
+              const float4 sv = srow[q4];                    // one 128-bit broadcast read for four columns
+              acc[4 * q4 + 0] = fmaf(m[u], sv.x, acc[4 * q4 + 0]);
+              acc[4 * q4 + 1] = fmaf(m[u], sv.y, acc[4 * q4 + 1]);
+              acc[4 * q4 + 2] = fmaf(m[u], sv.z, acc[4 * q4 + 2]);
+              acc[4 * q4 + 3] = fmaf(m[u], sv.w, acc[4 * q4 + 3]);
+            }
           }
         }
       }
