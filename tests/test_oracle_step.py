@@ -304,3 +304,40 @@ def test_train_run_tiny_shapes_loss_is_finite_and_sync_pulls_replicas_together()
     gap1 = np.abs(O.flatten(reps1[0]) - O.flatten(reps1[1])).max()
     assert gap1 < gap0            # elastic averaging keeps the replicas closer than no sync
     assert np.array_equal(np.array(l0[:2]), np.array(l1[:2]))   # identical until the first sync
+
+
+def test_gate_matching_recovers_planted_edge_gates_and_nothing_else():
+    """The helper that lets the oracle follow the kernels' ReLU decisions switches only units whose
+    pre-activation is within the stated distance of zero: planted switches at such units are found,
+    a switch at an ordinary unit is left unexplained (the caller's strict comparison then fails)."""
+    from parity import match_relu_gates
+    from paper_2003_03477_b200 import synth
+    cfg = synth.scaled(synth.CONFIGS["tiny"], B=24)
+    layers = synth.initial_weights(cfg)
+    nb = len(cfg.bottom) - 1
+    batch = synth.make_batch(cfg, 0, 0)
+    pooled = O.embbag_fwd(synth.tables_dense(cfg), batch.indices, batch.offsets, cfg.B)
+    fwd = O.mlp_fwd(layers, nb, batch.dense, pooled, batch.labels, False)
+    backward = lambda f: O.mlp_bwd(layers, nb, f, batch.labels, False)[1]
+    # move two pre-activations to the edge, then produce the "other side's" gradient with their gates switched
+    edge = dict(fwd); edge["pre"] = [p.copy() for p in fwd["pre"]]
+    planted = [(3, nb, 1), (17, nb, 40), (17, nb, 7)]
+    for b, l, j in planted:
+        edge["pre"][l][b, j] = 1e-9
+    other = dict(edge); other["pre"] = [p.copy() for p in edge["pre"]]
+    for b, l, j in planted:
+        other["pre"][l][b, j] = -1e-9
+    got = backward(other)
+    assert np.abs(got - backward(edge)).max() > 0
+    matched, flips = match_relu_gates(edge, backward, got, 1e-9, nb, len(layers))
+    assert sorted(flips) == sorted(planted)
+    np.testing.assert_allclose(backward(matched), got, rtol=1e-12, atol=0)
+    # a switched gate at a unit far from zero is a mistake, not a rounding decision
+    far = dict(fwd); far["pre"] = [p.copy() for p in fwd["pre"]]
+    b, l = 5, nb
+    j = int(np.argmax(np.abs(fwd["pre"][l][b])))
+    far["pre"][l][b, j] = -far["pre"][l][b, j]
+    wrong = backward(far)
+    assert np.abs(wrong - backward(fwd)).max() > 0
+    matched, flips = match_relu_gates(fwd, backward, wrong, 1e-9, nb, len(layers))
+    assert np.abs(backward(matched) - wrong)[b].max() > 0
