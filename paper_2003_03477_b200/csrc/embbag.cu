@@ -175,7 +175,8 @@ static BwdPlan make_plan(int T, int64_t N, int D, int64_t L) {
 __global__ void __launch_bounds__(256)
 build_keys_kernel(const int32_t* __restrict__ indices, const int32_t* __restrict__ offsets, int T, int64_t N,
                   int B, int64_t L, uint32_t* __restrict__ keys, int32_t* __restrict__ bag_of,
-                  int32_t* __restrict__ d_status) {
+                  int32_t* __restrict__ d_status, const int32_t* __restrict__ run_if) {
+  if (run_if && *run_if == 0) return;                     // the per-table sort already produced the result
   const int64_t bag = (int64_t)blockIdx.x * 256 + threadIdx.x;
   const int64_t nbags = (int64_t)T * B;
   if (bag >= nbags) return;
@@ -223,8 +224,9 @@ __device__ __forceinline__ uint32_t same_digit_lanes(uint32_t digit, int nbits) 
 // digit are counted together, so a hot row does not serialise on one counter.
 __global__ void __launch_bounds__(kSortThreads)
 sort_hist_kernel(const uint32_t* __restrict__ keys, int64_t L, int shift, int bins, int nblk,
-                 uint32_t* __restrict__ hist) {
+                 uint32_t* __restrict__ hist, const int32_t* __restrict__ run_if) {
   __shared__ uint32_t cnt[kMaxBins];
+  if (run_if && *run_if == 0) return;
   for (int i = threadIdx.x; i < bins; i += kSortThreads) cnt[i] = 0;
   __syncthreads();
   const int lane = threadIdx.x & 31;
@@ -249,7 +251,9 @@ sort_hist_kernel(const uint32_t* __restrict__ keys, int64_t L, int shift, int bi
 
 // One warp per bin: exclusive scan of that bin's per-tile counts in place, bin total to bintot[bin].
 __global__ void __launch_bounds__(256)
-bin_scan_kernel(uint32_t* __restrict__ hist, int bins, int nblk, uint32_t* __restrict__ bintot) {
+bin_scan_kernel(uint32_t* __restrict__ hist, int bins, int nblk, uint32_t* __restrict__ bintot,
+                const int32_t* __restrict__ run_if) {
+  if (run_if && *run_if == 0) return;
   const int bin = blockIdx.x * 8 + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
   if (bin >= bins) return;
@@ -322,8 +326,10 @@ scan_exclusive_kernel(uint32_t* __restrict__ data, int64_t m, uint32_t* __restri
 __global__ void __launch_bounds__(kSortThreads)
 sort_scatter_kernel(const uint32_t* __restrict__ keys_in, const int32_t* __restrict__ pos_in,
                     uint32_t* __restrict__ keys_out, int32_t* __restrict__ pos_out, int64_t L, int shift,
-                    int bins, int nblk, const uint32_t* __restrict__ hist_scanned, const uint32_t* __restrict__ bintot) {
+                    int bins, int nblk, const uint32_t* __restrict__ hist_scanned, const uint32_t* __restrict__ bintot,
+                    const int32_t* __restrict__ run_if) {
   extern __shared__ uint32_t cnt[];                       // [kSortWarps][bins], then binbase[bins], wtot[8]
+  if (run_if && *run_if == 0) return;
   uint32_t* binbase = cnt + kSortWarps * bins;
   uint32_t* wtot = binbase + bins;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -388,6 +394,158 @@ sort_scatter_kernel(const uint32_t* __restrict__ keys_in, const int32_t* __restr
       keys_out[dst] = key[k];
       pos_out[dst] = pos_in ? pos_in[i] : (int32_t)i;
     }
+  }
+}
+
+// ---- (2b) per-table sort in shared memory -------------------------------------------------
+// The lookups arrive grouped by table (bags are table-major), so the sort by key = t*N + row is T
+// independent sorts by row.  One block per table keeps the table's row ids and a 16-bit position payload
+// in shared memory and runs the stable LSD passes there: no global histogram, no scan launches, and only
+// T of the SMs are busy while the other streams use the rest.  The result is the same unique stable
+// order the tiled passes produce.  A block that cannot take this path (more than kTsCap lookups in its
+// table, offsets that are not monotone within [0, L], a row index outside the table) raises *fallback
+// and the tiled passes, launched after this kernel, run; otherwise they return at once.
+constexpr int kTsThreads = 1024;
+constexpr int kTsWarps = kTsThreads / 32;
+constexpr int kTsCap = 24576;                              // lookups of one table
+constexpr int kTsMaxBins = 256;
+constexpr size_t kTsSmem = (size_t)kTsCap * 8 + (size_t)kTsWarps * kTsMaxBins * 4;   // 229,376 bytes
+
+template <int NB>
+__device__ __forceinline__ uint32_t same_digit_lanes_n(uint32_t digit) {
+  uint32_t peers = 0xffffffffu;
+#pragma unroll
+  for (int b = 0; b < NB; ++b) {
+    const bool bit = (digit >> b) & 1u;
+    const uint32_t m = __ballot_sync(0xffffffffu, bit);
+    peers &= bit ? m : ~m;
+  }
+  return peers;
+}
+
+template <int NB>                                          // digit bits, 5..8
+__global__ void __launch_bounds__(kTsThreads, 1)
+table_sort_kernel(const int32_t* __restrict__ indices, const int32_t* __restrict__ offsets, int T, int64_t N, int B,
+                  int64_t L, int passes, uint32_t* __restrict__ keys_out, int32_t* __restrict__ perm_out,
+                  int32_t* __restrict__ bag_of, int32_t* __restrict__ fallback) {
+  extern __shared__ __align__(16) unsigned char ts_smem[];
+  uint32_t* okey = reinterpret_cast<uint32_t*>(ts_smem);              // row id of local position i
+  uint16_t* pa = reinterpret_cast<uint16_t*>(okey + kTsCap);          // payload ping
+  uint16_t* pb = pa + kTsCap;                                         // payload pong
+  uint32_t* cnt = reinterpret_cast<uint32_t*>(pb + kTsCap);           // [kTsWarps][bins]
+  __shared__ uint32_t wtot[kTsWarps];
+  constexpr int bins = 1 << NB;
+  constexpr uint32_t mask = (uint32_t)bins - 1u;
+  const int t = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int64_t bag0 = (int64_t)t * B;
+  const int seg0 = offsets[bag0], seg1 = offsets[bag0 + B];
+  // block-uniform checks of the table's segment
+  if (seg0 < 0 || seg1 < seg0 || (int64_t)seg1 > L || seg1 - seg0 > kTsCap || (t == 0 && seg0 != 0) ||
+      (t == T - 1 && (int64_t)seg1 != L)) {
+    if (tid == 0) atomicOr(fallback, 1);
+    return;
+  }
+  const int n = seg1 - seg0;
+  const int n32 = (n + 31) & ~31;                          // padded to whole rounds (kTsCap is a multiple of 32)
+  // bag of every local position (16 bits: B <= 65536 is checked by the host), parked in the pong array
+  int bad = 0;
+  for (int b = tid; b < B; b += kTsThreads) {
+    const int lo = offsets[bag0 + b], hi = offsets[bag0 + b + 1];
+    if (lo < seg0 || hi < lo || hi > seg1) { bad = 1; continue; }
+    for (int j = lo; j < hi; ++j) pb[j - seg0] = (uint16_t)b;
+  }
+  if (__syncthreads_or(bad)) {
+    if (tid == 0) atomicOr(fallback, 1);
+    return;
+  }
+  // pad items carry the largest key and the highest positions, so every stable pass leaves them at the end
+#pragma unroll 4
+  for (int i = tid; i < n32; i += kTsThreads) {
+    uint32_t row = 0xffffffffu;
+    if (i < n) {
+      const int idx = indices[seg0 + i];
+      if (idx < 0 || (int64_t)idx >= N) bad = 1;
+      row = (uint32_t)idx;
+      bag_of[seg0 + i] = (int32_t)(bag0 + pb[i]);
+    }
+    okey[i] = row;
+    pa[i] = (uint16_t)i;
+  }
+  if (__syncthreads_or(bad)) {
+    if (tid == 0) atomicOr(fallback, 1);
+    return;
+  }
+  const int rounds = (n32 + kTsThreads - 1) / kTsThreads;  // rounds of 32 consecutive items per warp
+  const int w0 = warp * rounds * 32;                       // warp w owns items [w0, w0 + 32*rounds)
+  const int wend = min(w0 + rounds * 32, n32);
+  uint32_t* mycnt = cnt + warp * bins;
+  uint16_t* src = pa;
+  uint16_t* dst = pb;
+  for (int pass = 0; pass < passes; ++pass) {
+    const int shift = pass * NB;
+    for (int i = tid; i < kTsWarps * bins; i += kTsThreads) cnt[i] = 0;
+    __syncthreads();
+    // counts per (warp, digit): warp-private counters, equal digits inside a round resolved by the atomic unit
+    for (int i = w0 + lane; i < wend; i += 32) atomicAdd(&mycnt[(okey[src[i]] >> shift) & mask], 1u);
+    __syncthreads();
+    // exclusive scan in (digit, warp) order: thread tid owns q = bins/32 consecutive entries of that order
+    {
+      constexpr int q = bins >> 5;
+      uint32_t c[q];
+      uint32_t sum = 0;
+#pragma unroll
+      for (int u = 0; u < q; ++u) {
+        const int e = tid * q + u;
+        c[u] = cnt[(e & 31) * bins + (e >> 5)];
+        sum += c[u];
+      }
+      uint32_t inc = sum;
+#pragma unroll
+      for (int off = 1; off < 32; off <<= 1) {
+        const uint32_t v = __shfl_up_sync(0xffffffffu, inc, off);
+        if (lane >= off) inc += v;
+      }
+      if (lane == 31) wtot[warp] = inc;
+      __syncthreads();
+      if (warp == 0) {
+        uint32_t v = wtot[lane];
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+          const uint32_t u = __shfl_up_sync(0xffffffffu, v, off);
+          if (lane >= off) v += u;
+        }
+        wtot[lane] = v;                                    // inclusive over warps
+      }
+      __syncthreads();
+      uint32_t run = (warp ? wtot[warp - 1] : 0u) + inc - sum;
+#pragma unroll
+      for (int u = 0; u < q; ++u) {
+        const int e = tid * q + u;
+        cnt[(e & 31) * bins + (e >> 5)] = run;
+        run += c[u];
+      }
+    }
+    __syncthreads();
+    // stable scatter: rank inside a round from the lanes holding the same digit, across rounds from the counter
+    for (int i = w0 + lane; i < wend; i += 32) {           // whole rounds: the bound is the same for all lanes
+      const uint32_t pay = src[i];
+      const uint32_t digit = (okey[pay] >> shift) & mask;
+      const uint32_t peers = same_digit_lanes_n<NB>(digit);
+      const uint32_t below = peers & ((1u << lane) - 1u);
+      const uint32_t base = mycnt[digit];
+      __syncwarp();
+      if (below == 0) mycnt[digit] = base + __popc(peers);
+      __syncwarp();
+      dst[base + __popc(below)] = (uint16_t)pay;
+    }
+    __syncthreads();
+    uint16_t* sw = src; src = dst; dst = sw;
+  }
+  const uint32_t key0 = (uint32_t)((uint64_t)t * (uint64_t)N);
+  for (int j = tid; j < n; j += kTsThreads) {
+    const int pay = src[j];
+    keys_out[seg0 + j] = key0 + okey[pay];
+    perm_out[seg0 + j] = seg0 + pay;
   }
 }
 
@@ -968,10 +1126,45 @@ static ss_status bwd_impl(bool do_sort, bool do_apply, float* tables, float* row
   const int32_t* perm_sorted = (p.passes & 1) ? pos_b : pos_a;
   if (do_sort) {
 
+  // (0) one block per table sorts that table's lookups in shared memory; scalars[4] stays 0 when every
+  // block could, and the tiled passes below then return at once
+  int32_t* fallback = scalars + 4;
+  const bool try_table_sort = B <= 65536;
+  SS_CUDA(cudaMemsetAsync(fallback, try_table_sort ? 0 : 1, 4, cs));
+  if (try_table_sort) {
+    int row_bits = 1;
+    while (((uint64_t)(N - 1) >> row_bits) != 0) ++row_bits;
+    const int t_passes = (row_bits + 7) / 8;
+    int t_digit = (row_bits + t_passes - 1) / t_passes;
+    if (t_digit < 5) t_digit = 5;                          // the in-block scan wants at least 32 bins
+    static bool attr_set[64];
+    int dev = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess && dev >= 0 && dev < 64 && !attr_set[dev]) {
+      cudaFuncSetAttribute(table_sort_kernel<5>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTsSmem);
+      cudaFuncSetAttribute(table_sort_kernel<6>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTsSmem);
+      cudaFuncSetAttribute(table_sort_kernel<7>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTsSmem);
+      cudaFuncSetAttribute(table_sort_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTsSmem);
+      attr_set[dev] = true;
+    }
+    SS_TIMED("table_sort_kernel", cs);
+#define SS_TS(NB_)                                                                                              \
+  table_sort_kernel<NB_><<<T, kTsThreads, kTsSmem, cs>>>(indices, offsets, T, N, B, L, t_passes,                \
+                                                         const_cast<uint32_t*>(keys_sorted),                    \
+                                                         const_cast<int32_t*>(perm_sorted), bag_of, fallback)
+    switch (t_digit) {
+      case 5: SS_TS(5); break;
+      case 6: SS_TS(6); break;
+      case 7: SS_TS(7); break;
+      default: SS_TS(8); break;
+    }
+#undef SS_TS
+  }
+  SS_LAUNCH_OK();
+
   // (1) keys
   { SS_TIMED("build_keys_kernel", cs);
   build_keys_kernel<<<(unsigned)(((int64_t)T * B + 255) / 256), 256, 0, cs>>>(indices, offsets, T, N, B, L, keys_a,
-                                                                                bag_of, d_status);
+                                                                                bag_of, d_status, fallback);
   }
   SS_LAUNCH_OK();
 
@@ -984,13 +1177,14 @@ static ss_status bwd_impl(bool do_sort, bool do_apply, float* tables, float* row
   for (int pass = 0; pass < p.passes; ++pass) {
     const int shift = pass * p.digit_bits;
     { SS_TIMED("sort_hist_kernel", cs);
-    sort_hist_kernel<<<p.nblk, kSortThreads, 0, cs>>>(kin, L, shift, p.bins, p.nblk, hist);
+    sort_hist_kernel<<<p.nblk, kSortThreads, 0, cs>>>(kin, L, shift, p.bins, p.nblk, hist, fallback);
     }
     { SS_TIMED("bin_scan_kernel", cs);
-    bin_scan_kernel<<<(p.bins + 7) / 8, 256, 0, cs>>>(hist, p.bins, p.nblk, bintot);
+    bin_scan_kernel<<<(p.bins + 7) / 8, 256, 0, cs>>>(hist, p.bins, p.nblk, bintot, fallback);
     }
     { SS_TIMED("sort_scatter_kernel", cs);
-    sort_scatter_kernel<<<p.nblk, kSortThreads, smem, cs>>>(kin, pin, kout, pout, L, shift, p.bins, p.nblk, hist, bintot);
+    sort_scatter_kernel<<<p.nblk, kSortThreads, smem, cs>>>(kin, pin, kout, pout, L, shift, p.bins, p.nblk, hist, bintot,
+                                                            fallback);
     }
     SS_LAUNCH_OK();
     uint32_t* tk = kin; kin = kout; kout = tk;
@@ -1129,7 +1323,7 @@ ss_status ss_embbag_bwd_sort_noalloc(int T, int64_t N, const int32_t* indices, c
     return SS_OK;
   }
   build_keys_kernel<<<(unsigned)(((int64_t)T * B + 255) / 256), 256, 0, cs>>>(indices, offsets, T, N, B, L, keys_a,
-                                                                                bag_of, d_status);
+                                                                                bag_of, d_status, nullptr);
   SS_LAUNCH_OK();
   uint32_t* kin = keys_a; uint32_t* kout = keys_b;
   int32_t* pin = nullptr;
@@ -1138,9 +1332,10 @@ ss_status ss_embbag_bwd_sort_noalloc(int T, int64_t N, const int32_t* indices, c
   const size_t smem = ((size_t)kSortWarps * bins + bins + 8) * 4;
   for (int pass = 0; pass < passes; ++pass) {
     const int shift = pass * digit_bits;
-    sort_hist_kernel<<<nblk, kSortThreads, 0, cs>>>(kin, L, shift, bins, nblk, hist);
-    bin_scan_kernel<<<(bins + 7) / 8, 256, 0, cs>>>(hist, bins, nblk, bintot);
-    sort_scatter_kernel<<<nblk, kSortThreads, smem, cs>>>(kin, pin, kout, pout, L, shift, bins, nblk, hist, bintot);
+    sort_hist_kernel<<<nblk, kSortThreads, 0, cs>>>(kin, L, shift, bins, nblk, hist, nullptr);
+    bin_scan_kernel<<<(bins + 7) / 8, 256, 0, cs>>>(hist, bins, nblk, bintot, nullptr);
+    sort_scatter_kernel<<<nblk, kSortThreads, smem, cs>>>(kin, pin, kout, pout, L, shift, bins, nblk, hist, bintot,
+                                                          nullptr);
     SS_LAUNCH_OK();
     uint32_t* tk = kin; kin = kout; kout = tk;
     pin = pout; pout = pnext; pnext = pin;
