@@ -433,8 +433,9 @@ def profile_pass(model, dev, cfg, steps=6, replicas=None):
 def roofline(kernels, model, host, cfg, peaks):
     """Roofline entry of the kernel with the largest share of the step's kernel time.
 
-    Algorithmic work per launch: embedding forward L(4D+4) + 4(TB+1) + TB*D*{2,4} bytes; window reduction
-    L(4D+16) + U*4D; row update U(3*4D+12); tensor-core GEMMs: the step's 2MNK summed over its GEMM launches.
+    Algorithmic work per launch: embedding forward L(4D+4) + 4(TB+1) + TB*D*{2,4} bytes; fused window kernel
+    L(4D+16) + U(2*4D+8) (gather plus row read-modify-write); unfused window reduction L(4D+16) + U*4D; row update
+    U(3*4D+12); tensor-core GEMMs: the step's 2MNK summed over its GEMM launches.
     L and U are the means over the batches of replica 0 (U read back from the device)."""
     T, D, B = cfg.T, cfg.D, cfg.B
     L = float(np.mean([b.L for b in host[0]]))
@@ -448,6 +449,7 @@ def roofline(kernels, model, host, cfg, peaks):
         gemm_flops += 6.0 * B * fin * fout   # forward, weight gradient, input gradient: 2*B*in*out each
     work = {
         "embbag_fwd_kernel": ("hbm", L * (4 * D + 4) + 4 * (T * B + 1) + T * B * D * (2 if cfg.bf16 else 4), 1),
+        "window_apply_kernel": ("hbm", L * (4 * D + 16) + U * (2 * 4 * D + 8), 1),
         "window_reduce_kernel": ("hbm", L * (4 * D + 16) + U * 4 * D, 1),
         "apply_rows_kernel": ("hbm", U * (3 * 4 * D + 12), 1),
         "gemm_tc_kernel": ("tensor", gemm_flops, None),

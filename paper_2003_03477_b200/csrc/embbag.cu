@@ -628,67 +628,19 @@ __device__ __forceinline__ bool ws_matches(const int32_t* scalars, int64_t L, ui
 }
 
 // ---- (4) windowed segment reduction ---------------------------------------------------------
-// A lane group owns a window of 32 consecutive sorted positions and adds the gradient rows of each
+// A lane group owns a window of kWin consecutive sorted positions and adds the gradient rows of each
 // run of equal keys in position order.  A run that lies inside the window is complete: its sum goes
 // to gsum[u].  A run that crosses a window edge leaves a partial sum in the window's slot 0 (run
-// covers the window's first position) or slot 1.
-// FUSE (rows of at most 128 floats): the sums of the complete runs stay in shared memory and the group applies
-// row-wise Adagrad to those rows itself, four rows' loads in flight, so their sums never travel through global
-// memory; only rows crossing window edges go through gsum and the kernels that follow.
-// Row-wise Adagrad on the nr rows a lane group has stashed in shared memory (sums in s_sum, keys in s_runkey),
-// the loads of four rows in flight at a time.  All lanes of the group call it together.
-template <int G>
-__device__ __forceinline__ void update_stashed_rows(int nr, const float4* __restrict__ s_sum, const uint32_t* __restrict__ s_runkey,
-                                                    int lane, int nvec, int D, unsigned gmask, float* __restrict__ tables,
-                                                    float* __restrict__ row_state, float lr, float eps) {
-  __syncwarp(gmask);
-  for (int r0 = 0; r0 < nr; r0 += 4) {
-    uint32_t rk[4];
-    float4 rw[4], g[4];
-    float st[4];
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      const bool ok = r0 + j < nr;
-      rk[j] = ok ? s_runkey[r0 + j] : 0u;
-      const float4* row = reinterpret_cast<const float4*>(tables + (int64_t)rk[j] * D);
-      rw[j] = (ok && lane < nvec) ? row[lane] : make_float4(0.f, 0.f, 0.f, 0.f);
-      g[j] = (ok && lane < nvec) ? s_sum[(size_t)(r0 + j) * nvec + lane] : make_float4(0.f, 0.f, 0.f, 0.f);
-      st[j] = ok ? row_state[rk[j]] : 0.f;
-    }
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      float ss = g[j].x * g[j].x + g[j].y * g[j].y + g[j].z * g[j].z + g[j].w * g[j].w;
-#pragma unroll
-      for (int off = G / 2; off >= 1; off >>= 1) ss += __shfl_down_sync(gmask, ss, off, G);
-      ss = __shfl_sync(gmask, ss, 0, G);                   // every lane uses lane 0's sum
-      if (r0 + j >= nr) continue;
-      const float sn = st[j] + ss / (float)D;
-      const float scale = lr / (sqrtf(sn) + eps);
-      if (lane < nvec) {
-        float4 o = rw[j];
-        o.x -= scale * g[j].x; o.y -= scale * g[j].y; o.z -= scale * g[j].z; o.w -= scale * g[j].w;
-        reinterpret_cast<float4*>(tables + (int64_t)rk[j] * D)[lane] = o;
-      }
-      if (lane == 0) row_state[rk[j]] = sn;
-    }
-  }
-  __syncwarp(gmask);
-}
-
-constexpr int kStash = kWin; // complete runs a group can keep in shared memory (a window holds at most kWin)
-
-template <int G, int NV, bool FUSE>
-__global__ void __launch_bounds__(256, FUSE ? 3 : 1)
+// covers the window's first position) or slot 1.  This kernel serves rows wider than 128 floats (several
+// float4 per lane); narrower rows take window_apply_kernel, which also updates the rows.
+template <int G, int NV>
+__global__ void __launch_bounds__(256)
 window_reduce_kernel(const uint32_t* __restrict__ keys, const int32_t* __restrict__ sbag,
                      const int32_t* __restrict__ uidx, int64_t L,
                      uint32_t sentinel, int64_t N, int D, int B, const float* __restrict__ grad, int64_t ld_grad,
                      int col0, float* __restrict__ gsum, float* __restrict__ partial, int32_t* __restrict__ long_list,
-                     int32_t* __restrict__ scalars, int nwin, int64_t umax, int32_t* __restrict__ d_status,
-                     float* __restrict__ tables, float* __restrict__ row_state, float lr, float eps) {
+                     int32_t* __restrict__ scalars, int nwin, int64_t umax, int32_t* __restrict__ d_status) {
   constexpr int kGroups = 256 / G;
-  extern __shared__ float4 s_sum[];                        // FUSE: [kGroups][kStash][D/4] sums of complete runs
-  __shared__ uint32_t s_runkey[FUSE ? kGroups : 1][kStash];
-  int nr = 0;
   __shared__ uint32_t s_key[kGroups][kWin + 2];            // [0] = key before the window, [kWin+1] = key after
   __shared__ int32_t s_row[kGroups][kWin];                 // float4 index of the lookup's gradient row
   __shared__ int32_t s_u[kGroups][kWin];
@@ -710,10 +662,10 @@ window_reduce_kernel(const uint32_t* __restrict__ keys, const int32_t* __restric
     const int u = (body && in_range) ? uidx[j] : 0;
     int32_t row = -1;
     if (body && key < sentinel) {
-      const int t = (int)(key / (uint64_t)N);
+      const int t = (int)((uint32_t)sb / (uint32_t)B);     // bags are table-major: bag = t*B + b (32-bit division)
       const int b = sb - t * B;
       // a consistent workspace never fails these; an inconsistent one must not turn into a wild access
-      if (b >= 0 && b < B && u >= 0 && u < umax)
+      if (sb >= 0 && (int64_t)key >= (int64_t)t * N && (int64_t)key < (int64_t)(t + 1) * N && u >= 0 && u < umax)
         row = (int32_t)((int64_t)b * ld4 + (int64_t)t * nvec);   // B * ld_grad / 4 < 2^31 is checked on the host
       else
         key = sentinel;
@@ -752,20 +704,13 @@ window_reduce_kernel(const uint32_t* __restrict__ keys, const int32_t* __restric
         const bool head_open = (run_start == 0) && (s_key[grp][0] == key);
         const bool tail_open = (next == key);              // only possible at the window's last position
         const bool complete = !head_open && !tail_open;
-        if (FUSE && complete) {
-          if (lane < nvec) s_sum[((size_t)grp * kStash + nr) * nvec + lane] = acc[0];
-          if (lane == 0) s_runkey[grp][nr] = key;
-          ++nr;
-          acc[0] = make_float4(0.f, 0.f, 0.f, 0.f);
-        } else {
-          float4* dst = complete ? reinterpret_cast<float4*>(gsum + (int64_t)s_u[grp][i] * D)
-                                 : reinterpret_cast<float4*>(partial + ((int64_t)win * 2 + (run_start == 0 ? 0 : 1)) * D);
+        float4* dst = complete ? reinterpret_cast<float4*>(gsum + (int64_t)s_u[grp][i] * D)
+                               : reinterpret_cast<float4*>(partial + ((int64_t)win * 2 + (run_start == 0 ? 0 : 1)) * D);
 #pragma unroll
-          for (int v = 0; v < NV; ++v) {
-            const int c = lane + v * G;
-            if (c < nvec) dst[c] = acc[v];
-            acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
-          }
+        for (int v = 0; v < NV; ++v) {
+          const int c = lane + v * G;
+          if (c < nvec) dst[c] = acc[v];
+          acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
         }
         // the window in which a multi-window run starts enters the row in the list of rows to combine
         if (!head_open && tail_open && lane == 0) {
@@ -776,8 +721,121 @@ window_reduce_kernel(const uint32_t* __restrict__ keys, const int32_t* __restric
       }
     }
   }
-  if (FUSE && nr > 0)
-    update_stashed_rows<G>(nr, s_sum + (size_t)grp * kStash * nvec, s_runkey[grp], lane, nvec, D, gmask, tables, row_state, lr, eps);
+}
+
+template <int G>
+__device__ __forceinline__ void adagrad_one_row(float4 g, uint32_t key, int lane, int nvec, int D, unsigned gmask,
+                                                float* __restrict__ tables, float* __restrict__ row_state, float lr,
+                                                float eps);
+
+__device__ __forceinline__ void prefetch_l2(const void* p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
+
+// ---- (4b) fused window kernel for rows of at most 4G floats ------------------------------------
+// Same windows, same order of additions and same outputs as window_reduce_kernel<G, 1, true>.  The run
+// structure of the window is three 16-bit masks (valid, head, tail) built once from the keys; while the
+// keys are looked at, the table rows of the window's runs are requested into L2, so that when a run ends
+// its row is updated on the spot from the sum in the lanes' registers.  No shared-memory stash: the number
+// of windows in flight on an SM is bounded by registers only.
+constexpr int kWaThreads = 128;
+
+template <int G>
+__global__ void __launch_bounds__(kWaThreads, 8)
+window_apply_kernel(const uint32_t* __restrict__ keys, const int32_t* __restrict__ sbag,
+                    const int32_t* __restrict__ uidx, int64_t L, uint32_t sentinel, int64_t N, int D, int B,
+                    const float* __restrict__ grad, int64_t ld_grad, int col0, float* __restrict__ partial,
+                    int32_t* __restrict__ long_list, int32_t* __restrict__ scalars, int nwin, int64_t umax,
+                    int32_t* __restrict__ d_status, float* __restrict__ tables, float* __restrict__ row_state,
+                    float lr, float eps) {
+  constexpr int kGroups = kWaThreads / G;
+  __shared__ uint32_t s_key[kGroups][kWin + 2];            // [0] = key before the window, [kWin+1] = key after
+  __shared__ int32_t s_row[kGroups][kWin];                 // float4 index of the lookup's gradient row
+  __shared__ int32_t s_u[kGroups][kWin];
+  const int grp = threadIdx.x / G, lane = threadIdx.x % G;
+  const int64_t win = (int64_t)blockIdx.x * kGroups + grp;
+  const unsigned gmask = (G == 32) ? 0xffffffffu : (((1u << G) - 1u) << ((threadIdx.x & 31) / G * G));
+  if (!ws_matches(scalars, L, sentinel, d_status)) return;
+  if (win >= nwin) return;
+  const int64_t w0 = win * kWin;
+  const int nvec = D >> 2;
+  const int64_t ld4 = ld_grad >> 2;
+  for (int e = lane; e < kWin + 2; e += G) {
+    const int64_t j = w0 - 1 + e;
+    const bool in_range = j >= 0 && j < L;
+    const bool body = e >= 1 && e <= kWin;
+    uint32_t key = in_range ? keys[j] : sentinel;
+    const int sb = (body && in_range) ? sbag[j] : 0;
+    const int u = (body && in_range) ? uidx[j] : 0;
+    int32_t row = -1;
+    if (body && key < sentinel) {
+      const int t = (int)((uint32_t)sb / (uint32_t)B);     // bags are table-major: bag = t*B + b
+      const int b = sb - t * B;
+      // a consistent workspace never fails these; an inconsistent one must not turn into a wild access
+      if (sb >= 0 && (int64_t)key >= (int64_t)t * N && (int64_t)key < (int64_t)(t + 1) * N && u >= 0 && u < umax) {
+        row = (int32_t)((int64_t)b * ld4 + (int64_t)t * nvec);   // B * ld_grad / 4 < 2^31 is checked on the host
+        const char* trow = reinterpret_cast<const char*>(tables + (int64_t)key * D);
+        for (int o = 0; o < D * 4; o += 128) prefetch_l2(trow + o);     // a repeated key asks for a line already on its way
+        prefetch_l2(row_state + key);
+      } else {
+        key = sentinel;
+      }
+    }
+    s_key[grp][e] = key;
+    if (body) { s_row[grp][e - 1] = row; s_u[grp][e - 1] = u; }
+  }
+  __syncwarp(gmask);
+  // valid (bits 16..31) and head (bits 0..15) of the positions this lane owns, then OR over the group
+  uint32_t bits = 0;
+  for (int i = lane; i < kWin; i += G) {
+    const uint32_t k = s_key[grp][1 + i];
+    if (k < sentinel) {
+      bits |= 0x10000u << i;
+      if (i == 0 || s_key[grp][i] != k) bits |= 1u << i;
+    }
+  }
+#pragma unroll
+  for (int off = G / 2; off >= 1; off >>= 1) bits |= __shfl_xor_sync(gmask, bits, off, G);
+  const uint32_t vm = bits >> 16, hm = bits & 0xffffu;
+  // a run ends where the next position starts another run, is a skipped lookup, or lies outside the window
+  const uint32_t tm = vm & ((hm >> 1) | (~vm >> 1) | 0x8000u);
+  const bool first_open = (vm & 1u) && s_key[grp][0] == s_key[grp][1];
+  const bool last_open = (vm >> (kWin - 1) & 1u) && s_key[grp][kWin + 1] == s_key[grp][kWin];
+  const float4* grad4 = reinterpret_cast<const float4*>(grad + col0);  // col0 is a multiple of 4
+
+  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+  constexpr int kBatch = 8;                                // gradient rows in flight per lane
+#pragma unroll
+  for (int i0 = 0; i0 < kWin; i0 += kBatch) {
+    float4 gv[kBatch];
+#pragma unroll
+    for (int u = 0; u < kBatch; ++u) {
+      const int32_t row = s_row[grp][i0 + u];
+      gv[u] = (row >= 0 && lane < nvec) ? __ldg(grad4 + row + lane) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+#pragma unroll
+    for (int u = 0; u < kBatch; ++u) {
+      const int i = i0 + u;
+      if ((hm >> i) & 1u) acc = make_float4(0.f, 0.f, 0.f, 0.f);
+      acc = add4(acc, gv[u]);                              // skipped lookups carry zeros and follow every run
+      if ((tm >> i) & 1u) {
+        const uint32_t key = s_key[grp][1 + i];
+        const bool first = (tm & ((1u << i) - 1u)) == 0u;  // the window's first run holds position 0
+        const bool head_open = first && first_open;
+        const bool tail_open = (i == kWin - 1) && last_open;
+        if (!head_open && !tail_open) {
+          adagrad_one_row<G>(acc, key, lane, nvec, D, gmask, tables, row_state, lr, eps);
+        } else {
+          // the run goes on in a neighbouring window: its part goes to the window's partial slot
+          // (slot 0 when the run holds the window's first position), the combine kernel adds the parts
+          float4* dst = reinterpret_cast<float4*>(partial + ((int64_t)win * 2 + (first ? 0 : 1)) * D);
+          if (lane < nvec) dst[lane] = acc;
+          if (!head_open && lane == 0) {                   // the window in which a multi-window run starts lists the row
+            const int slot = atomicAdd(&scalars[1], 1);
+            if (slot < nwin) long_list[slot] = s_u[grp][i];   // at most one such run per window
+          }
+        }
+      }
+    }
+  }
 }
 
 // Row-wise Adagrad on one row whose gradient slice is in the lanes' registers (rows of at most 4G floats).
@@ -792,8 +850,8 @@ __device__ __forceinline__ void adagrad_one_row(float4 g, uint32_t key, int lane
 #pragma unroll
   for (int off = G / 2; off >= 1; off >>= 1) ss += __shfl_down_sync(gmask, ss, off, G);
   ss = __shfl_sync(gmask, ss, 0, G);                       // every lane uses lane 0's sum
-  const float sn = st + ss / (float)D;
-  const float scale = lr / (sqrtf(sn) + eps);
+  const float sn = st + ss * (1.0f / (float)D);            // the reciprocal is loop-invariant at the call sites
+  const float scale = __fdividef(lr, sqrtf(sn) + eps);     // within 2 ulp of the quotient
   if (lane < nvec) {
     float4 o = r;
     o.x -= scale * g.x; o.y -= scale * g.y; o.z -= scale * g.z; o.w -= scale * g.w;
@@ -860,14 +918,29 @@ combine_rows_kernel(const int32_t* __restrict__ seg, const int32_t* __restrict__
       if (key < sentinel) adagrad_one_row<G>(t0, key, lane, nvec, D, gmask, tables, row_state, lr, eps);
     }
   }
-  // phase B: long spans, the whole block per row
-  for (int i = blockIdx.x; i < n; i += gridDim.x) {
-    const int u = long_list[i];
-    if (u < 0 || u >= umax) continue;                      // uniform over the block, like the tests below
+  // phase B: long spans, the whole block per row.  The block owns the list entries blockIdx.x + k*gridDim.x;
+  // its threads look at 256 of them at a time (one round of loads) and queue the long ones.
+  __shared__ int s_long[256];
+  __shared__ int s_nlong;
+  for (int64_t base = 0; (int64_t)blockIdx.x + base * gridDim.x < n; base += 256) {
+    if (threadIdx.x == 0) s_nlong = 0;
+    __syncthreads();
+    {
+      const int64_t i = (int64_t)blockIdx.x + (base + threadIdx.x) * gridDim.x;
+      if (i < n) {
+        const int u = long_list[i];
+        if (u >= 0 && u < umax) {
+          const int s0 = seg[u], s1 = seg[u + 1];
+          if (s0 >= 0 && s1 > s0 && s1 <= L && (s1 - 1) / kWin - s0 / kWin + 1 > kShort) s_long[atomicAdd(&s_nlong, 1)] = u;
+        }
+      }
+    }
+    __syncthreads();
+    const int nlong = s_nlong;
+  for (int q = 0; q < nlong; ++q) {
+    const int u = s_long[q];                               // checked above; uniform over the block
     const int s0 = seg[u], s1 = seg[u + 1];
-    if (s0 < 0 || s1 <= s0 || s1 > L) continue;
     const int k0 = s0 / kWin, k1 = (s1 - 1) / kWin;
-    if (k1 - k0 + 1 <= kShort) continue;
     float4 acc[NV];
 #pragma unroll
     for (int v = 0; v < NV; ++v) acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -906,6 +979,7 @@ combine_rows_kernel(const int32_t* __restrict__ seg, const int32_t* __restrict__
       }
     }
     __syncthreads();
+  }
   }
 }
 
@@ -998,22 +1072,18 @@ static void launch_reduce(const BwdPlan& p, char* ws, const uint32_t* keys, cons
   constexpr bool kFuse = (NV == 1);
   // the list of rows crossing window edges starts empty (the apply half may be repeated on one sort)
   cudaMemsetAsync(scalars + 1, 0, sizeof(int32_t), st);
-  {
+  if (kFuse) {
+    constexpr int kWaGroups = kWaThreads / G;
+    SS_TIMED("window_apply_kernel", st);
+    window_apply_kernel<G><<<(unsigned)((p.nwin + kWaGroups - 1) / kWaGroups), kWaThreads, 0, st>>>(
+        keys, reinterpret_cast<int32_t*>(ws + p.off_sbag), reinterpret_cast<int32_t*>(ws + p.off_uidx), p.L, sentinel,
+        N, D, B, grad, ld_grad, col0, partial, long_list, scalars, p.nwin, (int64_t)umax, d_status, tables, row_state,
+        lr, eps);
+  } else {
     SS_TIMED("window_reduce_kernel", st);
-    const size_t smem = kFuse ? (size_t)kGroups * kStash * D * 4 : 0;
-    if (kFuse) {
-      static bool attr_set[64];
-      int dev = 0;
-      if (cudaGetDevice(&dev) == cudaSuccess && dev >= 0 && dev < 64 && !attr_set[dev]) {
-        cudaFuncSetAttribute(window_reduce_kernel<G, NV, kFuse>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             65536);   // kGroups * kStash * (4G floats) * 4 bytes for every G
-        attr_set[dev] = true;
-      }
-    }
-    window_reduce_kernel<G, NV, kFuse><<<blocks, 256, smem, st>>>(
+    window_reduce_kernel<G, NV><<<blocks, 256, 0, st>>>(
         keys, reinterpret_cast<int32_t*>(ws + p.off_sbag), reinterpret_cast<int32_t*>(ws + p.off_uidx), p.L, sentinel, N, D,
-        B, grad, ld_grad, col0, gsum, partial, long_list, scalars, p.nwin, (int64_t)umax, d_status, tables, row_state, lr,
-        eps);
+        B, grad, ld_grad, col0, gsum, partial, long_list, scalars, p.nwin, (int64_t)umax, d_status);
   }
   {
     SS_TIMED("combine_rows_kernel", st);
