@@ -34,6 +34,41 @@ METRIC = "training examples/sec at 1 B200 with shadow sync on; sync HBM GB/s vs 
 UNIT = "examples/s"
 RING = 8            # pre-generated batches per replica, cycled through
 
+# DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum) from one ncu capture of the kernel, valid
+# for the named workload and for exactly the sources whose hashes are listed: once one of them changes the figure is
+# reported as null until the counters are taken again.
+NCU_TRAFFIC = {
+    "gemm_tc_kernel": {
+        "workload": "medium",
+        "bytes_per_launch": 3667904,      # mean over the 12 GEMM launches of a replica step
+        "capture": "profiles/step_medium_top_kernels.md",
+        "sources": {
+            "gemm_tc.cu": "b5bffd890cb45d12702fb5bb1f8241eba14bb7f5385abd222ef7e47c4ee3f121",
+            "mlp.cu": "d19c4b892161d5ed072e508a46f8c87a8581353428f85020fa705df9f385ed89",
+            "gemm.cuh": "da1df6183e23abbd5728584e558625d4dc65d14209886465342899cdf4a7a462",
+            "mlp_plan.cuh": "bc8b0ba72d2a7789979f8bd83bc7a7f74e710c88cebe970199f86206822370c5",
+        },
+    },
+}
+
+
+def ncu_traffic(kernel, workload):
+    """Bytes per launch from the stored ncu capture, or None when it does not cover this kernel, this workload
+    or the current sources."""
+    import hashlib
+    e = NCU_TRAFFIC.get(kernel)
+    if e is None or e["workload"] != workload:
+        return None
+    csrc = os.path.join(os.path.dirname(os.path.abspath(__file__)), "paper_2003_03477_b200", "csrc")
+    for name, want in e["sources"].items():
+        try:
+            with open(os.path.join(csrc, name), "rb") as f:
+                if hashlib.sha256(f.read()).hexdigest() != want:
+                    return None
+        except OSError:
+            return None
+    return e["bytes_per_launch"]
+
 
 def measured_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
@@ -469,7 +504,8 @@ def roofline(kernels, model, host, cfg, peaks):
         achieved = amount / (us_total * 1e-6) / 1e12
         peak, unit = peaks["bf16_tflops_sustained"], "TFLOP/s"
     return {"kernel": name, "bound": bound, "achieved": achieved, "peak": peak, "unit": unit, "frac": achieved / peak,
-            "traffic": None, "peak_source": peaks["source"], "launches_per_replica_step": n_launch,
+            "traffic": ncu_traffic(name, cfg.name), "traffic_unit": "bytes per launch (ncu, DRAM read + write)",
+            "peak_source": peaks["source"], "launches_per_replica_step": n_launch,
             "us_per_launch": k["us_per_launch"], "share_of_kernel_time": k["share"],
             "work_per_replica_step": amount,
             "timing": "CUDA events around every launch on its stream, all replicas training concurrently"}
