@@ -738,7 +738,37 @@ __device__ __forceinline__ void prefetch_l2(const void* p) { asm volatile("prefe
 // of windows in flight on an SM is bounded by registers only.
 constexpr int kWaThreads = 128;
 
-template <int G>
+// Row-wise Adagrad on one row whose gradient is in the lanes' registers, NV float4 per lane (column lane + v*G).
+template <int G, int NV>
+__device__ __forceinline__ void adagrad_row_nv(const float4 (&g)[NV], uint32_t key, int lane, int nvec, int D,
+                                               unsigned gmask, float* __restrict__ tables,
+                                               float* __restrict__ row_state, float lr, float eps) {
+  float4* row = reinterpret_cast<float4*>(tables + (int64_t)key * D);
+  float4 r[NV];
+#pragma unroll
+  for (int v = 0; v < NV; ++v) r[v] = (lane + v * G < nvec) ? row[lane + v * G] : make_float4(0.f, 0.f, 0.f, 0.f);
+  const float st = row_state[key];
+  float ss = 0.f;
+#pragma unroll
+  for (int v = 0; v < NV; ++v) ss += g[v].x * g[v].x + g[v].y * g[v].y + g[v].z * g[v].z + g[v].w * g[v].w;
+#pragma unroll
+  for (int off = G / 2; off >= 1; off >>= 1) ss += __shfl_down_sync(gmask, ss, off, G);
+  ss = __shfl_sync(gmask, ss, 0, G);                       // every lane uses lane 0's sum
+  const float sn = st + ss * (1.0f / (float)D);            // the reciprocal is loop-invariant at the call sites
+  const float scale = __fdividef(lr, sqrtf(sn) + eps);     // within 2 ulp of the quotient
+#pragma unroll
+  for (int v = 0; v < NV; ++v) {
+    if (lane + v * G < nvec) {
+      float4 o = r[v];
+      o.x -= scale * g[v].x; o.y -= scale * g[v].y; o.z -= scale * g[v].z; o.w -= scale * g[v].w;
+      row[lane + v * G] = o;
+    }
+  }
+  __syncwarp(gmask);
+  if (lane == 0) row_state[key] = sn;
+}
+
+template <int G, int NV>
 __global__ void __launch_bounds__(kWaThreads, 8)
 window_apply_kernel(const uint32_t* __restrict__ keys, const int32_t* __restrict__ sbag,
                     const int32_t* __restrict__ uidx, int64_t L, uint32_t sentinel, int64_t N, int D, int B,
@@ -801,33 +831,44 @@ window_apply_kernel(const uint32_t* __restrict__ keys, const int32_t* __restrict
   const bool last_open = (vm >> (kWin - 1) & 1u) && s_key[grp][kWin + 1] == s_key[grp][kWin];
   const float4* grad4 = reinterpret_cast<const float4*>(grad + col0);  // col0 is a multiple of 4
 
-  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-  constexpr int kBatch = 8;                                // gradient rows in flight per lane
+  float4 acc[NV];
+#pragma unroll
+  for (int v = 0; v < NV; ++v) acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
+  constexpr int kBatch = 8 / NV;                           // gradient rows in flight per lane (8 float4)
 #pragma unroll
   for (int i0 = 0; i0 < kWin; i0 += kBatch) {
-    float4 gv[kBatch];
+    float4 gv[kBatch][NV];
 #pragma unroll
     for (int u = 0; u < kBatch; ++u) {
       const int32_t row = s_row[grp][i0 + u];
-      gv[u] = (row >= 0 && lane < nvec) ? __ldg(grad4 + row + lane) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+      for (int v = 0; v < NV; ++v) {
+        const int c = lane + v * G;
+        gv[u][v] = (row >= 0 && c < nvec) ? __ldg(grad4 + row + c) : make_float4(0.f, 0.f, 0.f, 0.f);
+      }
     }
 #pragma unroll
     for (int u = 0; u < kBatch; ++u) {
       const int i = i0 + u;
-      if ((hm >> i) & 1u) acc = make_float4(0.f, 0.f, 0.f, 0.f);
-      acc = add4(acc, gv[u]);                              // skipped lookups carry zeros and follow every run
+#pragma unroll
+      for (int v = 0; v < NV; ++v) {
+        if ((hm >> i) & 1u) acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
+        acc[v] = add4(acc[v], gv[u][v]);                   // skipped lookups carry zeros and follow every run
+      }
       if ((tm >> i) & 1u) {
         const uint32_t key = s_key[grp][1 + i];
         const bool first = (tm & ((1u << i) - 1u)) == 0u;  // the window's first run holds position 0
         const bool head_open = first && first_open;
         const bool tail_open = (i == kWin - 1) && last_open;
         if (!head_open && !tail_open) {
-          adagrad_one_row<G>(acc, key, lane, nvec, D, gmask, tables, row_state, lr, eps);
+          adagrad_row_nv<G, NV>(acc, key, lane, nvec, D, gmask, tables, row_state, lr, eps);
         } else {
           // the run goes on in a neighbouring window: its part goes to the window's partial slot
           // (slot 0 when the run holds the window's first position), the combine kernel adds the parts
           float4* dst = reinterpret_cast<float4*>(partial + ((int64_t)win * 2 + (first ? 0 : 1)) * D);
-          if (lane < nvec) dst[lane] = acc;
+#pragma unroll
+          for (int v = 0; v < NV; ++v)
+            if (lane + v * G < nvec) dst[lane + v * G] = acc[v];
           if (!head_open && lane == 0) {                   // the window in which a multi-window run starts lists the row
             const int slot = atomicAdd(&scalars[1], 1);
             if (slot < nwin) long_list[slot] = s_u[grp][i];   // at most one such run per window
@@ -1073,9 +1114,11 @@ static void launch_reduce(const BwdPlan& p, char* ws, const uint32_t* keys, cons
   // the list of rows crossing window edges starts empty (the apply half may be repeated on one sort)
   cudaMemsetAsync(scalars + 1, 0, sizeof(int32_t), st);
   if (kFuse) {
-    constexpr int kWaGroups = kWaThreads / G;
+    // two float4 per lane (half as many lanes per window) wherever the row has at least eight
+    constexpr int WG = G >= 8 ? G / 2 : G, WNV = G >= 8 ? 2 : 1;
+    constexpr int kWaGroups = kWaThreads / WG;
     SS_TIMED("window_apply_kernel", st);
-    window_apply_kernel<G><<<(unsigned)((p.nwin + kWaGroups - 1) / kWaGroups), kWaThreads, 0, st>>>(
+    window_apply_kernel<WG, WNV><<<(unsigned)((p.nwin + kWaGroups - 1) / kWaGroups), kWaThreads, 0, st>>>(
         keys, reinterpret_cast<int32_t*>(ws + p.off_sbag), reinterpret_cast<int32_t*>(ws + p.off_uidx), p.L, sentinel,
         N, D, B, grad, ld_grad, col0, partial, long_list, scalars, p.nwin, (int64_t)umax, d_status, tables, row_state,
         lr, eps);
