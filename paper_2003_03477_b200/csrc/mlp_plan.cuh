@@ -71,8 +71,9 @@ inline ss_status make_mlp_plan(const ss_mlp_desc* d, int B, MlpPlan* p) {
   red_total += (size_t)p->layer[p->nl - 1].in;
   if (p->layer[0].in <= 16) red_total += (size_t)p->layer[0].in * p->layer[0].out;
   p->red_partial = take(red_total * 4 * (size_t)p->red_splits);
-  // weight-gradient GEMMs contract over the batch and have small outputs: cut K so that about one
-  // wave of CTAs works on each of them; the slices are added in order by the update kernel
+  // weight-gradient GEMMs contract over the batch and have small outputs: cut K into a few slices so that
+  // more CTAs work on each of them (measured on the 2048-sample step: 2 slices beat both 1 and 4..16 in
+  // whole-step throughput); the slices are added in order by the update kernel
   int64_t gp = 0;
   const int nk = (B + 63) / 64;
   for (int l = 0; l < p->nl; ++l) {
@@ -82,6 +83,7 @@ inline ss_status make_mlp_plan(const ss_mlp_desc* d, int B, MlpPlan* p) {
       const int tiles = ((L.out + 127) / 128) * ((L.in + 127) / 128);
       s = (148 + tiles - 1) / tiles;
       if (s > 16) s = 16;
+      if (s > nk / 16) s = nk / 16;                        // slices of at least 16 k-steps: a CTA's fixed cost outweighs shorter ones
       if (s > nk) s = nk;
       if (s < 1) s = 1;
     }
