@@ -41,6 +41,16 @@ bool gemm_tc_eligible(int M, int N, int K, const Operand& A, const Operand& B, c
 // out_lo + z * split_stride (plain stores only: no bias, ReLU, mask or bf16 output); the caller adds the slices.
 ss_status gemm_tc(int M, int N, int K, const Operand& A, const Operand& B, const Epilogue& ep, cudaStream_t st,
                   int k_splits, int64_t split_stride);
+// Several independent products (each eligible for gemm_tc, at most kTcMaxGroup) in ONE launch of 128 x 128 tiles.
+constexpr int kTcMaxGroup = 4;
+struct TcJob {
+  int M, N, K;
+  Operand A, B;
+  Epilogue ep;
+  int k_splits;
+  int64_t split_stride;
+};
+ss_status gemm_tc_group(const TcJob* jobs, int n, cudaStream_t st);
 // Tensor cores when eligible, SIMT otherwise.
 ss_status gemm(int M, int N, int K, const Operand& A, const Operand& B, const Epilogue& ep, cudaStream_t st);
 // The device error flag raised by a bounded wait that ran out (0 = none); synchronises the device.

@@ -2,7 +2,9 @@
 //
 //   C[m, n] = sum_k A(m, k) * B(n, k)
 //
-// One CTA computes a 128 x 128 (or, for large products, 128 x 256) tile.  Warp 0 (one lane) streams 128 x 64 / 64 x 128 operand tiles
+// One CTA computes a 128 x 128 tile (128 x 256 for large products, 128 x 64 for products with too few
+// tiles to occupy the SMs).  One launch may hold several independent products (a group): a CTA finds its
+// product from its block index.  Warp 0 (one lane) streams 128 x 64 / 64 x 128 operand tiles
 // into a ring of shared-memory stages (3 or 6 deep) with TMA (128-byte swizzle); warp 1 (one lane) issues
 // tcgen05.mma (M = 128, N = 128 or 256, K = 16, accumulators in tensor memory) and releases stages with
 // tcgen05.commit; warps 2-5 wait for the accumulator, read it with tcgen05.ld (one row per thread)
@@ -43,10 +45,23 @@ __device__ int g_device_error = 0;   // 0 ok; otherwise the code of the first wa
 struct TcParams {
   int M, N, K;
   int a_mn, b_mn;          // 1 = MN-major operand
-  int k_splits;            // the K range is cut into this many slices (grid.z); slice z writes out_lo + z*split_stride
+  int k_splits;            // the K range is cut into this many slices; slice z writes out_lo + z*split_stride
   int64_t split_stride;    // in floats
   Epilogue ep;
   int* err;
+};
+
+// One product of a launch: its tensor maps, its parameters and its share of the (one-dimensional) grid.
+// CTA `cta_begin + (z * grid_y + y) * grid_x + x` computes tile (row block y, column block x) of K slice z.
+struct TcProblem {
+  CUtensorMap map_a, map_b;
+  TcParams p;
+  int cta_begin, grid_x, grid_y;
+};
+template <int NP>
+struct TcGroup {
+  TcProblem prob[NP];
+  int n;
 };
 
 // ---------------------------------------------------------------------------------------- PTX wrappers
@@ -127,10 +142,22 @@ __device__ __forceinline__ uint32_t pack2(float a, float b) {
 }
 
 // ---------------------------------------------------------------------------------------- kernel
-template <int kStages, int kBN>
+template <int kStages, int kBN, int NP>
 __global__ void __launch_bounds__(kTcThreads, 1)
-gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, TcParams p) {
+gemm_tc_kernel(const __grid_constant__ TcGroup<NP> grp) {
   extern __shared__ uint8_t smem_raw[];
+  int pj = 0;
+  if (NP > 1) {
+    while (pj + 1 < grp.n && (int)blockIdx.x >= grp.prob[pj + 1].cta_begin) ++pj;
+  }
+  const TcProblem& prob = grp.prob[pj];
+  const TcParams& p = prob.p;
+  const CUtensorMap& map_a = prob.map_a;
+  const CUtensorMap& map_b = prob.map_b;
+  const int cta_local = (int)blockIdx.x - prob.cta_begin;
+  const int tile_x = cta_local % prob.grid_x;
+  const int tile_y = (cta_local / prob.grid_x) % prob.grid_y;
+  const int slice_z = cta_local / (prob.grid_x * prob.grid_y);
   constexpr int kStageBytes = stage_bytes(kBN);
   constexpr int kTmemCols = kBN;                           // one fp32 accumulator column per tile column
   const uint32_t raw = smem_u32(smem_raw);
@@ -146,10 +173,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   const uint32_t acc_bar = bar0 + 8u * (2 * kStages);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int m0 = blockIdx.y * kBM, n0 = blockIdx.x * kBN;
+  const int m0 = tile_y * kBM, n0 = tile_x * kBN;
   const int nk_all = (p.K + kBK - 1) / kBK;
-  const int kb_begin = (int)((int64_t)nk_all * blockIdx.z / p.k_splits);
-  const int nk = (int)((int64_t)nk_all * (blockIdx.z + 1) / p.k_splits) - kb_begin;   // >= 1: k_splits <= nk_all
+  const int kb_begin = (int)((int64_t)nk_all * slice_z / p.k_splits);
+  const int nk = (int)((int64_t)nk_all * (slice_z + 1) / p.k_splits) - kb_begin;   // >= 1: k_splits <= nk_all
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) { mbar_init(full(s), 1); mbar_init(empty(s), 1); }
@@ -264,7 +291,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             o.x = pack2(x[0], x[1]); o.y = pack2(x[2], x[3]); o.z = pack2(x[4], x[5]); o.w = pack2(x[6], x[7]);
             *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(ep.out_lo) + m * ep.ld_lo + n) = o;
           } else {
-            float4* o = reinterpret_cast<float4*>(reinterpret_cast<float*>(ep.out_lo) + (int64_t)blockIdx.z * p.split_stride + m * ep.ld_lo + n);
+            float4* o = reinterpret_cast<float4*>(reinterpret_cast<float*>(ep.out_lo) + (int64_t)slice_z * p.split_stride + m * ep.ld_lo + n);
             o[0] = make_float4(x[0], x[1], x[2], x[3]);
             o[1] = make_float4(x[4], x[5], x[6], x[7]);
           }
@@ -343,54 +370,103 @@ bool gemm_tc_eligible(int M, int N, int K, const Operand& A, const Operand& B, c
   return true;
 }
 
-ss_status gemm_tc(int M, int N, int K, const Operand& A, const Operand& B, const Epilogue& ep, cudaStream_t st,
-                  int k_splits, int64_t split_stride) {
+// Tile width and ring depth of a launch.
+enum TcVariant { TC_SMALL = 0, TC_LARGE = 1, TC_WIDE = 2, TC_NARROW = 3 };
+constexpr int kStagesNarrow = 4;   // 128 x 64 tiles: 4 stages of 24 KiB, two CTAs per SM
+
+template <int kStages, int kBN, int NP>
+static ss_status launch_group(const TcGroup<NP>& g, int total_ctas, cudaStream_t st) {
   static bool attr_set[64];
   int dev = 0;
   SS_CUDA(cudaGetDevice(&dev));
   if (dev >= 0 && dev < 64 && !attr_set[dev]) {
-    SS_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<kStagesSmall, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)tc_smem_bytes(kStagesSmall, 128)));
-    SS_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<kStagesLarge, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)tc_smem_bytes(kStagesLarge, 128)));
-    SS_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<kStagesWide, 256>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)tc_smem_bytes(kStagesWide, 256)));
+    SS_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<kStages, kBN, NP>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)tc_smem_bytes(kStages, kBN)));
     attr_set[dev] = true;
   }
-  TcParams p;
-  p.M = M; p.N = N; p.K = K;
-  p.a_mn = (A.s_k != 1);
-  p.b_mn = (B.s_k != 1);
-  const int nk_all = (K + kBK - 1) / kBK;
-  if (k_splits < 1) k_splits = 1;
-  if (k_splits > nk_all) k_splits = nk_all;
-  if (k_splits > 1 && (ep.lo_bf16 || ep.lo_cols < N || ep.bias || ep.relu || ep.mask)) return SS_ERR_SHAPE;   // slices are plain fp32 sums
-  p.k_splits = k_splits;
-  p.split_stride = split_stride;
-  p.ep = ep;
-  p.err = device_error_ptr();
-  if (!p.err) return SS_ERR_CUDA;
-  alignas(64) CUtensorMap ma, mb;
-  const bool oka = p.a_mn ? make_map(&ma, A.p, M, K, A.s_k, 64, 64) : make_map(&ma, A.p, K, M, A.s_row, 64, kBM);
-  const int nk_all2 = (K + kBK - 1) / kBK;
-  const int nk_slice = (nk_all2 + k_splits - 1) / k_splits;
-  const long long ctas128 = (long long)((N + 127) / 128) * ((M + kBM - 1) / kBM) * k_splits;
-  const long long ctas256 = (long long)((N + 255) / 256) * ((M + kBM - 1) / kBM) * k_splits;
-  const bool wide = N >= 256 && ctas256 >= 2ll * num_sms() && nk_slice >= 2 * kStagesWide;
-  const int bn = wide ? 256 : 128;
-  const bool okb = p.b_mn ? make_map(&mb, B.p, N, K, B.s_k, 64, 64) : make_map(&mb, B.p, K, N, B.s_row, 64, bn);
-  if (!oka || !okb) return SS_ERR_CUDA;
-  dim3 grid((N + bn - 1) / bn, (M + kBM - 1) / kBM, k_splits);
   { SS_TIMED("gemm_tc_kernel", st);
-  if (wide)
-    gemm_tc_kernel<kStagesWide, 256><<<grid, kTcThreads, tc_smem_bytes(kStagesWide, 256), st>>>(ma, mb, p);
-  else if (ctas128 >= 2ll * num_sms() && nk_slice >= 2 * kStagesLarge)
-    gemm_tc_kernel<kStagesLarge, 128><<<grid, kTcThreads, tc_smem_bytes(kStagesLarge, 128), st>>>(ma, mb, p);
-  else
-    gemm_tc_kernel<kStagesSmall, 128><<<grid, kTcThreads, tc_smem_bytes(kStagesSmall, 128), st>>>(ma, mb, p);
+  gemm_tc_kernel<kStages, kBN, NP><<<total_ctas, kTcThreads, tc_smem_bytes(kStages, kBN), st>>>(g);
   }
   SS_LAUNCH_OK();
   return SS_OK;
+}
+
+// Fills one problem of a group for tile width bn; returns its CTA count (0 on failure).
+static int fill_problem(TcProblem* pr, const TcJob& j, int bn, int cta_begin, int* err) {
+  TcParams& p = pr->p;
+  p.M = j.M; p.N = j.N; p.K = j.K;
+  p.a_mn = (j.A.s_k != 1);
+  p.b_mn = (j.B.s_k != 1);
+  const int nk_all = (j.K + kBK - 1) / kBK;
+  int ks = j.k_splits < 1 ? 1 : j.k_splits;
+  if (ks > nk_all) ks = nk_all;
+  p.k_splits = ks;
+  p.split_stride = j.split_stride;
+  p.ep = j.ep;
+  p.err = err;
+  const bool oka = p.a_mn ? make_map(&pr->map_a, j.A.p, j.M, j.K, j.A.s_k, 64, 64)
+                          : make_map(&pr->map_a, j.A.p, j.K, j.M, j.A.s_row, 64, kBM);
+  const bool okb = p.b_mn ? make_map(&pr->map_b, j.B.p, j.N, j.K, j.B.s_k, 64, 64)
+                          : make_map(&pr->map_b, j.B.p, j.K, j.N, j.B.s_row, 64, bn);
+  if (!oka || !okb) return 0;
+  pr->cta_begin = cta_begin;
+  pr->grid_x = (j.N + bn - 1) / bn;
+  pr->grid_y = (j.M + kBM - 1) / kBM;
+  return pr->grid_x * pr->grid_y * ks;
+}
+
+static bool splits_ok(const TcJob& j) {
+  const Epilogue& ep = j.ep;                 // slices are plain fp32 sums
+  return j.k_splits <= 1 || !(ep.lo_bf16 || ep.lo_cols < j.N || ep.bias || ep.relu || ep.mask);
+}
+
+ss_status gemm_tc_group(const TcJob* jobs, int n, cudaStream_t st) {
+  if (n < 1 || n > kTcMaxGroup) return SS_ERR_SHAPE;
+  for (int i = 0; i < n; ++i)
+    if (!splits_ok(jobs[i])) return SS_ERR_SHAPE;
+  int* err = device_error_ptr();
+  if (!err) return SS_ERR_CUDA;
+  if (n == 1) {
+    const TcJob& j = jobs[0];
+    const int nk_all = (j.K + kBK - 1) / kBK;
+    int ks = j.k_splits < 1 ? 1 : j.k_splits;
+    if (ks > nk_all) ks = nk_all;
+    const int nk_slice = (nk_all + ks - 1) / ks;
+    const long long mt = (j.M + kBM - 1) / kBM;
+    const long long ctas128 = (long long)((j.N + 127) / 128) * mt * ks;
+    const long long ctas256 = (long long)((j.N + 255) / 256) * mt * ks;
+    int variant = TC_SMALL;
+    if (j.N >= 256 && ctas256 >= 2ll * num_sms() && nk_slice >= 2 * kStagesWide) variant = TC_WIDE;
+    else if (ctas128 >= 2ll * num_sms() && nk_slice >= 2 * kStagesLarge) variant = TC_LARGE;
+    else if (j.N <= 64 || 2 * ctas128 <= num_sms()) variant = TC_NARROW;    // a narrow product, or too few 128-wide tiles to occupy the SMs
+    const int bn = variant == TC_WIDE ? 256 : (variant == TC_NARROW ? 64 : 128);
+    alignas(64) TcGroup<1> g;
+    g.n = 1;
+    const int ctas = fill_problem(&g.prob[0], j, bn, 0, err);
+    if (ctas < 1) return SS_ERR_CUDA;
+    switch (variant) {
+      case TC_WIDE: return launch_group<kStagesWide, 256, 1>(g, ctas, st);
+      case TC_LARGE: return launch_group<kStagesLarge, 128, 1>(g, ctas, st);
+      case TC_NARROW: return launch_group<kStagesNarrow, 64, 1>(g, ctas, st);
+      default: return launch_group<kStagesSmall, 128, 1>(g, ctas, st);
+    }
+  }
+  alignas(64) TcGroup<kTcMaxGroup> g;
+  g.n = n;
+  int total = 0;
+  for (int i = 0; i < n; ++i) {
+    const int ctas = fill_problem(&g.prob[i], jobs[i], 128, total, err);
+    if (ctas < 1) return SS_ERR_CUDA;
+    total += ctas;
+  }
+  for (int i = n; i < kTcMaxGroup; ++i) g.prob[i] = g.prob[n - 1];   // never selected; keeps the parameter block defined
+  return launch_group<kStagesSmall, 128, kTcMaxGroup>(g, total, st);
+}
+
+ss_status gemm_tc(int M, int N, int K, const Operand& A, const Operand& B, const Epilogue& ep, cudaStream_t st,
+                  int k_splits, int64_t split_stride) {
+  TcJob j{M, N, K, A, B, ep, k_splits, split_stride};
+  return gemm_tc_group(&j, 1, st);
 }
 
 int read_device_error(bool clear) {

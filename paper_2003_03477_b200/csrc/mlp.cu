@@ -379,6 +379,8 @@ ss_status ss_mlp_bwd(const ss_mlp_desc* desc, float* w, void* w_bf16, float* ada
     jobs.total += ncols * s_cols;
   };
 
+  TcJob dw_jobs[kMaxLayers];
+  int n_dw = 0;
   for (int l = last; l >= 0; --l) {
     const LayerInfo& L = p.layer[l];
     const void* G = ws + p.dact[l];
@@ -398,12 +400,20 @@ ss_status ss_mlp_bwd(const ss_mlp_desc* desc, float* w, void* w_bf16, float* ada
       Operand A{G, act_kind, 1, L.out};
       Epilogue ep;
       ep.out_lo = g + L.w_off; ep.lo_bf16 = 0; ep.ld_lo = L.in; ep.lo_cols = L.in;
-      if (p.k_splits[l] > 1 && gemm_tc_eligible(L.out, L.in, B, A, X, ep)) {
-        // K = batch cut into slices; the update kernel adds them in slice order
+      if (gemm_tc_eligible(L.out, L.in, B, A, X, ep)) {
+        // Nothing on the way back needs dW, so the weight-gradient products of all layers wait and go out
+        // together as one launch after the last input gradient.  K = batch may be cut into slices; the
+        // update kernel adds them in slice order.
         const int64_t size = (int64_t)L.in * L.out;
-        ep.out_lo = gpart + p.gpart_off[l];
-        st = gemm_tc(L.out, L.in, B, A, X, ep, cs, p.k_splits[l], size);
-        add_range(L.w_off, size, GRAD_SLICES, p.gpart_off[l], size, p.k_splits[l]);
+        const int ks = p.k_splits[l];
+        if (ks > 1) {
+          ep.out_lo = gpart + p.gpart_off[l];
+          add_range(L.w_off, size, GRAD_SLICES, p.gpart_off[l], size, ks);
+        } else {
+          add_range(L.w_off, size, GRAD_FLAT, 0, 0, 1);
+        }
+        if (n_dw == kMaxLayers) return SS_ERR_SHAPE;
+        dw_jobs[n_dw++] = TcJob{L.out, L.in, B, A, X, ep, ks, size};
       } else {
         st = gemm(L.out, L.in, B, A, X, ep, cs);
         add_range(L.w_off, (int64_t)L.in * L.out, GRAD_FLAT, 0, 0, 1);
@@ -438,6 +448,10 @@ ss_status ss_mlp_bwd(const ss_mlp_desc* desc, float* w, void* w_bf16, float* ada
       st = gemm(B, L.in, L.out, A, Wt, ep, cs);
       if (st != SS_OK) return st;
     }
+  }
+  for (int i = 0; i < n_dw; i += kTcMaxGroup) {
+    st = gemm_tc_group(dw_jobs + i, n_dw - i < kTcMaxGroup ? n_dw - i : kTcMaxGroup, cs);
+    if (st != SS_OK) return st;
   }
   {
     // all batch reductions of the pass in one launch; the update kernel adds the batch slices
