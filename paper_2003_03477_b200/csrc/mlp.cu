@@ -68,11 +68,42 @@ __device__ __forceinline__ float load_kind(const void* p, int kind, int64_t i) {
 }
 
 constexpr int kRedRows = 256;     // most rows of the batch a block takes (bounds the staged S tile)
+constexpr int kRedWide = 256;     // columns per block of a job without a second factor matrix (s_cols = 1)
+
+// Eight consecutive elements M[row, c .. c+7] as floats; elements at or beyond ncols read as zero.  One
+// 128-bit load (bf16) or two (float) when the address allows it, element loads otherwise.
+__device__ __forceinline__ void load8_kind(const void* p, int kind, int64_t row, int64_t ld, int c, int ncols, bool vec_ok,
+                                           float (&v)[8]) {
+  if (vec_ok && c + 8 <= ncols) {
+    if (kind == OP_BF16) {
+      const uint4 q = *reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(p) + row * ld + c);
+      const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        v[2 * j] = __uint_as_float(w[j] << 16);                // a bf16 is the upper half of a float
+        v[2 * j + 1] = __uint_as_float(w[j] & 0xFFFF0000u);
+      }
+    } else {
+      const float4* q = reinterpret_cast<const float4*>(reinterpret_cast<const float*>(p) + row * ld + c);
+      const float4 a = q[0], b = q[1];
+      v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w; v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+      if (kind == OP_F32_ROUND_BF16) {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) v[j] = __bfloat162float(__float2bfloat16_rn(v[j]));
+      }
+    }
+  } else {
+#pragma unroll
+    for (int j = 0; j < 8; ++j) v[j] = (c + j < ncols) ? load_kind(p, kind, row * ld + c + j) : 0.f;
+  }
+}
 
 __global__ void __launch_bounds__(256)
 batch_reduce_partial_kernel(const __grid_constant__ RedJobs jobs, int B, int rows_per_split, float* __restrict__ partial) {
-  __shared__ float part[8][32][kMaxSCols + 1];
-  __shared__ __align__(16) float s_tile[kRedRows * kMaxSCols];   // S rows of this block's batch slice, as float
+  // S rows of this block's batch slice, as float; then the row groups' sums (8 x 256 or 8 x 32 x 17 floats)
+  constexpr int kPartFloats = 8 * 32 * (kMaxSCols + 1);
+  static_assert(kPartFloats >= kRedRows * kMaxSCols && kPartFloats >= 8 * kRedWide, "one buffer serves all three uses");
+  __shared__ __align__(16) float s_tile[kPartFloats];
   __shared__ RedJob s_job;
   if (threadIdx.x == 0) {
     int j = 0;
@@ -82,19 +113,71 @@ batch_reduce_partial_kernel(const __grid_constant__ RedJobs jobs, int B, int row
   __syncthreads();
   const RedJob J = s_job;                                    // the job's fields in registers
   const int cx = threadIdx.x & 31, ry = threadIdx.x >> 5;
-  const int c = ((int)blockIdx.x - J.tile0) * 32 + cx;
   const int sc = J.s_cols;
   const int r0 = blockIdx.y * rows_per_split;
   const int r1 = min(B, r0 + rows_per_split);
   const int nrows = r1 - r0;
-  if (J.S != nullptr) {
-    // S rows as float, padded with zeros to kMaxSCols columns so that the inner product needs no column test
-    for (int i = threadIdx.x; i < nrows * kMaxSCols; i += 256) {
-      const int rr = i / kMaxSCols, q = i % kMaxSCols;
-      s_tile[i] = q < sc ? load_kind(J.S, J.s_kind, (int64_t)(r0 + rr) * J.lds + q) : 0.f;
+
+  if (sc == 1) {
+    // ---- no second factor, or a single column of one (S[b]): a warp reads 256 consecutive columns of a row,
+    // eight per lane; warp ry adds rows ry, ry+8, ... in ascending order, then the eight warps are added in order.
+    const int c = ((int)blockIdx.x - J.tile0) * kRedWide + 8 * cx;
+    const bool vec_ok = J.m_kind == OP_BF16 ? ((J.ldm & 7) == 0 && (reinterpret_cast<uintptr_t>(J.M) & 15u) == 0)
+                                            : ((J.ldm & 3) == 0 && (reinterpret_cast<uintptr_t>(J.M) & 15u) == 0);
+    float acc[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) acc[j] = 0.f;
+    if (c < J.ncols) {
+      for (int rr = ry; rr < nrows; rr += 32) {
+        float m[4][8], sv[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {                          // four rows in flight per thread
+          const int r = rr + 8 * u;
+          if (r < nrows) {
+            load8_kind(J.M, J.m_kind, r0 + r, J.ldm, c, J.ncols, vec_ok, m[u]);
+            sv[u] = J.S ? load_kind(J.S, J.s_kind, (int64_t)(r0 + r) * J.lds) : 1.f;
+          } else {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) m[u][j] = 0.f;
+            sv[u] = 0.f;
+          }
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          if (J.S) {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) acc[j] = fmaf(m[u][j], sv[u], acc[j]);
+          } else {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) acc[j] += m[u][j];
+          }
+        }
+      }
     }
+    float* part = s_tile;                                      // [8][256]
+    float4* pw = reinterpret_cast<float4*>(part + ry * kRedWide + 8 * cx);
+    pw[0] = make_float4(acc[0], acc[1], acc[2], acc[3]);
+    pw[1] = make_float4(acc[4], acc[5], acc[6], acc[7]);
     __syncthreads();
+    const int co = ((int)blockIdx.x - J.tile0) * kRedWide + (int)threadIdx.x;
+    if (co < J.ncols) {
+      float t = 0.f;
+#pragma unroll
+      for (int r = 0; r < 8; ++r) t += part[r * kRedWide + threadIdx.x];
+      partial[(int64_t)blockIdx.y * jobs.total + J.part_off + co] = t;
+    }
+    return;
   }
+
+  // ---- a second factor with several columns (the layer with few inputs): 32 columns c per block, each thread
+  // keeps one sum per column of S
+  const int c = ((int)blockIdx.x - J.tile0) * 32 + cx;
+  // S rows as float, padded with zeros to kMaxSCols columns so that the inner product needs no column test
+  for (int i = threadIdx.x; i < nrows * kMaxSCols; i += 256) {
+    const int rr = i / kMaxSCols, q = i % kMaxSCols;
+    s_tile[i] = q < sc ? load_kind(J.S, J.s_kind, (int64_t)(r0 + rr) * J.lds + q) : 0.f;
+  }
+  __syncthreads();
   float acc[kMaxSCols];
 #pragma unroll
   for (int q = 0; q < kMaxSCols; ++q) acc[q] = 0.f;
@@ -105,31 +188,24 @@ batch_reduce_partial_kernel(const __grid_constant__ RedJobs jobs, int B, int row
 #pragma unroll
       for (int u = 0; u < 4; ++u)
         m[u] = (rr + 8 * u < nrows) ? load_kind(J.M, J.m_kind, (int64_t)(r0 + rr + 8 * u) * J.ldm + c) : 0.f;
-      if (J.S == nullptr) {
 #pragma unroll
-        for (int u = 0; u < 4; ++u) acc[0] += m[u];
-      } else if (sc == 1) {
+      for (int u = 0; u < 4; ++u) {
+        if (rr + 8 * u < nrows) {
+          const float4* srow = reinterpret_cast<const float4*>(s_tile + (rr + 8 * u) * kMaxSCols);
 #pragma unroll
-        for (int u = 0; u < 4; ++u)
-          if (rr + 8 * u < nrows) acc[0] = fmaf(m[u], s_tile[(rr + 8 * u) * kMaxSCols], acc[0]);
-      } else {
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-          if (rr + 8 * u < nrows) {
-            const float4* srow = reinterpret_cast<const float4*>(s_tile + (rr + 8 * u) * kMaxSCols);
-#pragma unroll
-            for (int q4 = 0; q4 < kMaxSCols / 4; ++q4) {
-              const float4 sv = srow[q4];                    // one 128-bit broadcast read for four columns
-              acc[4 * q4 + 0] = fmaf(m[u], sv.x, acc[4 * q4 + 0]);
-              acc[4 * q4 + 1] = fmaf(m[u], sv.y, acc[4 * q4 + 1]);
-              acc[4 * q4 + 2] = fmaf(m[u], sv.z, acc[4 * q4 + 2]);
-              acc[4 * q4 + 3] = fmaf(m[u], sv.w, acc[4 * q4 + 3]);
-            }
+          for (int q4 = 0; q4 < kMaxSCols / 4; ++q4) {
+            const float4 sv = srow[q4];                    // one 128-bit broadcast read for four columns
+            acc[4 * q4 + 0] = fmaf(m[u], sv.x, acc[4 * q4 + 0]);
+            acc[4 * q4 + 1] = fmaf(m[u], sv.y, acc[4 * q4 + 1]);
+            acc[4 * q4 + 2] = fmaf(m[u], sv.z, acc[4 * q4 + 2]);
+            acc[4 * q4 + 3] = fmaf(m[u], sv.w, acc[4 * q4 + 3]);
           }
         }
       }
     }
   }
+  __syncthreads();                                           // the S tile is no longer read
+  float (*part)[32][kMaxSCols + 1] = reinterpret_cast<float (*)[32][kMaxSCols + 1]>(s_tile);   // [8][32][17]
 #pragma unroll
   for (int q = 0; q < kMaxSCols; ++q) part[ry][cx][q] = acc[q];
   __syncthreads();
@@ -158,17 +234,48 @@ rowdot_kernel(const void* __restrict__ X, int x_kind, int64_t ldx, const void* _
   if (lane == 0) logit[b] = s + bias[0];
 }
 
-// dX[b, k] = dz[b] * w[k], gated by X[b, k] > 0 (the backward of the single-logit layer).
+// The backward of the single-logit layer with the loss gradient folded in:
+//   dz[b] = (prob[b] - y[b]) / B   (rounded to bf16 in bf16 mode, and stored: the reductions read it)
+//   dX[b, k] = dz[b] * w[k], gated by X[b, k] > 0.
+// One thread per eight consecutive k of a row (K is a multiple of 8: hidden widths are).
+template <bool BF16>
 __global__ void __launch_bounds__(256)
-outer_mask_kernel(const void* __restrict__ dz, const void* __restrict__ w, const void* __restrict__ X, int kind_dz,
-                  int kind_w, int kind_x, int B, int K, void* __restrict__ dX, int out_bf16) {
+dz_outer_mask_kernel(const float* __restrict__ prob, const float* __restrict__ labels, const void* __restrict__ w,
+                     const void* __restrict__ X, int B, int K, void* __restrict__ dz, void* __restrict__ dX) {
+  const int kc = K >> 3;
   const int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x;
-  if (i >= (int64_t)B * K) return;
-  const int b = (int)(i / K), k = (int)(i - (int64_t)b * K);
-  float v = load_kind(dz, kind_dz, b) * load_kind(w, kind_w, k);
-  if (!(load_kind(X, kind_x, i) > 0.f)) v = 0.f;
-  if (out_bf16) reinterpret_cast<__nv_bfloat16*>(dX)[i] = __float2bfloat16_rn(v);
-  else reinterpret_cast<float*>(dX)[i] = v;
+  if (i >= (int64_t)B * kc) return;
+  const int b = (int)(i / kc), c = (int)(i - (int64_t)b * kc) * 8;
+  float d = (prob[b] - labels[b]) / (float)B;
+  if (BF16) {
+    const __nv_bfloat16 dh = __float2bfloat16_rn(d);
+    d = __bfloat162float(dh);
+    if (c == 0) reinterpret_cast<__nv_bfloat16*>(dz)[b] = dh;
+    const uint4 xq = *reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(X) + (int64_t)b * K + c);
+    const uint4 wq = *reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(w) + c);
+    const uint32_t xw[4] = {xq.x, xq.y, xq.z, xq.w}, ww[4] = {wq.x, wq.y, wq.z, wq.w};
+    uint32_t o[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const float x0 = __uint_as_float(xw[j] << 16), x1 = __uint_as_float(xw[j] & 0xFFFF0000u);
+      const float w0 = __uint_as_float(ww[j] << 16), w1 = __uint_as_float(ww[j] & 0xFFFF0000u);
+      const float v0 = x0 > 0.f ? d * w0 : 0.f, v1 = x1 > 0.f ? d * w1 : 0.f;
+      __nv_bfloat162 h = __floats2bfloat162_rn(v0, v1);
+      o[j] = *reinterpret_cast<uint32_t*>(&h);
+    }
+    *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(dX) + (int64_t)b * K + c) = make_uint4(o[0], o[1], o[2], o[3]);
+  } else {
+    if (c == 0) reinterpret_cast<float*>(dz)[b] = d;
+    const float4* xq = reinterpret_cast<const float4*>(reinterpret_cast<const float*>(X) + (int64_t)b * K + c);
+    const float4* wq = reinterpret_cast<const float4*>(reinterpret_cast<const float*>(w) + c);
+    float4* oq = reinterpret_cast<float4*>(reinterpret_cast<float*>(dX) + (int64_t)b * K + c);
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      const float4 x = xq[h], ww = wq[h];
+      oq[h] = make_float4(x.x > 0.f ? d * ww.x : 0.f, x.y > 0.f ? d * ww.y : 0.f, x.z > 0.f ? d * ww.z : 0.f,
+                          x.w > 0.f ? d * ww.w : 0.f);
+    }
+  }
 }
 
 // Where the gradient of each parameter tensor is found when the update kernel runs.
@@ -187,12 +294,12 @@ struct GradTable {
 // Element-wise Adagrad over the flat parameter vector; refreshes the bf16 mirror.  The slices of a
 // gradient are added in slice order.  A zero gradient (pads, dead units) leaves the element
 // untouched.  g_out (nullable, may alias g) receives the assembled gradient.
-__global__ void __launch_bounds__(256)
-adagrad_kernel(float* __restrict__ w, float* __restrict__ acc, const float* g, const float* __restrict__ gpart,
-               const float* __restrict__ bpart, const __grid_constant__ GradTable tab,
-               __nv_bfloat16* __restrict__ mirror, int64_t n4, float lr, float eps, float* g_out, int apply) {
-  const int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x;
-  if (i >= n4) return;
+// A thread owns two float4 positions, 256 apart; the parameter and accumulator loads of both go out
+// before the gradient is looked up, so one round of memory latency covers all of a thread's loads.
+constexpr int kAdaPerThread = 2;
+
+__device__ __forceinline__ float4 assemble_grad(const GradTable& tab, int64_t i, const float* g, const float* __restrict__ gpart,
+                                                const float* __restrict__ bpart) {
   const int64_t e = i * 4;
   float4 gv = make_float4(0.f, 0.f, 0.f, 0.f);
   for (int t = 0; t < tab.n; ++t) {
@@ -202,10 +309,17 @@ adagrad_kernel(float* __restrict__ w, float* __restrict__ acc, const float* g, c
         gv = reinterpret_cast<const float4*>(g)[i];
       } else if (tab.kind[t] == GRAD_SLICES) {               // sizes are multiples of 8: aligned float4 loads
         const float4* p = reinterpret_cast<const float4*>(gpart + tab.off[t] + rel);
+        const int ns = tab.nsplit[t];
+        const int64_t st4 = tab.stride[t] >> 2;
         gv = p[0];
-        for (int z = 1; z < tab.nsplit[t]; ++z) {
-          const float4 q = p[(int64_t)z * (tab.stride[t] >> 2)];
+        if (ns == 2) {
+          const float4 q = p[st4];
           gv.x += q.x; gv.y += q.y; gv.z += q.z; gv.w += q.w;
+        } else {
+          for (int z = 1; z < ns; ++z) {
+            const float4 q = p[(int64_t)z * st4];
+            gv.x += q.x; gv.y += q.y; gv.z += q.z; gv.w += q.w;
+          }
         }
       } else {                                               // any size: scalar loads, elements past the end stay zero
         const int64_t left = tab.end[t] - e;
@@ -221,25 +335,101 @@ adagrad_kernel(float* __restrict__ w, float* __restrict__ acc, const float* g, c
       break;
     }
   }
-  if (g_out) reinterpret_cast<float4*>(g_out)[i] = gv;
-  if (!apply) return;
-  float4 wv = reinterpret_cast<float4*>(w)[i];
-  float4 av = reinterpret_cast<float4*>(acc)[i];
-#define SS_UPD(F)                                  \
-  if (gv.F != 0.f) {                               \
-    av.F = fmaf(gv.F, gv.F, av.F);                 \
-    wv.F -= lr * gv.F / (sqrtf(av.F) + eps);       \
+  return gv;
+}
+
+__global__ void __launch_bounds__(256)
+adagrad_kernel(float* __restrict__ w, float* __restrict__ acc, const float* g, const float* __restrict__ gpart,
+               const float* __restrict__ bpart, const __grid_constant__ GradTable tab,
+               __nv_bfloat16* __restrict__ mirror, int64_t n4, float lr, float eps, float* g_out, int apply) {
+  const int64_t i0 = (int64_t)blockIdx.x * (256 * kAdaPerThread) + threadIdx.x;
+  float4 wv[kAdaPerThread], av[kAdaPerThread], gv[kAdaPerThread];
+#pragma unroll
+  for (int u = 0; u < kAdaPerThread; ++u) {
+    const int64_t i = i0 + 256 * u;
+    if (apply && i < n4) {
+      wv[u] = reinterpret_cast<float4*>(w)[i];
+      av[u] = reinterpret_cast<float4*>(acc)[i];
+    }
   }
-  SS_UPD(x) SS_UPD(y) SS_UPD(z) SS_UPD(w)
+#pragma unroll
+  for (int u = 0; u < kAdaPerThread; ++u) {
+    const int64_t i = i0 + 256 * u;
+    if (i < n4) gv[u] = assemble_grad(tab, i, g, gpart, bpart);
+  }
+#pragma unroll
+  for (int u = 0; u < kAdaPerThread; ++u) {
+    const int64_t i = i0 + 256 * u;
+    if (i >= n4) continue;
+    if (g_out) reinterpret_cast<float4*>(g_out)[i] = gv[u];
+    if (!apply) continue;
+#define SS_UPD(F)                                        \
+    if (gv[u].F != 0.f) {                                \
+      av[u].F = fmaf(gv[u].F, gv[u].F, av[u].F);         \
+      wv[u].F -= lr * gv[u].F / (sqrtf(av[u].F) + eps);  \
+    }
+    SS_UPD(x) SS_UPD(y) SS_UPD(z) SS_UPD(w)
 #undef SS_UPD
-  reinterpret_cast<float4*>(w)[i] = wv;
-  reinterpret_cast<float4*>(acc)[i] = av;
-  if (mirror) {
-    __nv_bfloat162 lo = __floats2bfloat162_rn(wv.x, wv.y), hi = __floats2bfloat162_rn(wv.z, wv.w);
-    uint2 r;
-    r.x = *reinterpret_cast<uint32_t*>(&lo);
-    r.y = *reinterpret_cast<uint32_t*>(&hi);
-    reinterpret_cast<uint2*>(mirror)[i] = r;
+    reinterpret_cast<float4*>(w)[i] = wv[u];
+    reinterpret_cast<float4*>(acc)[i] = av[u];
+    if (mirror) {
+      __nv_bfloat162 lo = __floats2bfloat162_rn(wv[u].x, wv[u].y), hi = __floats2bfloat162_rn(wv[u].z, wv[u].w);
+      uint2 r;
+      r.x = *reinterpret_cast<uint32_t*>(&lo);
+      r.y = *reinterpret_cast<uint32_t*>(&hi);
+      reinterpret_cast<uint2*>(mirror)[i] = r;
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// The layer that reads the dense features (at most 16 inputs) is no dense contraction either:
+//   Y[b, o] = ReLU( sum_k bf16(x[b, k]) * W[o, k] + bias[o] ),   stored as bf16.
+// The weights sit in shared memory as [k][o]; a thread computes eight consecutive outputs of one
+// sample with fp32 FMAs in ascending k.
+// ---------------------------------------------------------------------------------------------
+constexpr int kFewInputs = 16;
+constexpr int kFirstRows = 16;      // samples per block
+
+__global__ void __launch_bounds__(256)
+few_inputs_layer_kernel(const float* __restrict__ x, int K, const __nv_bfloat16* __restrict__ W, const float* __restrict__ bias,
+                        int relu, int B, int N, __nv_bfloat16* __restrict__ Y, int64_t ldy) {
+  extern __shared__ __align__(16) __nv_bfloat16 s_w[];       // [K][N]
+  for (int i = threadIdx.x; i < K * N; i += 256) {
+    const int o = i / K, k = i - o * K;                      // W is [o][k], read in memory order
+    s_w[k * N + o] = W[i];
+  }
+  __syncthreads();
+  const int nchunk = N >> 3;
+  const int b0 = blockIdx.x * kFirstRows;
+  const int rows = min(kFirstRows, B - b0);
+  for (int item = threadIdx.x; item < rows * nchunk; item += 256) {
+    const int r = item / nchunk, o = (item - r * nchunk) * 8;
+    const float* xr = x + (int64_t)(b0 + r) * K;
+    float acc[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) acc[j] = 0.f;
+    for (int k = 0; k < K; ++k) {
+      const float xv = __bfloat162float(__float2bfloat16_rn(xr[k]));
+      const uint4 q = *reinterpret_cast<const uint4*>(s_w + k * N + o);
+      const uint32_t ww[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        acc[2 * j] = fmaf(xv, __uint_as_float(ww[j] << 16), acc[2 * j]);
+        acc[2 * j + 1] = fmaf(xv, __uint_as_float(ww[j] & 0xFFFF0000u), acc[2 * j + 1]);
+      }
+    }
+    const float4 b0v = reinterpret_cast<const float4*>(bias + o)[0], b1v = reinterpret_cast<const float4*>(bias + o)[1];
+    const float bv[8] = {b0v.x, b0v.y, b0v.z, b0v.w, b1v.x, b1v.y, b1v.z, b1v.w};
+    uint32_t out[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      float v0 = acc[2 * j] + bv[2 * j], v1 = acc[2 * j + 1] + bv[2 * j + 1];
+      if (relu) { v0 = fmaxf(v0, 0.f); v1 = fmaxf(v1, 0.f); }
+      __nv_bfloat162 h = __floats2bfloat162_rn(v0, v1);
+      out[j] = *reinterpret_cast<uint32_t*>(&h);
+    }
+    *reinterpret_cast<uint4*>(Y + (int64_t)(b0 + r) * ldy + o) = make_uint4(out[0], out[1], out[2], out[3]);
   }
 }
 
@@ -320,6 +510,15 @@ ss_status ss_mlp_fwd(const ss_mlp_desc* desc, const float* w, const void* w_bf16
     } else {
       ep.out_lo = ws + p.act[l]; ep.lo_bf16 = p.bf16; ep.ld_lo = L.out;
     }
+    const size_t few_smem = (size_t)L.in * L.out * 2;
+    if (p.bf16 && l == 0 && L.in <= kFewInputs && few_smem <= 48 * 1024 && (ep.ld_lo & 7) == 0 && aligned16(ep.out_lo)) {
+      SS_TIMED("few_inputs_layer_kernel", cs);
+      few_inputs_layer_kernel<<<(B + kFirstRows - 1) / kFirstRows, 256, few_smem, cs>>>(
+          dense, L.in, reinterpret_cast<const __nv_bfloat16*>(w_bf16) + L.w_off, ep.bias, ep.relu, B, L.out,
+          reinterpret_cast<__nv_bfloat16*>(ep.out_lo), ep.ld_lo);
+      SS_LAUNCH_OK();
+      continue;
+    }
     st = gemm(B, L.out, L.in, A, Bm, ep, cs);
     if (st != SS_OK) return st;
   }
@@ -354,8 +553,9 @@ ss_status ss_mlp_bwd(const ss_mlp_desc* desc, float* w, void* w_bf16, float* ada
 
   const int last = p.nl - 1;
   const int dz_kind = p.bf16 ? OP_BF16 : OP_F32;
-  { SS_TIMED("dz_kernel", cs);
-  dz_kernel<<<(B + 255) / 256, 256, 0, cs>>>(prob, labels, B, ws + p.dact[last], p.bf16);
+  if (last == p.nb) {   // a single top layer: its input gradient is a GEMM's; otherwise dz comes out of the fused kernel below
+    SS_TIMED("dz_kernel", cs);
+    dz_kernel<<<(B + 255) / 256, 256, 0, cs>>>(prob, labels, B, ws + p.dact[last], p.bf16);
   }
   SS_LAUNCH_OK();
 
@@ -375,7 +575,7 @@ ss_status ss_mlp_bwd(const ss_mlp_desc* desc, float* w, void* w_bf16, float* ada
     J.M = M; J.m_kind = m_kind; J.ldm = ldm; J.ncols = ncols;
     J.S = S; J.s_kind = s_kind; J.lds = lds; J.s_cols = s_cols;
     J.tile0 = jobs.ntiles; J.part_off = jobs.total; J.out_off = out_off;
-    jobs.ntiles += (ncols + 31) / 32;
+    jobs.ntiles += s_cols == 1 ? (ncols + kRedWide - 1) / kRedWide : (ncols + 31) / 32;
     jobs.total += ncols * s_cols;
   };
 
@@ -424,10 +624,14 @@ ss_status ss_mlp_bwd(const ss_mlp_desc* desc, float* w, void* w_bf16, float* ada
     // dX[b, i] = sum_o G[b, o] * W[o, i], gated by the ReLU of the producing layer
     if (l == last && l != p.nb) {
       const void* wl = p.bf16 ? (const void*)(reinterpret_cast<const __nv_bfloat16*>(w_bf16) + L.w_off) : (const void*)(w + L.w_off);
-      const int64_t cnt = (int64_t)B * L.in;
-      { SS_TIMED("outer_mask_kernel", cs);
-      outer_mask_kernel<<<(unsigned)((cnt + 255) / 256), 256, 0, cs>>>(G, wl, ws + p.act[l - 1], dz_kind, act_kind, act_kind,
-                                                                       B, L.in, ws + p.dact[l - 1], p.bf16);
+      const int64_t cnt = (int64_t)B * (L.in >> 3);            // L.in is a hidden width: a multiple of 8
+      { SS_TIMED("dz_outer_mask_kernel", cs);
+      if (p.bf16)
+        dz_outer_mask_kernel<true><<<(unsigned)((cnt + 255) / 256), 256, 0, cs>>>(prob, labels, wl, ws + p.act[l - 1], B, L.in,
+                                                                                  ws + p.dact[last], ws + p.dact[l - 1]);
+      else
+        dz_outer_mask_kernel<false><<<(unsigned)((cnt + 255) / 256), 256, 0, cs>>>(prob, labels, wl, ws + p.act[l - 1], B, L.in,
+                                                                                   ws + p.dact[last], ws + p.dact[l - 1]);
       }
       SS_LAUNCH_OK();
     } else {
@@ -467,7 +671,7 @@ ss_status ss_mlp_bwd(const ss_mlp_desc* desc, float* w, void* w_bf16, float* ada
                 jobs.total, nsplit);
     const int64_t n4 = p.P / 4;
     SS_TIMED("adagrad_kernel", cs);
-    adagrad_kernel<<<(unsigned)((n4 + 255) / 256), 256, 0, cs>>>(w, adagrad_acc, g, gpart, partial, tab,
+    adagrad_kernel<<<(unsigned)((n4 + 256 * kAdaPerThread - 1) / (256 * kAdaPerThread)), 256, 0, cs>>>(w, adagrad_acc, g, gpart, partial, tab,
                                                                  reinterpret_cast<__nv_bfloat16*>(w_bf16), n4, lr, eps,
                                                                  (grads || !apply_update) ? g : nullptr, apply_update);
     SS_LAUNCH_OK();
