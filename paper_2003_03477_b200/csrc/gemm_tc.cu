@@ -36,6 +36,7 @@ constexpr int kStagesWide = 4;
 constexpr int kTileBytes = kBM * kBK * 2;                 // 16 KiB: the A tile, and every 128 columns of the B tile
 __host__ __device__ constexpr int stage_bytes(int bn) { return kTileBytes + bn * kBK * 2; }
 constexpr int kTcThreads = 192;
+constexpr int kStgLd = 36;                                // floats per row of an epilogue warp's 32 x 32 staging block
 constexpr size_t tc_smem_bytes(int stages, int bn) { return (size_t)stages * stage_bytes(bn) + 1024 /*alignment slack*/ + 256 /*barriers*/; }
 constexpr long long kWaitCycles = 400ll * 1000 * 1000;    // ~0.2 s: far beyond any legitimate wait
 constexpr long long kWaitCyclesAborted = 2ll * 1000 * 1000;
@@ -142,7 +143,7 @@ __device__ __forceinline__ uint32_t pack2(float a, float b) {
 }
 
 // ---------------------------------------------------------------------------------------- kernel
-template <int kStages, int kBN, int NP>
+template <int kStages, int kBN, int NP, bool kDirect>
 __global__ void __launch_bounds__(kTcThreads, 1)
 gemm_tc_kernel(const __grid_constant__ TcGroup<NP> grp) {
   extern __shared__ uint8_t smem_raw[];
@@ -178,11 +179,36 @@ gemm_tc_kernel(const __grid_constant__ TcGroup<NP> grp) {
   const int kb_begin = (int)((int64_t)nk_all * slice_z / p.k_splits);
   const int nk = (int)((int64_t)nk_all * (slice_z + 1) / p.k_splits) - kb_begin;   // >= 1: k_splits <= nk_all
 
+  // one stage of operand tiles for k block kb of this CTA's slice
+  auto load_stage = [&](int kb) {
+    const int s = kb % kStages;
+    mbar_expect_tx(full(s), kStageBytes);
+    const uint32_t sa = tiles + s * kStageBytes, sb = sa + kTileBytes;
+    const int k0 = (kb_begin + kb) * kBK;
+    if (p.a_mn) {                       // A stored [K, M]: two boxes of 64 k-rows x 64 m
+      tma_load_2d(sa, &map_a, full(s), m0, k0);
+      tma_load_2d(sa + kTileBytes / 2, &map_a, full(s), m0 + 64, k0);
+    } else {                            // A stored [M, K]: one box of 128 rows x 64 k
+      tma_load_2d(sa, &map_a, full(s), k0, m0);
+    }
+    if (p.b_mn) {
+#pragma unroll
+      for (int a = 0; a < kBN / 64; ++a) tma_load_2d(sb + a * (kTileBytes / 2), &map_b, full(s), n0 + 64 * a, k0);
+    } else {
+      tma_load_2d(sb, &map_b, full(s), k0, n0);
+    }
+  };
+  const int n_early = nk < kStages ? nk : kStages;           // the ring starts empty: its first round needs no wait
   if (threadIdx.x == 0) {
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_a)) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_b)) : "memory");
     for (int s = 0; s < kStages; ++s) { mbar_init(full(s), 1); mbar_init(empty(s), 1); }
     mbar_init(acc_bar, 1);
     *aborted = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    // the first round of loads goes out before tensor memory is allocated and the warps meet
+    for (int kb = 0; kb < n_early; ++kb) load_stage(kb);
   }
   if (warp == 1) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(kTmemCols) : "memory");
@@ -196,25 +222,11 @@ gemm_tc_kernel(const __grid_constant__ TcGroup<NP> grp) {
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
-      for (int kb = 0; kb < nk; ++kb) {
+      for (int kb = n_early; kb < nk; ++kb) {
         const int s = kb % kStages;
         const uint32_t ph = (kb / kStages) & 1;
-        mbar_wait(empty(s), ph ^ 1u, aborted, p.err, 1);
-        mbar_expect_tx(full(s), kStageBytes);
-        const uint32_t sa = tiles + s * kStageBytes, sb = sa + kTileBytes;
-        const int k0 = (kb_begin + kb) * kBK;
-        if (p.a_mn) {                       // A stored [K, M]: two boxes of 64 k-rows x 64 m
-          tma_load_2d(sa, &map_a, full(s), m0, k0);
-          tma_load_2d(sa + kTileBytes / 2, &map_a, full(s), m0 + 64, k0);
-        } else {                            // A stored [M, K]: one box of 128 rows x 64 k
-          tma_load_2d(sa, &map_a, full(s), k0, m0);
-        }
-        if (p.b_mn) {
-#pragma unroll
-          for (int a = 0; a < kBN / 64; ++a) tma_load_2d(sb + a * (kTileBytes / 2), &map_b, full(s), n0 + 64 * a, k0);
-        } else {
-          tma_load_2d(sb, &map_b, full(s), k0, n0);
-        }
+        if (!mbar_wait(empty(s), ph ^ 1u, aborted, p.err, 1)) break;
+        load_stage(kb);
       }
     }
   } else if (warp == 1) {
@@ -246,60 +258,117 @@ gemm_tc_kernel(const __grid_constant__ TcGroup<NP> grp) {
   } else {
     // ------------------------------------------------------------------ epilogue warps 2..5
     const int q = warp & 3;               // tensor-memory lane quadrant this warp may read
-    const int64_t m = (int64_t)m0 + 32 * q + lane;
-    const bool m_ok = m < p.M;
     const Epilogue& ep = p.ep;
     mbar_wait(acc_bar, 0, aborted, p.err, 3);
     tc_fence_after();
+    if constexpr (kDirect) {
+      // Machine-filling products (their epilogue is a small part of a long CTA): every thread stores the
+      // accumulator row it reads, 32 consecutive columns at a time.
+      const int64_t m = (int64_t)m0 + 32 * q + lane;
+      const bool m_ok = m < p.M;
 #pragma unroll 1
-    for (int c = 0; c < kBN / 32; ++c) {
-      const int nb = n0 + 32 * c;
-      if (nb >= p.N) break;
-      uint32_t r[32];
-      tc_ld32(tmem + ((uint32_t)(32 * q) << 16) + (uint32_t)(32 * c), r);
-      float v[32];
+      for (int c = 0; c < kBN / 32; ++c) {
+        const int nb = n0 + 32 * c;
+        if (nb >= p.N) break;
+        uint32_t r[32];
+        tc_ld32(tmem + ((uint32_t)(32 * q) << 16) + (uint32_t)(32 * c), r);
+        float v[32];
 #pragma unroll
-      for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
-      if (ep.bias) {
+        for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
+        if (ep.bias) {
 #pragma unroll
-        for (int j = 0; j < 32; ++j) if (nb + j < p.N) v[j] += __ldg(ep.bias + nb + j);
-      }
-      if (ep.relu) {
-#pragma unroll
-        for (int j = 0; j < 32; ++j) v[j] = fmaxf(v[j], 0.f);
-      }
-      if (!m_ok) continue;
-#pragma unroll
-      for (int g = 0; g < 4; ++g) {
-        const int n = nb + 8 * g;
-        if (n >= p.N) break;
-        float* x = v + 8 * g;
-        if (ep.mask && n < ep.mask_cols) {                       // bf16 activation of the producing layer
-          const uint4 mk = *reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(ep.mask) + m * ep.ld_mask + n);
-          const uint32_t w[4] = {mk.x, mk.y, mk.z, mk.w};
-#pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            // a bf16 is positive iff its sign bit is clear and it is not zero
-            const uint32_t lo = w[j] & 0xFFFFu, hi = w[j] >> 16;
-            if (!((lo & 0x8000u) == 0 && (lo & 0x7FFFu) != 0)) x[2 * j] = 0.f;
-            if (!((hi & 0x8000u) == 0 && (hi & 0x7FFFu) != 0)) x[2 * j + 1] = 0.f;
-          }
+          for (int j = 0; j < 32; ++j) if (nb + j < p.N) v[j] += __ldg(ep.bias + nb + j);
         }
-        if (n < ep.lo_cols) {
-          if (ep.lo_bf16) {
-            uint4 o;
-            o.x = pack2(x[0], x[1]); o.y = pack2(x[2], x[3]); o.z = pack2(x[4], x[5]); o.w = pack2(x[6], x[7]);
-            *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(ep.out_lo) + m * ep.ld_lo + n) = o;
-          } else {
-            float4* o = reinterpret_cast<float4*>(reinterpret_cast<float*>(ep.out_lo) + (int64_t)slice_z * p.split_stride + m * ep.ld_lo + n);
+        if (ep.relu) {
+#pragma unroll
+          for (int j = 0; j < 32; ++j) v[j] = fmaxf(v[j], 0.f);
+        }
+        if (!m_ok) continue;
+#pragma unroll
+        for (int g = 0; g < 4; ++g) {
+          const int n = nb + 8 * g;
+          if (n >= p.N) break;
+          float* x = v + 8 * g;
+          if (ep.mask && n < ep.mask_cols) {                       // bf16 activation of the producing layer
+            const uint4 mk = *reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(ep.mask) + m * ep.ld_mask + n);
+            const uint32_t w[4] = {mk.x, mk.y, mk.z, mk.w};
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              // a bf16 is positive iff its sign bit is clear and it is not zero
+              const uint32_t lo = w[j] & 0xFFFFu, hi = w[j] >> 16;
+              if (!((lo & 0x8000u) == 0 && (lo & 0x7FFFu) != 0)) x[2 * j] = 0.f;
+              if (!((hi & 0x8000u) == 0 && (hi & 0x7FFFu) != 0)) x[2 * j + 1] = 0.f;
+            }
+          }
+          if (n < ep.lo_cols) {
+            if (ep.lo_bf16) {
+              uint4 o;
+              o.x = pack2(x[0], x[1]); o.y = pack2(x[2], x[3]); o.z = pack2(x[4], x[5]); o.w = pack2(x[6], x[7]);
+              *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(ep.out_lo) + m * ep.ld_lo + n) = o;
+            } else {
+              float4* o = reinterpret_cast<float4*>(reinterpret_cast<float*>(ep.out_lo) + (int64_t)slice_z * p.split_stride + m * ep.ld_lo + n);
+              o[0] = make_float4(x[0], x[1], x[2], x[3]);
+              o[1] = make_float4(x[4], x[5], x[6], x[7]);
+            }
+          } else if (ep.out_hi) {
+            float4* o = reinterpret_cast<float4*>(ep.out_hi + m * ep.ld_hi + (n - ep.lo_cols));
             o[0] = make_float4(x[0], x[1], x[2], x[3]);
             o[1] = make_float4(x[4], x[5], x[6], x[7]);
           }
-        } else if (ep.out_hi) {
-          float4* o = reinterpret_cast<float4*>(ep.out_hi + m * ep.ld_hi + (n - ep.lo_cols));
-          o[0] = make_float4(x[0], x[1], x[2], x[3]);
-          o[1] = make_float4(x[4], x[5], x[6], x[7]);
         }
+      }
+    } else {
+      // tcgen05.ld hands a thread one accumulator row; stores of that shape put 32 different rows into one
+      // instruction.  For the short CTAs of a training step each warp turns its 32 x 32 block round in shared
+      // memory (the operand ring is idle once the accumulator is complete) and continues with four consecutive
+      // columns per lane, eight lanes per row: bias, ReLU, mask and stores touch whole 64- or 128-byte row segments.
+      float* stg = reinterpret_cast<float*>(gen) + q * (32 * kStgLd);   // rows of 36 floats: 128-bit accesses without bank conflicts
+      const int cl = 4 * (lane & 7), rl = lane >> 3;
+#pragma unroll 1
+      for (int c = 0; c < kBN / 32; ++c) {
+        const int nb = n0 + 32 * c;
+        if (nb >= p.N) break;
+        uint32_t r[32];
+        tc_ld32(tmem + ((uint32_t)(32 * q) << 16) + (uint32_t)(32 * c), r);
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+          *reinterpret_cast<uint4*>(stg + lane * kStgLd + 4 * j) = make_uint4(r[4 * j], r[4 * j + 1], r[4 * j + 2], r[4 * j + 3]);
+        __syncwarp();
+        const int n = nb + cl;
+        if (n < p.N) {                       // N is a multiple of 8: four columns are inside together or not at all
+          float4 bv = make_float4(0.f, 0.f, 0.f, 0.f);
+          if (ep.bias) bv = __ldg(reinterpret_cast<const float4*>(ep.bias + n));
+          const bool masked = ep.mask && n < ep.mask_cols;
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            const int row = rl + 4 * i;
+            const int64_t m = (int64_t)m0 + 32 * q + row;
+            if (m >= p.M) break;
+            const float4 sv = *reinterpret_cast<const float4*>(stg + row * kStgLd + cl);
+            float x0 = sv.x + bv.x, x1 = sv.y + bv.y, x2 = sv.z + bv.z, x3 = sv.w + bv.w;
+            if (ep.relu) { x0 = fmaxf(x0, 0.f); x1 = fmaxf(x1, 0.f); x2 = fmaxf(x2, 0.f); x3 = fmaxf(x3, 0.f); }
+            if (masked) {                    // bf16 activation of the producing layer: positive iff sign clear and not zero
+              const uint2 mk = *reinterpret_cast<const uint2*>(reinterpret_cast<const __nv_bfloat16*>(ep.mask) + m * ep.ld_mask + n);
+              if (!((mk.x & 0x8000u) == 0 && (mk.x & 0x7FFFu) != 0)) x0 = 0.f;
+              if (!((mk.x & 0x80000000u) == 0 && (mk.x & 0x7FFF0000u) != 0)) x1 = 0.f;
+              if (!((mk.y & 0x8000u) == 0 && (mk.y & 0x7FFFu) != 0)) x2 = 0.f;
+              if (!((mk.y & 0x80000000u) == 0 && (mk.y & 0x7FFF0000u) != 0)) x3 = 0.f;
+            }
+            if (n < ep.lo_cols) {
+              if (ep.lo_bf16) {
+                uint2 o;
+                o.x = pack2(x0, x1); o.y = pack2(x2, x3);
+                *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(ep.out_lo) + m * ep.ld_lo + n) = o;
+              } else {
+                *reinterpret_cast<float4*>(reinterpret_cast<float*>(ep.out_lo) + (int64_t)slice_z * p.split_stride + m * ep.ld_lo + n) =
+                    make_float4(x0, x1, x2, x3);
+              }
+            } else if (ep.out_hi) {
+              *reinterpret_cast<float4*>(ep.out_hi + m * ep.ld_hi + (n - ep.lo_cols)) = make_float4(x0, x1, x2, x3);
+            }
+          }
+        }
+        __syncwarp();                        // the block is read before the next one overwrites it
       }
     }
   }
@@ -372,20 +441,21 @@ bool gemm_tc_eligible(int M, int N, int K, const Operand& A, const Operand& B, c
 
 // Tile width and ring depth of a launch.
 enum TcVariant { TC_SMALL = 0, TC_LARGE = 1, TC_WIDE = 2, TC_NARROW = 3 };
-constexpr int kStagesNarrow = 4;   // 128 x 64 tiles: 4 stages of 24 KiB, two CTAs per SM
+constexpr int kStagesNarrow = 4;   // 128 x 64 tiles: 4 stages of 24 KiB, two CTAs per SM (measured: giving a launch of at most one CTA
+                                   // per SM the whole shared memory as a deeper ring lowers whole-step throughput by 3-5 %)
 
-template <int kStages, int kBN, int NP>
+template <int kStages, int kBN, int NP, bool kDirect>
 static ss_status launch_group(const TcGroup<NP>& g, int total_ctas, cudaStream_t st) {
   static bool attr_set[64];
   int dev = 0;
   SS_CUDA(cudaGetDevice(&dev));
   if (dev >= 0 && dev < 64 && !attr_set[dev]) {
-    SS_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<kStages, kBN, NP>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    SS_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<kStages, kBN, NP, kDirect>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  (int)tc_smem_bytes(kStages, kBN)));
     attr_set[dev] = true;
   }
   { SS_TIMED("gemm_tc_kernel", st);
-  gemm_tc_kernel<kStages, kBN, NP><<<total_ctas, kTcThreads, tc_smem_bytes(kStages, kBN), st>>>(g);
+  gemm_tc_kernel<kStages, kBN, NP, kDirect><<<total_ctas, kTcThreads, tc_smem_bytes(kStages, kBN), st>>>(g);
   }
   SS_LAUNCH_OK();
   return SS_OK;
@@ -445,10 +515,10 @@ ss_status gemm_tc_group(const TcJob* jobs, int n, cudaStream_t st) {
     const int ctas = fill_problem(&g.prob[0], j, bn, 0, err);
     if (ctas < 1) return SS_ERR_CUDA;
     switch (variant) {
-      case TC_WIDE: return launch_group<kStagesWide, 256, 1>(g, ctas, st);
-      case TC_LARGE: return launch_group<kStagesLarge, 128, 1>(g, ctas, st);
-      case TC_NARROW: return launch_group<kStagesNarrow, 64, 1>(g, ctas, st);
-      default: return launch_group<kStagesSmall, 128, 1>(g, ctas, st);
+      case TC_WIDE: return launch_group<kStagesWide, 256, 1, true>(g, ctas, st);
+      case TC_LARGE: return launch_group<kStagesLarge, 128, 1, true>(g, ctas, st);
+      case TC_NARROW: return launch_group<kStagesNarrow, 64, 1, false>(g, ctas, st);
+      default: return launch_group<kStagesSmall, 128, 1, false>(g, ctas, st);
     }
   }
   alignas(64) TcGroup<kTcMaxGroup> g;
@@ -460,7 +530,7 @@ ss_status gemm_tc_group(const TcJob* jobs, int n, cudaStream_t st) {
     total += ctas;
   }
   for (int i = n; i < kTcMaxGroup; ++i) g.prob[i] = g.prob[n - 1];   // never selected; keeps the parameter block defined
-  return launch_group<kStagesSmall, 128, kTcMaxGroup>(g, total, st);
+  return launch_group<kStagesSmall, 128, kTcMaxGroup, false>(g, total, st);
 }
 
 ss_status gemm_tc(int M, int N, int K, const Operand& A, const Operand& B, const Epilogue& ep, cudaStream_t st,

@@ -1,8 +1,9 @@
 """Host-side schedule of the ShadowSync hot path on one GPU (Algorithm 1).
 
-R trainer replicas live on the device as separate buffers.  Each replica owns a high-priority CUDA
-stream on which its training step is enqueued (four library calls: embedding forward, MLP forward,
-MLP backward + dense Adagrad, embedding backward + row-wise Adagrad).  The shadow thread of the
+R trainer replicas live on the device as separate buffers.  Each replica owns CUDA streams above the
+shadow stream's priority on which its training step is enqueued (four library calls: embedding forward,
+MLP forward, MLP backward + dense Adagrad, embedding backward + row-wise Adagrad; the MLP calls on the
+highest priority, the embedding calls one level below where the device has the levels).  The shadow thread of the
 paper (Section 3.2) is a host thread that keeps enqueuing one synchronisation kernel after another
 on a separate lowest-priority stream; it shares no event or dependency with the training streams.
 
@@ -64,8 +65,13 @@ class Replica:
             self.uniq_keys = torch.empty(max_L, dtype=torch.int32, device=dev)
             self.seg_off = torch.empty(max_L + 1, dtype=torch.int32, device=dev)
             self.perm = torch.empty(max_L, dtype=torch.int32, device=dev)
-        self.stream = torch.cuda.Stream(device=dev, priority=priority)
-        self.side = torch.cuda.Stream(device=dev, priority=priority)   # the index sort of the backward runs here
+        # The embedding calls are long kernels that fill the device and are bound by memory throughput; the MLP
+        # calls are chains of short kernels bound by latency.  The MLP chain therefore gets the highest priority
+        # and the embedding calls a level in between (still above the shadow stream): blocks of an MLP kernel
+        # are placed as soon as a slot frees up instead of queueing behind another replica's gather.
+        self.stream = torch.cuda.Stream(device=dev, priority=model.prio_embedding)
+        self.side = torch.cuda.Stream(device=dev, priority=model.prio_embedding)   # the index sort of the backward runs here
+        self.mlp = torch.cuda.Stream(device=dev, priority=priority)
         self.steps_done = 0
 
 
@@ -88,6 +94,7 @@ class Model:
         self.d_status = torch.zeros(1, dtype=torch.int32, device=device)
         lo, hi = torch.cuda.Stream.priority_range()   # (lowest priority value, highest), e.g. (0, -5)
         self.prio_low, self.prio_high = lo, hi
+        self.prio_embedding = hi + min(2, max(0, (lo - hi) - 1))   # between the two when the device has the levels
         self.replicas: List[Replica] = [Replica(self, w0_flat, hi, max_L, keep_sort_outputs) for _ in range(R)]
         # workers[r][k]: worker k of trainer r; worker 0 is the replica itself, further workers share its parameters
         # (the paper's intra-trainer Hogwild: m threads, each on its own batch, updating one local copy)
@@ -121,10 +128,20 @@ class Model:
             join.record(rep.side)
         ss.ss_embbag_fwd(self.tables, T, N, D, batch.indices, batch.offsets, B, rep.concat_f32, sp.W,
                          rep.concat_bf16, sp.W, D, self.d_status, s)
+        # on the replica's own stream the MLP calls move to its high-priority stream (a caller's stream is kept)
+        m = rep.mlp if s is rep.stream else s
+        if m is not s:
+            e = torch.cuda.Event()
+            e.record(s)
+            m.wait_event(e)
         ss.ss_mlp_fwd(sp, rep.w, rep.w_bf16, batch.dense, rep.concat_f32, rep.concat_bf16, B, batch.labels,
-                      rep.logit, rep.prob, rep.loss, rep.mlp_ws, s)
+                      rep.logit, rep.prob, rep.loss, rep.mlp_ws, m)
         ss.ss_mlp_bwd(sp, rep.w, rep.w_bf16, rep.acc, None, batch.dense, rep.concat_f32, rep.concat_bf16,
-                      batch.labels, rep.prob, B, self.lr, self.eps, 1, rep.grad_pooled, T * D, rep.mlp_ws, s)
+                      batch.labels, rep.prob, B, self.lr, self.eps, 1, rep.grad_pooled, T * D, rep.mlp_ws, m)
+        if m is not s:
+            e = torch.cuda.Event()
+            e.record(m)
+            s.wait_event(e)
         if overlap_sort:
             s.wait_event(join)
             ss.ss_embbag_bwd_apply(self.tables, self.row_state, T, N, D, B, batch.L, rep.grad_pooled, T * D, 0,
