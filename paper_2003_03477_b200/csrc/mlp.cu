@@ -389,34 +389,41 @@ adagrad_kernel(float* __restrict__ w, float* __restrict__ acc, const float* g, c
 // sample with fp32 FMAs in ascending k.
 // ---------------------------------------------------------------------------------------------
 constexpr int kFewInputs = 16;
-constexpr int kFirstRows = 16;      // samples per block
+constexpr int kFirstRows = 8;       // samples per block
 
 __global__ void __launch_bounds__(256)
 few_inputs_layer_kernel(const float* __restrict__ x, int K, const __nv_bfloat16* __restrict__ W, const float* __restrict__ bias,
                         int relu, int B, int N, __nv_bfloat16* __restrict__ Y, int64_t ldy) {
   extern __shared__ __align__(16) __nv_bfloat16 s_w[];       // [K][N]
-  for (int i = threadIdx.x; i < K * N; i += 256) {
-    const int o = i / K, k = i - o * K;                      // W is [o][k], read in memory order
-    s_w[k * N + o] = W[i];
+  __shared__ float s_x[kFirstRows][kFewInputs];              // the block's samples, rounded to bf16, zero beyond K
+  const int b0 = blockIdx.x * kFirstRows;
+  const int rows = min(kFirstRows, B - b0);
+  for (int o = threadIdx.x; o < N; o += 256) {               // W is [o][k]
+#pragma unroll 4
+    for (int k = 0; k < K; ++k) s_w[k * N + o] = W[(int64_t)o * K + k];
+  }
+  if (threadIdx.x < kFirstRows * kFewInputs) {
+    const int r = threadIdx.x / kFewInputs, k = threadIdx.x % kFewInputs;
+    s_x[r][k] = (r < rows && k < K) ? __bfloat162float(__float2bfloat16_rn(x[(int64_t)(b0 + r) * K + k])) : 0.f;
   }
   __syncthreads();
   const int nchunk = N >> 3;
-  const int b0 = blockIdx.x * kFirstRows;
-  const int rows = min(kFirstRows, B - b0);
   for (int item = threadIdx.x; item < rows * nchunk; item += 256) {
     const int r = item / nchunk, o = (item - r * nchunk) * 8;
-    const float* xr = x + (int64_t)(b0 + r) * K;
     float acc[8];
 #pragma unroll
     for (int j = 0; j < 8; ++j) acc[j] = 0.f;
-    for (int k = 0; k < K; ++k) {
-      const float xv = __bfloat162float(__float2bfloat16_rn(xr[k]));
-      const uint4 q = *reinterpret_cast<const uint4*>(s_w + k * N + o);
-      const uint32_t ww[4] = {q.x, q.y, q.z, q.w};
 #pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        acc[2 * j] = fmaf(xv, __uint_as_float(ww[j] << 16), acc[2 * j]);
-        acc[2 * j + 1] = fmaf(xv, __uint_as_float(ww[j] & 0xFFFF0000u), acc[2 * j + 1]);
+    for (int k = 0; k < kFewInputs; ++k) {
+      if (k < K) {
+        const float xv = s_x[r][k];
+        const uint4 q = *reinterpret_cast<const uint4*>(s_w + k * N + o);
+        const uint32_t ww[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          acc[2 * j] = fmaf(xv, __uint_as_float(ww[j] << 16), acc[2 * j]);
+          acc[2 * j + 1] = fmaf(xv, __uint_as_float(ww[j] & 0xFFFF0000u), acc[2 * j + 1]);
+        }
       }
     }
     const float4 b0v = reinterpret_cast<const float4*>(bias + o)[0], b1v = reinterpret_cast<const float4*>(bias + o)[1];
