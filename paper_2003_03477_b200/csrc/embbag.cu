@@ -1245,7 +1245,8 @@ static ss_status bwd_impl(bool do_sort, bool do_apply, float* tables, float* row
   // (0) one block per table sorts that table's lookups in shared memory; scalars[4] stays 0 when every
   // block could, and the tiled passes below then return at once
   int32_t* fallback = scalars + 4;
-  const bool try_table_sort = B <= 65536;
+  // more lookups than T tables of kTsCap can hold: some table is too large for its block, the tiled passes are certain
+  const bool try_table_sort = B <= 65536 && L <= (int64_t)T * kTsCap;
   SS_CUDA(cudaMemsetAsync(fallback, try_table_sort ? 0 : 1, 4, cs));
   if (try_table_sort) {
     int row_bits = 1;

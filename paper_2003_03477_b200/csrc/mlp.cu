@@ -389,21 +389,21 @@ adagrad_kernel(float* __restrict__ w, float* __restrict__ acc, const float* g, c
 // sample with fp32 FMAs in ascending k.
 // ---------------------------------------------------------------------------------------------
 constexpr int kFewInputs = 16;
-constexpr int kFirstRows = 8;       // samples per block
+constexpr int kFirstRowsMax = 32;   // most samples per block (the launch picks 8, 16 or 32 so that the grid is about two blocks per SM)
 
 __global__ void __launch_bounds__(256)
 few_inputs_layer_kernel(const float* __restrict__ x, int K, const __nv_bfloat16* __restrict__ W, const float* __restrict__ bias,
-                        int relu, int B, int N, __nv_bfloat16* __restrict__ Y, int64_t ldy) {
+                        int relu, int B, int N, __nv_bfloat16* __restrict__ Y, int64_t ldy, int rows_per_block) {
   extern __shared__ __align__(16) __nv_bfloat16 s_w[];       // [K][N]
-  __shared__ float s_x[kFirstRows][kFewInputs];              // the block's samples, rounded to bf16, zero beyond K
-  const int b0 = blockIdx.x * kFirstRows;
-  const int rows = min(kFirstRows, B - b0);
+  __shared__ float s_x[kFirstRowsMax][kFewInputs];           // the block's samples, rounded to bf16, zero beyond K
+  const int b0 = blockIdx.x * rows_per_block;
+  const int rows = min(rows_per_block, B - b0);
   for (int o = threadIdx.x; o < N; o += 256) {               // W is [o][k]
 #pragma unroll 4
     for (int k = 0; k < K; ++k) s_w[k * N + o] = W[(int64_t)o * K + k];
   }
-  if (threadIdx.x < kFirstRows * kFewInputs) {
-    const int r = threadIdx.x / kFewInputs, k = threadIdx.x % kFewInputs;
+  for (int i = threadIdx.x; i < rows_per_block * kFewInputs; i += 256) {
+    const int r = i / kFewInputs, k = i % kFewInputs;
     s_x[r][k] = (r < rows && k < K) ? __bfloat162float(__float2bfloat16_rn(x[(int64_t)(b0 + r) * K + k])) : 0.f;
   }
   __syncthreads();
@@ -519,10 +519,12 @@ ss_status ss_mlp_fwd(const ss_mlp_desc* desc, const float* w, const void* w_bf16
     }
     const size_t few_smem = (size_t)L.in * L.out * 2;
     if (p.bf16 && l == 0 && L.in <= kFewInputs && few_smem <= 48 * 1024 && (ep.ld_lo & 7) == 0 && aligned16(ep.out_lo)) {
+      int rows = 8;                                            // every block stages the whole weight matrix
+      while (rows < kFirstRowsMax && (B + rows - 1) / rows > 2 * num_sms()) rows *= 2;
       SS_TIMED("few_inputs_layer_kernel", cs);
-      few_inputs_layer_kernel<<<(B + kFirstRows - 1) / kFirstRows, 256, few_smem, cs>>>(
+      few_inputs_layer_kernel<<<(B + rows - 1) / rows, 256, few_smem, cs>>>(
           dense, L.in, reinterpret_cast<const __nv_bfloat16*>(w_bf16) + L.w_off, ep.bias, ep.relu, B, L.out,
-          reinterpret_cast<__nv_bfloat16*>(ep.out_lo), ep.ld_lo);
+          reinterpret_cast<__nv_bfloat16*>(ep.out_lo), ep.ld_lo, rows);
       SS_LAUNCH_OK();
       continue;
     }
