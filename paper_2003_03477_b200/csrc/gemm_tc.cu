@@ -339,21 +339,28 @@ gemm_tc_kernel(const __grid_constant__ TcGroup<NP> grp) {
           float4 bv = make_float4(0.f, 0.f, 0.f, 0.f);
           if (ep.bias) bv = __ldg(reinterpret_cast<const float4*>(ep.bias + n));
           const bool masked = ep.mask && n < ep.mask_cols;
+          // the mask words of all eight rows are requested before any is used: one round of load latency, not eight
+          uint2 mk[8];
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            const int64_t m = (int64_t)m0 + 32 * q + rl + 4 * i;
+            mk[i] = make_uint2(0x3F803F80u, 0x3F803F80u);   // four positive values: nothing is masked
+            if (masked && m < p.M)
+              mk[i] = *reinterpret_cast<const uint2*>(reinterpret_cast<const __nv_bfloat16*>(ep.mask) + m * ep.ld_mask + n);
+          }
 #pragma unroll
           for (int i = 0; i < 8; ++i) {
             const int row = rl + 4 * i;
             const int64_t m = (int64_t)m0 + 32 * q + row;
-            if (m >= p.M) break;
+            if (m >= p.M) continue;
             const float4 sv = *reinterpret_cast<const float4*>(stg + row * kStgLd + cl);
             float x0 = sv.x + bv.x, x1 = sv.y + bv.y, x2 = sv.z + bv.z, x3 = sv.w + bv.w;
             if (ep.relu) { x0 = fmaxf(x0, 0.f); x1 = fmaxf(x1, 0.f); x2 = fmaxf(x2, 0.f); x3 = fmaxf(x3, 0.f); }
-            if (masked) {                    // bf16 activation of the producing layer: positive iff sign clear and not zero
-              const uint2 mk = *reinterpret_cast<const uint2*>(reinterpret_cast<const __nv_bfloat16*>(ep.mask) + m * ep.ld_mask + n);
-              if (!((mk.x & 0x8000u) == 0 && (mk.x & 0x7FFFu) != 0)) x0 = 0.f;
-              if (!((mk.x & 0x80000000u) == 0 && (mk.x & 0x7FFF0000u) != 0)) x1 = 0.f;
-              if (!((mk.y & 0x8000u) == 0 && (mk.y & 0x7FFFu) != 0)) x2 = 0.f;
-              if (!((mk.y & 0x80000000u) == 0 && (mk.y & 0x7FFF0000u) != 0)) x3 = 0.f;
-            }
+            // bf16 activation of the producing layer: positive iff sign clear and not zero
+            if (!((mk[i].x & 0x8000u) == 0 && (mk[i].x & 0x7FFFu) != 0)) x0 = 0.f;
+            if (!((mk[i].x & 0x80000000u) == 0 && (mk[i].x & 0x7FFF0000u) != 0)) x1 = 0.f;
+            if (!((mk[i].y & 0x8000u) == 0 && (mk[i].y & 0x7FFFu) != 0)) x2 = 0.f;
+            if (!((mk[i].y & 0x80000000u) == 0 && (mk[i].y & 0x7FFF0000u) != 0)) x3 = 0.f;
             if (n < ep.lo_cols) {
               if (ep.lo_bf16) {
                 uint2 o;
