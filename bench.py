@@ -40,13 +40,13 @@ RING = 8            # pre-generated batches per replica, cycled through
 NCU_TRAFFIC = {
     "gemm_tc_kernel": {
         "workload": "medium",
-        "bytes_per_launch": 3667904,      # mean over the 12 GEMM launches of a replica step
+        "bytes_per_launch": 4887011,      # mean over the 9 GEMM launches of a replica step
         "capture": "profiles/step_medium_top_kernels.md",
         "sources": {
-            "gemm_tc.cu": "b5bffd890cb45d12702fb5bb1f8241eba14bb7f5385abd222ef7e47c4ee3f121",
-            "mlp.cu": "d19c4b892161d5ed072e508a46f8c87a8581353428f85020fa705df9f385ed89",
-            "gemm.cuh": "da1df6183e23abbd5728584e558625d4dc65d14209886465342899cdf4a7a462",
-            "mlp_plan.cuh": "bc8b0ba72d2a7789979f8bd83bc7a7f74e710c88cebe970199f86206822370c5",
+            "gemm_tc.cu": "d2e358fd5c31e8fc1c3d78389618a122201e165dbf62652aa8cfe46616c3001e",
+            "mlp.cu": "1c63eda249700af7d8a428f91ce25d1018427f7b1592706555d5eeab65df660c",
+            "gemm.cuh": "7491d2079ed234aeda8b58fdac00e6c5965a825b21e58246e8fc0e3b9a32b6f8",
+            "mlp_plan.cuh": "40fc89d02a018eefd85fb14d8606d76b7c19e763b529208b4af61f8b88819181",
         },
     },
 }
@@ -396,6 +396,9 @@ def bench_gpu(args):
     torch.cuda.synchronize()
     if cfg.bf16:
         out["gemm_alone"] = gemm_alone(s, peaks)
+    if cfg.D <= 128:
+        out["embedding_alone"] = embedding_alone(model, host, dev, cfg, peaks)
+        torch.cuda.synchronize()
 
     # ---- end to end through the public API with host buffers ------------------------------------
     if not args.quick:
@@ -434,6 +437,67 @@ def gemm_alone(stream, peaks):
         tf = 2.0 * M * N * K / us / 1e6
         res.append({"M": M, "N": N, "K": K, "us": us, "TFLOP/s": tf, "frac_of_bf16_peak": tf / peaks["bf16_tflops"]})
     return res
+
+
+def embedding_alone(model, host, dev, cfg, peaks):
+    """The embedding kernels on their own: the forward gather, and the reduction half of the backward (fused
+    window kernel + combine kernel, which also update the rows), each timed with events around a captured graph
+    of `reps` launches with an L2 flush (a 256 MiB fill) before every launch; the time of a graph of the flushes
+    alone is subtracted.  Algorithmic bytes as in roofline(); fractions are of the measured copy peak."""
+    import torch
+    from paper_2003_03477_b200 import binding as ss
+    rep, sp = model.replicas[0], model.spec
+    s = rep.stream
+    T, N, D, B = model.T, model.N, model.D, model.B
+    b, hb = dev[0][0], host[0][0]
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=b.indices.device)
+    reps = 8
+    with torch.cuda.stream(s):
+        # the workspace holds the sort of this batch; the gradient is whatever the last step left (any values do)
+        ss.ss_embbag_bwd_sort(T, N, D, b.indices, b.offsets, B, b.L, rep.emb_ws, None, None, None, rep.num_unique,
+                              model.d_status, s)
+    torch.cuda.synchronize()
+    U = float(rep.num_unique.item())
+
+    def fwd():
+        ss.ss_embbag_fwd(model.tables, T, N, D, b.indices, b.offsets, B, rep.concat_f32, sp.W, rep.concat_bf16, sp.W, D,
+                         model.d_status, s)
+
+    def apply():
+        ss.ss_embbag_bwd_apply(model.tables, model.row_state, T, N, D, B, b.L, rep.grad_pooled, T * D, 0, model.lr,
+                               model.eps, rep.emb_ws, model.d_status, s)
+
+    def graph_ms(fn):
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=s):
+            for _ in range(reps):
+                flush.fill_(1)
+                if fn is not None:
+                    fn()
+        best = None
+        with torch.cuda.stream(s):
+            g.replay()
+            for _ in range(3):
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(s)
+                g.replay()
+                e1.record(s)
+                e1.synchronize()
+                ms = e0.elapsed_time(e1)
+                best = ms if best is None else min(best, ms)
+        return best
+
+    base = graph_ms(None)
+    out = {}
+    for name, fn, nbytes in (
+            ("embbag_fwd", fwd, hb.L * (4 * D + 4) + 4 * (T * B + 1) + T * B * D * (2 if cfg.bf16 else 4)),
+            ("embbag_bwd_apply", apply, hb.L * (4 * D + 16) + U * (2 * 4 * D + 8))):
+        us = (graph_ms(fn) - base) * 1e3 / reps
+        gbs = nbytes / (us * 1e-6) / 1e9
+        out[name] = {"us": us, "algorithmic_bytes": nbytes, "GB/s": gbs, "frac_of_hbm_peak": gbs / peaks["hbm_gbs"]}
+    out["note"] = ("L2 flushed before every launch; Zipf-hot rows and the gathered gradient rows are re-read through L2 "
+                   "within a launch; embbag_bwd_apply = fused window kernel + combine kernel")
+    return out
 
 
 def profile_pass(model, dev, cfg, steps=6, replicas=None):
