@@ -448,6 +448,10 @@ bool gemm_tc_eligible(int M, int N, int K, const Operand& A, const Operand& B, c
 
 // Tile width and ring depth of a launch.
 enum TcVariant { TC_SMALL = 0, TC_LARGE = 1, TC_WIDE = 2, TC_NARROW = 3 };
+// Products of at least this many flops (4096 x 1024 x 1024) take the 128 x 256 tiles even when they fill the SMs less than
+// twice: their CTAs run long enough for the tile's lower shared-memory traffic per flop to outweigh the smaller grid
+// (the 3.6 GFLOP products of a 2048-sample step are below it: wide tiles cost that step 3 %).
+constexpr double kHeavyFlops = 8589934592.0;
 constexpr int kStagesNarrow = 4;   // 128 x 64 tiles: 4 stages of 24 KiB, two CTAs per SM (measured: giving a launch of at most one CTA
                                    // per SM the whole shared memory as a deeper ring lowers whole-step throughput by 3-5 %)
 
@@ -513,7 +517,8 @@ ss_status gemm_tc_group(const TcJob* jobs, int n, cudaStream_t st) {
     const long long ctas128 = (long long)((j.N + 127) / 128) * mt * ks;
     const long long ctas256 = (long long)((j.N + 255) / 256) * mt * ks;
     int variant = TC_SMALL;
-    if (j.N >= 256 && ctas256 >= 2ll * num_sms() && nk_slice >= 2 * kStagesWide) variant = TC_WIDE;
+    const bool heavy = 2.0 * j.M * j.N * j.K >= kHeavyFlops;
+    if (j.N >= 256 && (ctas256 >= 2ll * num_sms() || heavy) && nk_slice >= 2 * kStagesWide) variant = TC_WIDE;
     else if (ctas128 >= 2ll * num_sms() && nk_slice >= 2 * kStagesLarge) variant = TC_LARGE;
     else if (j.N <= 64 || 2 * ctas128 <= num_sms()) variant = TC_NARROW;    // a narrow product, or too few 128-wide tiles to occupy the SMs
     const int bn = variant == TC_WIDE ? 256 : (variant == TC_NARROW ? 64 : 128);
@@ -528,15 +533,27 @@ ss_status gemm_tc_group(const TcJob* jobs, int n, cudaStream_t st) {
       default: return launch_group<kStagesSmall, 128, 1, false>(g, ctas, st);
     }
   }
+  // a group made of wide products that is heavy as a whole takes the 128 x 256 tiles as well
+  double flops = 0.0;
+  bool wide = true;
+  for (int i = 0; i < n; ++i) {
+    const TcJob& j = jobs[i];
+    flops += 2.0 * j.M * j.N * j.K;
+    const int nk_all = (j.K + kBK - 1) / kBK;
+    const int ks = j.k_splits < 1 ? 1 : (j.k_splits > nk_all ? nk_all : j.k_splits);
+    if (j.N < 256 || (nk_all + ks - 1) / ks < 2 * kStagesWide) wide = false;
+  }
+  wide = wide && flops >= 2.0 * kHeavyFlops;
   alignas(64) TcGroup<kTcMaxGroup> g;
   g.n = n;
   int total = 0;
   for (int i = 0; i < n; ++i) {
-    const int ctas = fill_problem(&g.prob[i], jobs[i], 128, total, err);
+    const int ctas = fill_problem(&g.prob[i], jobs[i], wide ? 256 : 128, total, err);
     if (ctas < 1) return SS_ERR_CUDA;
     total += ctas;
   }
   for (int i = n; i < kTcMaxGroup; ++i) g.prob[i] = g.prob[n - 1];   // never selected; keeps the parameter block defined
+  if (wide) return launch_group<kStagesWide, 256, kTcMaxGroup, true>(g, total, st);
   return launch_group<kStagesSmall, 128, kTcMaxGroup, false>(g, total, st);
 }
 
