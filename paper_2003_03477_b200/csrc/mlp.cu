@@ -5,27 +5,6 @@
 
 namespace ss {
 
-// prob = sigmoid(z); loss = mean_b( max(z,0) - z*y + log(1+exp(-|z|)) ); one block, fixed reduction tree.
-__global__ void __launch_bounds__(1024)
-bce_loss_kernel(const float* __restrict__ logit, const float* __restrict__ labels, int B,
-                float* __restrict__ prob, float* __restrict__ loss) {
-  __shared__ float red[1024];
-  float s = 0.f;
-  for (int b = threadIdx.x; b < B; b += 1024) {
-    const float z = logit[b], y = labels[b];
-    const float e = expf(-fabsf(z));
-    prob[b] = (z >= 0.f) ? 1.f / (1.f + e) : e / (1.f + e);
-    s += fmaxf(z, 0.f) - z * y + log1pf(e);
-  }
-  red[threadIdx.x] = s;
-  __syncthreads();
-  for (int off = 512; off >= 1; off >>= 1) {
-    if (threadIdx.x < off) red[threadIdx.x] += red[threadIdx.x + off];
-    __syncthreads();
-  }
-  if (threadIdx.x == 0) loss[0] = red[0] / (float)B;
-}
-
 // dz[b] = (prob[b] - y[b]) / B, stored as float or bf16 (a [B,1] gradient matrix).
 __global__ void dz_kernel(const float* __restrict__ prob, const float* __restrict__ labels, int B, void* __restrict__ dz,
                           int as_bf16) {
@@ -220,18 +199,70 @@ batch_reduce_partial_kernel(const __grid_constant__ RedJobs jobs, int B, int row
   }
 }
 
-// logit[b] = sum_k X[b, k] * w[k] + bias: one warp per row, lanes stride k, fixed shuffle tree.
+// The single-logit layer, the sigmoid and the loss in one launch:
+//   logit[b] = sum_k X[b, k] * w[k] + bias;  prob[b] = sigmoid(logit[b]);
+//   loss = mean_b( max(z,0) - z*y + log(1+exp(-|z|)) ).
+// One warp per sample (eight consecutive k per lane and round, fixed shuffle tree); a block adds the loss terms of
+// its eight samples in order and leaves the sum in part[block]; the block that draws the last ticket adds the
+// blocks' sums in a fixed order (which block that is does not matter) and clears the ticket for the next call.
 __global__ void __launch_bounds__(256)
-rowdot_kernel(const void* __restrict__ X, int x_kind, int64_t ldx, const void* __restrict__ w, int w_kind, int K,
-              const float* __restrict__ bias, int B, float* __restrict__ logit) {
-  const int b = blockIdx.x * 8 + (threadIdx.x >> 5);
-  const int lane = threadIdx.x & 31;
-  if (b >= B) return;
+logit_loss_kernel(const void* __restrict__ X, int x_kind, int64_t ldx, const void* __restrict__ w, int w_kind, int K,
+                  const float* __restrict__ bias, const float* __restrict__ labels, int B, float* __restrict__ logit,
+                  float* __restrict__ prob, float* __restrict__ loss, float* part, unsigned int* ticket) {
+  __shared__ float s_term[8];
+  __shared__ float s_red[256];
+  __shared__ int s_last;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int b = blockIdx.x * 8 + warp;
   float s = 0.f;
-  for (int k = lane; k < K; k += 32) s = fmaf(load_kind(X, x_kind, (int64_t)b * ldx + k), load_kind(w, w_kind, k), s);
+  if (b < B) {
+    const bool al_x = (reinterpret_cast<uintptr_t>(X) & 15u) == 0, al_w = (reinterpret_cast<uintptr_t>(w) & 15u) == 0;
+    const bool vec_x = al_x && (x_kind == OP_BF16 ? (ldx & 7) == 0 : (ldx & 3) == 0);
+    for (int k0 = 8 * lane; k0 < K; k0 += 256) {
+      float xv[8], wv[8];
+      load8_kind(X, x_kind, b, ldx, k0, K, vec_x, xv);
+      load8_kind(w, w_kind, 0, 0, k0, K, al_w, wv);
+#pragma unroll
+      for (int j = 0; j < 8; ++j) s = fmaf(xv[j], wv[j], s);
+    }
+  }
 #pragma unroll
   for (int off = 16; off >= 1; off >>= 1) s += __shfl_down_sync(0xffffffffu, s, off);
-  if (lane == 0) logit[b] = s + bias[0];
+  if (lane == 0) {
+    float t = 0.f;
+    if (b < B) {
+      const float z = s + bias[0], y = labels[b];
+      const float e = expf(-fabsf(z));
+      logit[b] = z;
+      prob[b] = (z >= 0.f) ? 1.f / (1.f + e) : e / (1.f + e);
+      t = fmaxf(z, 0.f) - z * y + log1pf(e);
+    }
+    s_term[warp] = t;
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    float t = 0.f;
+#pragma unroll
+    for (int r = 0; r < 8; ++r) t += s_term[r];
+    part[blockIdx.x] = t;
+    __threadfence();
+    s_last = atomicAdd(ticket, 1u) == gridDim.x - 1;
+  }
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+  float a = 0.f;
+  for (int i = threadIdx.x; i < (int)gridDim.x; i += 256) a += __ldcg(part + i);
+  s_red[threadIdx.x] = a;
+  __syncthreads();
+  for (int off = 128; off >= 1; off >>= 1) {
+    if (threadIdx.x < off) s_red[threadIdx.x] += s_red[threadIdx.x + off];
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) {
+    loss[0] = s_red[0] / (float)B;
+    *ticket = 0u;
+  }
 }
 
 // The backward of the single-logit layer with the loss gradient folded in:
@@ -492,6 +523,8 @@ ss_status ss_mlp_fwd(const ss_mlp_desc* desc, const float* w, const void* w_bf16
   cudaStream_t cs = as_stream(stream);
   char* ws = reinterpret_cast<char*>(workspace);
   const int act_kind = p.bf16 ? OP_BF16 : OP_F32;
+  // the loss kernel's ticket starts at zero (the workspace arrives uninitialised); it clears itself after use
+  SS_CUDA(cudaMemsetAsync(ws + p.loss_part, 0, 4, cs));
 
   for (int l = 0; l < p.nl; ++l) {
     const LayerInfo& L = p.layer[l];
@@ -502,8 +535,10 @@ ss_status ss_mlp_fwd(const ss_mlp_desc* desc, const float* w, const void* w_bf16
     Bm = p.bf16 ? Operand{reinterpret_cast<const __nv_bfloat16*>(w_bf16) + L.w_off, OP_BF16, L.in, 1}
                 : Operand{w + L.w_off, OP_F32, L.in, 1};
     if (l == p.nl - 1) {   // one output unit: a dot product per sample
-      { SS_TIMED("rowdot_kernel", cs);
-      rowdot_kernel<<<(B + 7) / 8, 256, 0, cs>>>(A.p, A.kind, A.s_row, Bm.p, Bm.kind, L.in, w + L.b_off, B, logit);
+      unsigned int* ticket = reinterpret_cast<unsigned int*>(ws + p.loss_part);
+      { SS_TIMED("logit_loss_kernel", cs);
+      logit_loss_kernel<<<(B + 7) / 8, 256, 0, cs>>>(A.p, A.kind, A.s_row, Bm.p, Bm.kind, L.in, w + L.b_off, labels, B, logit,
+                                                     prob, loss, reinterpret_cast<float*>(ticket + 4), ticket);
       }
       SS_LAUNCH_OK();
       break;
@@ -531,10 +566,6 @@ ss_status ss_mlp_fwd(const ss_mlp_desc* desc, const float* w, const void* w_bf16
     st = gemm(B, L.out, L.in, A, Bm, ep, cs);
     if (st != SS_OK) return st;
   }
-  { SS_TIMED("bce_loss_kernel", cs);
-  bce_loss_kernel<<<1, 1024, 0, cs>>>(logit, labels, B, prob, loss);
-  }
-  SS_LAUNCH_OK();
   return SS_OK;
 }
 

@@ -22,7 +22,7 @@ struct MlpPlan {
   // respect to it after the ReLU mask.  The last bottom layer's output lives in the concat buffer and
   // the last top layer's in logit[], so act[] is unused for those two.
   size_t act[kMaxLayers], dact[kMaxLayers];
-  size_t grads, red_partial, gpart, total;
+  size_t grads, red_partial, gpart, loss_part, total;   // loss_part: a ticket word, then one partial loss per 8 samples
   int k_splits[kMaxLayers];      // K slices of the weight-gradient GEMM of each layer (1 = none)
   int64_t gpart_off[kMaxLayers]; // float offset of the layer's slice buffer inside the gpart region
   int red_splits;         // batch slices of the two-stage reductions (bias and skinny weight gradients)
@@ -71,17 +71,24 @@ inline ss_status make_mlp_plan(const ss_mlp_desc* d, int B, MlpPlan* p) {
   red_total += (size_t)p->layer[p->nl - 1].in;
   if (p->layer[0].in <= 16) red_total += (size_t)p->layer[0].in * p->layer[0].out;
   p->red_partial = take(red_total * 4 * (size_t)p->red_splits);
-  // weight-gradient GEMMs contract over the batch and have small outputs: cut K into a few slices so that
-  // more CTAs work on each of them (measured on the 2048-sample step: 2 slices beat both 1 and 4..16 in
-  // whole-step throughput); the slices are added in order by the update kernel
+  // Weight-gradient GEMMs contract over the batch and have small outputs.  They go out together as one launch, so the
+  // K range is cut into slices only while all their tiles together fill less than half the SMs (measured on the
+  // 2048-sample step, 74 tiles: 1 slice 15.1 M examples/s, 2 slices 14.8 M, 4 slices 14.1 M: the update kernel adds the
+  // slices in order and reads each of them).
   int64_t gp = 0;
   const int nk = (B + 63) / 64;
+  auto sliced = [&](int l) {
+    const LayerInfo& L = p->layer[l];
+    return p->bf16 && l != p->nl - 1 && !(l == 0 && L.in <= 16) && B >= 16;
+  };
+  int64_t all_tiles = 0;
+  for (int l = 0; l < p->nl; ++l)
+    if (sliced(l)) all_tiles += (int64_t)((p->layer[l].out + 127) / 128) * ((p->layer[l].in + 127) / 128);
   for (int l = 0; l < p->nl; ++l) {
     const LayerInfo& L = p->layer[l];
     int s = 1;
-    if (p->bf16 && l != p->nl - 1 && !(l == 0 && L.in <= 16) && B >= 16) {
-      const int tiles = ((L.out + 127) / 128) * ((L.in + 127) / 128);
-      s = (148 + tiles - 1) / tiles;
+    if (sliced(l)) {
+      s = (int)(148 / (2 * all_tiles));
       if (s > 16) s = 16;
       if (s > nk / 16) s = nk / 16;                        // slices of at least 16 k-steps: a CTA's fixed cost outweighs shorter ones
       if (s > nk) s = nk;
@@ -92,6 +99,7 @@ inline ss_status make_mlp_plan(const ss_mlp_desc* d, int B, MlpPlan* p) {
     if (s > 1) gp += (int64_t)s * L.in * L.out;
   }
   p->gpart = take((size_t)gp * 4);
+  p->loss_part = take(((size_t)(B + 7) / 8 + 4) * 4);
   p->total = o;
   return SS_OK;
 }
