@@ -40,13 +40,13 @@ RING = 8            # pre-generated batches per replica, cycled through
 NCU_TRAFFIC = {
     "gemm_tc_kernel": {
         "workload": "medium",
-        "bytes_per_launch": 4887011,      # mean over the 9 GEMM launches of a replica step
+        "bytes_per_launch": 4887836,      # mean over the 9 GEMM launches of a replica step
         "capture": "profiles/step_medium_top_kernels.md",
         "sources": {
-            "gemm_tc.cu": "d2e358fd5c31e8fc1c3d78389618a122201e165dbf62652aa8cfe46616c3001e",
-            "mlp.cu": "1c63eda249700af7d8a428f91ce25d1018427f7b1592706555d5eeab65df660c",
+            "gemm_tc.cu": "5f9de5bcdb37f0ff4599f4caabb1334cf391928d2d14d0fce9b71869917ac138",
+            "mlp.cu": "9ebfdc7cb9de27e940592657a1445a3989af3655ecfafc592519c4e215891479",
             "gemm.cuh": "7491d2079ed234aeda8b58fdac00e6c5965a825b21e58246e8fc0e3b9a32b6f8",
-            "mlp_plan.cuh": "40fc89d02a018eefd85fb14d8606d76b7c19e763b529208b4af61f8b88819181",
+            "mlp_plan.cuh": "0c026b6ce9a10e26eec5b857317a2fda0152cc17fa8989500e7fba16f35a7bbb",
         },
     },
 }
