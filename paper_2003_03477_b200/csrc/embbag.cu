@@ -906,7 +906,7 @@ __device__ __forceinline__ void adagrad_one_row(float4 g, uint32_t key, int lane
 }
 
 // ---- (5) rows whose run crosses window edges: add their window partials ---------------------------
-// Rows spanning up to four windows: one lane group adds the partials in window order.  Longer rows: one
+// Rows spanning up to 32 windows: one lane group adds the partials in window order.  Longer rows: one
 // block per row, lane group j adds the partials of windows k0+j, k0+j+groups, ... in ascending order and
 // the group sums are then added in group order.  The association is fixed by the
 // segment's position alone (the order of the list does not matter).
@@ -925,8 +925,12 @@ combine_rows_kernel(const int32_t* __restrict__ seg, const int32_t* __restrict__
   const int nvec = D >> 2;
   if (!ws_matches(scalars, L, sentinel, nullptr)) return;
   const int n = min(scalars[1], nwin);
-  constexpr int kShort = 4;                                // spans up to this many windows: one group per row
-  // phase A: short spans, one lane group per listed row, all partial loads issued together
+  // Spans of up to kShort windows: one lane group per row, which requests kBatch partials at a time and adds them in
+  // window order.  Only the few rows with longer spans (the hottest of a skewed table) take a whole block each: a
+  // block works through its rows one after the other, so that path must stay short.
+  constexpr int kShort = 32;
+  constexpr int kBatch = NV <= 1 ? 8 : (NV <= 2 ? 4 : 2);
+  // phase A
   for (int i = blockIdx.x * kGroups + grp; i < n; i += gridDim.x * kGroups) {
     const int u = long_list[i];
     if (u < 0 || u >= umax) continue;
@@ -934,32 +938,38 @@ combine_rows_kernel(const int32_t* __restrict__ seg, const int32_t* __restrict__
     if (s0 < 0 || s1 <= s0 || s1 > L) continue;
     const int k0 = s0 / kWin, k1 = (s1 - 1) / kWin;
     if (k1 - k0 + 1 > kShort) continue;
-    float4 pv[kShort][NV];
+    float4 t[NV];
 #pragma unroll
-    for (int j = 0; j < kShort; ++j) {
-      const int k = k0 + j;
-      const int slot = (s0 <= k * kWin) ? 0 : 1;           // the run covers the window's first position -> slot 0
-      const float4* p = reinterpret_cast<const float4*>(partial + ((int64_t)k * 2 + slot) * D);
+    for (int v = 0; v < NV; ++v) t[v] = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int kb = k0; kb <= k1; kb += kBatch) {
+      float4 pv[kBatch][NV];
+#pragma unroll
+      for (int j = 0; j < kBatch; ++j) {
+        const int k = kb + j;
+        const int slot = (s0 <= k * kWin) ? 0 : 1;         // the run covers the window's first position -> slot 0
+        const float4* p = reinterpret_cast<const float4*>(partial + ((int64_t)k * 2 + slot) * D);
+#pragma unroll
+        for (int v = 0; v < NV; ++v) {
+          const int c = lane + v * G;
+          pv[j][v] = (k <= k1 && c < nvec) ? p[c] : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+      }
+#pragma unroll
+      for (int j = 0; j < kBatch; ++j)
+#pragma unroll
+        for (int v = 0; v < NV; ++v) t[v] = add4(t[v], pv[j][v]);   // adding zeros for absent windows changes nothing
+    }
+    if (!FUSE) {
+      float4* dst = reinterpret_cast<float4*>(gsum + (int64_t)u * D);
 #pragma unroll
       for (int v = 0; v < NV; ++v) {
         const int c = lane + v * G;
-        pv[j][v] = (k <= k1 && c < nvec) ? p[c] : make_float4(0.f, 0.f, 0.f, 0.f);
+        if (c < nvec) dst[c] = t[v];
       }
-    }
-    float4* dst = reinterpret_cast<float4*>(gsum + (int64_t)u * D);
-    float4 t0 = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-    for (int v = 0; v < NV; ++v) {
-      const int c = lane + v * G;
-      float4 t = pv[0][v];
-#pragma unroll
-      for (int j = 1; j < kShort; ++j) t = add4(t, pv[j][v]);   // adding zeros for absent windows changes nothing
-      if (!FUSE && c < nvec) dst[c] = t;
-      if (v == 0) t0 = t;
     }
     if (FUSE) {
       const uint32_t key = (uint32_t)uniq[u];
-      if (key < sentinel) adagrad_one_row<G>(t0, key, lane, nvec, D, gmask, tables, row_state, lr, eps);
+      if (key < sentinel) adagrad_row_nv<G, NV>(t, key, lane, nvec, D, gmask, tables, row_state, lr, eps);
     }
   }
   // phase B: long spans, the whole block per row.  The block owns the list entries blockIdx.x + k*gridDim.x;
@@ -1006,20 +1016,21 @@ combine_rows_kernel(const int32_t* __restrict__ seg, const int32_t* __restrict__
     if (grp == 0) {
       const int used = min(kGroups, k1 - k0 + 1);
       float4* dst = reinterpret_cast<float4*>(gsum + (int64_t)u * D);
-      float4 t0 = make_float4(0.f, 0.f, 0.f, 0.f);
+      float4 tt[NV];
 #pragma unroll
       for (int v = 0; v < NV; ++v) {
         const int c = lane + v * G;
+        tt[v] = make_float4(0.f, 0.f, 0.f, 0.f);
         if (c < nvec) {
           float4 t = s_part[c];
           for (int j = 1; j < used; ++j) t = add4(t, s_part[j * nvec + c]);
           if (!FUSE) dst[c] = t;
-          if (v == 0) t0 = t;
+          tt[v] = t;
         }
       }
       if (FUSE) {
         const uint32_t key = (uint32_t)uniq[u];
-        if (key < sentinel) adagrad_one_row<G>(t0, key, lane, nvec, D, gmask, tables, row_state, lr, eps);
+        if (key < sentinel) adagrad_row_nv<G, NV>(tt, key, lane, nvec, D, gmask, tables, row_state, lr, eps);
       }
     }
     __syncthreads();
@@ -1134,7 +1145,9 @@ static void launch_reduce(const BwdPlan& p, char* ws, const uint32_t* keys, cons
   {
     SS_TIMED("combine_rows_kernel", st);
     const int cblocks = p.nwin < num_sms() * 8 ? p.nwin : num_sms() * 8;
-    combine_rows_kernel<G, NV, kFuse><<<cblocks, 256, (size_t)kGroups * D * 4, st>>>(
+    // fused rows of at least eight float4: two float4 per lane, half as many lanes per row, twice as many rows in flight
+    constexpr int CG = (kFuse && G >= 8) ? G / 2 : G, CNV = (kFuse && G >= 8) ? 2 : NV;
+    combine_rows_kernel<CG, CNV, kFuse><<<cblocks, 256, (size_t)(256 / CG) * D * 4, st>>>(
         seg, scalars, long_list, p.nwin, D, partial, gsum, p.L, sentinel, (int64_t)umax, uniq, tables, row_state, lr, eps);
   }
   if (!kFuse) {
