@@ -40,7 +40,7 @@ RING = 8            # pre-generated batches per replica, cycled through
 NCU_TRAFFIC = {
     "gemm_tc_kernel": {
         "workload": "medium",
-        "bytes_per_launch": 4887836,      # mean over the 9 GEMM launches of a replica step
+        "bytes_per_launch": 4887352,      # mean over the 9 GEMM launches of a replica step
         "capture": "profiles/step_medium_top_kernels.md",
         "sources": {
             "gemm_tc.cu": "5f9de5bcdb37f0ff4599f4caabb1334cf391928d2d14d0fce9b71869917ac138",
