@@ -43,7 +43,7 @@ NCU_TRAFFIC = {
         "bytes_per_launch": 4887352,      # mean over the 9 GEMM launches of a replica step
         "capture": "profiles/step_medium_top_kernels.md",
         "sources": {
-            "gemm_tc.cu": "5f9de5bcdb37f0ff4599f4caabb1334cf391928d2d14d0fce9b71869917ac138",
+            "gemm_tc.cu": "14567cfb0dbd4a7a16394e5e5b169de194ea2f38254bf0ec44ffbb10551c1479",
             "mlp.cu": "9ebfdc7cb9de27e940592657a1445a3989af3655ecfafc592519c4e215891479",
             "gemm.cuh": "7491d2079ed234aeda8b58fdac00e6c5965a825b21e58246e8fc0e3b9a32b6f8",
             "mlp_plan.cuh": "0c026b6ce9a10e26eec5b857317a2fda0152cc17fa8989500e7fba16f35a7bbb",

@@ -5,10 +5,11 @@
 // One CTA computes a 128 x 128 tile (128 x 256 for large products, 128 x 64 for products with too few
 // tiles to occupy the SMs).  One launch may hold several independent products (a group): a CTA finds its
 // product from its block index.  Warp 0 (one lane) streams 128 x 64 / 64 x 128 operand tiles
-// into a ring of shared-memory stages (3 or 6 deep) with TMA (128-byte swizzle); warp 1 (one lane) issues
-// tcgen05.mma (M = 128, N = 128 or 256, K = 16, accumulators in tensor memory) and releases stages with
-// tcgen05.commit; warps 2-5 wait for the accumulator, read it with tcgen05.ld (one row per thread)
-// and apply the epilogue (bias, ReLU, ReLU-gradient mask, bf16 / fp32 stores).
+// into a ring of shared-memory stages (3, 4 or 6 deep) with TMA (128-byte swizzle), the first round before the
+// warps meet; warp 1 (one lane) issues tcgen05.mma (M = 128, N = 64, 128 or 256, K = 16, accumulators in tensor
+// memory) and releases stages with tcgen05.commit; warps 2-5 wait for the accumulator, read it with tcgen05.ld
+// (one row per thread) and apply the epilogue (bias, ReLU, ReLU-gradient mask, bf16 / fp32 stores), through a
+// transposition in shared memory for the short CTAs of a training step.
 //
 // Either operand may be K-major (k contiguous in memory: the forward pass reads activations [B, in]
 // and weights [out, in] this way) or MN-major (m or n contiguous: the backward pass reads the same
@@ -25,7 +26,7 @@
 
 namespace ss {
 
-constexpr int kBM = 128, kBK = 64;   // tile rows and k depth; the tile width kBN (128 or 256) is a template parameter
+constexpr int kBM = 128, kBK = 64;   // tile rows and k depth; the tile width kBN (64, 128 or 256) is a template parameter
 // Ring depth: 3 stages (97 KiB, two CTAs per SM) for the small GEMMs of a training step, where several
 // replicas' kernels share the SMs and a second resident CTA hides more latency than a deeper ring does;
 // 6 stages (193 KiB, one CTA per SM) for large products that fill the machine on their own.
