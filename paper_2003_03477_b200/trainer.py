@@ -70,7 +70,9 @@ class Replica:
         # and the embedding calls a level in between (still above the shadow stream): blocks of an MLP kernel
         # are placed as soon as a slot frees up instead of queueing behind another replica's gather.
         self.stream = torch.cuda.Stream(device=dev, priority=model.prio_embedding)
-        self.side = torch.cuda.Stream(device=dev, priority=model.prio_embedding)   # the index sort of the backward runs here
+        # the index sort of the backward runs here: one block per table on few SMs, and the reduction waits for it,
+        # so it goes in between where the device has a level left (measured +2 % examples/s)
+        self.side = torch.cuda.Stream(device=dev, priority=model.prio_sort)
         self.mlp = torch.cuda.Stream(device=dev, priority=priority)
         self.steps_done = 0
 
@@ -95,6 +97,7 @@ class Model:
         lo, hi = torch.cuda.Stream.priority_range()   # (lowest priority value, highest), e.g. (0, -5)
         self.prio_low, self.prio_high = lo, hi
         self.prio_embedding = hi + min(2, max(0, (lo - hi) - 1))   # between the two when the device has the levels
+        self.prio_sort = self.prio_embedding - 1 if self.prio_embedding - 1 > hi else self.prio_embedding
         self.replicas: List[Replica] = [Replica(self, w0_flat, hi, max_L, keep_sort_outputs) for _ in range(R)]
         # workers[r][k]: worker k of trainer r; worker 0 is the replica itself, further workers share its parameters
         # (the paper's intra-trainer Hogwild: m threads, each on its own batch, updating one local copy)
