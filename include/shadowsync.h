@@ -103,6 +103,11 @@ ss_status ss_embbag_bwd_adagrad(float* tables, float* row_state, int T, int64_t 
                                 int32_t* uniq_keys, int32_t* seg_off, int32_t* perm,
                                 int32_t* d_num_unique, int32_t* d_status, ss_stream stream);
 
+/* The sort half handles a table with at most this many lookups in a call with one thread block that sorts in shared
+ * memory (a light kernel on T SMs); when the lookups of a call exceed T times this number, or a table exceeds it, tiled
+ * passes over all SMs sort instead.  Callers that schedule the sort beside other work can plan with it. */
+#define SS_TABLE_SORT_CAP 24576
+
 /* The same operation in two calls, so that its first half can be enqueued early on another stream:
  * steps 1-2 depend only on the batch's indices, steps 3-4 also on the gradient.
  *   ss_embbag_bwd_sort   steps 1-2 into the workspace (and the optional uniq_keys / seg_off / perm outputs)

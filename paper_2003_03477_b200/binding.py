@@ -20,6 +20,7 @@ SS_OK = 0
 STATUS_NAMES = {0: "SS_OK", -1: "SS_ERR_NULL", -2: "SS_ERR_SHAPE", -3: "SS_ERR_ALIGN", -4: "SS_ERR_DTYPE",
                 -5: "SS_ERR_WORKSPACE", -6: "SS_ERR_ARCH", -7: "SS_ERR_CUDA", -8: "SS_ERR_RANGE"}
 SS_DEV_BAD_INDEX, SS_DEV_BAD_OFFSET, SS_DEV_BAD_WORKSPACE = 1, 2, 4
+SS_TABLE_SORT_CAP = 24576          # lookups of one table that the light per-table sort takes (shadowsync.h)
 SS_SYNC_EASGD_LITERAL = 1
 SS_SYNC_BMUF_NESTEROV = 2
 

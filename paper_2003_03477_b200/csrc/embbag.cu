@@ -410,7 +410,7 @@ sort_scatter_kernel(const uint32_t* __restrict__ keys_in, const int32_t* __restr
 // and the tiled passes, launched after this kernel, run; otherwise they return at once.
 constexpr int kTsThreads = 1024;
 constexpr int kTsWarps = kTsThreads / 32;
-constexpr int kTsCap = 24576;                              // lookups of one table
+constexpr int kTsCap = SS_TABLE_SORT_CAP;                  // lookups of one table (24576)
 constexpr int kTsMaxBins = 256;
 constexpr size_t kTsSmem = (size_t)kTsCap * 8 + (size_t)kTsWarps * kTsMaxBins * 4;   // 229,376 bytes
 

@@ -97,7 +97,10 @@ class Model:
         lo, hi = torch.cuda.Stream.priority_range()   # (lowest priority value, highest), e.g. (0, -5)
         self.prio_low, self.prio_high = lo, hi
         self.prio_embedding = hi + min(2, max(0, (lo - hi) - 1))   # between the two when the device has the levels
-        self.prio_sort = self.prio_embedding - 1 if self.prio_embedding - 1 > hi else self.prio_embedding
+        # only while the sort is the light per-table kernel: the tiled passes of larger batches fill the device and,
+        # given precedence over the other replicas' embedding calls, cost a quarter of the throughput (measured)
+        light_sort = 0 < max_L <= T * ss.SS_TABLE_SORT_CAP
+        self.prio_sort = self.prio_embedding - 1 if (light_sort and self.prio_embedding - 1 > hi) else self.prio_embedding
         self.replicas: List[Replica] = [Replica(self, w0_flat, hi, max_L, keep_sort_outputs) for _ in range(R)]
         # workers[r][k]: worker k of trainer r; worker 0 is the replica itself, further workers share its parameters
         # (the paper's intra-trainer Hogwild: m threads, each on its own batch, updating one local copy)

@@ -72,3 +72,11 @@ def test_null_and_range_checks_need_no_gpu(lib):
     assert lib.ss_sync_ma(bad, 2, None, 16, 0.1, 0, None, None) == -3
     assert lib.ss_embbag_fwd(0x1000, 2, 10, 6, 0x1000, 0x1000, 4, 0x1000, 16, None, 0, 0, None, None) == -2  # D % 4
     assert lib.ss_embbag_fwd(None, 2, 10, 8, 0x1000, 0x1000, 4, 0x1000, 16, None, 0, 0, None, None) == -1
+
+
+def test_binding_constants_match_the_header():
+    import os
+    import re
+    hdr = open(os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "include", "shadowsync.h")).read()
+    m = re.search(r"#define\s+SS_TABLE_SORT_CAP\s+(\d+)", hdr)
+    assert m and int(m.group(1)) == ss.SS_TABLE_SORT_CAP
