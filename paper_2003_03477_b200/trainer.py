@@ -99,7 +99,9 @@ class Model:
         self.prio_embedding = hi + min(2, max(0, (lo - hi) - 1))   # between the two when the device has the levels
         # only while the sort is the light per-table kernel: the tiled passes of larger batches fill the device and,
         # given precedence over the other replicas' embedding calls, cost a quarter of the throughput (measured)
-        light_sort = 0 < max_L <= T * ss.SS_TABLE_SORT_CAP
+        # ... and while the sorts of all replicas together (one SM per table each) leave SMs free: with R*T beyond the
+        # SM count the raised level costs 2 % instead of gaining 2 % (measured at R=8, T=26)
+        light_sort = 0 < max_L <= T * ss.SS_TABLE_SORT_CAP and R * workers * T <= ss.ss_num_sms()
         self.prio_sort = self.prio_embedding - 1 if (light_sort and self.prio_embedding - 1 > hi) else self.prio_embedding
         self.replicas: List[Replica] = [Replica(self, w0_flat, hi, max_L, keep_sort_outputs) for _ in range(R)]
         # workers[r][k]: worker k of trainer r; worker 0 is the replica itself, further workers share its parameters
