@@ -11,8 +11,14 @@ kernel (S-EASGD / S-MA / S-BMUF as the workload says) on the lowest-priority str
 With N > 1 (launched under torchrun) every rank runs the same job on its own GPU: the path does not
 shard across GPUs, so these are independent replicas of the job and the values add (weak scaling).
 
+The K-step region is repeated (sync off and sync on alternating) until at least a second has been timed, and the
+median region gives `value`; the spread is reported beside it.  The same line carries, as legs, the other
+single-GPU workloads (`workloads.medium_bmuf`, `workloads.large`) and the sync-kernel sweep running concurrently with
+this training (`sync.concurrent_sweep`).
+
 `--impl reference` times the CPU oracle (oracle/, test infrastructure) on a bounded sample of the same
 workload on the host cores; it is deliberately slow and is a reported baseline, not a target.
+`--plain` runs a few un-captured replica steps (every kernel its own launch) for profilers.
 """
 from __future__ import annotations
 
@@ -38,17 +44,6 @@ RING = 8            # pre-generated batches per replica, cycled through
 # for the named workload and for exactly the sources whose hashes are listed: once one of them changes the figure is
 # reported as null until the counters are taken again.
 NCU_TRAFFIC = {
-    "gemm_tc_kernel": {
-        "workload": "medium",
-        "bytes_per_launch": 4887352,      # mean over the 9 GEMM launches of a replica step
-        "capture": "profiles/step_medium_top_kernels.md",
-        "sources": {
-            "gemm_tc.cu": "14567cfb0dbd4a7a16394e5e5b169de194ea2f38254bf0ec44ffbb10551c1479",
-            "mlp.cu": "9ebfdc7cb9de27e940592657a1445a3989af3655ecfafc592519c4e215891479",
-            "gemm.cuh": "7491d2079ed234aeda8b58fdac00e6c5965a825b21e58246e8fc0e3b9a32b6f8",
-            "mlp_plan.cuh": "0c026b6ce9a10e26eec5b857317a2fda0152cc17fa8989500e7fba16f35a7bbb",
-        },
-    },
 }
 
 
@@ -125,18 +120,20 @@ class ClockSampler:
                 if v.lower().startswith("active"):
                     reasons.add(name)
         return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "reasons": sorted(reasons), "samples": len(sm)}
+                "reasons": sorted(reasons), "samples": len(sm),
+                "sm_mhz_min": min(sm) if sm else None, "sm_mhz_highest_seen": max(sm) if sm else None,
+                "sampled": "nvidia-smi every 100 ms across all repeated timed regions"}
 
 
 # ----------------------------------------------------------------------------------------------
-def build_job(cfg, device, workers=1):
+def build_job(cfg, device, workers=1, ring=RING):
     """Tables, replicas and a ring of device-resident batches for one GPU."""
     import torch
     from paper_2003_03477_b200 import binding as ss, synth, trainer
     tables = trainer.device_tables(cfg, device)
     spec = ss.MlpSpec(cfg.bottom, cfg.top, cfg.bf16)
     w0 = torch.from_numpy(trainer.pack_params(spec, synth.initial_weights(cfg))).to(device)
-    host = [[synth.make_batch(cfg, r, t) for t in range(RING)] for r in range(cfg.R)]
+    host = [[synth.make_batch(cfg, r, t) for t in range(ring)] for r in range(cfg.R)]
     max_L = max(b.L for bs in host for b in bs)
     model = trainer.Model(cfg.T, cfg.N, cfg.D, cfg.B, cfg.bottom, cfg.top, cfg.bf16, cfg.R, w0, tables, cfg.lr, cfg.eps,
                           max_L=max_L, device=device, workers=workers)
@@ -162,28 +159,37 @@ def capture_graphs(model, dev):
 STEPS_AHEAD = 16   # set from --steps-ahead
 
 
-def run_steps(model, graphs, first_step, n_steps):
+def run_steps(model, graphs, first_step, n_steps, paced=None):
     """Replays the replicas' step graphs.  The host keeps at most STEPS_AHEAD steps of a replica queued on the device
     (it waits for the event of step t - STEPS_AHEAD before it enqueues step t; 0 = no bound).  An unbounded queue
     changes nothing for training but makes the shadow thread's launches wait behind thousands of queued graph
     launches: measured 76 sync rounds/s (a pass every 25 steps) unbounded, 312/s (every 6 steps) with 16, 1416/s
-    (every 1.3 steps, training -1 %) with 4."""
+    (every 1.3 steps, training -1 %) with 4.
+    paced = (every, fn): the paced form of the background sync (one pass after each round of `every` local steps):
+    fn() enqueues a pass on the low-priority sync stream, with no dependency on the training streams.
+    Returns the number of paced passes enqueued."""
     import torch
+    ring = len(graphs[0])
     evs = [[] for _ in model.replicas]
+    passes = 0
     for t in range(first_step, first_step + n_steps):
         for r, rep in enumerate(model.replicas):
             if STEPS_AHEAD and len(evs[r]) >= STEPS_AHEAD:
                 evs[r].pop(0).synchronize()
             with torch.cuda.stream(rep.stream):
-                graphs[r][t % RING].replay()
+                graphs[r][t % ring].replay()
                 if STEPS_AHEAD:
                     e = torch.cuda.Event()
                     e.record(rep.stream)
                     evs[r].append(e)
+        if paced and (t - first_step + 1) % paced[0] == 0:
+            paced[1]()
+            passes += 1
+    return passes
 
 
-def timed_region(model, graphs, first_step, n_steps):
-    """Device time of n_steps steps over all replica streams (ms)."""
+def timed_region(model, graphs, first_step, n_steps, paced=None):
+    """Device time of n_steps steps over all replica streams (ms), and the paced sync passes enqueued in it."""
     import torch
     main = torch.cuda.current_stream()
     torch.cuda.synchronize()
@@ -191,14 +197,14 @@ def timed_region(model, graphs, first_step, n_steps):
     start.record(main)
     for rep in model.replicas:
         rep.stream.wait_event(start)
-    run_steps(model, graphs, first_step, n_steps)
+    passes = run_steps(model, graphs, first_step, n_steps, paced)
     for rep in model.replicas:
         e = torch.cuda.Event()
         e.record(rep.stream)
         main.wait_event(e)
     stop.record(main)
     stop.synchronize()
-    return start.elapsed_time(stop)
+    return start.elapsed_time(stop), passes
 
 
 def reduce_over_ranks(ms_list, examples, device):
@@ -213,6 +219,18 @@ def reduce_over_ranks(ms_list, examples, device):
     n = torch.tensor([examples], dtype=torch.int64, device=device)
     dist.all_reduce(n, op=dist.ReduceOp.SUM)
     return [float(x) for x in t], int(n[0])
+
+
+def region_stats(ms):
+    """Median, extremes and count of repeated timed regions."""
+    return {"median_ms": statistics.median(ms), "min_ms": min(ms), "max_ms": max(ms), "repeats": len(ms)}
+
+
+def repeats_for(region_ms, min_total_s, min_reps, max_reps):
+    """How often the K-step region is repeated so that at least min_total_s are timed (clocks settle, and a sync
+    loss of a fraction of a per cent is above the spread)."""
+    need = int(np.ceil(min_total_s * 1e3 / max(region_ms, 1e-3)))
+    return max(min_reps, min(max_reps, need))
 
 
 def sync_args(cfg):
@@ -233,6 +251,95 @@ def time_kernel_call(fn, stream, reps):
     return sum(a.elapsed_time(b) for a, b in evs) / reps
 
 
+class Barrier:
+    def __init__(self, world):
+        self.world = world
+
+    def __call__(self):
+        import torch
+        import torch.distributed as dist
+        torch.cuda.synchronize()
+        if self.world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+
+def measure_training(model, graphs, cfg, K, W, barrier, device, args, sampler=None):
+    """Sync-off and sync-on regions of exactly K steps each, alternating, repeated until args.min_seconds have been
+    timed per arm (at least args.min_repeats times).  Background sync: the native shadow thread, paused (drained)
+    during the off regions so that the pass count of an on region is the number of passes that completed in it; for a
+    workload with a paced sync (one pass after each round of k local steps) the host enqueues that pass on the
+    low-priority sync stream instead.  Returns a dict of lists (max over ranks per region) and totals."""
+    import torch
+    from paper_2003_03477_b200 import trainer
+    paced = (cfg.sync_every, lambda: model.sync(**sync_args(cfg))) if cfg.sync_every else None
+    loop = None
+    if paced is None:
+        loop = trainer.ShadowLoop(model, max_in_flight=args.sync_in_flight, pause_s=args.sync_pause, **sync_args(cfg)).start()
+        loop.pause()
+    run_steps(model, graphs, 0, W)
+    barrier()
+    # one probe region sizes the repeat count (every rank takes the same count: the max over ranks decides)
+    probe, _ = timed_region(model, graphs, W, K)
+    (probe,), _ = reduce_over_ranks([probe], 0, device)
+    reps = repeats_for(probe, args.min_seconds, args.min_repeats, 400)
+    ms_on, ms_off, rounds = [], [], []
+    if sampler is not None:
+        sampler.start()
+    for i in range(reps):
+        barrier()
+        t_off, _ = timed_region(model, graphs, W + i * K, K)
+        barrier()
+        if loop is not None:
+            r0 = loop.rounds
+            loop.resume()
+            t_on, _ = timed_region(model, graphs, W + i * K, K)
+            r1 = loop.pause()
+            rounds.append(r1 - r0)
+        else:
+            t_on, n_pass = timed_region(model, graphs, W + i * K, K, paced)
+            model.sync_stream.synchronize()
+            rounds.append(n_pass)
+        ms_on.append(t_on)
+        ms_off.append(t_off)
+    clocks = sampler.stop() if sampler is not None else None
+    barrier()
+    if loop is not None:
+        loop.stop()
+    torch.cuda.synchronize()
+    both, examples = reduce_over_ranks(ms_on + ms_off, cfg.R * cfg.B * K, device)
+    return {"ms_on": both[:reps], "ms_off": both[reps:], "rounds": rounds, "examples_per_region": examples,
+            "clocks": clocks, "paced": paced is not None}
+
+
+def summarise_training(m, K):
+    """examples/s from the median region of each arm, the spread, the sync loss and the sync rate."""
+    on, off = region_stats(m["ms_on"]), region_stats(m["ms_off"])
+    ex = m["examples_per_region"]
+    value, value_off = ex / (on["median_ms"] * 1e-3), ex / (off["median_ms"] * 1e-3)
+    total_rounds, total_s = sum(m["rounds"]), sum(m["ms_on"]) * 1e-3
+    # loss from the medians, and the median of the per-pair losses (regions alternate, so a pair shares its clocks)
+    pair = [100.0 * (1.0 - b / a) for a, b in zip(m["ms_on"], m["ms_off"])]
+    return value, on, {
+        "rounds_per_s": total_rounds / total_s if total_s > 0 else None,
+        "avg_sync_gap_steps": (K * len(m["ms_on"]) / total_rounds) if total_rounds else None,
+        "passes_counted": total_rounds, "counting": "passes completed inside the sync-on regions (the shadow thread is "
+        "paused and drained outside them)" if not m["paced"] else "one pass enqueued on the sync stream per round of local steps",
+        "examples_per_s_sync_off": value_off,
+        "throughput_loss_pct": 100.0 * (1.0 - value / value_off),
+        "throughput_loss_pct_median_of_pairs": statistics.median(pair),
+        "regions_sync_on": on, "regions_sync_off": off,
+        "examples_per_s_sync_on_best_region": ex / (on["min_ms"] * 1e-3),
+    }
+
+
+def workload_text(cfg):
+    return (f"{cfg.name}: R={cfg.R} T={cfg.T} N={cfg.N} D={cfg.D} B={cfg.B} "
+            f"bottom={'-'.join(map(str, cfg.bottom))} top={'-'.join(map(str, cfg.top))} "
+            f"sync={cfg.sync} alpha={cfg.alpha} "
+            + (f"one background pass per {cfg.sync_every} local steps" if cfg.sync_every else "background, continuous"))
+
+
 def bench_gpu(args):
     import torch
     import torch.distributed as dist
@@ -250,6 +357,7 @@ def bench_gpu(args):
         cfg = synth.scaled(cfg, R=args.replicas)
     K, W = args.steps, max(args.warmup, 3)
     peaks = measured_peaks()
+    barrier = Barrier(world)
 
     model, host, dev, max_L = build_job(cfg, device, workers=max(1, args.workers))
     # un-captured warm-up: first-use set-up inside the library (function attributes, symbol addresses)
@@ -259,29 +367,9 @@ def bench_gpu(args):
     torch.cuda.synchronize()
     graphs = capture_graphs(model, dev)
 
-    def barrier():
-        torch.cuda.synchronize()
-        if world > 1:
-            dist.barrier()
-            torch.cuda.synchronize()
-
-    # ---- sync off ------------------------------------------------------------------------
-    run_steps(model, graphs, 0, W)
-    barrier()
-    ms_off = timed_region(model, graphs, W, K)
-
-    # ---- sync on (the headline) -------------------------------------------------------------
-    loop = trainer.ShadowLoop(model, max_in_flight=args.sync_in_flight, pause_s=args.sync_pause, **sync_args(cfg)).start()
-    run_steps(model, graphs, 0, W)
-    barrier()
-    sampler = ClockSampler(local).start()
-    rounds0 = loop.rounds
-    ms_on = timed_region(model, graphs, W, K)
-    rounds = loop.rounds - rounds0
-    clocks = sampler.stop()
-    barrier()
-    loop.stop()
-    torch.cuda.synchronize()
+    m = measure_training(model, graphs, cfg, K, W, barrier, device, args, sampler=ClockSampler(local))
+    value, on, sync_info = summarise_training(m, K)
+    clocks = m["clocks"]
     # ---- foreground variant (the paper's FR-* baselines): the sync pass inside the training loop every k steps
     ms_fg = None
     if args.foreground > 0:
@@ -307,15 +395,15 @@ def bench_gpu(args):
     # ---- intra-trainer Hogwild: m workers per replica, each on its own batches, sharing the replica's parameters
     ms_hw = None
     if args.workers > 1:
-        m = args.workers
+        mw = args.workers
         for r in range(cfg.R):
-            for k in range(1, m):
+            for k in range(1, mw):
                 model.step(r, dev[r][k % RING], worker=k)
         torch.cuda.synchronize()
         wg = []
         for r in range(cfg.R):
             per_worker = []
-            for k in range(m):
+            for k in range(mw):
                 wk, row = model.workers[r][k], []
                 for slot in range(RING):
                     g = torch.cuda.CUDAGraph()
@@ -328,7 +416,7 @@ def bench_gpu(args):
         def hw_steps(first, n):
             for t in range(first, first + n):
                 for r in range(cfg.R):
-                    for k in range(m):
+                    for k in range(mw):
                         with torch.cuda.stream(model.workers[r][k].stream):
                             wg[r][k][t % RING].replay()
         hw_steps(0, W)
@@ -348,21 +436,20 @@ def bench_gpu(args):
         e1.record(main)
         e1.synchronize()
         ms_hw = e0.elapsed_time(e1)
-    (ms_on, ms_off), examples = reduce_over_ranks([ms_on, ms_off], cfg.R * cfg.B * K, device)
-    value = examples / (ms_on * 1e-3)
-    value_off = examples / (ms_off * 1e-3)
-    status = model.status() | (ss.ss_device_error() << 8)
+    status = model.status()
 
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
-        "ms_per_step": ms_on / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "ms_per_step": on["median_ms"] / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16" if cfg.bf16 else "f32", "data": "synthetic",
-        "config": {"workload": f"{cfg.name}: R={cfg.R} T={cfg.T} N={cfg.N} D={cfg.D} B={cfg.B} "
-                               f"bottom={'-'.join(map(str, cfg.bottom))} top={'-'.join(map(str, cfg.top))} "
-                               f"sync={cfg.sync} alpha={cfg.alpha} background",
-                   "l2": "inputs larger than L2: tables 6.7 GB gathered by Zipf indices, 8 rotating batches per replica",
+        "config": {"workload": workload_text(cfg),
+                   "l2": f"inputs larger than L2: tables {cfg.T * cfg.N * cfg.D * 4 / 1e9:.1f} GB gathered by skewed "
+                         f"indices, {RING} rotating batches per replica",
                    "multi_gpu": "replicas only (no cross-GPU exchange on this path)",
-                   "steps_ahead": STEPS_AHEAD},
+                   "steps_ahead": STEPS_AHEAD,
+                   "timing": f"CUDA events around exactly {K} steps, barrier + synchronise on both sides, max over "
+                             f"ranks; the region is repeated {on['repeats']} times (sync off / on alternating) and "
+                             f"value is examples / median region"},
         "clocks": clocks,
         "status_word": status,
     }
@@ -372,8 +459,7 @@ def bench_gpu(args):
         return
 
     # ---- extra measurements on rank 0 ---------------------------------------------------------
-    out["sync"] = {"rounds_per_s": rounds / (ms_on * 1e-3), "avg_sync_gap_steps": (K / rounds) if rounds else None,
-                   "examples_per_s_sync_off": value_off, "throughput_loss_pct": 100.0 * (1.0 - value / value_off)}
+    out["sync"] = sync_info
 
     if ms_fg is not None:
         out["sync"]["foreground"] = {"every_k_steps": args.foreground, "examples_per_s": cfg.R * cfg.B * K / (ms_fg * 1e-3),
@@ -383,7 +469,8 @@ def bench_gpu(args):
                           "examples_per_s": cfg.R * args.workers * cfg.B * K / (ms_hw * 1e-3)}
     kernels, per_step = profile_pass(model, dev, cfg)
     out["kernels"] = kernels
-    out["gpu_launches"] = int(round(per_step * cfg.R * K)) + int(rounds)
+    out["gpu_launches"] = int(round(per_step * cfg.R * K)) + int(round(sum(m["rounds"]) / len(m["rounds"])))
+    out["gpu_launches_note"] = "kernel launches of this library inside one timed K-step region (sync on)"
     out["roofline"] = roofline(kernels, model, host, cfg, peaks)
     # the same kernel with one replica training alone (no other replica's kernels competing for the SMs)
     k1, _ = profile_pass(model, dev, cfg, replicas=[0])
@@ -405,8 +492,7 @@ def bench_gpu(args):
         with torch.cuda.stream(s):
             time_kernel_call(fn, s, 3)
             ms = time_kernel_call(fn, s, 20)
-        per = {"easgd": 2 * R + 2, "ma": 2 * R + 1, "bmuf": 2 * R + 4}[cfg.sync]
-        gbs = per * 4 * n / (ms * 1e-3) / 1e9
+        gbs = SYNC_VECTORS[cfg.sync](R) * 4 * n / (ms * 1e-3) / 1e9
         return {"n": n, "R": R, "us": ms * 1e3, "GB/s": gbs, "frac_of_hbm_peak": gbs / peaks["hbm_gbs"]}
     out["sync"]["kernel_alone_64M"] = time_sync(1 << 26, cfg.R)
     torch.cuda.synchronize()
@@ -416,13 +502,96 @@ def bench_gpu(args):
         out["embedding_alone"] = embedding_alone(model, host, dev, cfg, peaks)
         torch.cuda.synchronize()
 
+    # ---- the sync-kernel sweep running concurrently with this training ---------------------------
+    if not args.quick and not args.no_sweep:
+        out["sync"]["concurrent_sweep"] = concurrent_sweep(model, graphs, cfg, K, W, args, peaks,
+                                                           value_off=sync_info["examples_per_s_sync_off"])
     # ---- end to end through the public API with host buffers ------------------------------------
     if not args.quick:
-        out["e2e"] = bench_e2e(model, host, dev, graphs, cfg, K, W)
+        out["e2e"] = bench_e2e(model, host, dev, graphs, cfg, K, W, args)
         out["cpu_baseline"] = cpu_baseline(cfg, budget_s=args.cpu_budget)
+    # ---- the other single-GPU workloads, as legs of the same line ---------------------------------
+    if not args.quick and not args.no_legs and world == 1 and args.workload == "medium" and not args.replicas:
+        del graphs, dev, host, model
+        torch.cuda.empty_cache()
+        out["workloads"] = {}
+        for name in ("medium_bmuf", "large"):
+            out["workloads"][name] = bench_leg(synth.CONFIGS[name], K, W, device, args, peaks)
+            torch.cuda.empty_cache()
     print(json.dumps(out))
     if world > 1:
         dist.destroy_process_group()
+
+
+SYNC_VECTORS = {"easgd": lambda R: 2 * R + 2, "ma": lambda R: 2 * R + 1, "bmuf": lambda R: 2 * R + 4}
+
+
+def bench_leg(cfg, K, W, device, args, peaks):
+    """Another workload measured the same way (K-step regions, sync off / on alternating, median), reported as a leg:
+    examples/s, sync loss, sync gap and the roofline entry of its dominant kernel."""
+    import torch
+    ring = 4 if cfg.R * cfg.B >= 32768 else RING           # fewer pre-generated batches where one is ~850 k lookups
+    model, host, dev, max_L = build_job(cfg, device, ring=ring)
+    for r in range(cfg.R):
+        model.step(r, dev[r][0])
+    model.sync(**sync_args(cfg))
+    torch.cuda.synchronize()
+    graphs = capture_graphs(model, dev)
+    m = measure_training(model, graphs, cfg, K, W, Barrier(1), device, args)
+    value, on, info = summarise_training(m, K)
+    kernels, per_step = profile_pass(model, dev, cfg, steps=3)
+    leg = {"value": value, "unit": UNIT, "ms_per_step": on["median_ms"] / K, "config": {"workload": workload_text(cfg)},
+           "sync": info, "roofline": roofline(kernels, model, host, cfg, peaks),
+           "kernel_launches_per_replica_step": per_step, "status_word": model.status()}
+    del graphs, dev, host, model
+    return leg
+
+
+def concurrent_sweep(model, graphs, cfg, K, W, args, peaks, value_off):
+    """The sync-kernel sweep run concurrently with this workload's training: the shadow thread loops a sync pass
+    over R vectors of n floats each (separate buffers, N(0, 0.02^2)) on the lowest-priority stream while the
+    replicas train; per point the training throughput, its loss against the sync-off figure and the sync traffic
+    the passes got under that contention (algorithmic bytes of the completed passes / time)."""
+    import torch
+    from paper_2003_03477_b200 import binding as ss
+    device = model.center.device
+    rows = []
+    Rs = (2, 4, 8, 16) if args.sweep_all_r else (cfg.R,)
+    gen = torch.Generator(device=device).manual_seed(20030347)
+    for n in (1 << 20, 1 << 23, 1 << 26, 1 << 28):
+        for R in Rs:
+            if (R + 2) * n * 4 > 40e9:
+                continue
+            ws = [torch.randn(n, device=device, generator=gen) * 0.02 for _ in range(R)]
+            c = ws[0].clone()
+            d = torch.zeros(n, device=device)
+            for rule, alpha, eta, mu in (("easgd", 0.1, 1.0, 0.0), ("ma", 0.1, 1.0, 0.0), ("bmuf", 0.1, 1.0, 0.9)):
+                h = ss.ss_shadow_start(rule, ws, c, d, n, alpha, eta, mu, 0, None, model.sync_stream, args.sync_in_flight, 0)
+                ss.ss_shadow_pause(h, True)
+                run_steps(model, graphs, 0, W)
+                torch.cuda.synchronize()
+                reps = 0
+                t_ms = 0.0
+                r0 = ss.ss_shadow_rounds(h)
+                ss.ss_shadow_pause(h, False)
+                while t_ms < 1e3 * args.sweep_seconds or reps < 2:
+                    ms, _ = timed_region(model, graphs, W + reps * K, K)
+                    t_ms += ms
+                    reps += 1
+                ss.ss_shadow_pause(h, True)
+                passes = ss.ss_shadow_rounds(h) - r0
+                ss.ss_shadow_stop(h)
+                ex = cfg.R * cfg.B * K * reps / (t_ms * 1e-3)
+                gbs = SYNC_VECTORS[rule](R) * 4 * n * passes / (t_ms * 1e-3) / 1e9
+                rows.append({"rule": rule, "R": R, "n": n, "train_examples_per_s": ex,
+                             "train_loss_pct": 100.0 * (1.0 - ex / value_off), "sync_passes_per_s": passes / (t_ms * 1e-3),
+                             "sync_GB/s": gbs, "sync_frac_of_hbm_peak": gbs / peaks["hbm_gbs"],
+                             "timed_s": t_ms * 1e-3})
+            del ws, c, d
+            torch.cuda.empty_cache()
+    return {"training": workload_text(cfg), "rows": rows,
+            "note": "sync vectors are separate buffers; passes counted as completed (thread paused and drained at both "
+                    "ends); train_loss_pct is against examples_per_s_sync_off of the same run"}
 
 
 def gemm_alone(stream, peaks):
@@ -505,14 +674,28 @@ def embedding_alone(model, host, dev, cfg, peaks):
 
     base = graph_ms(None)
     out = {}
-    for name, fn, nbytes in (
-            ("embbag_fwd", fwd, hb.L * (4 * D + 4) + 4 * (T * B + 1) + T * B * D * (2 if cfg.bf16 else 4)),
-            ("embbag_bwd_apply", apply, hb.L * (4 * D + 16) + U * (2 * 4 * D + 8))):
+    obytes = T * B * D * (2 if cfg.bf16 else 4)
+    for name, fn, nbytes, compulsory, kernels in (
+            ("embbag_fwd", fwd, hb.L * (4 * D + 4) + 4 * (T * B + 1) + obytes,
+             U * 4 * D + 4 * hb.L + 4 * (T * B + 1) + obytes, ("embbag_fwd_kernel",)),
+            ("embbag_bwd_apply", apply, hb.L * (4 * D + 16) + U * (2 * 4 * D + 8),
+             U * (2 * 4 * D + 8) + T * B * 4 * D + 16 * hb.L, ("window_apply_kernel", "combine_rows_kernel"))):
         us = (graph_ms(fn) - base) * 1e3 / reps
         gbs = nbytes / (us * 1e-6) / 1e9
-        out[name] = {"us": us, "algorithmic_bytes": nbytes, "GB/s": gbs, "frac_of_hbm_peak": gbs / peaks["hbm_gbs"]}
-    out["note"] = ("L2 flushed before every launch; Zipf-hot rows and the gathered gradient rows are re-read through L2 "
-                   "within a launch; embbag_bwd_apply = fused window kernel + combine kernel")
+        cgbs = compulsory / (us * 1e-6) / 1e9
+        dram = [ncu_traffic(k, cfg.name) for k in kernels]
+        dram = sum(dram) if all(d is not None for d in dram) else None
+        out[name] = {"us": us, "algorithmic_bytes": nbytes, "GB/s": gbs, "frac_of_hbm_peak": gbs / peaks["hbm_gbs"],
+                     "compulsory_bytes": compulsory, "compulsory_GB/s": cgbs,
+                     "compulsory_frac_of_hbm_peak": cgbs / peaks["hbm_gbs"],
+                     "dram_bytes_ncu": dram,
+                     "dram_GB/s_ncu_bytes_over_this_time": (dram / (us * 1e-6) / 1e9) if dram else None}
+    out["note"] = ("L2 flushed before every launch.  algorithmic_bytes counts every lookup's row (forward) or gradient row "
+                   "(backward) once per lookup, which is what the kernels move between L2 and the SMs: Zipf-hot rows and the "
+                   "gathered gradient rows are served from L2 within a launch, so this is an effective figure and is the one "
+                   "the 0.70 target is read against; compulsory_bytes counts each distinct row, the gradient matrix and the "
+                   "index / sort metadata once (what must cross DRAM); dram_bytes_ncu is dram__bytes_read + write of one ncu "
+                   "capture (null when the kernels changed since).  embbag_bwd_apply = window kernel + combine kernel")
     return out
 
 
@@ -523,14 +706,15 @@ def profile_pass(model, dev, cfg, steps=6, replicas=None):
     import torch
     from paper_2003_03477_b200 import binding as ss
     reps = list(range(cfg.R)) if replicas is None else list(replicas)
+    ring = len(dev[0])
     for t in range(2):
         for r in reps:
-            model.step(r, dev[r][t % RING])
+            model.step(r, dev[r][t % ring])
     torch.cuda.synchronize()
     ss.ss_profile(True)
     for t in range(steps):
         for r in reps:
-            model.step(r, dev[r][t % RING])
+            model.step(r, dev[r][t % ring])
     recs = ss.ss_profile_collect()
     ss.ss_profile(False)
     agg = {}
@@ -591,20 +775,24 @@ def roofline(kernels, model, host, cfg, peaks):
             "timing": "CUDA events around every launch on its stream, all replicas training concurrently"}
 
 
-def bench_e2e(model, host, dev, graphs, cfg, K, W):
+def bench_e2e(model, host, dev, graphs, cfg, K, W, args):
     """Same metric with the step's inputs in pinned host memory: every step copies its batch host->device
-    into the ring slot's device buffers, replays that slot's captured step and reads the loss back."""
+    into the ring slot's device buffers, replays that slot's captured step and reads the loss back.  Host wall
+    clock around exactly K steps (ending with a synchronise of every replica stream), the region repeated until
+    half of args.min_seconds has been timed; the median region gives the value."""
     import torch
     from paper_2003_03477_b200 import trainer
     pinned = [[tuple(torch.from_numpy(np.ascontiguousarray(a)).pin_memory() for a in
                      (b.indices, b.offsets, b.dense, b.labels)) for b in bs] for bs in host]
     loss_host = [torch.zeros(1).pin_memory() for _ in range(cfg.R)]
     h2d = d2h = 0
+    ring = len(dev[0])
+    paced = cfg.sync_every
 
     def step(t):
         nonlocal h2d, d2h
         for r, rep in enumerate(model.replicas):
-            slot = t % RING
+            slot = t % ring
             src, dst = pinned[r][slot], dev[r][slot]
             with torch.cuda.stream(rep.stream):
                 dst.indices.copy_(src[0], non_blocking=True)
@@ -615,22 +803,29 @@ def bench_e2e(model, host, dev, graphs, cfg, K, W):
                 loss_host[r].copy_(rep.loss, non_blocking=True)
             h2d += sum(x.numel() * x.element_size() for x in src)
             d2h += 4
+        if paced and (t + 1) % paced == 0:
+            model.sync(**sync_args(cfg))
 
-    loop = trainer.ShadowLoop(model, cfg.sync, cfg.alpha, cfg.eta, cfg.mu).start()
+    loop = None if paced else trainer.ShadowLoop(model, cfg.sync, cfg.alpha, cfg.eta, cfg.mu).start()
     for t in range(W):
         step(t)
     torch.cuda.synchronize()
-    h2d = d2h = 0
-    t0 = time.perf_counter()
-    for t in range(W, W + K):
-        step(t)
-    for rep in model.replicas:
-        rep.stream.synchronize()
-    dt = time.perf_counter() - t0
-    loop.stop()
+    times = []
+    while len(times) < 3 or (sum(times) < 0.5 * args.min_seconds and len(times) < 200):
+        h2d = d2h = 0
+        t0 = time.perf_counter()
+        for t in range(W, W + K):
+            step(t)
+        for rep in model.replicas:
+            rep.stream.synchronize()
+        times.append(time.perf_counter() - t0)
+    if loop is not None:
+        loop.stop()
     torch.cuda.synchronize()
+    dt = statistics.median(times)
     return {"value": cfg.R * cfg.B * K / dt, "unit": UNIT, "h2d_bytes_per_step": h2d // K, "d2h_bytes_per_step": d2h // K,
-            "timing": "host wall clock around K steps, ending with a synchronise of every replica stream"}
+            "regions": {"median_ms": dt * 1e3, "min_ms": min(times) * 1e3, "max_ms": max(times) * 1e3, "repeats": len(times)},
+            "timing": "host wall clock around K steps, ending with a synchronise of every replica stream; median of the repeats"}
 
 
 # ----------------------------------------------------------------------------------------------
@@ -670,7 +865,11 @@ def oracle_sample(cfg, budget_s):
 
 def cpu_baseline(cfg, budget_s):
     n, dt, what = oracle_sample(cfg, budget_s)
-    return {"value": n / dt, "unit": UNIT, "cores": threads_used(), "kind": "oracle", "sample": what}
+    blas = threads_used()
+    return {"value": n / dt, "unit": UNIT, "cores": blas, "kind": "oracle",
+            "threads": {"python": 1, "blas": blas},
+            "sample": what + f"; one Python thread (pooling, sort and segment loops), numpy matrix products on up to "
+                             f"{blas} BLAS threads"}
 
 
 def threads_used():
@@ -704,7 +903,9 @@ def bench_reference(args):
         "steps": K, "warmup": W, "ms_per_step": 1e3 * dt / K, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": {"workload": f"{cfg.name} (CPU oracle on a bounded sample)"},
-        "cpu_baseline": {"value": v, "unit": UNIT, "cores": threads_used(), "kind": "oracle", "sample": what + " per step"},
+        "cpu_baseline": {"value": v, "unit": UNIT, "cores": threads_used(), "kind": "oracle",
+                         "threads": {"python": 1, "blas": threads_used()},
+                         "sample": what + " per step; one Python thread, numpy matrix products on the BLAS threads"},
         "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0}))
 
@@ -739,10 +940,37 @@ def bench_sweep(args):
     print(json.dumps({"sweep": "sync kernels alone", "peak_gbs": peaks["hbm_gbs"], "peak_source": peaks["source"], "rows": rows}))
 
 
+def plain_steps(args):
+    """A few plain (un-captured) replica steps of a workload on one GPU, every library call launched directly on the
+    replica's stream so that each kernel shows up as its own launch: the program profilers are pointed at.
+    --tables / --rows / --batch shrink the workload (fewer or shorter tables, smaller batch) while keeping its layer
+    widths, bag-length mix and index skew; --plain-sync adds one synchronisation pass after every step."""
+    import torch
+    from paper_2003_03477_b200 import binding as ss, synth, trainer
+    cfg = synth.CONFIGS[args.workload]
+    if args.tables:
+        cfg = synth.scaled(cfg, T=args.tables, top=((1 + args.tables) * cfg.D,) + tuple(cfg.top[1:]))
+    if args.rows:
+        cfg = synth.scaled(cfg, N=args.rows)
+    if args.batch:
+        cfg = synth.scaled(cfg, B=args.batch)
+    cfg = synth.scaled(cfg, R=args.replicas or 1)
+    torch.cuda.set_device(0)
+    model, host, dev, _ = build_job(cfg, torch.device("cuda", 0), ring=2)
+    for t in range(args.steps):
+        for r in range(cfg.R):
+            model.step(r, dev[r][t % 2])
+        if args.plain_sync:
+            model.sync(cfg.sync, cfg.alpha, cfg.eta, cfg.mu)
+    torch.cuda.synchronize()
+    print(json.dumps({"plain": workload_text(cfg), "steps": args.steps, "loss": float(model.replicas[0].loss.item()),
+                      "status_word": model.status()}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=1000)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="medium", choices=["tiny", "medium", "medium_bmuf", "large"])
@@ -750,18 +978,32 @@ def main():
     ap.add_argument("--sync-pause", type=float, default=0.0)
     ap.add_argument("--steps-ahead", type=int, default=16,
                     help="steps of a replica the host keeps queued on the device (0 = unbounded)")
+    ap.add_argument("--min-seconds", type=float, default=1.0,
+                    help="the K-step region is repeated until this much has been timed per arm (sync on, sync off)")
+    ap.add_argument("--min-repeats", type=int, default=10)
     ap.add_argument("--cpu-budget", type=float, default=15.0)
     ap.add_argument("--replicas", type=int, default=0, help="override the workload's replica count (experiments)")
-    ap.add_argument("--quick", action="store_true", help="skip the e2e and CPU-baseline legs (experiments)")
+    ap.add_argument("--quick", action="store_true", help="skip the e2e, CPU-baseline, concurrent-sweep and other-workload legs")
+    ap.add_argument("--no-legs", action="store_true", help="skip the medium_bmuf and large legs")
+    ap.add_argument("--no-sweep", action="store_true", help="skip the sync sweep concurrent with training")
+    ap.add_argument("--sweep-seconds", type=float, default=0.25, help="training time per point of the concurrent sweep")
+    ap.add_argument("--sweep-all-r", action="store_true", help="concurrent sweep over R = 2, 4, 8, 16 instead of the workload's R")
     ap.add_argument("--foreground", type=int, default=0,
                     help="also time the foreground variant: one sync pass on the training streams every k steps")
     ap.add_argument("--workers", type=int, default=1,
                     help="also time m lock-free workers per replica sharing its parameters (intra-trainer Hogwild)")
     ap.add_argument("--sweep", action="store_true", help="isolated sync-kernel sweep instead of the training benchmark")
+    ap.add_argument("--plain", action="store_true", help="run --steps un-captured replica steps and exit (for profilers)")
+    ap.add_argument("--tables", type=int, default=0, help="--plain: number of tables")
+    ap.add_argument("--rows", type=int, default=0, help="--plain: rows per table")
+    ap.add_argument("--batch", type=int, default=0, help="--plain: per-replica batch")
+    ap.add_argument("--plain-sync", action="store_true", help="--plain: one sync pass after every step")
     args = ap.parse_args()
     global STEPS_AHEAD
     STEPS_AHEAD = max(0, args.steps_ahead)
-    if args.sweep:
+    if args.plain:
+        plain_steps(args)
+    elif args.sweep:
         bench_sweep(args)
     elif args.impl == "reference":
         bench_reference(args)

@@ -249,13 +249,17 @@ ss_status ss_sync_bmuf(float* const* w, int R, float* global, float* delta, int6
  * device runs the passes in whatever room training leaves.  The pointer arrays are copied; the
  * buffers they point to must outlive ss_shadow_stop, which joins the thread, waits for the queued
  * passes, stores the number of passes in *rounds_out (nullable), frees the handle and returns the
- * first error the thread met (SS_OK if none).  ss_shadow_rounds reads the running count.
+ * first error the thread met (SS_OK if none).  ss_shadow_rounds reads the running count of passes
+ * enqueued.  ss_shadow_pause(h, 1) makes the thread stop enqueuing and returns once every pass it
+ * had enqueued has completed on the device (ss_shadow_rounds is then the number of completed
+ * passes); ss_shadow_pause(h, 0) lets it loop again.  A paused thread still ends on ss_shadow_stop.
  * ---------------------------------------------------------------------------------------- */
 typedef struct ss_shadow ss_shadow;
 ss_status ss_shadow_start(ss_shadow** out, int rule, float* const* w, int R, float* center, float* delta, int64_t n,
                           float alpha, float eta, float mu, int flags, void* const* w_bf16, ss_stream stream,
                           int max_in_flight, int pause_us, int64_t max_rounds);
 int64_t ss_shadow_rounds(const ss_shadow* h);
+ss_status ss_shadow_pause(ss_shadow* h, int paused);
 ss_status ss_shadow_stop(ss_shadow* h, int64_t* rounds_out);
 
 /* ------------------------------------------------------------------------------------------

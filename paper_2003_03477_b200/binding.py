@@ -26,7 +26,7 @@ SS_SYNC_BMUF_NESTEROV = 2
 
 EXPORTS = ["ss_status_str", "ss_last_cuda_error", "ss_num_sms", "ss_embbag_fwd", "ss_embbag_bwd_workspace_bytes",
            "ss_embbag_bwd_adagrad", "ss_embbag_bwd_sort", "ss_embbag_bwd_apply", "ss_embbag_bwd_sort_noalloc", "ss_mlp_param_count", "ss_mlp_param_offsets", "ss_mlp_workspace_bytes",
-           "ss_mlp_fwd", "ss_mlp_bwd", "ss_ne_accumulate", "ss_ne_value", "ss_sync_easgd", "ss_sync_ma", "ss_sync_bmuf", "ss_shadow_start", "ss_shadow_rounds", "ss_shadow_stop", "ss_to_bf16",
+           "ss_mlp_fwd", "ss_mlp_bwd", "ss_ne_accumulate", "ss_ne_value", "ss_sync_easgd", "ss_sync_ma", "ss_sync_bmuf", "ss_shadow_start", "ss_shadow_rounds", "ss_shadow_pause", "ss_shadow_stop", "ss_to_bf16",
            "ss_gemm_bf16", "ss_device_error", "ssh_fill_uniform", "ss_profile", "ss_profile_collect"]
 
 
@@ -86,6 +86,7 @@ def lib() -> C.CDLL:
                                       i32, i32, i64]
         L.ss_shadow_rounds.argtypes = [vp]
         L.ss_shadow_rounds.restype = i64
+        L.ss_shadow_pause.argtypes = [vp, i32]
         L.ss_shadow_stop.argtypes = [vp, C.POINTER(i64)]
         L.ss_to_bf16.argtypes = [vp, vp, i64, vp]
         L.ss_gemm_bf16.argtypes = [vp, i32, i64, vp, i32, i64, vp, i64, i32, i32, i32, i32, vp]
@@ -282,6 +283,11 @@ def ss_shadow_start(rule, w, center, delta, n, alpha, eta=1.0, mu=0.0, flags=0, 
 
 def ss_shadow_rounds(handle) -> int:
     return int(lib().ss_shadow_rounds(handle))
+
+
+def ss_shadow_pause(handle, paused: bool) -> None:
+    """paused=True: stop enqueuing and return once every enqueued pass has completed; False: loop again."""
+    _check("ss_shadow_pause", lib().ss_shadow_pause(handle, 1 if paused else 0))
 
 
 def ss_shadow_stop(handle) -> int:

@@ -48,8 +48,10 @@ embbag_fwd_kernel(const float* __restrict__ tables, int T, int64_t N, int D,
   const int t = (int)(bag / B);
   const int b = (int)(bag - (int64_t)t * B);
   int lo = offsets[bag], hi = offsets[bag + 1];
+  // the index list ends where the last bag ends; a bag that is not inside [0, L] in ascending order is treated as empty
+  const int L = __ldg(offsets + (int64_t)T * B);
   int bad = 0;
-  if (lo < 0 || hi < lo) { bad |= SS_DEV_BAD_OFFSET; hi = lo; }
+  if (lo < 0 || hi < lo || hi > L) { bad |= SS_DEV_BAD_OFFSET; lo = hi = 0; }
   const float4* tab = reinterpret_cast<const float4*>(tables + (int64_t)t * N * D);
   const int nvec = D >> 2;
 

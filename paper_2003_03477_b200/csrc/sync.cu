@@ -233,6 +233,8 @@ struct ss_shadow {
   cudaStream_t stream;
   std::atomic<int64_t> rounds{0};
   std::atomic<int> stop{0};
+  std::atomic<int> paused{0};      // set by ss_shadow_pause; the thread drains its passes and idles while it is set
+  std::atomic<int> idle{0};        // the thread's answer: 1 while it idles with nothing queued
   std::atomic<int> status{SS_OK};
   std::thread thread;
 };
@@ -245,6 +247,15 @@ static void shadow_main(ss_shadow* h) {
     if (cudaEventCreateWithFlags(&ev[i], cudaEventDisableTiming) != cudaSuccess) { h->status = SS_ERR_CUDA; return; }
   int64_t k = 0;
   while (!h->stop.load(std::memory_order_relaxed) && k < h->max_rounds) {
+    if (h->paused.load(std::memory_order_acquire)) {
+      // every pass enqueued so far has completed before the pause is acknowledged
+      for (int i = 0; i < depth && i < k; ++i) cudaEventSynchronize(ev[i]);
+      h->idle.store(1, std::memory_order_release);
+      while (h->paused.load(std::memory_order_acquire) && !h->stop.load(std::memory_order_relaxed))
+        std::this_thread::sleep_for(std::chrono::microseconds(20));
+      h->idle.store(0, std::memory_order_release);
+      continue;
+    }
     const int slot = (int)(k % depth);
     if (k >= depth && cudaEventSynchronize(ev[slot]) != cudaSuccess) { h->status = SS_ERR_CUDA; break; }
     ss_status st;
@@ -261,6 +272,7 @@ static void shadow_main(ss_shadow* h) {
     cudaEventSynchronize(ev[i]);
     cudaEventDestroy(ev[i]);
   }
+  h->idle.store(1, std::memory_order_release);             // ended: nothing in flight
 }
 
 extern "C" {
@@ -288,6 +300,19 @@ ss_status ss_shadow_start(ss_shadow** out, int rule, float* const* w, int R, flo
 }
 
 int64_t ss_shadow_rounds(const ss_shadow* h) { return h ? h->rounds.load(std::memory_order_relaxed) : -1; }
+
+ss_status ss_shadow_pause(ss_shadow* h, int paused) {
+  if (!h) return SS_ERR_NULL;
+  h->paused.store(paused ? 1 : 0, std::memory_order_release);
+  if (!paused) return SS_OK;
+  // wait (at most ~30 s) until the thread has drained its queued passes and idles, or has ended by itself
+  for (int i = 0; i < 1500000; ++i) {
+    if (h->idle.load(std::memory_order_acquire) || h->status.load() != SS_OK)
+      return (ss_status)h->status.load();
+    std::this_thread::sleep_for(std::chrono::microseconds(20));
+  }
+  return SS_ERR_CUDA;
+}
 
 ss_status ss_shadow_stop(ss_shadow* h, int64_t* rounds_out) {
   if (!h) return SS_ERR_NULL;

@@ -202,7 +202,9 @@ class Model:
             rep.stream.wait_event(done)
 
     def status(self) -> int:
-        return int(self.d_status.item())
+        """Device-detected problems so far: the SS_DEV_* bits of malformed input in the low byte, and from bit 8
+        up the code of a tensor-core kernel's bounded wait that ran out (0 = none).  Synchronises the device."""
+        return int(self.d_status.item()) | (ss.ss_device_error(False) << 8)
 
 
 class ShadowLoop:
@@ -232,6 +234,14 @@ class ShadowLoop:
                                           self.mu, 0, mirrors, m.sync_stream, self.max_in_flight,
                                           int(self.pause_s * 1e6), self.max_rounds)
         return self
+
+    def pause(self) -> int:
+        """Stop enqueuing, wait for the queued passes; returns the number of passes completed so far."""
+        ss.ss_shadow_pause(self._handle, True)
+        return self.rounds
+
+    def resume(self) -> None:
+        ss.ss_shadow_pause(self._handle, False)
 
     def stop(self) -> int:
         if self._handle is not None:

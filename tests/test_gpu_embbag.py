@@ -69,6 +69,25 @@ def test_fwd_edge_cases_empty_bags_single_row_duplicates_and_bad_index():
     assert st == 0 and np.array_equal(got[:, 0], [0, 1, 3]) and np.array_equal(got[:, 8], [2, 0, 2])
 
 
+def test_fwd_malformed_offsets_give_empty_bags_and_a_status_bit():
+    """Offsets that decrease, are negative or point beyond the end of the index list (offsets[T*B]) must not
+    become reads outside the list: such a bag pools to zero and SS_DEV_BAD_OFFSET is raised; the well-formed
+    bags of the same call are unaffected."""
+    tables = np.random.default_rng(1).normal(size=(1, 7, 8)).astype(np.float32)
+    idx = np.array([3, 5, 6, 1], np.int32)
+    for off, bad_bags in ((np.array([0, 1, 1 << 30, 3, 4], np.int32), (1, 2)),     # far beyond the list
+                          (np.array([0, 2, 1, 3, 4], np.int32), (1,)),              # decreasing
+                          (np.array([0, -5, 2, 3, 4], np.int32), (0, 1))):          # negative
+        got, _, st = _fwd(tables, idx, off, 4, col0=0)
+        assert st & ss.SS_DEV_BAD_OFFSET, off
+        for b in range(4):
+            if b in bad_bags:
+                assert not got[b].any(), (off, b)
+            else:
+                want = tables[0, idx[off[b]:off[b + 1]]].astype(np.float64).sum(axis=0)
+                assert_close(got[b], want, RTOL_F32, f"bag {b}", floor=1.0)
+
+
 def _bwd(cfg, batch, tables, state, gp, keep=True):
     T, N, D, B, L = cfg.T, cfg.N, cfg.D, cfg.B, batch.L
     dt, ds = _cuda(tables), _cuda(state.reshape(-1))
@@ -115,8 +134,9 @@ def test_bwd_parity_small_uniform(D):
 
 
 def test_bwd_parity_skewed_long_segments_cross_windows_and_sort_tiles():
-    # Zipf rows: the hottest row of each table has hundreds of lookups -> runs spanning many 32-wide windows;
-    # L is about 21k -> several 4096-item sort tiles with a ragged last one
+    # Zipf rows: the hottest row of each table has hundreds of lookups -> runs spanning many 16-wide windows;
+    # about 5k lookups per table: the per-table shared-memory sort takes them (the tiled passes are covered by the
+    # malformed-input cases, the no-scratch entry point and the full-size test of the large workload)
     cfg = synth.scaled(synth.CONFIGS["medium"], T=4, N=20_000, D=64, B=512, bottom=(13, 64, 64), top=(320, 64, 1))
     U, L = _check_bwd(cfg)
     assert L > 4 * 4096 and U < L // 2

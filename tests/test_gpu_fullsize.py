@@ -77,7 +77,7 @@ def test_medium_workload_first_step_full_size_as_benchmarked():
                                              cfg.eps, cfg.bf16, rep.grad_pooled.cpu().numpy(), RTOL_BF16)
     assert len(flips) <= 1e-4 * cfg.B * (sum(cfg.bottom[1:]) + sum(cfg.top[1:-1])), flips
 
-    # integer outputs, bit-exact at full size (560k lookups, 3 radix passes, 137 sort tiles)
+    # integer outputs, bit-exact at full size (560k lookups: 26 per-table sorts in shared memory, 3 digit passes each)
     U = int(rep.num_unique.item())
     assert U == len(uniq) == len(out["uniq_keys"])
     assert np.array_equal(rep.uniq_keys.cpu().numpy()[:U], uniq)
@@ -104,6 +104,91 @@ def test_medium_workload_first_step_full_size_as_benchmarked():
         rows = np.setdiff1d(rng.integers(0, cfg.N, 400), uniq[t_of == t] % cfg.N)
         got = model.tables[t][torch.from_numpy(rows).cuda()].cpu().numpy()
         assert np.array_equal(got, synth.table_rows(cfg, t, rows))
+
+
+def test_large_workload_embedding_path_full_size():
+    """The embedding calls of the large workload at its full size (26 tables of 4 M rows x 128 floats = 53 GB filled
+    on the device, batch 4096, about 852 k lookups with 27-bit keys): more lookups than the per-table shared-memory
+    sort can hold, so the tiled radix passes run (three digits, about 208 tiles), the hottest row of a table has
+    thousands of lookups (runs spanning hundreds of reduction windows) and rows are 128 floats wide.  Forward, sort
+    (integers bit-exact) and reduction + row-wise Adagrad against the oracle on the compact table of touched rows;
+    the gradient is a seeded synthetic matrix, so no MLP (and no ReLU gate) is involved."""
+    cfg = synth.scaled(synth.CONFIGS["large"], R=1)
+    T, N, D, B = cfg.T, cfg.N, cfg.D, cfg.B
+    batch = synth.make_batch(cfg, 0, 0)
+    L = batch.L
+    assert L > T * ss.SS_TABLE_SORT_CAP                      # the tiled passes are certain
+    tables_c, small, uniq, t_of, local, nmax = _compact(cfg, batch)
+    tables = trainer.device_tables(cfg)
+    state = torch.zeros(T * N, dtype=torch.float32, device="cuda")
+    idx, off = torch.from_numpy(batch.indices).cuda(), torch.from_numpy(batch.offsets).cuda()
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    W = (1 + T) * D
+    concat = torch.zeros(B, W, device="cuda")
+    ss.ss_embbag_fwd(tables, T, N, D, idx, off, B, concat, W, None, W, D, status)
+    want_pooled = O.embbag_fwd(tables_c, small.indices, small.offsets, B)
+    assert_close(concat.cpu().numpy()[:, D:], want_pooled.reshape(B, -1), RTOL_F32, "pooled")
+
+    ws = torch.empty(ss.ss_embbag_bwd_workspace_bytes(T, N, D, B, L), dtype=torch.uint8, device="cuda")
+    uk = torch.empty(L, dtype=torch.int32, device="cuda")
+    so = torch.empty(L + 1, dtype=torch.int32, device="cuda")
+    pm = torch.empty(L, dtype=torch.int32, device="cuda")
+    nu = torch.zeros(1, dtype=torch.int32, device="cuda")
+    ss.ss_embbag_bwd_sort(T, N, D, idx, off, B, L, ws, uk, so, pm, nu, status)
+    torch.cuda.synchronize()
+    want_uniq, want_seg, want_perm = O.sort_unique(batch.indices, batch.offsets, T, N, B)
+    U = int(nu.item())
+    assert U == len(want_uniq) == len(uniq)
+    assert np.array_equal(uk.cpu().numpy()[:U], want_uniq)
+    assert np.array_equal(so.cpu().numpy()[:U + 1], want_seg)
+    assert np.array_equal(pm.cpu().numpy(), want_perm)
+    assert int(np.diff(want_seg).max()) > 2000               # a run over hundreds of 16-position windows
+
+    gp = (synth.normal_f32(synth.stream_key(cfg.seed, synth.stream_id(synth.KIND_VEC, 77)), B * T * D, 1e-3)
+          .reshape(B, T * D))
+    ss.ss_embbag_bwd_apply(tables, state, T, N, D, B, L, torch.from_numpy(gp).cuda(), T * D, 0, cfg.lr, cfg.eps, ws, status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    t_before = tables_c.copy()
+    state_c = np.zeros((T, nmax), np.float32)
+    O.embbag_bwd_adagrad(tables_c, state_c, small.indices, small.offsets, B, gp, cfg.lr, cfg.eps)
+    ukeys = torch.from_numpy(uniq).cuda()
+    rows_dev = tables.view(-1, D)[ukeys].cpu().numpy()
+    # the row step is lr * g / (sqrt(s) + eps): compared on the step, 2e-5 (a sum of up to thousands of float terms)
+    assert_close(rows_dev - t_before[t_of, local], tables_c[t_of, local].astype(np.float64) - t_before[t_of, local],
+                 2e-5, "row updates")
+    assert_close(state[ukeys].cpu().numpy(), state_c[t_of, local], 2e-5, "row state")
+    rng = np.random.default_rng(1)
+    for t in (0, 12, 25):                                    # untouched rows keep their initial values
+        rows = np.setdiff1d(rng.integers(0, N, 300), uniq[t_of == t] % N)
+        assert np.array_equal(tables[t][torch.from_numpy(rows).cuda()].cpu().numpy(), synth.table_rows(cfg, t, rows))
+
+
+def test_sort_with_one_table_beyond_the_shared_memory_sort_beside_tables_within_it():
+    """Three tables in one call: the middle one has more lookups than one block of the per-table sort holds
+    (its block raises the fallback word and the tiled passes redo the whole call), the outer two would fit."""
+    T, N, B = 3, 1 << 20, 4096
+    rng = np.random.default_rng(11)
+    lens = np.concatenate([rng.integers(1, 4, B), rng.integers(6, 12, B), rng.integers(0, 3, B)])
+    off = np.zeros(T * B + 1, np.int32)
+    off[1:] = np.cumsum(lens)
+    L = int(off[-1])
+    assert int(off[2 * B] - off[B]) > ss.SS_TABLE_SORT_CAP and L <= T * ss.SS_TABLE_SORT_CAP
+    idx = (rng.zipf(1.3, L) % N).astype(np.int32)
+    ws = torch.empty(ss.ss_embbag_bwd_workspace_bytes(T, N, 64, B, L), dtype=torch.uint8, device="cuda")
+    uk = torch.empty(L, dtype=torch.int32, device="cuda")
+    so = torch.empty(L + 1, dtype=torch.int32, device="cuda")
+    pm = torch.empty(L, dtype=torch.int32, device="cuda")
+    nu = torch.zeros(1, dtype=torch.int32, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    ss.ss_embbag_bwd_sort(T, N, 64, torch.from_numpy(idx).cuda(), torch.from_numpy(off).cuda(), B, L, ws, uk, so, pm, nu, status)
+    torch.cuda.synchronize()
+    want_uniq, want_seg, want_perm = O.sort_unique(idx, off, T, N, B)
+    U = int(nu.item())
+    assert int(status.item()) == 0 and U == len(want_uniq)
+    assert np.array_equal(uk.cpu().numpy()[:U], want_uniq)
+    assert np.array_equal(so.cpu().numpy()[:U + 1], want_seg)
+    assert np.array_equal(pm.cpu().numpy(), want_perm)
 
 
 @pytest.mark.parametrize("rule", ["easgd", "ma", "bmuf"])

@@ -165,6 +165,34 @@ def test_shadow_loop_free_running_keeps_invariants():
     assert float((m.replicas[0].w - m.center).abs().max()) < 0.5
 
 
+def test_shadow_loop_pause_counts_completed_passes_and_resume_continues():
+    """A paused shadow thread has no pass in flight: the vectors stay put until it is resumed, and the pass count
+    read while paused equals the number of S-EASGD passes the vectors have actually been through."""
+    n, R, alpha = 1 << 16, 2, 0.25
+    ws = [torch.full((n,), float(r + 1), device="cuda") for r in range(R)]
+    c = torch.zeros(n, device="cuda")
+    s = torch.cuda.Stream()
+    h = ss.ss_shadow_start("easgd", ws, c, None, n, alpha, stream=s, max_in_flight=2, max_rounds=1 << 40)
+    import time
+    time.sleep(0.02)
+    ss.ss_shadow_pause(h, True)
+    k = ss.ss_shadow_rounds(h)
+    snap = [w.clone() for w in ws] + [c.clone()]
+    time.sleep(0.02)
+    assert ss.ss_shadow_rounds(h) == k and all(torch.equal(a, b) for a, b in zip(snap, ws + [c]))
+    # k passes of Algorithm 2 on the scalars (1, 2 | 0), in the oracle
+    w0 = [np.full(1, float(r + 1), np.float32) for r in range(R)]
+    c0 = np.zeros(1, np.float32)
+    for _ in range(k):
+        O.sync_easgd(w0, c0, alpha)
+    assert k >= 1
+    for r in range(R):
+        assert_close(ws[r][:1].cpu().numpy(), w0[r], 1e-5, "replica after k passes", floor=1.0)
+    ss.ss_shadow_pause(h, False)
+    time.sleep(0.02)
+    assert ss.ss_shadow_stop(h) > k
+
+
 def test_foreground_sync_variants_match_the_oracle_rules():
     # FR-EASGD: each replica interpolates with the centre on its own stream; FR-MA / FR-BMUF: one joint pass
     cfg = synth.scaled(synth.CONFIGS["tiny"], R=3)

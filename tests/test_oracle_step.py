@@ -2,6 +2,7 @@
 Adagrad, MLP forward/backward, dense Adagrad.  CPU only; the pins are library routines (torch in
 float64), finite differences, brute force and closed forms."""
 import math
+import os
 
 import numpy as np
 import pytest
@@ -341,3 +342,55 @@ def test_gate_matching_recovers_planted_edge_gates_and_nothing_else():
     assert np.abs(wrong - backward(fwd)).max() > 0
     matched, flips = match_relu_gates(fwd, backward, wrong, 1e-9, nb, len(layers))
     assert np.abs(backward(matched) - wrong)[b].max() > 0
+
+
+# ---------------------------------------------------------------- bf16 backward: which tensors are rounded, and where
+def _hand_bf16_case():
+    """The hand-computed case of tests/golden/mlp_bwd_bf16_hand.txt (inputs typed in here, results read from the file)."""
+    layers = [(np.array([[0.5]], np.float32), np.zeros(1, np.float32)),
+              (np.array([[1.0078125, 1.005859375], [-1.0, 3.0]], np.float32), np.zeros(2, np.float32)),
+              (np.array([[1.005859375, -0.75]], np.float32), np.zeros(1, np.float32))]
+    fwd = dict(inputs=[np.array([[1.005859375], [5.0]]),
+                       np.array([[0.75, 1.005859375], [0.0, -2.0078125]]),
+                       np.array([[1.005859375, 0.0], [0.5, 2.0078125]])],
+               pre=[np.array([[0.75], [-1.0]]), np.array([[1.005859375, -0.5], [0.5, 2.0078125]]), np.zeros((2, 1))],
+               prob=np.array([0.25, 0.5029296875]), logit=np.zeros(2))
+    want = {}
+    with open(os.path.join(os.path.dirname(__file__), "golden", "mlp_bwd_bf16_hand.txt")) as f:
+        for line in f:
+            if line.strip() and not line.startswith("#"):
+                name, *vals = line.split()
+                want[name] = np.array([float(v) for v in vals])
+    return layers, fwd, np.array([1.0, 0.0]), want
+
+
+def test_mlp_bwd_bf16_matches_the_hand_computed_case():
+    """Pins the bf16 branch of the backward pass: gradients are rounded after the ReLU mask where they enter a
+    product, weights and saved inputs are rounded as operands, bias gradients sum the rounded values, and the
+    gradient of the pooled embeddings leaves unrounded.  All values are dyadic, so the comparison is exact."""
+    layers, fwd, y, want = _hand_bf16_case()
+    grads, gp = O.mlp_bwd(layers, 1, fwd, y, bf16=True)
+    for l in range(3):
+        assert np.array_equal(grads[l][0].ravel(), want[f"dW{l}"]), (l, grads[l][0])
+        assert np.array_equal(grads[l][1].ravel(), want[f"db{l}"]), (l, grads[l][1])
+    assert np.array_equal(gp.ravel(), want["grad_pooled"])
+    # the case separates the readings: without any rounding every quantity but the masked zeros differs,
+    # a rounded grad_pooled or bias gradients summed before rounding would differ too
+    g64, gp64 = O.mlp_bwd(layers, 1, fwd, y, bf16=False)
+    assert abs(g64[2][1][0] - want["db2"][0]) > 1e-4 and abs(g64[1][1][0] - want["db1"][0]) > 1e-4
+    assert abs(g64[0][0][0, 0] - want["dW0"][0]) > 1e-3
+    assert not np.array_equal(O.round_bf16(want["grad_pooled"]), want["grad_pooled"])
+    d1 = np.array([[-0.3779296875, 0.0], [0.2539215087890625, -0.18896484375]])      # layer-1 gradient before rounding
+    assert not np.array_equal(d1.sum(axis=0), want["db1"])
+
+
+def test_mlp_fwd_bf16_rounds_operands_but_neither_bias_nor_pre_activation():
+    """Forward, one unit by hand: r(1.005859375) * r(0.50390625) + 2^-12 with r(1.005859375) = 1.0078125 and
+    0.50390625 = 0.5 * (1 + 2^-7) on the bf16 grid: 0.5078430175781250 + 0.000244140625, a value off the grid."""
+    layers = [(np.array([[0.50390625]], np.float32), np.array([2.0 ** -12], np.float32)),
+              (np.array([[1.0, 1.0]], np.float32), np.zeros(1, np.float32))]
+    f = O.mlp_fwd(layers, 1, np.array([[1.005859375]], np.float32), np.zeros((1, 1, 1), np.float32),
+                  np.array([1.0], np.float32), bf16=True)
+    assert f["pre"][0][0, 0] == 1.0078125 * 0.50390625 + 2.0 ** -12
+    # the next layer reads the activation rounded to bf16: r(0.508087158203125) = 0.5078125
+    assert f["logit"][0] == 0.5078125
