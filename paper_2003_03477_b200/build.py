@@ -50,7 +50,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
                 sys.stderr.write(res.stdout + res.stderr)
                 raise RuntimeError(f"nvcc failed on {src}")
     objs = [os.path.join(OBJ, s[:-3] + ".o") for s in _sources()]
-    if jobs or not os.path.exists(LIB):
+    if jobs or not os.path.exists(LIB) or os.path.getmtime(LIB) < max(os.path.getmtime(o) for o in objs):
         res = subprocess.run([nvcc, "-shared", "-o", LIB] + objs + ["-gencode", "arch=compute_100a,code=sm_100a"],
                              capture_output=True, text=True)
         if res.returncode != 0:

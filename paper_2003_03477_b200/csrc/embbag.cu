@@ -177,12 +177,11 @@ static BwdPlan make_plan(int T, int64_t N, int D, int64_t L) {
 // [0, L] (consecutive bags share an end, so the clamped ranges tile [clamp(off[0]), clamp(off[T*B])) even
 // when the offsets are not monotone), the first and the last bag also take what lies before and after.
 // Positions of a malformed bag, and lookups with a row index outside the table, get the sentinel key.
-__global__ void __launch_bounds__(256)
-build_keys_kernel(const int32_t* __restrict__ indices, const int32_t* __restrict__ offsets, int T, int64_t N,
-                  int B, int64_t L, uint32_t* __restrict__ keys, int32_t* __restrict__ bag_of,
-                  int32_t* __restrict__ d_status, const int32_t* __restrict__ run_if) {
-  if (run_if && *run_if == 0) return;                     // the per-table sort already produced the result
-  const int64_t bag = (int64_t)blockIdx.x * 256 + threadIdx.x;
+__device__ __forceinline__ void build_keys_block(int blk, const int32_t* __restrict__ indices,
+                                                 const int32_t* __restrict__ offsets, int T, int64_t N, int B, int64_t L,
+                                                 uint32_t* __restrict__ keys, int32_t* __restrict__ bag_of,
+                                                 int32_t* __restrict__ d_status) {
+  const int64_t bag = (int64_t)blk * 256 + threadIdx.x;
   const int64_t nbags = (int64_t)T * B;
   if (bag >= nbags) return;
   const uint32_t sentinel = (uint32_t)((uint64_t)T * (uint64_t)N);
@@ -212,6 +211,14 @@ build_keys_kernel(const int32_t* __restrict__ indices, const int32_t* __restrict
   if (bad && d_status) atomicOr(d_status, bad);
 }
 
+__global__ void __launch_bounds__(256)
+build_keys_kernel(const int32_t* __restrict__ indices, const int32_t* __restrict__ offsets, int T, int64_t N,
+                  int B, int64_t L, uint32_t* __restrict__ keys, int32_t* __restrict__ bag_of,
+                  int32_t* __restrict__ d_status, const int32_t* __restrict__ run_if) {
+  if (run_if && *run_if == 0) return;                     // the per-table sort already produced the result
+  build_keys_block(blockIdx.x, indices, offsets, T, N, B, L, keys, bag_of, d_status);
+}
+
 // ---- (2) radix sort pass ----------------------------------------------------------------
 // Lanes of the warp that hold the same digit, from one ballot per digit bit (cost independent of how many
 // distinct digits the warp holds).  `digit` is below 2^nbits, or exactly 2^nbits for a lane past the end.
@@ -227,22 +234,20 @@ __device__ __forceinline__ uint32_t same_digit_lanes(uint32_t digit, int nbits) 
 
 // hist[bin * nblk + blk] = number of keys of tile blk whose digit is bin.  Lanes holding the same
 // digit are counted together, so a hot row does not serialise on one counter.
-__global__ void __launch_bounds__(kSortThreads)
-sort_hist_kernel(const uint32_t* __restrict__ keys, int64_t L, int shift, int bins, int nblk,
-                 uint32_t* __restrict__ hist, const int32_t* __restrict__ run_if) {
-  __shared__ uint32_t cnt[kMaxBins];
-  if (run_if && *run_if == 0) return;
+// Reads of data that other blocks of the same launch may have written (the single-launch form below) bypass L1.
+__device__ __forceinline__ void sort_hist_block(int blk, uint32_t* cnt /*shared, kMaxBins*/, const uint32_t* keys, int64_t L,
+                                                int shift, int bins, int nblk, uint32_t* hist) {
   for (int i = threadIdx.x; i < bins; i += kSortThreads) cnt[i] = 0;
   __syncthreads();
   const int lane = threadIdx.x & 31;
-  const int64_t base = (int64_t)blockIdx.x * kSortTile;
+  const int64_t base = (int64_t)blk * kSortTile;
   const uint32_t mask = (uint32_t)bins - 1u;
   const int nbits = 31 - __clz(bins);
   uint32_t digit[kSortIPT];
 #pragma unroll
   for (int k = 0; k < kSortIPT; ++k) {                      // all loads first, then the counting
     const int64_t i = base + (int64_t)k * kSortThreads + threadIdx.x;
-    digit[k] = (i < L) ? ((keys[i] >> shift) & mask) : (uint32_t)bins;
+    digit[k] = (i < L) ? ((__ldcg(keys + i) >> shift) & mask) : (uint32_t)bins;
   }
 #pragma unroll
   for (int k = 0; k < kSortIPT; ++k) {
@@ -251,22 +256,27 @@ sort_hist_kernel(const uint32_t* __restrict__ keys, int64_t L, int shift, int bi
       atomicAdd(&cnt[digit[k]], (uint32_t)__popc(peers));   // integer counts: order-free
   }
   __syncthreads();
-  for (int i = threadIdx.x; i < bins; i += kSortThreads) hist[(int64_t)i * nblk + blockIdx.x] = cnt[i];
+  for (int i = threadIdx.x; i < bins; i += kSortThreads) hist[(int64_t)i * nblk + blk] = cnt[i];
+}
+
+__global__ void __launch_bounds__(kSortThreads)
+sort_hist_kernel(const uint32_t* __restrict__ keys, int64_t L, int shift, int bins, int nblk,
+                 uint32_t* __restrict__ hist, const int32_t* __restrict__ run_if) {
+  __shared__ uint32_t cnt[kMaxBins];
+  if (run_if && *run_if == 0) return;
+  sort_hist_block(blockIdx.x, cnt, keys, L, shift, bins, nblk, hist);
 }
 
 // One warp per bin: exclusive scan of that bin's per-tile counts in place, bin total to bintot[bin].
-__global__ void __launch_bounds__(256)
-bin_scan_kernel(uint32_t* __restrict__ hist, int bins, int nblk, uint32_t* __restrict__ bintot,
-                const int32_t* __restrict__ run_if) {
-  if (run_if && *run_if == 0) return;
-  const int bin = blockIdx.x * 8 + (threadIdx.x >> 5);
+__device__ __forceinline__ void bin_scan_block(int blk, uint32_t* hist, int bins, int nblk, uint32_t* bintot) {
+  const int bin = blk * 8 + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
   if (bin >= bins) return;
   uint32_t* row = hist + (int64_t)bin * nblk;
   uint32_t carry = 0;
   for (int b0 = 0; b0 < nblk; b0 += 32) {
     const int b = b0 + lane;
-    const uint32_t v = (b < nblk) ? row[b] : 0u;
+    const uint32_t v = (b < nblk) ? __ldcg(row + b) : 0u;
     uint32_t inc = v;
 #pragma unroll
     for (int off = 1; off < 32; off <<= 1) {
@@ -277,6 +287,13 @@ bin_scan_kernel(uint32_t* __restrict__ hist, int bins, int nblk, uint32_t* __res
     carry += __shfl_sync(0xffffffffu, inc, 31);
   }
   if (lane == 0) bintot[bin] = carry;
+}
+
+__global__ void __launch_bounds__(256)
+bin_scan_kernel(uint32_t* __restrict__ hist, int bins, int nblk, uint32_t* __restrict__ bintot,
+                const int32_t* __restrict__ run_if) {
+  if (run_if && *run_if == 0) return;
+  bin_scan_block(blockIdx.x, hist, bins, nblk, bintot);
 }
 
 // Exclusive scan of m values in place by one block (m is a few thousand at most).
@@ -328,13 +345,10 @@ scan_exclusive_kernel(uint32_t* __restrict__ data, int64_t m, uint32_t* __restri
 // Stable scatter: warp w of the block owns the contiguous items [w*512, (w+1)*512) of the tile and
 // walks them 32 at a time; rank inside a round comes from the lanes holding the same digit, across rounds and warps from
 // per-warp running counters that start at (bins before this digit) + (this digit in earlier tiles).
-__global__ void __launch_bounds__(kSortThreads)
-sort_scatter_kernel(const uint32_t* __restrict__ keys_in, const int32_t* __restrict__ pos_in,
-                    uint32_t* __restrict__ keys_out, int32_t* __restrict__ pos_out, int64_t L, int shift,
-                    int bins, int nblk, const uint32_t* __restrict__ hist_scanned, const uint32_t* __restrict__ bintot,
-                    const int32_t* __restrict__ run_if) {
-  extern __shared__ uint32_t cnt[];                       // [kSortWarps][bins], then binbase[bins], wtot[8]
-  if (run_if && *run_if == 0) return;
+__device__ __forceinline__ void sort_scatter_block(int blk, uint32_t* cnt /*shared: [kSortWarps][bins], binbase[bins], wtot[8]*/,
+                                                   const uint32_t* keys_in, const int32_t* pos_in, uint32_t* keys_out,
+                                                   int32_t* pos_out, int64_t L, int shift, int bins, int nblk,
+                                                   const uint32_t* hist_scanned, const uint32_t* bintot) {
   uint32_t* binbase = cnt + kSortWarps * bins;
   uint32_t* wtot = binbase + bins;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -342,7 +356,7 @@ sort_scatter_kernel(const uint32_t* __restrict__ keys_in, const int32_t* __restr
   // exclusive scan of the bin totals (bins <= 512 = 2 per thread)
   {
     const int i0 = 2 * threadIdx.x, i1 = i0 + 1;
-    const uint32_t v0 = (i0 < bins) ? bintot[i0] : 0u, v1 = (i1 < bins) ? bintot[i1] : 0u;
+    const uint32_t v0 = (i0 < bins) ? __ldcg(bintot + i0) : 0u, v1 = (i1 < bins) ? __ldcg(bintot + i1) : 0u;
     uint32_t inc = v0 + v1;
 #pragma unroll
     for (int off = 1; off < 32; off <<= 1) {
@@ -360,14 +374,14 @@ sort_scatter_kernel(const uint32_t* __restrict__ keys_in, const int32_t* __restr
   __syncthreads();
   const uint32_t mask = (uint32_t)bins - 1u;
   const int nbits = 31 - __clz(bins);
-  const int64_t wbase = (int64_t)blockIdx.x * kSortTile + (int64_t)warp * (32 * kSortIPT);
+  const int64_t wbase = (int64_t)blk * kSortTile + (int64_t)warp * (32 * kSortIPT);
   uint32_t key[kSortIPT];
   uint32_t* mycnt = cnt + warp * bins;
 #pragma unroll
   for (int k = 0; k < kSortIPT; ++k) {
     const int64_t i = wbase + k * 32 + lane;
     const bool valid = i < L;
-    key[k] = valid ? keys_in[i] : 0u;
+    key[k] = valid ? __ldcg(keys_in + i) : 0u;
     const uint32_t digit = valid ? ((key[k] >> shift) & mask) : (uint32_t)bins;   // invalid lanes pair up apart
     const uint32_t peers = same_digit_lanes(digit, nbits);
     if (valid && lane == (__ffs(peers) - 1)) mycnt[digit] += __popc(peers);
@@ -375,7 +389,7 @@ sort_scatter_kernel(const uint32_t* __restrict__ keys_in, const int32_t* __restr
   }
   __syncthreads();
   for (int bin = threadIdx.x; bin < bins; bin += kSortThreads) {
-    uint32_t run = binbase[bin] + hist_scanned[(int64_t)bin * nblk + blockIdx.x];
+    uint32_t run = binbase[bin] + __ldcg(hist_scanned + (int64_t)bin * nblk + blk);
 #pragma unroll
     for (int w = 0; w < kSortWarps; ++w) {
       const uint32_t c = cnt[w * bins + bin];
@@ -397,8 +411,92 @@ sort_scatter_kernel(const uint32_t* __restrict__ keys_in, const int32_t* __restr
     __syncwarp();
     if (valid) {
       keys_out[dst] = key[k];
-      pos_out[dst] = pos_in ? pos_in[i] : (int32_t)i;
+      pos_out[dst] = pos_in ? __ldcg(pos_in + i) : (int32_t)i;
     }
+  }
+}
+
+__global__ void __launch_bounds__(kSortThreads)
+sort_scatter_kernel(const uint32_t* __restrict__ keys_in, const int32_t* __restrict__ pos_in,
+                    uint32_t* __restrict__ keys_out, int32_t* __restrict__ pos_out, int64_t L, int shift,
+                    int bins, int nblk, const uint32_t* __restrict__ hist_scanned, const uint32_t* __restrict__ bintot,
+                    const int32_t* __restrict__ run_if) {
+  extern __shared__ uint32_t cnt[];                       // [kSortWarps][bins], then binbase[bins], wtot[8]
+  if (run_if && *run_if == 0) return;
+  sort_scatter_block(blockIdx.x, cnt, keys_in, pos_in, keys_out, pos_out, L, shift, bins, nblk, hist_scanned, bintot);
+}
+
+// ---- (2a) the tiled sort as ONE launch -------------------------------------------------------
+// Work items -- key building per 256 bags, then per digit pass: a histogram per tile, a scan per 8 bins, a ranked
+// scatter per tile -- are numbered in that order and drawn by the blocks from a counter.  An item of one phase needs
+// every item of the phases before it; it waits until that many items have been reported complete.  The items it
+// waits for have lower numbers, so they were drawn earlier by blocks that are running: the wait ends however few
+// blocks the device keeps resident.  run_if (nullable): the launch does nothing when the word it points to is zero
+// (the per-table sort has produced the result).  ctl = {next item, items complete, blocks gone}, zero at launch and
+// left zero.  The wait is bounded (about a second); when it runs out the block reports SS_DEV_BAD_WORKSPACE and leaves.
+struct TiledSort {
+  const int32_t* indices; const int32_t* offsets;
+  int T, B; int64_t N, L;
+  uint32_t *keys_a, *keys_b; int32_t *pos_a, *pos_b, *bag_of;
+  uint32_t *hist, *bintot;
+  int32_t* d_status; const int32_t* run_if; int* ctl;
+  int passes, digit_bits, bins, nblk, n_key_items, n_scan_items;
+};
+
+__global__ void __launch_bounds__(kSortThreads)
+tiled_sort_kernel(const TiledSort a) {
+  __shared__ uint32_t smem[kSortWarps * kMaxBins + kMaxBins + 8];
+  __shared__ int s_item;
+  if (a.run_if && *a.run_if == 0) return;
+  const int per_pass = 2 * a.nblk + a.n_scan_items;
+  const int total = a.n_key_items + a.passes * per_pass;
+  for (;;) {
+    __syncthreads();                                       // the previous item's shared memory is no longer in use
+    if (threadIdx.x == 0) s_item = atomicAdd(a.ctl, 1);
+    __syncthreads();
+    const int item = s_item;
+    if (item >= total) break;
+    // phase of the item, and how many items precede that phase
+    int need = 0, pass = -1, phase = 0, idx = item;
+    if (item >= a.n_key_items) {
+      const int r = item - a.n_key_items;
+      pass = r / per_pass;
+      idx = r - pass * per_pass;
+      need = a.n_key_items + pass * per_pass;
+      if (idx >= a.nblk) { idx -= a.nblk; need += a.nblk; phase = 1; }
+      if (phase == 1 && idx >= a.n_scan_items) { idx -= a.n_scan_items; need += a.n_scan_items; phase = 2; }
+    }
+    if (threadIdx.x == 0 && need > 0) {
+      const long long t0 = clock64();
+      int seen;
+      do {
+        asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(seen) : "l"(a.ctl + 1) : "memory");
+        if (seen < need && clock64() - t0 > 2000000000ll) { s_item = -1; break; }
+      } while (seen < need);
+    }
+    __syncthreads();
+    if (s_item < 0) {                                      // gave up: report, and do not touch the item
+      if (threadIdx.x == 0 && a.d_status) atomicOr(a.d_status, SS_DEV_BAD_WORKSPACE);
+      break;
+    }
+    // buffers of this pass: pass 0 reads keys_a (positions = indices), every pass swaps
+    const uint32_t* kin = (pass & 1) ? a.keys_b : a.keys_a;
+    uint32_t* kout = (pass & 1) ? a.keys_a : a.keys_b;
+    const int32_t* pin = pass <= 0 ? nullptr : ((pass & 1) ? a.pos_b : a.pos_a);
+    int32_t* pout = (pass & 1) ? a.pos_a : a.pos_b;
+    const int shift = pass * a.digit_bits;
+    if (pass < 0) build_keys_block(idx, a.indices, a.offsets, a.T, a.N, a.B, a.L, a.keys_a, a.bag_of, a.d_status);
+    else if (phase == 0) sort_hist_block(idx, smem, kin, a.L, shift, a.bins, a.nblk, a.hist);
+    else if (phase == 1) bin_scan_block(idx, a.hist, a.bins, a.nblk, a.bintot);
+    else sort_scatter_block(idx, smem, kin, pin, kout, pout, a.L, shift, a.bins, a.nblk, a.hist, a.bintot);
+    __threadfence();                                       // this thread's stores, before the item is reported
+    __syncthreads();
+    if (threadIdx.x == 0) atomicAdd(a.ctl + 1, 1);
+  }
+  // the last block to leave clears the control words for the next launch
+  if (threadIdx.x == 0) {
+    __threadfence();
+    if (atomicAdd(a.ctl + 2, 1) == (int)gridDim.x - 1) { a.ctl[0] = 0; a.ctl[1] = 0; a.ctl[2] = 0; __threadfence(); }
   }
 }
 
@@ -1258,11 +1356,12 @@ static ss_status bwd_impl(bool do_sort, bool do_apply, float* tables, float* row
   if (do_sort) {
 
   // (0) one block per table sorts that table's lookups in shared memory; scalars[4] stays 0 when every
-  // block could, and the tiled passes below then return at once
+  // block could, and the tiled sort below then returns at once
   int32_t* fallback = scalars + 4;
-  // more lookups than T tables of kTsCap can hold: some table is too large for its block, the tiled passes are certain
+  int* sort_ctl = scalars + 8;                             // control words of the tiled sort: zero at launch, left zero
+  // more lookups than T tables of kTsCap can hold: some table is too large for its block, the tiled sort is certain
   const bool try_table_sort = B <= 65536 && L <= (int64_t)T * kTsCap;
-  SS_CUDA(cudaMemsetAsync(fallback, try_table_sort ? 0 : 1, 4, cs));
+  SS_CUDA(cudaMemsetAsync(fallback, 0, 8 * sizeof(int32_t), cs));
   if (try_table_sort) {
     int row_bits = 1;
     while (((uint64_t)(N - 1) >> row_bits) != 0) ++row_bits;
@@ -1293,35 +1392,23 @@ static ss_status bwd_impl(bool do_sort, bool do_apply, float* tables, float* row
   }
   SS_LAUNCH_OK();
 
-  // (1) keys
-  { SS_TIMED("build_keys_kernel", cs);
-  build_keys_kernel<<<(unsigned)(((int64_t)T * B + 255) / 256), 256, 0, cs>>>(indices, offsets, T, N, B, L, keys_a,
-                                                                                bag_of, d_status, fallback);
+  // (1) keys and (2) LSD radix sort, `passes` digits of `digit_bits` bits, as one launch (see tiled_sort_kernel)
+  {
+    TiledSort ts;
+    ts.indices = indices; ts.offsets = offsets; ts.T = T; ts.B = B; ts.N = N; ts.L = L;
+    ts.keys_a = keys_a; ts.keys_b = keys_b; ts.pos_a = pos_a; ts.pos_b = pos_b; ts.bag_of = bag_of;
+    ts.hist = hist; ts.bintot = bintot; ts.d_status = d_status;
+    ts.run_if = try_table_sort ? fallback : nullptr;
+    ts.ctl = sort_ctl;
+    ts.passes = p.passes; ts.digit_bits = p.digit_bits; ts.bins = p.bins; ts.nblk = p.nblk;
+    ts.n_key_items = (int)(((int64_t)T * B + 255) / 256);
+    ts.n_scan_items = (p.bins + 7) / 8;
+    int grid = ts.n_key_items > p.nblk ? ts.n_key_items : p.nblk;
+    if (grid > 4 * num_sms()) grid = 4 * num_sms();
+    SS_TIMED("tiled_sort_kernel", cs);
+    tiled_sort_kernel<<<grid, kSortThreads, 0, cs>>>(ts);
   }
   SS_LAUNCH_OK();
-
-  // (2) LSD radix sort, `passes` digits of `digit_bits` bits
-  uint32_t* kin = keys_a; uint32_t* kout = keys_b;
-  int32_t* pin = nullptr;  // first pass: position = index
-  int32_t* pout = pos_b;
-  int32_t* pnext = pos_a;
-  const size_t smem = ((size_t)kSortWarps * p.bins + p.bins + 8) * 4;
-  for (int pass = 0; pass < p.passes; ++pass) {
-    const int shift = pass * p.digit_bits;
-    { SS_TIMED("sort_hist_kernel", cs);
-    sort_hist_kernel<<<p.nblk, kSortThreads, 0, cs>>>(kin, L, shift, p.bins, p.nblk, hist, fallback);
-    }
-    { SS_TIMED("bin_scan_kernel", cs);
-    bin_scan_kernel<<<(p.bins + 7) / 8, 256, 0, cs>>>(hist, p.bins, p.nblk, bintot, fallback);
-    }
-    { SS_TIMED("sort_scatter_kernel", cs);
-    sort_scatter_kernel<<<p.nblk, kSortThreads, smem, cs>>>(kin, pin, kout, pout, L, shift, p.bins, p.nblk, hist, bintot,
-                                                            fallback);
-    }
-    SS_LAUNCH_OK();
-    uint32_t* tk = kin; kin = kout; kout = tk;
-    pin = pout; pout = pnext; pnext = pin;
-  }
   if (perm) SS_CUDA(cudaMemcpyAsync(perm, perm_sorted, (size_t)L * 4, cudaMemcpyDeviceToDevice, cs));
 
   // (3) unique keys and segment offsets

@@ -41,16 +41,37 @@ bool gemm_tc_eligible(int M, int N, int K, const Operand& A, const Operand& B, c
 // out_lo + z * split_stride (plain stores only: no bias, ReLU, mask or bf16 output); the caller adds the slices.
 ss_status gemm_tc(int M, int N, int K, const Operand& A, const Operand& B, const Epilogue& ep, cudaStream_t st,
                   int k_splits, int64_t split_stride);
-// Several independent products (each eligible for gemm_tc, at most kTcMaxGroup) in ONE launch of 128 x 128 tiles.
-constexpr int kTcMaxGroup = 4;
+
+// A flow: several products (each eligible for gemm_tc, at most kTcMaxFlow) in ONE persistent launch whose CTAs draw
+// output tiles from a shared counter, in the order the products are listed.  A product may read, as its A operand,
+// what an EARLIER product of the same flow writes (out_lo); its tiles then wait for the row blocks they need:
+//   dep_mode 1  A(m, k) rows are the producer's output rows (a layer reading the previous layer's activations, an
+//               input gradient reading the gradient above it): tile row block y waits for the producer's row block y.
+//               dep_k_blocks > 0: only the first dep_k_blocks 64-wide k blocks of A come from the producer (the
+//               concat buffer, whose first columns are the bottom MLP's output): the tile contracts the other
+//               k blocks first and waits only then.
+//   dep_mode 2  A is the producer's output read transposed (a weight gradient contracting over the batch): k block
+//               kb waits for the producer's row block holding batch rows 64 kb .. 64 kb + 63.
+// signal_cols: only output tiles that start below this column report completion (0 = all): what later products read.
+// Waiting never deadlocks: a tile only waits for tiles that were drawn before it, by CTAs that are running.
+constexpr int kTcMaxFlow = 12;
 struct TcJob {
   int M, N, K;
   Operand A, B;
   Epilogue ep;
-  int k_splits;
-  int64_t split_stride;
+  int k_splits = 1;
+  int64_t split_stride = 0;
+  int dep = -1;            // index of the producing job in the same flow, -1: A is complete before the launch
+  int dep_mode = 0;
+  int dep_k_blocks = 0;
+  int signal_cols = 0;
 };
-ss_status gemm_tc_group(const TcJob* jobs, int n, cudaStream_t st);
+// Control words of a flow in device memory: the tile counter, the exit ticket and per (job, 128-row block) completion
+// counts (plus one total per job).  They must be zero when the launch starts; the kernel leaves them zero when it ends without an error.
+inline size_t tc_flow_ctrl_ints(int max_rows) { return 2 + (size_t)kTcMaxFlow * (size_t)((max_rows + 127) / 128 + 1); }
+// ctrl == nullptr: tiles are assigned round-robin instead (only for flows without dependencies).
+// max_ctas <= 0: one CTA per SM at most.
+ss_status gemm_tc_flow(const TcJob* jobs, int n, int* ctrl, int max_rows, int max_ctas, cudaStream_t st);
 // Tensor cores when eligible, SIMT otherwise.
 ss_status gemm(int M, int N, int K, const Operand& A, const Operand& B, const Epilogue& ep, cudaStream_t st);
 // The device error flag raised by a bounded wait that ran out (0 = none); synchronises the device.

@@ -1,46 +1,65 @@
-// bf16 x bf16 -> fp32 GEMM on the 5th-generation tensor cores (tcgen05) of sm_100a.
+// bf16 x bf16 -> fp32 GEMM on the 5th-generation tensor cores (tcgen05) of sm_100a, as a persistent kernel.
 //
 //   C[m, n] = sum_k A(m, k) * B(n, k)
 //
-// One CTA computes a 128 x 128 tile (128 x 256 for large products, 128 x 64 for products with too few
-// tiles to occupy the SMs).  One launch may hold several independent products (a group): a CTA finds its
-// product from its block index.  Warp 0 (one lane) streams 128 x 64 / 64 x 128 operand tiles
-// into a ring of shared-memory stages (3, 4 or 6 deep) with TMA (128-byte swizzle), the first round before the
-// warps meet; warp 1 (one lane) issues tcgen05.mma (M = 128, N = 64, 128 or 256, K = 16, accumulators in tensor
-// memory) and releases stages with tcgen05.commit; warps 2-5 wait for the accumulator, read it with tcgen05.ld
-// (one row per thread) and apply the epilogue (bias, ReLU, ReLU-gradient mask, bf16 / fp32 stores), through a
-// transposition in shared memory for the short CTAs of a training step.
+// One launch (a "flow") holds one or several products.  Its CTAs (at most one per SM) stay resident and draw
+// 128 x kBN output tiles from a counter in device memory, in the order the products are listed.  Inside a CTA
+// three roles run concurrently on their own warps:
+//   warp 0 (one lane)  draws tiles and streams 128 x 64 / 64 x kBN operand tiles into a ring of shared-memory
+//                      stages with TMA (128-byte swizzle), running ahead into the next tile;
+//   warp 1 (one lane)  issues tcgen05.mma (M = 128, N = 16..kBN, K = 16) into one of TWO accumulators in tensor
+//                      memory and releases stages with tcgen05.commit;
+//   warps 2-5          read a finished accumulator with tcgen05.ld (one row per thread) and apply the epilogue
+//                      (bias, ReLU, ReLU-gradient mask, bf16 / fp32 stores), while the MMA warp already fills the
+//                      other accumulator.
+// Set-up (barriers, tensor memory, descriptor prefetch) is paid once per CTA, not once per tile.
+//
+// A product may read what an earlier product of the same flow writes (a layer reading the previous layer's
+// activations, a weight gradient reading the gradient tensor an input-gradient product produces).  Finished tiles
+// count up a per-(product, row block) word in device memory; the TMA role of a dependent tile waits for the words
+// it needs before it loads the operand (release / acquire at device scope, plus a proxy fence because the data is
+// written through the generic proxy and read by TMA).  A tile only ever waits for tiles drawn before it, by CTAs
+// that are running, so the wait ends whatever else occupies the device.
 //
 // Either operand may be K-major (k contiguous in memory: the forward pass reads activations [B, in]
 // and weights [out, in] this way) or MN-major (m or n contiguous: the backward pass reads the same
 // buffers transposed, dW = dY^T X and dX = dY W), so no transposed copy of any matrix is ever made.
-// K-major tiles are one TMA box of 128 rows x 64 k; MN-major tiles are two boxes of 64 k x 64 m, the
+// K-major tiles are one TMA box of 128 rows x 64 k; MN-major tiles are boxes of 64 k x 64 m, the
 // canonical 128-byte-swizzle layouts of the shared-memory matrix descriptor in both cases.
 //
-// Every mbarrier wait is bounded: when it runs out the kernel raises a device error flag, stops
-// waiting, drains, frees its tensor memory and returns; the host reads the flag (ss_device_error).
+// Every wait (mbarrier or dependency word) is bounded: when it runs out the kernel raises a device error flag,
+// every role stops, nothing more is stored, outstanding copies are awaited, tensor memory is freed and the kernel
+// returns; the host reads the flag (ss_device_error).
 #include <cuda.h>
 #include <cudaTypedefs.h>
 #include "gemm.cuh"
 #include "profile.cuh"
 
+// Hook for a time-stamp trace of the roles (a development harness defines it before including this file); no code here.
+#ifndef SS_TC_TRACE
+#define SS_TC_TRACE(id, tile)
+#endif
+
 namespace ss {
 
-constexpr int kBM = 128, kBK = 64;   // tile rows and k depth; the tile width kBN (64, 128 or 256) is a template parameter
-// Ring depth: 3 stages (97 KiB, two CTAs per SM) for the small GEMMs of a training step, where several
-// replicas' kernels share the SMs and a second resident CTA hides more latency than a deeper ring does;
-// 6 stages (193 KiB, one CTA per SM) for large products that fill the machine on their own.
-constexpr int kStagesSmall = 3, kStagesLarge = 6;
-// 128 x 256 tiles (4 stages of 48 KiB) for products large enough to fill the machine with them: a quarter less
-// shared-memory traffic per flop than 128 x 128, which is what bounds the 128-wide tile.
-constexpr int kStagesWide = 4;
+constexpr int kBM = 128, kBK = 64;   // tile rows and k depth; the tile width kBN (128 or 256) is a template parameter
 constexpr int kTileBytes = kBM * kBK * 2;                 // 16 KiB: the A tile, and every 128 columns of the B tile
 __host__ __device__ constexpr int stage_bytes(int bn) { return kTileBytes + bn * kBK * 2; }
-constexpr int kTcThreads = 192;
-constexpr int kStgLd = 36;                                // floats per row of an epilogue warp's 32 x 32 staging block
-constexpr size_t tc_smem_bytes(int stages, int bn) { return (size_t)stages * stage_bytes(bn) + 1024 /*alignment slack*/ + 256 /*barriers*/; }
+constexpr int kEpiWarps = 4;                              // one per tensor-memory lane quadrant
+constexpr int kTcThreads = 64 + 32 * kEpiWarps;
+constexpr int kQueue = 4;                                 // tiles a CTA may have drawn and not yet finished
+// Ring depth: 5 stages of 32 KiB for 128-wide tiles, 3 stages of 48 KiB for 256-wide tiles (a quarter less
+// shared-memory traffic per flop, for products that fill the machine); one CTA per SM either way.
+constexpr int kStagesNarrow = 5, kStagesWide = 3;
+constexpr int kCtlBytes = 512;                            // barriers, tile queue, tensor-memory address, abort flag
+// Per epilogue warp: one 4 KiB slab (32 rows x 128 bytes, 128-byte swizzle) from which TMA stores a piece of the
+// output, and one slab into which TMA loads the warp's rows of the ReLU-gradient mask, 64 columns at a time.
+constexpr int kSlabBytes = 32 * 128;
+constexpr int kEpiWarpBytes = 2 * kSlabBytes;
+constexpr size_t tc_smem_bytes(int stages, int bn, size_t meta_bytes) {
+  return (size_t)stages * stage_bytes(bn) + kEpiWarps * kEpiWarpBytes + 1024 /*alignment slack*/ + kCtlBytes + meta_bytes;
+}
 constexpr long long kWaitCycles = 400ll * 1000 * 1000;    // ~0.2 s: far beyond any legitimate wait
-constexpr long long kWaitCyclesAborted = 2ll * 1000 * 1000;
 
 __device__ int g_device_error = 0;   // 0 ok; otherwise the code of the first wait that ran out
 
@@ -49,21 +68,34 @@ struct TcParams {
   int a_mn, b_mn;          // 1 = MN-major operand
   int k_splits;            // the K range is cut into this many slices; slice z writes out_lo + z*split_stride
   int64_t split_stride;    // in floats
+  int dep, dep_mode, dep_k_blocks, dep_need;   // see TcJob; dep_need = arrivals that complete a row block of `dep`
+  int dep_need_all;        // arrivals that complete all of `dep`
+  int signal_x;            // tiles with x < signal_x report completion
+  int tma_out;             // 1: outputs leave through shared memory and TMA stores, the mask arrives by TMA
   Epilogue ep;
-  int* err;
 };
 
-// One product of a launch: its tensor maps, its parameters and its share of the (one-dimensional) grid.
-// CTA `cta_begin + (z * grid_y + y) * grid_x + x` computes tile (row block y, column block x) of K slice z.
+// One product of a flow: its tensor maps, its parameters and its share of the tile sequence.
+// Tile `tile_begin + (z * grid_y + y) * grid_x + x` is (row block y, column block x) of K slice z.
+// Everything but the tensor maps is copied into shared memory when a CTA starts and from there into registers when a
+// role takes up a tile: the parameter block is indexed by a run-time product number, and reading it field by field
+// inside the loops would put a constant-bank load in front of every use.
+struct TcMeta {
+  TcParams p;
+  int tile_begin, grid_x, grid_y, pad;
+};
 struct TcProblem {
   CUtensorMap map_a, map_b;
-  TcParams p;
-  int cta_begin, grid_x, grid_y;
+  CUtensorMap map_lo, map_hi, map_mask;   // out_lo (3-d for float: column, row, K slice), out_hi, mask; used when tma_out
+  TcMeta meta;
 };
 template <int NP>
-struct TcGroup {
+struct TcFlow {
   TcProblem prob[NP];
-  int n;
+  int n, total_tiles;
+  int* ctrl;               // [0] tile counter, [1] exit ticket, [2 + j * rb_stride + rb] completions; nullptr: round-robin
+  int rb_stride;
+  int* err;
 };
 
 // ---------------------------------------------------------------------------------------- PTX wrappers
@@ -75,6 +107,9 @@ __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
 __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
@@ -84,13 +119,13 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
       : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
   return ok;
 }
-// Bounded wait.  Returns false (and records `code`) when the limit is reached.
+// Bounded wait.  Returns false when the limit is reached (records `code`) or another role has given up.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* aborted, int* err, int code) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
-  const long long limit = *aborted ? kWaitCyclesAborted : kWaitCycles;
   while (!mbar_try_wait(bar, parity)) {
-    if (clock64() - t0 > limit) {
+    if (*aborted) return false;
+    if (clock64() - t0 > kWaitCycles) {
       *aborted = 1;
       atomicCAS(err, 0, code);
       return false;
@@ -98,11 +133,44 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   }
   return true;
 }
+__device__ __forceinline__ int ld_acquire(const int* p) {
+  int v;
+  asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+// Bounded wait for a completion word of the flow to reach `need`.
+__device__ __forceinline__ bool wait_count(const int* word, int need, volatile int* aborted, int* err) {
+  if (ld_acquire(word) < need) {
+    const long long t0 = clock64();
+    while (ld_acquire(word) < need) {
+      if (*aborted) return false;
+      if (clock64() - t0 > kWaitCycles) {
+        *aborted = 1;
+        atomicCAS(err, 0, 4);
+        return false;
+      }
+    }
+  }
+  // what the other CTAs stored through the generic proxy is read by TMA (async proxy) from here on
+  asm volatile("fence.proxy.async;" ::: "memory");
+  return true;
+}
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y) {
   asm volatile(
       "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
       ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(x), "r"(y) : "memory");
 }
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t src, int x, int y) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+               ::"l"(reinterpret_cast<uint64_t>(map)), "r"(src), "r"(x), "r"(y) : "memory");
+}
+__device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, uint32_t src, int x, int y, int z) {
+  asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%2, %3, %4}], [%1];"
+               ::"l"(reinterpret_cast<uint64_t>(map)), "r"(src), "r"(x), "r"(y), "r"(z) : "memory");
+}
+__device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
@@ -143,73 +211,76 @@ __device__ __forceinline__ uint32_t pack2(float a, float b) {
   return *reinterpret_cast<uint32_t*>(&h);
 }
 
+// A tile of the flow: which product, which block, which K range.
+struct TileAt {
+  int j, x, y, z, kb_begin, nk;
+};
+__device__ __forceinline__ TileAt locate_tile(const TcMeta* meta, int n, int t) {
+  int j = 0;
+  while (j + 1 < n && t >= meta[j + 1].tile_begin) ++j;
+  const int gx = meta[j].grid_x, gy = meta[j].grid_y, K = meta[j].p.K, ks = meta[j].p.k_splits;
+  const int local = t - meta[j].tile_begin;
+  TileAt a;
+  a.j = j;
+  a.x = local % gx;
+  a.y = (local / gx) % gy;
+  a.z = local / (gx * gy);
+  const int nk_all = (K + kBK - 1) / kBK;
+  a.kb_begin = (int)((int64_t)nk_all * a.z / ks);
+  a.nk = (int)((int64_t)nk_all * (a.z + 1) / ks) - a.kb_begin;   // >= 1: k_splits <= nk_all
+  return a;
+}
+
 // ---------------------------------------------------------------------------------------- kernel
-template <int kStages, int kBN, int NP, bool kDirect>
+template <int kStages, int kBN, int NP>
 __global__ void __launch_bounds__(kTcThreads, 1)
-gemm_tc_kernel(const __grid_constant__ TcGroup<NP> grp) {
+gemm_tc_kernel(const __grid_constant__ TcFlow<NP> flow) {
   extern __shared__ uint8_t smem_raw[];
-  int pj = 0;
-  if (NP > 1) {
-    while (pj + 1 < grp.n && (int)blockIdx.x >= grp.prob[pj + 1].cta_begin) ++pj;
-  }
-  const TcProblem& prob = grp.prob[pj];
-  const TcParams& p = prob.p;
-  const CUtensorMap& map_a = prob.map_a;
-  const CUtensorMap& map_b = prob.map_b;
-  const int cta_local = (int)blockIdx.x - prob.cta_begin;
-  const int tile_x = cta_local % prob.grid_x;
-  const int tile_y = (cta_local / prob.grid_x) % prob.grid_y;
-  const int slice_z = cta_local / (prob.grid_x * prob.grid_y);
   constexpr int kStageBytes = stage_bytes(kBN);
-  constexpr int kTmemCols = kBN;                           // one fp32 accumulator column per tile column
+  constexpr int kTmemCols = 2 * kBN;                       // two accumulators of kBN fp32 columns
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t tiles = (raw + 1023u) & ~1023u;                 // 1024-byte aligned swizzle atoms
   uint8_t* gen = smem_raw + (tiles - raw);
-  uint64_t* bars = reinterpret_cast<uint64_t*>(gen + (size_t)kStages * kStageBytes);
-  const uint32_t bar0 = tiles + kStages * kStageBytes;
-  // bars: [0,S) full, [S,2S) empty, [2S] accumulator ready; then tmem base and the abort flag
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kStages + 1);
+  const uint32_t epi0 = tiles + kStages * kStageBytes;            // 1024-byte aligned: stages are multiples of 1 KiB
+  uint8_t* epi_gen = gen + (size_t)kStages * kStageBytes;
+  uint8_t* ctl = epi_gen + kEpiWarps * kEpiWarpBytes;
+  const uint32_t bar0 = epi0 + kEpiWarps * kEpiWarpBytes;
+  // barriers: [0,S) full, [S,2S) empty, then accumulator full[2], empty[2], queue full[kQueue], empty[kQueue],
+  // mask slab full [epilogue warp]
+  constexpr int kNumBars = 2 * kStages + 4 + 2 * kQueue + kEpiWarps;
+  int* tile_q = reinterpret_cast<int*>(ctl + 8 * kNumBars);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tile_q + kQueue);
   volatile int* aborted = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  TcMeta* meta = reinterpret_cast<TcMeta*>(ctl + kCtlBytes);
+  static_assert(8 * kNumBars + 4 * kQueue + 8 <= kCtlBytes, "control region");
+  static_assert(sizeof(TcMeta) % 4 == 0, "copied word by word");
+  const int n_prob = flow.n;
+  for (int j = 0; j < n_prob; ++j) {
+    const uint32_t* src = reinterpret_cast<const uint32_t*>(&flow.prob[j].meta);
+    uint32_t* dst = reinterpret_cast<uint32_t*>(meta + j);
+    for (int i = threadIdx.x; i < (int)(sizeof(TcMeta) / 4); i += kTcThreads) dst[i] = src[i];
+  }
   auto full = [&](int s) { return bar0 + 8u * s; };
   auto empty = [&](int s) { return bar0 + 8u * (kStages + s); };
-  const uint32_t acc_bar = bar0 + 8u * (2 * kStages);
+  auto acc_full = [&](int b) { return bar0 + 8u * (2 * kStages + b); };
+  auto acc_empty = [&](int b) { return bar0 + 8u * (2 * kStages + 2 + b); };
+  auto q_full = [&](int s) { return bar0 + 8u * (2 * kStages + 4 + s); };
+  auto q_empty = [&](int s) { return bar0 + 8u * (2 * kStages + 4 + kQueue + s); };
+  auto mask_full = [&](int w) { return bar0 + 8u * (2 * kStages + 4 + 2 * kQueue + w); };
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int m0 = tile_y * kBM, n0 = tile_x * kBN;
-  const int nk_all = (p.K + kBK - 1) / kBK;
-  const int kb_begin = (int)((int64_t)nk_all * slice_z / p.k_splits);
-  const int nk = (int)((int64_t)nk_all * (slice_z + 1) / p.k_splits) - kb_begin;   // >= 1: k_splits <= nk_all
-
-  // one stage of operand tiles for k block kb of this CTA's slice
-  auto load_stage = [&](int kb) {
-    const int s = kb % kStages;
-    mbar_expect_tx(full(s), kStageBytes);
-    const uint32_t sa = tiles + s * kStageBytes, sb = sa + kTileBytes;
-    const int k0 = (kb_begin + kb) * kBK;
-    if (p.a_mn) {                       // A stored [K, M]: two boxes of 64 k-rows x 64 m
-      tma_load_2d(sa, &map_a, full(s), m0, k0);
-      tma_load_2d(sa + kTileBytes / 2, &map_a, full(s), m0 + 64, k0);
-    } else {                            // A stored [M, K]: one box of 128 rows x 64 k
-      tma_load_2d(sa, &map_a, full(s), k0, m0);
-    }
-    if (p.b_mn) {
-#pragma unroll
-      for (int a = 0; a < kBN / 64; ++a) tma_load_2d(sb + a * (kTileBytes / 2), &map_b, full(s), n0 + 64 * a, k0);
-    } else {
-      tma_load_2d(sb, &map_b, full(s), k0, n0);
-    }
-  };
-  const int n_early = nk < kStages ? nk : kStages;           // the ring starts empty: its first round needs no wait
   if (threadIdx.x == 0) {
-    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_a)) : "memory");
-    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_b)) : "memory");
+    for (int j = 0; j < flow.n; ++j) {
+      asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&flow.prob[j].map_a)) : "memory");
+      asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&flow.prob[j].map_b)) : "memory");
+    }
     for (int s = 0; s < kStages; ++s) { mbar_init(full(s), 1); mbar_init(empty(s), 1); }
-    mbar_init(acc_bar, 1);
+    for (int b = 0; b < 2; ++b) { mbar_init(acc_full(b), 1); mbar_init(acc_empty(b), kEpiWarps); }
+    for (int s = 0; s < kQueue; ++s) { mbar_init(q_full(s), 1); mbar_init(q_empty(s), 1 + kEpiWarps); }
+    for (int w = 0; w < kEpiWarps; ++w) mbar_init(mask_full(w), 1);
     *aborted = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    // the first round of loads goes out before tensor memory is allocated and the warps meet
-    for (int kb = 0; kb < n_early; ++kb) load_stage(kb);
   }
   if (warp == 1) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(kTmemCols) : "memory");
@@ -219,72 +290,298 @@ gemm_tc_kernel(const __grid_constant__ TcGroup<NP> grp) {
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
+  int* const done0 = flow.ctrl ? flow.ctrl + 2 : nullptr;
+  if (threadIdx.x == 0) SS_TC_TRACE(1, -1);
 
   if (warp == 0) {
-    // ------------------------------------------------------------------ TMA producer
+    // ------------------------------------------------------------------ tile scheduler + TMA producer
     if (lane == 0) {
-      for (int kb = n_early; kb < nk; ++kb) {
-        const int s = kb % kStages;
-        const uint32_t ph = (kb / kStages) & 1;
-        if (!mbar_wait(empty(s), ph ^ 1u, aborted, p.err, 1)) break;
-        load_stage(kb);
+      uint32_t it = 0;                                     // stages filled so far (over all tiles)
+      // the ticket of the next tile is drawn while the current one is loaded (the counter is a round trip to L2 away);
+      // tickets are still drawn in order by a running CTA and worked off in order, which is all the waiting needs
+      int t_next = flow.ctrl ? atomicAdd(flow.ctrl, 1) : (int)blockIdx.x;
+      for (uint32_t qi = 0;; ++qi) {
+        const int qs = qi % kQueue;
+        if (!mbar_wait(q_empty(qs), ((qi / kQueue) & 1) ^ 1u, aborted, flow.err, 5)) break;
+        int t = t_next;
+        if (t >= flow.total_tiles) t = -1;
+        if (t >= 0) t_next = flow.ctrl ? atomicAdd(flow.ctrl, 1) : (int)(blockIdx.x + (qi + 1) * gridDim.x);
+        tile_q[qs] = t;
+        mbar_arrive(q_full(qs));
+        if (t < 0) break;
+        SS_TC_TRACE(2, t);
+        const TileAt a = locate_tile(meta, n_prob, t);
+        const TcProblem& pr = flow.prob[a.j];
+        const int m0 = a.y * kBM, n0 = a.x * kBN;
+        int dep_mode = 0, dep_need = 0, dep_kb = 0;
+        const int* dep_words = nullptr;
+        const int a_mn = meta[a.j].p.a_mn, b_mn = meta[a.j].p.b_mn, K = meta[a.j].p.K;
+        if (meta[a.j].p.dep >= 0) {
+          dep_mode = meta[a.j].p.dep_mode; dep_need = meta[a.j].p.dep_need;
+          dep_kb = meta[a.j].p.k_splits == 1 ? meta[a.j].p.dep_k_blocks : 0;
+          dep_words = done0 + meta[a.j].p.dep * flow.rb_stride;
+        }
+        // k blocks [0, nd) of this tile's range wait for the producing product (taken last); the others do not
+        int nd = 0;
+        if (dep_mode == 1) nd = (dep_kb > 0 && dep_kb < a.nk) ? dep_kb : a.nk;
+        bool dep_ok = (nd == 0);
+        int rb_ready = -1;                                 // dep_mode 2: the producer's row blocks up to here are complete
+        if (dep_mode == 2 && ld_acquire(dep_words + flow.rb_stride - 1) >= meta[a.j].p.dep_need_all) {
+          asm volatile("fence.proxy.async;" ::: "memory");
+          rb_ready = 0x7fffffff;                           // the producing product is complete: nothing to wait for
+        }
+        bool failed = false;
+        for (int i = 0; i < a.nk; ++i) {
+          int kb = i + nd;
+          if (kb >= a.nk) kb -= a.nk;                      // independent k blocks first
+          if (!dep_ok && kb < nd) {
+            if (!wait_count(dep_words + a.y, dep_need, aborted, flow.err)) { failed = true; break; }
+            dep_ok = true;
+          }
+          const int k0 = (a.kb_begin + kb) * kBK;
+          if (dep_mode == 2) {
+            int rb = (k0 + kBK - 1) / kBM;                 // a 64-row k block lies inside one 128-row block
+            const int rb_last = (K - 1) / kBM;
+            if (rb > rb_last) rb = rb_last;
+            if (rb > rb_ready) {
+              if (!wait_count(dep_words + rb, dep_need, aborted, flow.err)) { failed = true; break; }
+              rb_ready = rb;
+            }
+          }
+          const int s = it % kStages;
+          if (!mbar_wait(empty(s), ((it / kStages) & 1) ^ 1u, aborted, flow.err, 1)) { failed = true; break; }
+          mbar_expect_tx(full(s), kStageBytes);
+          const uint32_t sa = tiles + s * kStageBytes, sb = sa + kTileBytes;
+          if (a_mn) {                         // A stored [K, M]: two boxes of 64 k-rows x 64 m
+            tma_load_2d(sa, &pr.map_a, full(s), m0, k0);
+            tma_load_2d(sa + kTileBytes / 2, &pr.map_a, full(s), m0 + 64, k0);
+          } else {                            // A stored [M, K]: one box of 128 rows x 64 k
+            tma_load_2d(sa, &pr.map_a, full(s), k0, m0);
+          }
+          if (b_mn) {
+#pragma unroll
+            for (int h = 0; h < kBN / 64; ++h) tma_load_2d(sb + h * (kTileBytes / 2), &pr.map_b, full(s), n0 + 64 * h, k0);
+          } else {
+#pragma unroll
+            for (int h = 0; h < kBN / 128; ++h) tma_load_2d(sb + h * kTileBytes, &pr.map_b, full(s), k0, n0 + 128 * h);
+          }
+          ++it;
+          if (i == 0) SS_TC_TRACE(3, t);
+        }
+        if (failed) break;
+        SS_TC_TRACE(4, t);
+      }
+      if (*aborted) {
+        // the copies still in flight land in this CTA's shared memory: wait for them (bounded) before leaving
+        const uint32_t first = it > (uint32_t)kStages ? it - kStages : 0u;
+        for (uint32_t i = first; i < it; ++i) {
+          const long long t0 = clock64();
+          while (!mbar_try_wait(full(i % kStages), (i / kStages) & 1) && clock64() - t0 < 4000000ll) {}
+        }
       }
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
-      // instruction descriptor: D = f32, A = B = bf16, majors, N >> 3, M >> 4
-      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)p.a_mn << 15) | ((uint32_t)p.b_mn << 16) |
-                             ((uint32_t)(kBN >> 3) << 17) | ((uint32_t)(kBM >> 4) << 24);
-      // K-major: 8-row groups 1024 B apart (SBO), K step of 16 elements = 32 B inside the swizzle span.
-      // MN-major: 64-wide m atoms 8192 B apart (LBO), 8-k groups 1024 B apart (SBO), K step of 16 = 2048 B.
-      const uint32_t a_lbo = p.a_mn ? 8192u : 16u, a_step = p.a_mn ? 2048u : 32u;
-      const uint32_t b_lbo = p.b_mn ? 8192u : 16u, b_step = p.b_mn ? 2048u : 32u;
-      for (int kb = 0; kb < nk; ++kb) {
-        const int s = kb % kStages;
-        const uint32_t ph = (kb / kStages) & 1;
-        mbar_wait(full(s), ph, aborted, p.err, 2);
+      uint32_t it = 0, at = 0;                             // stages consumed, tiles accumulated
+      for (uint32_t qi = 0;; ++qi) {
+        const int qs = qi % kQueue;
+        if (!mbar_wait(q_full(qs), (qi / kQueue) & 1, aborted, flow.err, 6)) break;
+        const int t = tile_q[qs];
+        mbar_arrive(q_empty(qs));
+        if (t < 0) break;
+        const TileAt a = locate_tile(meta, n_prob, t);
+        const int a_mn = meta[a.j].p.a_mn, b_mn = meta[a.j].p.b_mn;
+        int n_mma = meta[a.j].p.N - a.x * kBN;             // columns of this tile, rounded up to the instruction's granule
+        n_mma = n_mma >= kBN ? kBN : ((n_mma + 15) & ~15);
+        // instruction descriptor: D = f32, A = B = bf16, majors, N >> 3, M >> 4
+        const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)a_mn << 15) | ((uint32_t)b_mn << 16) |
+                               ((uint32_t)(n_mma >> 3) << 17) | ((uint32_t)(kBM >> 4) << 24);
+        // K-major: 8-row groups 1024 B apart (SBO), K step of 16 elements = 32 B inside the swizzle span.
+        // MN-major: 64-wide m atoms 8192 B apart (LBO), 8-k groups 1024 B apart (SBO), K step of 16 = 2048 B.
+        const uint32_t a_lbo = a_mn ? 8192u : 16u, a_step = a_mn ? 2048u : 32u;
+        const uint32_t b_lbo = b_mn ? 8192u : 16u, b_step = b_mn ? 2048u : 32u;
+        const int buf = at & 1;
+        if (!mbar_wait(acc_empty(buf), ((at >> 1) & 1) ^ 1u, aborted, flow.err, 7)) break;
         tc_fence_after();
-        const uint32_t sa = tiles + s * kStageBytes, sb = sa + kTileBytes;
+        const uint32_t d_tmem = tmem + (uint32_t)(buf * kBN);
+        bool failed = false;
+        for (int i = 0; i < a.nk; ++i) {
+          const int s = it % kStages;
+          if (!mbar_wait(full(s), (it / kStages) & 1, aborted, flow.err, 2)) { failed = true; break; }
+          if (i == 0) SS_TC_TRACE(5, t);
+          tc_fence_after();
+          const uint32_t sa = tiles + s * kStageBytes, sb = sa + kTileBytes;
 #pragma unroll
-        for (int k = 0; k < kBK / 16; ++k) {
-          const uint64_t ad = smem_desc(sa + k * a_step, a_lbo, 1024u);
-          const uint64_t bd = smem_desc(sb + k * b_step, b_lbo, 1024u);
-          tc_mma(tmem, ad, bd, idesc, (kb > 0 || k > 0) ? 1u : 0u);
+          for (int k = 0; k < kBK / 16; ++k) {
+            const uint64_t ad = smem_desc(sa + k * a_step, a_lbo, 1024u);
+            const uint64_t bd = smem_desc(sb + k * b_step, b_lbo, 1024u);
+            tc_mma(d_tmem, ad, bd, idesc, (i > 0 || k > 0) ? 1u : 0u);
+          }
+          tc_commit(empty(s));              // frees the stage when these MMAs have read it
+          ++it;
         }
-        tc_commit(empty(s));              // frees the stage when these MMAs have read it
+        if (failed) break;
+        tc_commit(acc_full(buf));           // accumulator complete
+        SS_TC_TRACE(6, t);
+        ++at;
       }
-      tc_commit(acc_bar);                 // accumulator complete
     }
   } else {
     // ------------------------------------------------------------------ epilogue warps 2..5
     const int q = warp & 3;               // tensor-memory lane quadrant this warp may read
-    const Epilogue& ep = p.ep;
-    mbar_wait(acc_bar, 0, aborted, p.err, 3);
-    tc_fence_after();
-    if constexpr (kDirect) {
-      // Machine-filling products (their epilogue is a small part of a long CTA): every thread stores the
-      // accumulator row it reads, 32 consecutive columns at a time.
+    uint8_t* const slab_gen = epi_gen + q * kEpiWarpBytes;
+    const uint32_t slab_out = epi0 + q * kEpiWarpBytes, slab_mask = slab_out + kSlabBytes;
+    uint32_t mask_uses = 0;               // completed phases of this warp's mask barrier
+    uint32_t at = 0;
+    for (uint32_t qi = 0;; ++qi) {
+      const int qs = qi % kQueue;
+      if (!mbar_wait(q_full(qs), (qi / kQueue) & 1, aborted, flow.err, 8)) break;
+      const int t = tile_q[qs];
+      __syncwarp();
+      if (lane == 0) mbar_arrive(q_empty(qs));
+      if (t < 0) break;
+      const TileAt a = locate_tile(meta, n_prob, t);
+      const Epilogue ep = meta[a.j].p.ep;                  // by value: registers
+      struct { int M, N, signal_x; int64_t split_stride; } p = {meta[a.j].p.M, meta[a.j].p.N, meta[a.j].p.signal_x,
+                                                                 meta[a.j].p.split_stride};
+      const int m0 = a.y * kBM, n0 = a.x * kBN;
+      const int buf = at & 1;
+      const bool tma_out = meta[a.j].p.tma_out != 0;
+      const TcProblem& pr = flow.prob[a.j];
+      // this warp's rows of the mask (the producing layer's bf16 activation), 64 columns per slab, requested as soon
+      // as the tile is known: they arrive while the tensor cores still work on the tile
+      const bool masked = tma_out && ep.mask != nullptr;
+      auto request_mask = [&](int h) {                     // the mask of columns 64 h .. 64 h + 63 of the tile, rows of this warp
+        if (lane == 0) {
+          mbar_expect_tx(mask_full(q), kSlabBytes);
+          tma_load_2d(slab_mask, &pr.map_mask, mask_full(q), n0 + 64 * h, m0 + 32 * q);
+        }
+      };
+      if (masked && n0 < ep.mask_cols) request_mask(0);
+      if (!mbar_wait(acc_full(buf), (at >> 1) & 1, aborted, flow.err, 3)) break;
+      if (threadIdx.x == 64) SS_TC_TRACE(7, t);
+      tc_fence_after();
+      if (tma_out) {
+        // The thread holds 32 consecutive columns of its accumulator row at a time.  It applies bias / ReLU / mask,
+        // writes the row piece into the warp's slab in the 128-byte-swizzle layout, and one lane hands the slab to
+        // TMA, which stores whole rows of it (and clips what lies beyond the matrix).  A slab is 64 columns of bf16
+        // output (two pieces) or 32 columns of float output.
+        const int sw = lane & 7;
+        const uint32_t row_off = (uint32_t)lane * 128u;
+        bool failed = false;
+#pragma unroll 1
+        for (int c = 0; c < kBN / 32; ++c) {
+          const int nb = n0 + 32 * c;
+          if (nb >= p.N) break;
+          const int odd = c & 1;
+          uint32_t r[32];
+          tc_ld32(tmem + ((uint32_t)(32 * q) << 16) + (uint32_t)(buf * kBN + 32 * c), r);
+          float v[32];
+#pragma unroll
+          for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
+          if (ep.bias) {
+#pragma unroll
+            for (int j = 0; j < 32; j += 4) {
+              if (nb + j < p.N) {            // N is a multiple of 8: four columns are inside together or not at all
+                const float4 bv = __ldg(reinterpret_cast<const float4*>(ep.bias + nb + j));
+                v[j] += bv.x; v[j + 1] += bv.y; v[j + 2] += bv.z; v[j + 3] += bv.w;
+              }
+            }
+          }
+          if (ep.relu) {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) v[j] = fmaxf(v[j], 0.f);
+          }
+          if (masked && nb < ep.mask_cols) {
+            // the mask slab holds the 64 columns of this piece and its neighbour
+            if (!odd && !mbar_wait(mask_full(q), (mask_uses++) & 1, aborted, flow.err, 9)) { failed = true; break; }
+#pragma unroll
+            for (int g = 0; g < 4; ++g) {
+              if (nb + 8 * g >= ep.mask_cols) break;
+              const uint4 mk = *reinterpret_cast<const uint4*>(slab_gen + kSlabBytes + row_off + ((uint32_t)((g + 4 * odd) ^ sw) << 4));
+              const uint32_t w[4] = {mk.x, mk.y, mk.z, mk.w};
+#pragma unroll
+              for (int j = 0; j < 4; ++j) {
+                // a bf16 is positive iff its sign bit is clear and it is not zero
+                const uint32_t lo = w[j] & 0xFFFFu, hi = w[j] >> 16;
+                if (!((lo & 0x8000u) == 0 && (lo & 0x7FFFu) != 0)) v[8 * g + 2 * j] = 0.f;
+                if (!((hi & 0x8000u) == 0 && (hi & 0x7FFFu) != 0)) v[8 * g + 2 * j + 1] = 0.f;
+              }
+            }
+            // the slab's 64 columns are used up: ask for the tile's next 64
+            const bool last_of_slab = odd || nb + 32 >= p.N || nb + 32 >= ep.mask_cols;
+            if (last_of_slab && c + 1 < kBN / 32 && n0 + 32 * (c + 1) < ep.mask_cols && n0 + 32 * (c + 1) < p.N) {
+              __syncwarp();                                // every lane has read the slab
+              request_mask((c + 1) >> 1);
+            }
+          }
+          const bool to_lo = nb < ep.lo_cols;
+          if (to_lo && ep.lo_bf16) {
+            if (!odd) {
+              if (lane == 0) tma_store_wait_read();        // the slab's previous contents have been read
+              __syncwarp();
+            }
+#pragma unroll
+            for (int g = 0; g < 4; ++g) {
+              uint4 o;
+              o.x = pack2(v[8 * g], v[8 * g + 1]); o.y = pack2(v[8 * g + 2], v[8 * g + 3]);
+              o.z = pack2(v[8 * g + 4], v[8 * g + 5]); o.w = pack2(v[8 * g + 6], v[8 * g + 7]);
+              *reinterpret_cast<uint4*>(slab_gen + row_off + ((uint32_t)((g + 4 * odd) ^ sw) << 4)) = o;
+            }
+            if (odd || nb + 32 >= p.N || nb + 32 >= ep.lo_cols) {   // the slab is complete (or the output ends here)
+              asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+              __syncwarp();
+              if (lane == 0 && !*aborted) {
+                tma_store_2d(&pr.map_lo, slab_out, nb - 32 * odd, m0 + 32 * q);
+                tma_store_commit();
+              }
+            }
+          } else {
+            if (lane == 0) tma_store_wait_read();
+            __syncwarp();
+#pragma unroll
+            for (int g = 0; g < 8; ++g)
+              *reinterpret_cast<float4*>(slab_gen + row_off + ((uint32_t)(g ^ sw) << 4)) =
+                  make_float4(v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            __syncwarp();
+            if (lane == 0 && !*aborted) {
+              if (to_lo) tma_store_3d(&pr.map_lo, slab_out, nb, m0 + 32 * q, a.z);
+              else tma_store_2d(&pr.map_hi, slab_out, nb - ep.lo_cols, m0 + 32 * q);
+              tma_store_commit();
+            }
+          }
+        }
+        if (failed) break;
+      } else {
+      // tcgen05.ld hands a thread one accumulator row, 32 consecutive columns at a time: the thread applies the
+      // epilogue to its row and stores 16-byte pieces of it (whole 32-byte sectors per pair of stores).
       const int64_t m = (int64_t)m0 + 32 * q + lane;
-      const bool m_ok = m < p.M;
+      const bool m_ok = m < p.M && !*aborted;
 #pragma unroll 1
       for (int c = 0; c < kBN / 32; ++c) {
         const int nb = n0 + 32 * c;
         if (nb >= p.N) break;
         uint32_t r[32];
-        tc_ld32(tmem + ((uint32_t)(32 * q) << 16) + (uint32_t)(32 * c), r);
+        tc_ld32(tmem + ((uint32_t)(32 * q) << 16) + (uint32_t)(buf * kBN + 32 * c), r);
+        if (!m_ok) continue;
         float v[32];
 #pragma unroll
         for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
         if (ep.bias) {
 #pragma unroll
-          for (int j = 0; j < 32; ++j) if (nb + j < p.N) v[j] += __ldg(ep.bias + nb + j);
+          for (int j = 0; j < 32; j += 4) {
+            if (nb + j < p.N) {              // N is a multiple of 8: four columns are inside together or not at all
+              const float4 bv = __ldg(reinterpret_cast<const float4*>(ep.bias + nb + j));
+              v[j] += bv.x; v[j + 1] += bv.y; v[j + 2] += bv.z; v[j + 3] += bv.w;
+            }
+          }
         }
         if (ep.relu) {
 #pragma unroll
           for (int j = 0; j < 32; ++j) v[j] = fmaxf(v[j], 0.f);
         }
-        if (!m_ok) continue;
 #pragma unroll
         for (int g = 0; g < 4; ++g) {
           const int n = nb + 8 * g;
@@ -307,7 +604,7 @@ gemm_tc_kernel(const __grid_constant__ TcGroup<NP> grp) {
               o.x = pack2(x[0], x[1]); o.y = pack2(x[2], x[3]); o.z = pack2(x[4], x[5]); o.w = pack2(x[6], x[7]);
               *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(ep.out_lo) + m * ep.ld_lo + n) = o;
             } else {
-              float4* o = reinterpret_cast<float4*>(reinterpret_cast<float*>(ep.out_lo) + (int64_t)slice_z * p.split_stride + m * ep.ld_lo + n);
+              float4* o = reinterpret_cast<float4*>(reinterpret_cast<float*>(ep.out_lo) + (int64_t)a.z * p.split_stride + m * ep.ld_lo + n);
               o[0] = make_float4(x[0], x[1], x[2], x[3]);
               o[1] = make_float4(x[4], x[5], x[6], x[7]);
             }
@@ -318,66 +615,29 @@ gemm_tc_kernel(const __grid_constant__ TcGroup<NP> grp) {
           }
         }
       }
-    } else {
-      // tcgen05.ld hands a thread one accumulator row; stores of that shape put 32 different rows into one
-      // instruction.  For the short CTAs of a training step each warp turns its 32 x 32 block round in shared
-      // memory (the operand ring is idle once the accumulator is complete) and continues with four consecutive
-      // columns per lane, eight lanes per row: bias, ReLU, mask and stores touch whole 64- or 128-byte row segments.
-      float* stg = reinterpret_cast<float*>(gen) + q * (32 * kStgLd);   // rows of 36 floats: 128-bit accesses without bank conflicts
-      const int cl = 4 * (lane & 7), rl = lane >> 3;
-#pragma unroll 1
-      for (int c = 0; c < kBN / 32; ++c) {
-        const int nb = n0 + 32 * c;
-        if (nb >= p.N) break;
-        uint32_t r[32];
-        tc_ld32(tmem + ((uint32_t)(32 * q) << 16) + (uint32_t)(32 * c), r);
-#pragma unroll
-        for (int j = 0; j < 8; ++j)
-          *reinterpret_cast<uint4*>(stg + lane * kStgLd + 4 * j) = make_uint4(r[4 * j], r[4 * j + 1], r[4 * j + 2], r[4 * j + 3]);
-        __syncwarp();
-        const int n = nb + cl;
-        if (n < p.N) {                       // N is a multiple of 8: four columns are inside together or not at all
-          float4 bv = make_float4(0.f, 0.f, 0.f, 0.f);
-          if (ep.bias) bv = __ldg(reinterpret_cast<const float4*>(ep.bias + n));
-          const bool masked = ep.mask && n < ep.mask_cols;
-          // the mask words of all eight rows are requested before any is used: one round of load latency, not eight
-          uint2 mk[8];
-#pragma unroll
-          for (int i = 0; i < 8; ++i) {
-            const int64_t m = (int64_t)m0 + 32 * q + rl + 4 * i;
-            mk[i] = make_uint2(0x3F803F80u, 0x3F803F80u);   // four positive values: nothing is masked
-            if (masked && m < p.M)
-              mk[i] = *reinterpret_cast<const uint2*>(reinterpret_cast<const __nv_bfloat16*>(ep.mask) + m * ep.ld_mask + n);
-          }
-#pragma unroll
-          for (int i = 0; i < 8; ++i) {
-            const int row = rl + 4 * i;
-            const int64_t m = (int64_t)m0 + 32 * q + row;
-            if (m >= p.M) continue;
-            const float4 sv = *reinterpret_cast<const float4*>(stg + row * kStgLd + cl);
-            float x0 = sv.x + bv.x, x1 = sv.y + bv.y, x2 = sv.z + bv.z, x3 = sv.w + bv.w;
-            if (ep.relu) { x0 = fmaxf(x0, 0.f); x1 = fmaxf(x1, 0.f); x2 = fmaxf(x2, 0.f); x3 = fmaxf(x3, 0.f); }
-            // bf16 activation of the producing layer: positive iff sign clear and not zero
-            if (!((mk[i].x & 0x8000u) == 0 && (mk[i].x & 0x7FFFu) != 0)) x0 = 0.f;
-            if (!((mk[i].x & 0x80000000u) == 0 && (mk[i].x & 0x7FFF0000u) != 0)) x1 = 0.f;
-            if (!((mk[i].y & 0x8000u) == 0 && (mk[i].y & 0x7FFFu) != 0)) x2 = 0.f;
-            if (!((mk[i].y & 0x80000000u) == 0 && (mk[i].y & 0x7FFF0000u) != 0)) x3 = 0.f;
-            if (n < ep.lo_cols) {
-              if (ep.lo_bf16) {
-                uint2 o;
-                o.x = pack2(x0, x1); o.y = pack2(x2, x3);
-                *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(ep.out_lo) + m * ep.ld_lo + n) = o;
-              } else {
-                *reinterpret_cast<float4*>(reinterpret_cast<float*>(ep.out_lo) + (int64_t)slice_z * p.split_stride + m * ep.ld_lo + n) =
-                    make_float4(x0, x1, x2, x3);
-              }
-            } else if (ep.out_hi) {
-              *reinterpret_cast<float4*>(ep.out_hi + m * ep.ld_hi + (n - ep.lo_cols)) = make_float4(x0, x1, x2, x3);
-            }
-          }
-        }
-        __syncwarp();                        // the block is read before the next one overwrites it
       }
+      // the accumulator may be overwritten: this warp's reads of it are complete
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(acc_empty(buf));
+      if (threadIdx.x == 64) SS_TC_TRACE(8, t);
+      // completion word of the row block, for the products that read this output
+      if (done0 && a.x < p.signal_x) {
+        if (tma_out && lane == 0) tma_store_wait_all();    // what this warp's TMA stores wrote is complete in memory
+        __threadfence();
+        asm volatile("fence.proxy.async;" ::: "memory");
+        __syncwarp();
+        if (lane == 0) {
+          atomicAdd(done0 + a.j * flow.rb_stride + a.y, 1);
+          __threadfence();
+          atomicAdd(done0 + a.j * flow.rb_stride + flow.rb_stride - 1, 1);   // after the row block's own word
+        }
+      }
+      ++at;
+    }
+    if (lane == 0) tma_store_wait_all();                   // the slabs are read before the CTA gives up its shared memory
+    if (*aborted) {
+      for (int i = 0; i < 64; ++i) __nanosleep(1000);      // mask slabs still on their way land in this CTA's memory
     }
   }
 
@@ -386,6 +646,15 @@ gemm_tc_kernel(const __grid_constant__ TcGroup<NP> grp) {
   if (warp == 1) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
+  }
+  // the last CTA to leave clears the control words for the next launch (every other CTA is past its last access)
+  if (flow.ctrl && threadIdx.x == 0 && !*aborted) {
+    __threadfence();
+    if (atomicAdd(flow.ctrl + 1, 1) == (int)gridDim.x - 1) {
+      const int words = 2 + flow.n * flow.rb_stride;
+      for (int i = 0; i < words; ++i) flow.ctrl[i] = 0;
+      __threadfence();
+    }
   }
 }
 
@@ -402,19 +671,23 @@ static PFN_cuTensorMapEncodeTiled_v12000 encode_fn() {
   return fn;
 }
 
-// bf16 matrix with `inner` contiguous elements per row, `outer` rows, row pitch ld elements.
-static bool make_map(CUtensorMap* map, const void* base, int64_t inner, int64_t outer, int64_t ld, int box_inner,
-                     int box_outer) {
+// Matrix with `inner` contiguous elements per row, `outer` rows, row pitch ld elements (and `planes` such matrices
+// plane_stride elements apart when rank is 3); 128-byte swizzle, so box_inner * element size is at most 128 bytes.
+static bool make_map_any(CUtensorMap* map, CUtensorMapDataType dt, int esize, const void* base, int64_t inner, int64_t outer,
+                         int64_t ld, int box_inner, int box_outer, int rank = 2, int64_t planes = 1, int64_t plane_stride = 0) {
   PFN_cuTensorMapEncodeTiled_v12000 fn = encode_fn();
   if (!fn) return false;
-  cuuint64_t dims[2] = {(cuuint64_t)inner, (cuuint64_t)outer};
-  cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
-  cuuint32_t box[2] = {(cuuint32_t)box_inner, (cuuint32_t)box_outer};
-  cuuint32_t estr[2] = {1, 1};
-  CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
-                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  cuuint64_t dims[3] = {(cuuint64_t)inner, (cuuint64_t)outer, (cuuint64_t)planes};
+  cuuint64_t strides[2] = {(cuuint64_t)ld * esize, (cuuint64_t)plane_stride * esize};
+  cuuint32_t box[3] = {(cuuint32_t)box_inner, (cuuint32_t)box_outer, 1};
+  cuuint32_t estr[3] = {1, 1, 1};
+  CUresult r = fn(map, dt, rank, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                  CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS;
+}
+static bool make_map(CUtensorMap* map, const void* base, int64_t inner, int64_t outer, int64_t ld, int box_inner,
+                     int box_outer) {
+  return make_map_any(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, inner, outer, ld, box_inner, box_outer);
 }
 
 static int* device_error_ptr() {
@@ -447,35 +720,26 @@ bool gemm_tc_eligible(int M, int N, int K, const Operand& A, const Operand& B, c
   return true;
 }
 
-// Tile width and ring depth of a launch.
-enum TcVariant { TC_SMALL = 0, TC_LARGE = 1, TC_WIDE = 2, TC_NARROW = 3 };
-// Products of at least this many flops (4096 x 1024 x 1024) take the 128 x 256 tiles even when they fill the SMs less than
-// twice: their CTAs run long enough for the tile's lower shared-memory traffic per flop to outweigh the smaller grid
-// (the 3.6 GFLOP products of a 2048-sample step are below it: wide tiles cost that step 3 %).
-constexpr double kHeavyFlops = 8589934592.0;
-constexpr int kStagesNarrow = 4;   // 128 x 64 tiles: 4 stages of 24 KiB, two CTAs per SM (measured: giving a launch of at most one CTA
-                                   // per SM the whole shared memory as a deeper ring lowers whole-step throughput by 3-5 %)
-
-template <int kStages, int kBN, int NP, bool kDirect>
-static ss_status launch_group(const TcGroup<NP>& g, int total_ctas, cudaStream_t st) {
+template <int kStages, int kBN>
+static ss_status launch_flow(const TcFlow<kTcMaxFlow>& f, int ctas, cudaStream_t st) {
   static bool attr_set[64];
   int dev = 0;
   SS_CUDA(cudaGetDevice(&dev));
   if (dev >= 0 && dev < 64 && !attr_set[dev]) {
-    SS_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<kStages, kBN, NP, kDirect>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)tc_smem_bytes(kStages, kBN)));
+    SS_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<kStages, kBN, kTcMaxFlow>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)tc_smem_bytes(kStages, kBN, sizeof(TcMeta) * kTcMaxFlow)));
     attr_set[dev] = true;
   }
   { SS_TIMED("gemm_tc_kernel", st);
-  gemm_tc_kernel<kStages, kBN, NP, kDirect><<<total_ctas, kTcThreads, tc_smem_bytes(kStages, kBN), st>>>(g);
+  gemm_tc_kernel<kStages, kBN, kTcMaxFlow><<<ctas, kTcThreads, tc_smem_bytes(kStages, kBN, sizeof(TcMeta) * kTcMaxFlow), st>>>(f);
   }
   SS_LAUNCH_OK();
   return SS_OK;
 }
 
-// Fills one problem of a group for tile width bn; returns its CTA count (0 on failure).
-static int fill_problem(TcProblem* pr, const TcJob& j, int bn, int cta_begin, int* err) {
-  TcParams& p = pr->p;
+// Fills one problem of a flow for tile width bn; returns its tile count (0 on failure).
+static int fill_problem(TcProblem* pr, const TcJob& j, int bn, int tile_begin) {
+  TcParams& p = pr->meta.p;
   p.M = j.M; p.N = j.N; p.K = j.K;
   p.a_mn = (j.A.s_k != 1);
   p.b_mn = (j.B.s_k != 1);
@@ -485,16 +749,41 @@ static int fill_problem(TcProblem* pr, const TcJob& j, int bn, int cta_begin, in
   p.k_splits = ks;
   p.split_stride = j.split_stride;
   p.ep = j.ep;
-  p.err = err;
+  p.dep = -1; p.dep_mode = 0; p.dep_k_blocks = 0; p.dep_need = 0; p.dep_need_all = 0;
   const bool oka = p.a_mn ? make_map(&pr->map_a, j.A.p, j.M, j.K, j.A.s_k, 64, 64)
                           : make_map(&pr->map_a, j.A.p, j.K, j.M, j.A.s_row, 64, kBM);
   const bool okb = p.b_mn ? make_map(&pr->map_b, j.B.p, j.N, j.K, j.B.s_k, 64, 64)
-                          : make_map(&pr->map_b, j.B.p, j.K, j.N, j.B.s_row, 64, bn);
+                          : make_map(&pr->map_b, j.B.p, j.K, j.N, j.B.s_row, 64, 128);
   if (!oka || !okb) return 0;
-  pr->cta_begin = cta_begin;
-  pr->grid_x = (j.N + bn - 1) / bn;
-  pr->grid_y = (j.M + kBM - 1) / kBM;
-  return pr->grid_x * pr->grid_y * ks;
+  // Outputs through TMA stores: every 64-column piece of a tile lies on one side of the lo / hi boundary.
+  const Epilogue& ep = j.ep;
+  p.tma_out = 0;
+  pr->map_lo = pr->map_a; pr->map_hi = pr->map_a; pr->map_mask = pr->map_a;   // defined, unused unless tma_out
+  if (ep.out_lo && ep.lo_cols > 0 && ((ep.lo_cols & 63) == 0 || ep.lo_cols >= j.N) && (!ep.mask || ep.mask_bf16)) {
+    bool ok = true;
+    if (ep.lo_bf16) {
+      ok = make_map_any(&pr->map_lo, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, ep.out_lo, ep.lo_cols < j.N ? ep.lo_cols : j.N, j.M,
+                        ep.ld_lo, 64, 32);
+    } else {
+      const int64_t plane = ks > 1 ? j.split_stride : (int64_t)ep.ld_lo * j.M;
+      ok = (plane & 3) == 0 && make_map_any(&pr->map_lo, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, ep.out_lo,
+                                            ep.lo_cols < j.N ? ep.lo_cols : j.N, j.M, ep.ld_lo, 32, 32, 3, ks, plane);
+    }
+    if (ok && ep.lo_cols < j.N)
+      ok = ep.out_hi && make_map_any(&pr->map_hi, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, ep.out_hi, j.N - ep.lo_cols, j.M, ep.ld_hi, 32, 32);
+    if (ok && ep.mask)
+      ok = make_map_any(&pr->map_mask, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, ep.mask, ep.mask_cols < j.N ? ep.mask_cols : j.N, j.M,
+                        ep.ld_mask, 64, 32);
+    p.tma_out = ok ? 1 : 0;
+  }
+  pr->meta.tile_begin = tile_begin;
+  pr->meta.grid_x = (j.N + bn - 1) / bn;
+  pr->meta.grid_y = (j.M + kBM - 1) / kBM;
+  pr->meta.pad = 0;
+  int sx = pr->meta.grid_x;
+  if (j.signal_cols > 0 && (j.signal_cols + bn - 1) / bn < sx) sx = (j.signal_cols + bn - 1) / bn;
+  p.signal_x = sx;
+  return pr->meta.grid_x * pr->meta.grid_y * ks;
 }
 
 static bool splits_ok(const TcJob& j) {
@@ -502,66 +791,66 @@ static bool splits_ok(const TcJob& j) {
   return j.k_splits <= 1 || !(ep.lo_bf16 || ep.lo_cols < j.N || ep.bias || ep.relu || ep.mask);
 }
 
-ss_status gemm_tc_group(const TcJob* jobs, int n, cudaStream_t st) {
-  if (n < 1 || n > kTcMaxGroup) return SS_ERR_SHAPE;
-  for (int i = 0; i < n; ++i)
-    if (!splits_ok(jobs[i])) return SS_ERR_SHAPE;
-  int* err = device_error_ptr();
-  if (!err) return SS_ERR_CUDA;
-  if (n == 1) {
-    const TcJob& j = jobs[0];
-    const int nk_all = (j.K + kBK - 1) / kBK;
-    int ks = j.k_splits < 1 ? 1 : j.k_splits;
-    if (ks > nk_all) ks = nk_all;
-    const int nk_slice = (nk_all + ks - 1) / ks;
-    const long long mt = (j.M + kBM - 1) / kBM;
-    const long long ctas128 = (long long)((j.N + 127) / 128) * mt * ks;
-    const long long ctas256 = (long long)((j.N + 255) / 256) * mt * ks;
-    int variant = TC_SMALL;
-    const bool heavy = 2.0 * j.M * j.N * j.K >= kHeavyFlops;
-    if (j.N >= 256 && (ctas256 >= 2ll * num_sms() || heavy) && nk_slice >= 2 * kStagesWide) variant = TC_WIDE;
-    else if (ctas128 >= 2ll * num_sms() && nk_slice >= 2 * kStagesLarge) variant = TC_LARGE;
-    else if (j.N <= 64 || 2 * ctas128 <= num_sms()) variant = TC_NARROW;    // a narrow product, or too few 128-wide tiles to occupy the SMs
-    const int bn = variant == TC_WIDE ? 256 : (variant == TC_NARROW ? 64 : 128);
-    alignas(64) TcGroup<1> g;
-    g.n = 1;
-    const int ctas = fill_problem(&g.prob[0], j, bn, 0, err);
-    if (ctas < 1) return SS_ERR_CUDA;
-    switch (variant) {
-      case TC_WIDE: return launch_group<kStagesWide, 256, 1, true>(g, ctas, st);
-      case TC_LARGE: return launch_group<kStagesLarge, 128, 1, true>(g, ctas, st);
-      case TC_NARROW: return launch_group<kStagesNarrow, 64, 1, false>(g, ctas, st);
-      default: return launch_group<kStagesSmall, 128, 1, false>(g, ctas, st);
-    }
-  }
-  // a group made of wide products that is heavy as a whole takes the 128 x 256 tiles as well
-  double flops = 0.0;
+ss_status gemm_tc_flow(const TcJob* jobs, int n, int* ctrl, int max_rows, int max_ctas, cudaStream_t st) {
+  if (n < 1 || n > kTcMaxFlow) return SS_ERR_SHAPE;
   bool wide = true;
+  double flops = 0.0;
   for (int i = 0; i < n; ++i) {
     const TcJob& j = jobs[i];
+    if (!splits_ok(j)) return SS_ERR_SHAPE;
+    if (j.dep >= i || (j.dep >= 0 && (!ctrl || j.dep_mode < 1 || j.dep_mode > 2 || jobs[j.dep].k_splits > 1))) return SS_ERR_SHAPE;
+    if (j.dep >= 0 && jobs[j.dep].M > max_rows) return SS_ERR_SHAPE;
     flops += 2.0 * j.M * j.N * j.K;
-    const int nk_all = (j.K + kBK - 1) / kBK;
-    const int ks = j.k_splits < 1 ? 1 : (j.k_splits > nk_all ? nk_all : j.k_splits);
-    if (j.N < 256 || (nk_all + ks - 1) / ks < 2 * kStagesWide) wide = false;
+    if (j.N < 256) wide = false;
   }
-  wide = wide && flops >= 2.0 * kHeavyFlops;
-  alignas(64) TcGroup<kTcMaxGroup> g;
-  g.n = n;
+  int* err = device_error_ptr();
+  if (!err) return SS_ERR_CUDA;
+  // 128 x 256 tiles where every product is at least that wide and the flow fills the SMs with them
+  if (wide) {
+    long long t256 = 0;
+    for (int i = 0; i < n; ++i)
+      t256 += (long long)((jobs[i].N + 255) / 256) * ((jobs[i].M + kBM - 1) / kBM) * (jobs[i].k_splits < 1 ? 1 : jobs[i].k_splits);
+    wide = t256 >= num_sms();
+  }
+  const int bn = wide ? 256 : 128;
+  alignas(64) TcFlow<kTcMaxFlow> f;
+  f.n = n;
   int total = 0;
   for (int i = 0; i < n; ++i) {
-    const int ctas = fill_problem(&g.prob[i], jobs[i], wide ? 256 : 128, total, err);
-    if (ctas < 1) return SS_ERR_CUDA;
-    total += ctas;
+    const int tiles = fill_problem(&f.prob[i], jobs[i], bn, total);
+    if (tiles < 1) return SS_ERR_CUDA;
+    total += tiles;
   }
-  for (int i = n; i < kTcMaxGroup; ++i) g.prob[i] = g.prob[n - 1];   // never selected; keeps the parameter block defined
-  if (wide) return launch_group<kStagesWide, 256, kTcMaxGroup, true>(g, total, st);
-  return launch_group<kStagesSmall, 128, kTcMaxGroup, false>(g, total, st);
+  for (int i = 0; i < n; ++i) {
+    const TcJob& j = jobs[i];
+    if (j.dep < 0) continue;
+    TcParams& p = f.prob[i].meta.p;
+    p.dep = j.dep; p.dep_mode = j.dep_mode; p.dep_k_blocks = j.dep_k_blocks;
+    p.dep_need = kEpiWarps * f.prob[j.dep].meta.p.signal_x;  // every epilogue warp reports per tile
+    p.dep_need_all = p.dep_need * f.prob[j.dep].meta.grid_y;
+  }
+  for (int i = n; i < kTcMaxFlow; ++i) f.prob[i] = f.prob[n - 1];   // never selected; keeps the parameter block defined
+  f.total_tiles = total;
+  f.ctrl = ctrl;
+  f.rb_stride = (max_rows + kBM - 1) / kBM + 1;    // per product: one word per row block, then their total
+  f.err = err;
+  // A flow with dependencies keeps CTAs waiting for one another, and a waiting CTA still holds its SM's shared
+  // memory and a third of its registers, which the other streams' kernels then lack (measured with four replicas
+  // training: 13.9 M examples/s with a CTA on every SM, 15.6 M with 64, 15.9 M with 32, while the flows themselves
+  // get slower: 55 / 63 / 81 us).  So a flow takes 64 CTAs, more only when it has more than eight tiles for each.
+  int ctas = num_sms();
+  if (ctrl && max_ctas <= 0) max_ctas = total / 8 > 64 ? total / 8 : 64;
+  if (max_ctas > 0 && max_ctas < ctas) ctas = max_ctas;
+  if (total < ctas) ctas = total;
+  if (wide) return launch_flow<kStagesWide, 256>(f, ctas, st);
+  return launch_flow<kStagesNarrow, 128>(f, ctas, st);
 }
 
 ss_status gemm_tc(int M, int N, int K, const Operand& A, const Operand& B, const Epilogue& ep, cudaStream_t st,
                   int k_splits, int64_t split_stride) {
-  TcJob j{M, N, K, A, B, ep, k_splits, split_stride};
-  return gemm_tc_group(&j, 1, st);
+  TcJob j;
+  j.M = M; j.N = N; j.K = K; j.A = A; j.B = B; j.ep = ep; j.k_splits = k_splits; j.split_stride = split_stride;
+  return gemm_tc_flow(&j, 1, nullptr, 0, 0, st);
 }
 
 int read_device_error(bool clear) {

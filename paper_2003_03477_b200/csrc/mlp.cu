@@ -471,6 +471,42 @@ few_inputs_layer_kernel(const float* __restrict__ x, int K, const __nv_bfloat16*
   }
 }
 
+// Collects the tensor-core products of a pass into flows (one persistent launch each, see gemm.cuh) and remembers
+// which job of the open flow writes which tensor, so that a later product reading that tensor waits for its row
+// blocks inside the launch instead of for a kernel boundary.
+static_assert(kTcMaxFlow == 12, "the control-word region of the workspace is sized for 12 products per flow");
+struct FlowBuilder {
+  TcJob jobs[kTcMaxFlow];
+  int n = 0;
+  int writer[kMaxLayers];      // writer[l]: job of the open flow whose output is the tensor attached to layer l, or -1
+  int* ctrl;
+  int max_rows;
+  cudaStream_t st;
+  FlowBuilder(int* ctrl_, int max_rows_, cudaStream_t st_) : ctrl(ctrl_), max_rows(max_rows_), st(st_) {
+    for (int l = 0; l < kMaxLayers; ++l) writer[l] = -1;
+  }
+  // launches what has been collected; everything it writes is complete for whatever follows on the stream
+  ss_status flush() {
+    if (n == 0) return SS_OK;
+    const ss_status r = gemm_tc_flow(jobs, n, ctrl, max_rows, 0, st);
+    n = 0;
+    for (int l = 0; l < kMaxLayers; ++l) writer[l] = -1;
+    return r;
+  }
+  // adds a job; `reads` is the layer whose tensor is its A operand (or -1); returns the job's index or a negative status
+  int add(TcJob j, int reads, int dep_mode, int dep_k_blocks) {
+    if (n == kTcMaxFlow) {
+      const ss_status r = flush();
+      if (r != SS_OK) return r;
+    }
+    if (reads >= 0 && writer[reads] >= 0) {
+      j.dep = writer[reads]; j.dep_mode = dep_mode; j.dep_k_blocks = dep_k_blocks;
+    }
+    jobs[n] = j;
+    return n++;
+  }
+};
+
 static ss_status check_common(const MlpPlan& p, int B, const void* concat_f32, const void* concat_bf16,
                               const void* w_bf16, void* ws, size_t ws_bytes) {
   if (B < 1) return SS_ERR_SHAPE;
@@ -523,8 +559,10 @@ ss_status ss_mlp_fwd(const ss_mlp_desc* desc, const float* w, const void* w_bf16
   cudaStream_t cs = as_stream(stream);
   char* ws = reinterpret_cast<char*>(workspace);
   const int act_kind = p.bf16 ? OP_BF16 : OP_F32;
-  // the loss kernel's ticket starts at zero (the workspace arrives uninitialised); it clears itself after use
-  SS_CUDA(cudaMemsetAsync(ws + p.loss_part, 0, 4, cs));
+  // the loss kernel's ticket and the control words of the tensor-core flows start at zero (the workspace arrives
+  // uninitialised); both clear themselves after use
+  SS_CUDA(cudaMemsetAsync(ws + p.loss_part, 0, p.ctrl + p.ctrl_bytes - p.loss_part, cs));
+  FlowBuilder flow(reinterpret_cast<int*>(ws + p.ctrl), p.ctrl_rows, cs);
 
   for (int l = 0; l < p.nl; ++l) {
     const LayerInfo& L = p.layer[l];
@@ -535,6 +573,8 @@ ss_status ss_mlp_fwd(const ss_mlp_desc* desc, const float* w, const void* w_bf16
     Bm = p.bf16 ? Operand{reinterpret_cast<const __nv_bfloat16*>(w_bf16) + L.w_off, OP_BF16, L.in, 1}
                 : Operand{w + L.w_off, OP_F32, L.in, 1};
     if (l == p.nl - 1) {   // one output unit: a dot product per sample
+      st = flow.flush();
+      if (st != SS_OK) return st;
       unsigned int* ticket = reinterpret_cast<unsigned int*>(ws + p.loss_part);
       { SS_TIMED("logit_loss_kernel", cs);
       logit_loss_kernel<<<(B + 7) / 8, 256, 0, cs>>>(A.p, A.kind, A.s_row, Bm.p, Bm.kind, L.in, w + L.b_off, labels, B, logit,
@@ -563,7 +603,20 @@ ss_status ss_mlp_fwd(const ss_mlp_desc* desc, const float* w, const void* w_bf16
       SS_LAUNCH_OK();
       continue;
     }
-    st = gemm(B, L.out, L.in, A, Bm, ep, cs);
+    if (gemm_tc_eligible(B, L.out, L.in, A, Bm, ep)) {
+      // The whole chain of tensor-core layers is ONE launch: layer l's tiles wait for the row blocks of layer l - 1
+      // they read.  The first top layer reads the concat buffer, of which only the first D0 columns come from the
+      // bottom MLP: it contracts the pooled embeddings first and waits for the bottom output only then.
+      TcJob j;
+      j.M = B; j.N = L.out; j.K = L.in; j.A = A; j.B = Bm; j.ep = ep;
+      const int idx = flow.add(j, l - 1, 1, l == p.nb ? (p.D0 + 63) / 64 : 0);
+      if (idx < 0) return (ss_status)idx;
+      flow.writer[l] = idx;
+      continue;
+    }
+    st = flow.flush();
+    if (st != SS_OK) return st;
+    st = gemm_simt(B, L.out, L.in, A, Bm, ep, cs);
     if (st != SS_OK) return st;
   }
   return SS_OK;
@@ -619,8 +672,10 @@ ss_status ss_mlp_bwd(const ss_mlp_desc* desc, float* w, void* w_bf16, float* ada
     jobs.total += ncols * s_cols;
   };
 
-  TcJob dw_jobs[kMaxLayers];
-  int n_dw = 0;
+  // All tensor-core products of the pass -- per layer the input gradient dX = dY W (which produces the next dY) and
+  // the weight gradient dW = dY^T X -- form ONE flow, input gradient first: a product that reads a dY written inside
+  // the flow waits for the row blocks it needs (dX by tile row, dW by k block, since it contracts over the batch).
+  FlowBuilder flow(reinterpret_cast<int*>(ws + p.ctrl), p.ctrl_rows, cs);   // writer[l]: the job that writes dact[l]
   for (int l = last; l >= 0; --l) {
     const LayerInfo& L = p.layer[l];
     const void* G = ws + p.dact[l];
@@ -629,40 +684,9 @@ ss_status ss_mlp_bwd(const ss_mlp_desc* desc, float* w, void* w_bf16, float* ada
     if (l == 0) X = Operand{dense, p.bf16 ? OP_F32_ROUND_BF16 : OP_F32, 1, p.n_dense};
     else if (l == p.nb) X = Operand{p.bf16 ? concat_bf16 : (const void*)concat_f32, act_kind, 1, p.W};
     else X = Operand{ws + p.act[l - 1], act_kind, 1, L.in};
-    // db[o] = sum_b G[b, o]
-    add_job(G, act_kind, L.out, L.out, nullptr, 0, 0, 1, L.b_off);
-    // dW[o, i] = sum_b G[b, o] * X[b, i]
-    if (l == last) {
-      add_job(X.p, X.kind, X.s_k, L.in, G, dz_kind, 1, 1, L.w_off);          // out = 1: dW[i] = sum_b X[b,i] dz[b]
-    } else if (l == 0 && L.in <= kMaxSCols) {
-      add_job(G, act_kind, L.out, L.out, X.p, X.kind, X.s_k, L.in, L.w_off);  // few inputs: dW[o, :] per column o
-    } else {
-      Operand A{G, act_kind, 1, L.out};
-      Epilogue ep;
-      ep.out_lo = g + L.w_off; ep.lo_bf16 = 0; ep.ld_lo = L.in; ep.lo_cols = L.in;
-      if (gemm_tc_eligible(L.out, L.in, B, A, X, ep)) {
-        // Nothing on the way back needs dW, so the weight-gradient products of all layers wait and go out
-        // together as one launch after the last input gradient.  K = batch may be cut into slices; the
-        // update kernel adds them in slice order.
-        const int64_t size = (int64_t)L.in * L.out;
-        const int ks = p.k_splits[l];
-        if (ks > 1) {
-          ep.out_lo = gpart + p.gpart_off[l];
-          add_range(L.w_off, size, GRAD_SLICES, p.gpart_off[l], size, ks);
-        } else {
-          add_range(L.w_off, size, GRAD_FLAT, 0, 0, 1);
-        }
-        if (n_dw == kMaxLayers) return SS_ERR_SHAPE;
-        dw_jobs[n_dw++] = TcJob{L.out, L.in, B, A, X, ep, ks, size};
-      } else {
-        st = gemm(L.out, L.in, B, A, X, ep, cs);
-        add_range(L.w_off, (int64_t)L.in * L.out, GRAD_FLAT, 0, 0, 1);
-      }
-      if (st != SS_OK) return st;
-    }
-    if (l == 0) break;
     // dX[b, i] = sum_o G[b, o] * W[o, i], gated by the ReLU of the producing layer
-    if (l == last && l != p.nb) {
+    if (l == 0) {
+    } else if (l == last && l != p.nb) {
       const void* wl = p.bf16 ? (const void*)(reinterpret_cast<const __nv_bfloat16*>(w_bf16) + L.w_off) : (const void*)(w + L.w_off);
       const int64_t cnt = (int64_t)B * (L.in >> 3);            // L.in is a hidden width: a multiple of 8
       { SS_TIMED("dz_outer_mask_kernel", cs);
@@ -689,14 +713,59 @@ ss_status ss_mlp_bwd(const ss_mlp_desc* desc, float* w, void* w_bf16, float* ada
         ep.mask = ws + p.act[l - 1]; ep.ld_mask = L.in; ep.mask_cols = L.in;
         ep.ld_lo = L.in; ep.lo_cols = L.in;
       }
-      st = gemm(B, L.in, L.out, A, Wt, ep, cs);
-      if (st != SS_OK) return st;
+      if (gemm_tc_eligible(B, L.in, L.out, A, Wt, ep)) {
+        TcJob j;
+        j.M = B; j.N = L.in; j.K = L.out; j.A = A; j.B = Wt; j.ep = ep;
+        if (l == p.nb) j.signal_cols = p.D0;                   // later products read the bottom MLP's part only
+        const int idx = flow.add(j, l, 1, 0);
+        if (idx < 0) return (ss_status)idx;
+        // the weight gradient below reads dact[l] as well: the entry of layer l stays as it is
+        const int keep = flow.writer[l];
+        flow.writer[l - 1] = idx;
+        flow.writer[l] = keep;
+      } else {
+        st = flow.flush();
+        if (st != SS_OK) return st;
+        st = gemm_simt(B, L.in, L.out, A, Wt, ep, cs);
+        if (st != SS_OK) return st;
+      }
+    }
+    // db[o] = sum_b G[b, o]
+    add_job(G, act_kind, L.out, L.out, nullptr, 0, 0, 1, L.b_off);
+    // dW[o, i] = sum_b G[b, o] * X[b, i]
+    if (l == last) {
+      add_job(X.p, X.kind, X.s_k, L.in, G, dz_kind, 1, 1, L.w_off);          // out = 1: dW[i] = sum_b X[b,i] dz[b]
+    } else if (l == 0 && L.in <= kMaxSCols) {
+      add_job(G, act_kind, L.out, L.out, X.p, X.kind, X.s_k, L.in, L.w_off);  // few inputs: dW[o, :] per column o
+    } else {
+      Operand A{G, act_kind, 1, L.out};
+      Epilogue ep;
+      ep.out_lo = g + L.w_off; ep.lo_bf16 = 0; ep.ld_lo = L.in; ep.lo_cols = L.in;
+      if (gemm_tc_eligible(L.out, L.in, B, A, X, ep)) {
+        // K = batch may be cut into slices; the update kernel adds them in slice order.
+        const int64_t size = (int64_t)L.in * L.out;
+        const int ks = p.k_splits[l];
+        if (ks > 1) {
+          ep.out_lo = gpart + p.gpart_off[l];
+          add_range(L.w_off, size, GRAD_SLICES, p.gpart_off[l], size, ks);
+        } else {
+          add_range(L.w_off, size, GRAD_FLAT, 0, 0, 1);
+        }
+        TcJob j;
+        j.M = L.out; j.N = L.in; j.K = B; j.A = A; j.B = X; j.ep = ep; j.k_splits = ks; j.split_stride = size;
+        const int idx = flow.add(j, l, 2, 0);
+        if (idx < 0) return (ss_status)idx;
+      } else {
+        st = flow.flush();
+        if (st != SS_OK) return st;
+        st = gemm_simt(L.out, L.in, B, A, X, ep, cs);
+        if (st != SS_OK) return st;
+        add_range(L.w_off, (int64_t)L.in * L.out, GRAD_FLAT, 0, 0, 1);
+      }
     }
   }
-  for (int i = 0; i < n_dw; i += kTcMaxGroup) {
-    st = gemm_tc_group(dw_jobs + i, n_dw - i < kTcMaxGroup ? n_dw - i : kTcMaxGroup, cs);
-    if (st != SS_OK) return st;
-  }
+  st = flow.flush();
+  if (st != SS_OK) return st;
   {
     // all batch reductions of the pass in one launch; the update kernel adds the batch slices
     int rows = ((B + p.red_splits - 1) / p.red_splits + 7) & ~7;   // <= kRedRows by the choice of red_splits

@@ -22,7 +22,9 @@ struct MlpPlan {
   // respect to it after the ReLU mask.  The last bottom layer's output lives in the concat buffer and
   // the last top layer's in logit[], so act[] is unused for those two.
   size_t act[kMaxLayers], dact[kMaxLayers];
-  size_t grads, red_partial, gpart, loss_part, total;   // loss_part: a ticket word, then one partial loss per 8 samples
+  size_t grads, red_partial, gpart, loss_part, ctrl, total;   // loss_part: a ticket word, then one partial loss per 8 samples
+  int ctrl_rows;          // most rows of a product that another product of a tensor-core flow may wait for
+  size_t ctrl_bytes;      // control words of the tensor-core flows (directly behind the loss ticket: one memset clears both)
   int k_splits[kMaxLayers];      // K slices of the weight-gradient GEMM of each layer (1 = none)
   int64_t gpart_off[kMaxLayers]; // float offset of the layer's slice buffer inside the gpart region
   int red_splits;         // batch slices of the two-stage reductions (bias and skinny weight gradients)
@@ -71,10 +73,10 @@ inline ss_status make_mlp_plan(const ss_mlp_desc* d, int B, MlpPlan* p) {
   red_total += (size_t)p->layer[p->nl - 1].in;
   if (p->layer[0].in <= 16) red_total += (size_t)p->layer[0].in * p->layer[0].out;
   p->red_partial = take(red_total * 4 * (size_t)p->red_splits);
-  // Weight-gradient GEMMs contract over the batch and have small outputs.  They go out together as one launch, so the
-  // K range is cut into slices only while all their tiles together fill less than half the SMs (measured on the
-  // 2048-sample step, 74 tiles: 1 slice 15.1 M examples/s, 2 slices 14.8 M, 4 slices 14.1 M: the update kernel adds the
-  // slices in order and reads each of them).
+  // Weight-gradient GEMMs contract over the batch (K = B: dozens of k steps per tile) and have small outputs: few,
+  // long tiles.  They are part of the backward flow, where they are what the tail of the launch waits for, so K is cut
+  // into slices until their tiles are about as many as the SMs (slices of at least 8 k steps); the update kernel adds
+  // the slices in order.
   int64_t gp = 0;
   const int nk = (B + 63) / 64;
   auto sliced = [&](int l) {
@@ -88,9 +90,9 @@ inline ss_status make_mlp_plan(const ss_mlp_desc* d, int B, MlpPlan* p) {
     const LayerInfo& L = p->layer[l];
     int s = 1;
     if (sliced(l)) {
-      s = (int)(148 / (2 * all_tiles));
-      if (s > 16) s = 16;
-      if (s > nk / 16) s = nk / 16;                        // slices of at least 16 k-steps: a CTA's fixed cost outweighs shorter ones
+      s = (int)((148 + all_tiles / 2) / all_tiles);
+      if (s > 8) s = 8;
+      if (s > nk / 8) s = nk / 8;                          // slices of at least 8 k-steps: a tile's fixed cost outweighs shorter ones
       if (s > nk) s = nk;
       if (s < 1) s = 1;
     }
@@ -100,6 +102,11 @@ inline ss_status make_mlp_plan(const ss_mlp_desc* d, int B, MlpPlan* p) {
   }
   p->gpart = take((size_t)gp * 4);
   p->loss_part = take(((size_t)(B + 7) / 8 + 4) * 4);
+  int widest = B;
+  for (int l = 0; l < p->nl; ++l) widest = p->layer[l].out > widest ? p->layer[l].out : widest;
+  p->ctrl_rows = widest;
+  p->ctrl_bytes = (2 + (size_t)12 * (size_t)((widest + 127) / 128 + 1)) * 4;
+  p->ctrl = take(p->ctrl_bytes);
   p->total = o;
   return SS_OK;
 }
