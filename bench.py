@@ -596,12 +596,13 @@ def concurrent_sweep(model, graphs, cfg, K, W, args, peaks, value_off):
 
 def gemm_alone(stream, peaks):
     """The tensor-core GEMM kernel on its own (ss_gemm_bf16, bf16 in, fp32 out), timed with events around a
-    captured graph of back-to-back launches: a product large enough to fill the machine, and the largest
+    captured graph of back-to-back launches: two products large enough to fill the machine (256 x 256 tiles on CTA
+    pairs: 4096^3 is 256 such tiles on 74 pairs, i.e. 3.5 rounds; 8192 x 8192 x 4096 is 13.8 rounds), and the largest
     product of the medium model's step, against the measured burst bf16 peak."""
     import torch
     from paper_2003_03477_b200 import binding as ss
     res = []
-    for M, N, K, reps in ((4096, 4096, 4096, 10), (2048, 1728, 512, 20)):
+    for M, N, K, reps in ((4096, 4096, 4096, 10), (8192, 8192, 4096, 5), (2048, 1728, 512, 20)):
         a = torch.randn(M, K, device="cuda").to(torch.bfloat16)
         b = torch.randn(N, K, device="cuda").to(torch.bfloat16)
         c = torch.empty(M, N, device="cuda")

@@ -48,16 +48,19 @@ __host__ __device__ constexpr int stage_bytes(int bn) { return kTileBytes + bn *
 constexpr int kEpiWarps = 4;                              // one per tensor-memory lane quadrant
 constexpr int kTcThreads = 64 + 32 * kEpiWarps;
 constexpr int kQueue = 4;                                 // tiles a CTA may have drawn and not yet finished
-// Ring depth: 5 stages of 32 KiB for 128-wide tiles, 3 stages of 48 KiB for 256-wide tiles (a quarter less
-// shared-memory traffic per flop, for products that fill the machine); one CTA per SM either way.
-constexpr int kStagesNarrow = 5, kStagesWide = 3;
+// Ring depth: 4 stages of 32 KiB for 128-wide tiles, 3 stages of 48 KiB for 256-wide tiles (a quarter less
+// shared-memory traffic per flop, for products that fill the machine), 5 stages of 32 KiB for CTA pairs (which carry
+// no mask slabs); one CTA per SM in every case.
+constexpr int kStagesNarrow = 4, kStagesWide = 3, kStagesPair = 5;
 constexpr int kCtlBytes = 512;                            // barriers, tile queue, tensor-memory address, abort flag
-// Per epilogue warp: one 4 KiB slab (32 rows x 128 bytes, 128-byte swizzle) from which TMA stores a piece of the
-// output, and one slab into which TMA loads the warp's rows of the ReLU-gradient mask, 64 columns at a time.
+// Per epilogue warp: two 4 KiB slabs (32 rows x 128 bytes, 128-byte swizzle) from which TMA stores pieces of the
+// output (one is filled while the other is being read), kMaskSlabs (0 or 2) slabs into which TMA loads the warp's rows
+// of the ReLU-gradient mask, 64 columns each, and the tile's bias values.
 constexpr int kSlabBytes = 32 * 128;
-constexpr int kEpiWarpBytes = 2 * kSlabBytes;
-constexpr size_t tc_smem_bytes(int stages, int bn, size_t meta_bytes) {
-  return (size_t)stages * stage_bytes(bn) + kEpiWarps * kEpiWarpBytes + 1024 /*alignment slack*/ + kCtlBytes + meta_bytes;
+constexpr int kBiasBytes = 256 * 4;
+__host__ __device__ constexpr int epi_warp_bytes(int mask_slabs) { return (2 + mask_slabs) * kSlabBytes + kBiasBytes; }
+constexpr size_t tc_smem_bytes(int stages, int load_n, int mask_slabs, size_t meta_bytes) {
+  return (size_t)stages * stage_bytes(load_n) + kEpiWarps * epi_warp_bytes(mask_slabs) + 1024 /*alignment slack*/ + kCtlBytes + meta_bytes;
 }
 constexpr long long kWaitCycles = 400ll * 1000 * 1000;    // ~0.2 s: far beyond any legitimate wait
 
@@ -169,8 +172,45 @@ __device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, uint32_t sr
                ::"l"(reinterpret_cast<uint64_t>(map)), "r"(src), "r"(x), "r"(y), "r"(z) : "memory");
 }
 __device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
-__device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void tma_store_wait_read1() { asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); }
 __device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+// ---- CTA pairs (cta_group::2): two CTAs of a cluster share one 256-row MMA
+__device__ __forceinline__ uint32_t cluster_rank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t smem_addr, uint32_t rank) {   // the same offset in another CTA of the cluster
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// TMA load of one CTA of a pair; the bytes are counted on a barrier that may live in the other CTA (no multicast:
+// each CTA fetches its own tiles)
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, uint32_t bar_cluster, int x, int y) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar_cluster), "r"(x), "r"(y) : "memory");
+}
+__device__ __forceinline__ void tc_commit_pair(uint32_t bar) {          // arrives on the barrier at this offset in both CTAs
+  const uint16_t mask = 3;
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(bar), "h"(mask) : "memory");
+}
+__device__ __forceinline__ void tc_mma_pair(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
@@ -232,12 +272,21 @@ __device__ __forceinline__ TileAt locate_tile(const TcMeta* meta, int n, int t) 
 }
 
 // ---------------------------------------------------------------------------------------- kernel
-template <int kStages, int kBN, int NP>
+// kPair: the CTAs come in pairs (clusters of two).  A pair computes a 256 x kBN tile with one tcgen05.mma.cta_group::2
+// per k step, issued by the pair's first CTA: each CTA holds its 128 rows of A, HALF of the B tile (the tensor cores of
+// both SMs read both halves) and the accumulator of its own 128 rows.  Per flop a CTA loads and reads a third less
+// shared memory than with 128 x 256 tiles of its own, which is what bounds those.  Tiles are assigned round-robin to
+// the pairs (no dependencies between products in this mode).
+template <int kStages, int kBN, int NP, bool kPair, int kMaskSlabs>
 __global__ void __launch_bounds__(kTcThreads, 1)
 gemm_tc_kernel(const __grid_constant__ TcFlow<NP> flow) {
   extern __shared__ uint8_t smem_raw[];
-  constexpr int kStageBytes = stage_bytes(kBN);
+  constexpr int kLoadN = kPair ? kBN / 2 : kBN;            // columns of B this CTA loads
+  constexpr int kTileM = kPair ? 2 * kBM : kBM;            // rows of a tile
+  constexpr int kStageBytes = stage_bytes(kLoadN);
   constexpr int kTmemCols = 2 * kBN;                       // two accumulators of kBN fp32 columns
+  constexpr int kEpiWarpBytes = epi_warp_bytes(kMaskSlabs);
+  const uint32_t rank = kPair ? cluster_rank() : 0u;       // 0: the CTA that issues the pair's MMAs
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t tiles = (raw + 1023u) & ~1023u;                 // 1024-byte aligned swizzle atoms
   uint8_t* gen = smem_raw + (tiles - raw);
@@ -246,8 +295,8 @@ gemm_tc_kernel(const __grid_constant__ TcFlow<NP> flow) {
   uint8_t* ctl = epi_gen + kEpiWarps * kEpiWarpBytes;
   const uint32_t bar0 = epi0 + kEpiWarps * kEpiWarpBytes;
   // barriers: [0,S) full, [S,2S) empty, then accumulator full[2], empty[2], queue full[kQueue], empty[kQueue],
-  // mask slab full [epilogue warp]
-  constexpr int kNumBars = 2 * kStages + 4 + 2 * kQueue + kEpiWarps;
+  // mask slab full [epilogue warp][2]
+  constexpr int kNumBars = 2 * kStages + 4 + 2 * kQueue + 2 * kEpiWarps;
   int* tile_q = reinterpret_cast<int*>(ctl + 8 * kNumBars);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tile_q + kQueue);
   volatile int* aborted = reinterpret_cast<volatile int*>(tmem_slot + 1);
@@ -275,19 +324,25 @@ gemm_tc_kernel(const __grid_constant__ TcFlow<NP> flow) {
       asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&flow.prob[j].map_b)) : "memory");
     }
     for (int s = 0; s < kStages; ++s) { mbar_init(full(s), 1); mbar_init(empty(s), 1); }
-    for (int b = 0; b < 2; ++b) { mbar_init(acc_full(b), 1); mbar_init(acc_empty(b), kEpiWarps); }
+    for (int b = 0; b < 2; ++b) { mbar_init(acc_full(b), 1); mbar_init(acc_empty(b), kPair ? 2 * kEpiWarps : kEpiWarps); }
     for (int s = 0; s < kQueue; ++s) { mbar_init(q_full(s), 1); mbar_init(q_empty(s), 1 + kEpiWarps); }
-    for (int w = 0; w < kEpiWarps; ++w) mbar_init(mask_full(w), 1);
+    for (int w = 0; w < 2 * kEpiWarps; ++w) mbar_init(mask_full(w), 1);
     *aborted = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
   if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(kTmemCols) : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    if (kPair) {
+      asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(kTmemCols) : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    } else {
+      asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(kTmemCols) : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
   }
   tc_fence_before();
   __syncthreads();
+  if (kPair) cluster_sync_all();                           // the other CTA's barriers exist before anything arrives on them
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
   int* const done0 = flow.ctrl ? flow.ctrl + 2 : nullptr;
@@ -299,20 +354,21 @@ gemm_tc_kernel(const __grid_constant__ TcFlow<NP> flow) {
       uint32_t it = 0;                                     // stages filled so far (over all tiles)
       // the ticket of the next tile is drawn while the current one is loaded (the counter is a round trip to L2 away);
       // tickets are still drawn in order by a running CTA and worked off in order, which is all the waiting needs
-      int t_next = flow.ctrl ? atomicAdd(flow.ctrl, 1) : (int)blockIdx.x;
+      const int unit = kPair ? (int)(blockIdx.x >> 1) : (int)blockIdx.x, n_units = kPair ? (int)(gridDim.x >> 1) : (int)gridDim.x;
+      int t_next = flow.ctrl ? atomicAdd(flow.ctrl, 1) : unit;
       for (uint32_t qi = 0;; ++qi) {
         const int qs = qi % kQueue;
         if (!mbar_wait(q_empty(qs), ((qi / kQueue) & 1) ^ 1u, aborted, flow.err, 5)) break;
         int t = t_next;
         if (t >= flow.total_tiles) t = -1;
-        if (t >= 0) t_next = flow.ctrl ? atomicAdd(flow.ctrl, 1) : (int)(blockIdx.x + (qi + 1) * gridDim.x);
+        if (t >= 0) t_next = flow.ctrl ? atomicAdd(flow.ctrl, 1) : (int)(unit + (qi + 1) * n_units);
         tile_q[qs] = t;
         mbar_arrive(q_full(qs));
         if (t < 0) break;
         SS_TC_TRACE(2, t);
         const TileAt a = locate_tile(meta, n_prob, t);
         const TcProblem& pr = flow.prob[a.j];
-        const int m0 = a.y * kBM, n0 = a.x * kBN;
+        const int m0 = a.y * kTileM + (int)rank * kBM, n0 = a.x * kBN + (int)rank * kLoadN;   // this CTA's rows, its part of B
         int dep_mode = 0, dep_need = 0, dep_kb = 0;
         const int* dep_words = nullptr;
         const int a_mn = meta[a.j].p.a_mn, b_mn = meta[a.j].p.b_mn, K = meta[a.j].p.K;
@@ -350,8 +406,26 @@ gemm_tc_kernel(const __grid_constant__ TcFlow<NP> flow) {
           }
           const int s = it % kStages;
           if (!mbar_wait(empty(s), ((it / kStages) & 1) ^ 1u, aborted, flow.err, 1)) { failed = true; break; }
-          mbar_expect_tx(full(s), kStageBytes);
           const uint32_t sa = tiles + s * kStageBytes, sb = sa + kTileBytes;
+          if (kPair) {
+            // both CTAs' tiles are counted on the first CTA's barrier, which its MMA thread waits on
+            const uint32_t bar = map_to_cta(full(s), 0);
+            if (rank == 0) mbar_expect_tx(full(s), 2 * kStageBytes);
+            if (a_mn) {
+              tma_load_2d_pair(sa, &pr.map_a, bar, m0, k0);
+              tma_load_2d_pair(sa + kTileBytes / 2, &pr.map_a, bar, m0 + 64, k0);
+            } else {
+              tma_load_2d_pair(sa, &pr.map_a, bar, k0, m0);
+            }
+            if (b_mn) {
+#pragma unroll
+              for (int h = 0; h < kLoadN / 64; ++h) tma_load_2d_pair(sb + h * (kTileBytes / 2), &pr.map_b, bar, n0 + 64 * h, k0);
+            } else {
+#pragma unroll
+              for (int h = 0; h < kLoadN / 128; ++h) tma_load_2d_pair(sb + h * kTileBytes, &pr.map_b, bar, k0, n0 + 128 * h);
+            }
+          } else {
+          mbar_expect_tx(full(s), kStageBytes);
           if (a_mn) {                         // A stored [K, M]: two boxes of 64 k-rows x 64 m
             tma_load_2d(sa, &pr.map_a, full(s), m0, k0);
             tma_load_2d(sa + kTileBytes / 2, &pr.map_a, full(s), m0 + 64, k0);
@@ -364,6 +438,7 @@ gemm_tc_kernel(const __grid_constant__ TcFlow<NP> flow) {
           } else {
 #pragma unroll
             for (int h = 0; h < kBN / 128; ++h) tma_load_2d(sb + h * kTileBytes, &pr.map_b, full(s), k0, n0 + 128 * h);
+          }
           }
           ++it;
           if (i == 0) SS_TC_TRACE(3, t);
@@ -390,13 +465,15 @@ gemm_tc_kernel(const __grid_constant__ TcFlow<NP> flow) {
         const int t = tile_q[qs];
         mbar_arrive(q_empty(qs));
         if (t < 0) break;
+        if (kPair && rank != 0) continue;                  // the pair's MMAs are issued by its first CTA
         const TileAt a = locate_tile(meta, n_prob, t);
         const int a_mn = meta[a.j].p.a_mn, b_mn = meta[a.j].p.b_mn;
         int n_mma = meta[a.j].p.N - a.x * kBN;             // columns of this tile, rounded up to the instruction's granule
         n_mma = n_mma >= kBN ? kBN : ((n_mma + 15) & ~15);
+        if (kPair) n_mma = kBN;                            // each CTA holds exactly half of the instruction's columns
         // instruction descriptor: D = f32, A = B = bf16, majors, N >> 3, M >> 4
         const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)a_mn << 15) | ((uint32_t)b_mn << 16) |
-                               ((uint32_t)(n_mma >> 3) << 17) | ((uint32_t)(kBM >> 4) << 24);
+                               ((uint32_t)(n_mma >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
         // K-major: 8-row groups 1024 B apart (SBO), K step of 16 elements = 32 B inside the swizzle span.
         // MN-major: 64-wide m atoms 8192 B apart (LBO), 8-k groups 1024 B apart (SBO), K step of 16 = 2048 B.
         const uint32_t a_lbo = a_mn ? 8192u : 16u, a_step = a_mn ? 2048u : 32u;
@@ -416,13 +493,16 @@ gemm_tc_kernel(const __grid_constant__ TcFlow<NP> flow) {
           for (int k = 0; k < kBK / 16; ++k) {
             const uint64_t ad = smem_desc(sa + k * a_step, a_lbo, 1024u);
             const uint64_t bd = smem_desc(sb + k * b_step, b_lbo, 1024u);
-            tc_mma(d_tmem, ad, bd, idesc, (i > 0 || k > 0) ? 1u : 0u);
+            if (kPair) tc_mma_pair(d_tmem, ad, bd, idesc, (i > 0 || k > 0) ? 1u : 0u);
+            else tc_mma(d_tmem, ad, bd, idesc, (i > 0 || k > 0) ? 1u : 0u);
           }
-          tc_commit(empty(s));              // frees the stage when these MMAs have read it
+          if (kPair) tc_commit_pair(empty(s));   // frees the stage in both CTAs when these MMAs have read it
+          else tc_commit(empty(s));
           ++it;
         }
         if (failed) break;
-        tc_commit(acc_full(buf));           // accumulator complete
+        if (kPair) tc_commit_pair(acc_full(buf));   // accumulator complete, in both CTAs
+        else tc_commit(acc_full(buf));
         SS_TC_TRACE(6, t);
         ++at;
       }
@@ -430,9 +510,11 @@ gemm_tc_kernel(const __grid_constant__ TcFlow<NP> flow) {
   } else {
     // ------------------------------------------------------------------ epilogue warps 2..5
     const int q = warp & 3;               // tensor-memory lane quadrant this warp may read
-    uint8_t* const slab_gen = epi_gen + q * kEpiWarpBytes;
-    const uint32_t slab_out = epi0 + q * kEpiWarpBytes, slab_mask = slab_out + kSlabBytes;
-    uint32_t mask_uses = 0;               // completed phases of this warp's mask barrier
+    uint8_t* const slab_gen = epi_gen + q * kEpiWarpBytes;              // [out 0][out 1][mask 0][mask 1][bias]
+    const uint32_t slab_out = epi0 + q * kEpiWarpBytes, slab_mask = slab_out + 2 * kSlabBytes;
+    float* const s_bias = reinterpret_cast<float*>(slab_gen + (2 + kMaskSlabs) * kSlabBytes);
+    uint32_t mask_uses[2] = {0, 0};       // completed phases of this warp's two mask barriers
+    uint32_t n_stores = 0;                // slabs handed to TMA so far (they alternate)
     uint32_t at = 0;
     for (uint32_t qi = 0;; ++qi) {
       const int qs = qi % kQueue;
@@ -445,20 +527,36 @@ gemm_tc_kernel(const __grid_constant__ TcFlow<NP> flow) {
       const Epilogue ep = meta[a.j].p.ep;                  // by value: registers
       struct { int M, N, signal_x; int64_t split_stride; } p = {meta[a.j].p.M, meta[a.j].p.N, meta[a.j].p.signal_x,
                                                                  meta[a.j].p.split_stride};
-      const int m0 = a.y * kBM, n0 = a.x * kBN;
+      const int m0 = a.y * kTileM + (int)rank * kBM, n0 = a.x * kBN;
       const int buf = at & 1;
-      const bool tma_out = meta[a.j].p.tma_out != 0;
+      const bool tma_out = meta[a.j].p.tma_out != 0 && (kMaskSlabs > 0 || ep.mask == nullptr);
       const TcProblem& pr = flow.prob[a.j];
-      // this warp's rows of the mask (the producing layer's bf16 activation), 64 columns per slab, requested as soon
-      // as the tile is known: they arrive while the tensor cores still work on the tile
+      // Everything the epilogue needs from memory is requested as soon as the tile is known, so that it arrives while
+      // the tensor cores still work on the tile: the tile's bias values (every thread needs all of them: one 16-byte
+      // load per lane into the warp's shared memory), and this warp's rows of the mask (the producing layer's bf16
+      // activation), 64 columns per slab.
+      if (ep.bias) {
+#pragma unroll
+        for (int i = 0; i < kBN / 128; ++i) {
+          const int n = n0 + 128 * i + 4 * lane;
+          float4 bv = make_float4(0.f, 0.f, 0.f, 0.f);
+          if (n < p.N) bv = __ldg(reinterpret_cast<const float4*>(ep.bias + n));   // N is a multiple of 8
+          *reinterpret_cast<float4*>(s_bias + 128 * i + 4 * lane) = bv;
+        }
+      }
       const bool masked = tma_out && ep.mask != nullptr;
       auto request_mask = [&](int h) {                     // the mask of columns 64 h .. 64 h + 63 of the tile, rows of this warp
-        if (lane == 0) {
-          mbar_expect_tx(mask_full(q), kSlabBytes);
-          tma_load_2d(slab_mask, &pr.map_mask, mask_full(q), n0 + 64 * h, m0 + 32 * q);
+        if (kMaskSlabs > 0 && lane == 0) {
+          mbar_expect_tx(mask_full(2 * q + (h & 1)), kSlabBytes);
+          tma_load_2d(slab_mask + (h & 1) * kSlabBytes, &pr.map_mask, mask_full(2 * q + (h & 1)), n0 + 64 * h, m0 + 32 * q);
         }
       };
-      if (masked && n0 < ep.mask_cols) request_mask(0);
+      if (masked) {
+#pragma unroll
+        for (int h = 0; h < 2; ++h)
+          if (n0 + 64 * h < ep.mask_cols && n0 + 64 * h < p.N) request_mask(h);
+      }
+      __syncwarp();                                        // the bias values are in shared memory
       if (!mbar_wait(acc_full(buf), (at >> 1) & 1, aborted, flow.err, 3)) break;
       if (threadIdx.x == 64) SS_TC_TRACE(7, t);
       tc_fence_after();
@@ -483,10 +581,8 @@ gemm_tc_kernel(const __grid_constant__ TcFlow<NP> flow) {
           if (ep.bias) {
 #pragma unroll
             for (int j = 0; j < 32; j += 4) {
-              if (nb + j < p.N) {            // N is a multiple of 8: four columns are inside together or not at all
-                const float4 bv = __ldg(reinterpret_cast<const float4*>(ep.bias + nb + j));
-                v[j] += bv.x; v[j + 1] += bv.y; v[j + 2] += bv.z; v[j + 3] += bv.w;
-              }
+              const float4 bv = *reinterpret_cast<const float4*>(s_bias + 32 * c + j);   // the same address in every lane
+              v[j] += bv.x; v[j + 1] += bv.y; v[j + 2] += bv.z; v[j + 3] += bv.w;
             }
           }
           if (ep.relu) {
@@ -494,12 +590,13 @@ gemm_tc_kernel(const __grid_constant__ TcFlow<NP> flow) {
             for (int j = 0; j < 32; ++j) v[j] = fmaxf(v[j], 0.f);
           }
           if (masked && nb < ep.mask_cols) {
-            // the mask slab holds the 64 columns of this piece and its neighbour
-            if (!odd && !mbar_wait(mask_full(q), (mask_uses++) & 1, aborted, flow.err, 9)) { failed = true; break; }
+            // mask slab (c / 2) & 1 holds the 64 columns of this piece and its neighbour
+            const int h = c >> 1, ms = h & 1;
+            if (!odd && !mbar_wait(mask_full(2 * q + ms), (mask_uses[ms]++) & 1, aborted, flow.err, 9)) { failed = true; break; }
 #pragma unroll
             for (int g = 0; g < 4; ++g) {
               if (nb + 8 * g >= ep.mask_cols) break;
-              const uint4 mk = *reinterpret_cast<const uint4*>(slab_gen + kSlabBytes + row_off + ((uint32_t)((g + 4 * odd) ^ sw) << 4));
+              const uint4 mk = *reinterpret_cast<const uint4*>(slab_gen + (2 + ms) * kSlabBytes + row_off + ((uint32_t)((g + 4 * odd) ^ sw) << 4));
               const uint32_t w[4] = {mk.x, mk.y, mk.z, mk.w};
 #pragma unroll
               for (int j = 0; j < 4; ++j) {
@@ -509,17 +606,18 @@ gemm_tc_kernel(const __grid_constant__ TcFlow<NP> flow) {
                 if (!((hi & 0x8000u) == 0 && (hi & 0x7FFFu) != 0)) v[8 * g + 2 * j + 1] = 0.f;
               }
             }
-            // the slab's 64 columns are used up: ask for the tile's next 64
+            // the slab's 64 columns are used up: it takes the 64 columns after the other slab's (256-wide tiles)
             const bool last_of_slab = odd || nb + 32 >= p.N || nb + 32 >= ep.mask_cols;
-            if (last_of_slab && c + 1 < kBN / 32 && n0 + 32 * (c + 1) < ep.mask_cols && n0 + 32 * (c + 1) < p.N) {
+            if (kBN > 128 && last_of_slab && h + 2 < kBN / 64 && n0 + 64 * (h + 2) < ep.mask_cols && n0 + 64 * (h + 2) < p.N) {
               __syncwarp();                                // every lane has read the slab
-              request_mask((c + 1) >> 1);
+              request_mask(h + 2);
             }
           }
           const bool to_lo = nb < ep.lo_cols;
           if (to_lo && ep.lo_bf16) {
+            uint8_t* const slab = slab_gen + (n_stores & 1) * kSlabBytes;
             if (!odd) {
-              if (lane == 0) tma_store_wait_read();        // the slab's previous contents have been read
+              if (lane == 0) tma_store_wait_read1();       // this slab's previous contents have been read (the other may be in flight)
               __syncwarp();
             }
 #pragma unroll
@@ -527,30 +625,33 @@ gemm_tc_kernel(const __grid_constant__ TcFlow<NP> flow) {
               uint4 o;
               o.x = pack2(v[8 * g], v[8 * g + 1]); o.y = pack2(v[8 * g + 2], v[8 * g + 3]);
               o.z = pack2(v[8 * g + 4], v[8 * g + 5]); o.w = pack2(v[8 * g + 6], v[8 * g + 7]);
-              *reinterpret_cast<uint4*>(slab_gen + row_off + ((uint32_t)((g + 4 * odd) ^ sw) << 4)) = o;
+              *reinterpret_cast<uint4*>(slab + row_off + ((uint32_t)((g + 4 * odd) ^ sw) << 4)) = o;
             }
             if (odd || nb + 32 >= p.N || nb + 32 >= ep.lo_cols) {   // the slab is complete (or the output ends here)
               asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
               __syncwarp();
               if (lane == 0 && !*aborted) {
-                tma_store_2d(&pr.map_lo, slab_out, nb - 32 * odd, m0 + 32 * q);
+                tma_store_2d(&pr.map_lo, slab_out + (n_stores & 1) * kSlabBytes, nb - 32 * odd, m0 + 32 * q);
                 tma_store_commit();
               }
+              ++n_stores;
             }
           } else {
-            if (lane == 0) tma_store_wait_read();
+            uint8_t* const slab = slab_gen + (n_stores & 1) * kSlabBytes;
+            if (lane == 0) tma_store_wait_read1();
             __syncwarp();
 #pragma unroll
             for (int g = 0; g < 8; ++g)
-              *reinterpret_cast<float4*>(slab_gen + row_off + ((uint32_t)(g ^ sw) << 4)) =
+              *reinterpret_cast<float4*>(slab + row_off + ((uint32_t)(g ^ sw) << 4)) =
                   make_float4(v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             __syncwarp();
             if (lane == 0 && !*aborted) {
-              if (to_lo) tma_store_3d(&pr.map_lo, slab_out, nb, m0 + 32 * q, a.z);
-              else tma_store_2d(&pr.map_hi, slab_out, nb - ep.lo_cols, m0 + 32 * q);
+              if (to_lo) tma_store_3d(&pr.map_lo, slab_out + (n_stores & 1) * kSlabBytes, nb, m0 + 32 * q, a.z);
+              else tma_store_2d(&pr.map_hi, slab_out + (n_stores & 1) * kSlabBytes, nb - ep.lo_cols, m0 + 32 * q);
               tma_store_commit();
             }
+            ++n_stores;
           }
         }
         if (failed) break;
@@ -572,10 +673,8 @@ gemm_tc_kernel(const __grid_constant__ TcFlow<NP> flow) {
         if (ep.bias) {
 #pragma unroll
           for (int j = 0; j < 32; j += 4) {
-            if (nb + j < p.N) {              // N is a multiple of 8: four columns are inside together or not at all
-              const float4 bv = __ldg(reinterpret_cast<const float4*>(ep.bias + nb + j));
-              v[j] += bv.x; v[j + 1] += bv.y; v[j + 2] += bv.z; v[j + 3] += bv.w;
-            }
+            const float4 bv = *reinterpret_cast<const float4*>(s_bias + 32 * c + j);   // the same address in every lane
+            v[j] += bv.x; v[j + 1] += bv.y; v[j + 2] += bv.z; v[j + 3] += bv.w;
           }
         }
         if (ep.relu) {
@@ -619,7 +718,10 @@ gemm_tc_kernel(const __grid_constant__ TcFlow<NP> flow) {
       // the accumulator may be overwritten: this warp's reads of it are complete
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(acc_empty(buf));
+      if (lane == 0) {
+        if (kPair) mbar_arrive_cluster(map_to_cta(acc_empty(buf), 0));   // the MMA thread of the pair's first CTA waits for both
+        else mbar_arrive(acc_empty(buf));
+      }
       if (threadIdx.x == 64) SS_TC_TRACE(8, t);
       // completion word of the row block, for the products that read this output
       if (done0 && a.x < p.signal_x) {
@@ -643,9 +745,11 @@ gemm_tc_kernel(const __grid_constant__ TcFlow<NP> flow) {
 
   tc_fence_before();
   __syncthreads();
+  if (kPair) cluster_sync_all();                           // neither CTA leaves while the other may still signal it
   if (warp == 1) {
     tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
+    if (kPair) asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
+    else asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
   }
   // the last CTA to leave clears the control words for the next launch (every other CTA is past its last access)
   if (flow.ctrl && threadIdx.x == 0 && !*aborted) {
@@ -720,25 +824,40 @@ bool gemm_tc_eligible(int M, int N, int K, const Operand& A, const Operand& B, c
   return true;
 }
 
-template <int kStages, int kBN>
+template <int kStages, int kBN, bool kPair, int kMaskSlabs>
 static ss_status launch_flow(const TcFlow<kTcMaxFlow>& f, int ctas, cudaStream_t st) {
   static bool attr_set[64];
   int dev = 0;
   SS_CUDA(cudaGetDevice(&dev));
+  const size_t smem = tc_smem_bytes(kStages, kPair ? kBN / 2 : kBN, kMaskSlabs, sizeof(TcMeta) * kTcMaxFlow);
   if (dev >= 0 && dev < 64 && !attr_set[dev]) {
-    SS_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<kStages, kBN, kTcMaxFlow>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)tc_smem_bytes(kStages, kBN, sizeof(TcMeta) * kTcMaxFlow)));
+    SS_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<kStages, kBN, kTcMaxFlow, kPair, kMaskSlabs>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)smem));
     attr_set[dev] = true;
   }
   { SS_TIMED("gemm_tc_kernel", st);
-  gemm_tc_kernel<kStages, kBN, kTcMaxFlow><<<ctas, kTcThreads, tc_smem_bytes(kStages, kBN, sizeof(TcMeta) * kTcMaxFlow), st>>>(f);
+  if (kPair) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)ctas, 1, 1);
+    cfg.blockDim = dim3(kTcThreads, 1, 1);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    SS_CUDA(cudaLaunchKernelEx(&cfg, gemm_tc_kernel<kStages, kBN, kTcMaxFlow, kPair, kMaskSlabs>, f));
+  } else {
+    gemm_tc_kernel<kStages, kBN, kTcMaxFlow, kPair, kMaskSlabs><<<ctas, kTcThreads, smem, st>>>(f);
+  }
   }
   SS_LAUNCH_OK();
   return SS_OK;
 }
 
 // Fills one problem of a flow for tile width bn; returns its tile count (0 on failure).
-static int fill_problem(TcProblem* pr, const TcJob& j, int bn, int tile_begin) {
+static int fill_problem(TcProblem* pr, const TcJob& j, int bn, int tile_begin, int tile_m = kBM) {
   TcParams& p = pr->meta.p;
   p.M = j.M; p.N = j.N; p.K = j.K;
   p.a_mn = (j.A.s_k != 1);
@@ -778,7 +897,7 @@ static int fill_problem(TcProblem* pr, const TcJob& j, int bn, int tile_begin) {
   }
   pr->meta.tile_begin = tile_begin;
   pr->meta.grid_x = (j.N + bn - 1) / bn;
-  pr->meta.grid_y = (j.M + kBM - 1) / kBM;
+  pr->meta.grid_y = (j.M + tile_m - 1) / tile_m;
   pr->meta.pad = 0;
   int sx = pr->meta.grid_x;
   if (j.signal_cols > 0 && (j.signal_cols + bn - 1) / bn < sx) sx = (j.signal_cols + bn - 1) / bn;
@@ -805,19 +924,26 @@ ss_status gemm_tc_flow(const TcJob* jobs, int n, int* ctrl, int max_rows, int ma
   }
   int* err = device_error_ptr();
   if (!err) return SS_ERR_CUDA;
-  // 128 x 256 tiles where every product is at least that wide and the flow fills the SMs with them
+  // 128 x 256 tiles where every product is at least that wide and the flow fills the SMs with them; 256 x 256 tiles on
+  // CTA pairs where, in addition, no product waits for another (tiles then go round-robin) and there is no K slicing
+  long long t256 = 0, t_pair = 0;
+  bool pair = wide && ctrl == nullptr;
   if (wide) {
-    long long t256 = 0;
-    for (int i = 0; i < n; ++i)
-      t256 += (long long)((jobs[i].N + 255) / 256) * ((jobs[i].M + kBM - 1) / kBM) * (jobs[i].k_splits < 1 ? 1 : jobs[i].k_splits);
+    for (int i = 0; i < n; ++i) {
+      const long long ks = jobs[i].k_splits < 1 ? 1 : jobs[i].k_splits;
+      t256 += (long long)((jobs[i].N + 255) / 256) * ((jobs[i].M + kBM - 1) / kBM) * ks;
+      t_pair += (long long)((jobs[i].N + 255) / 256) * ((jobs[i].M + 2 * kBM - 1) / (2 * kBM));
+      if (ks > 1 || jobs[i].dep >= 0) pair = false;
+    }
     wide = t256 >= num_sms();
+    pair = pair && t_pair >= num_sms() / 2;
   }
   const int bn = wide ? 256 : 128;
   alignas(64) TcFlow<kTcMaxFlow> f;
   f.n = n;
   int total = 0;
   for (int i = 0; i < n; ++i) {
-    const int tiles = fill_problem(&f.prob[i], jobs[i], bn, total);
+    const int tiles = fill_problem(&f.prob[i], jobs[i], bn, total, pair ? 2 * kBM : kBM);
     if (tiles < 1) return SS_ERR_CUDA;
     total += tiles;
   }
@@ -841,9 +967,14 @@ ss_status gemm_tc_flow(const TcJob* jobs, int n, int* ctrl, int max_rows, int ma
   int ctas = num_sms();
   if (ctrl && max_ctas <= 0) max_ctas = total / 8 > 64 ? total / 8 : 64;
   if (max_ctas > 0 && max_ctas < ctas) ctas = max_ctas;
+  if (pair) {
+    ctas &= ~1;                                            // whole pairs
+    if (2 * total < ctas) ctas = 2 * total;
+    return launch_flow<kStagesPair, 256, true, 0>(f, ctas, st);
+  }
   if (total < ctas) ctas = total;
-  if (wide) return launch_flow<kStagesWide, 256>(f, ctas, st);
-  return launch_flow<kStagesNarrow, 128>(f, ctas, st);
+  if (wide) return launch_flow<kStagesWide, 256, false, 2>(f, ctas, st);
+  return launch_flow<kStagesNarrow, 128, false, 2>(f, ctas, st);
 }
 
 ss_status gemm_tc(int M, int N, int K, const Operand& A, const Operand& B, const Epilogue& ep, cudaStream_t st,
