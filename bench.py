@@ -359,6 +359,8 @@ def bench_gpu(args):
     peaks = measured_peaks()
     barrier = Barrier(world)
 
+    if args.flow_ctas:
+        ss.ss_mlp_set_flow_ctas(args.flow_ctas)
     model, host, dev, max_L = build_job(cfg, device, workers=max(1, args.workers))
     # un-captured warm-up: first-use set-up inside the library (function attributes, symbol addresses)
     for r in range(cfg.R):
@@ -989,6 +991,8 @@ def main():
     ap.add_argument("--no-sweep", action="store_true", help="skip the sync sweep concurrent with training")
     ap.add_argument("--sweep-seconds", type=float, default=0.25, help="training time per point of the concurrent sweep")
     ap.add_argument("--sweep-all-r", action="store_true", help="concurrent sweep over R = 2, 4, 8, 16 instead of the workload's R")
+    ap.add_argument("--flow-ctas", type=int, default=0,
+                    help="CTAs of the persistent tensor-core launches of the MLP (0 = the library's rule)")
     ap.add_argument("--foreground", type=int, default=0,
                     help="also time the foreground variant: one sync pass on the training streams every k steps")
     ap.add_argument("--workers", type=int, default=1,

@@ -27,7 +27,7 @@ SS_SYNC_BMUF_NESTEROV = 2
 EXPORTS = ["ss_status_str", "ss_last_cuda_error", "ss_num_sms", "ss_embbag_fwd", "ss_embbag_bwd_workspace_bytes",
            "ss_embbag_bwd_adagrad", "ss_embbag_bwd_sort", "ss_embbag_bwd_apply", "ss_embbag_bwd_sort_noalloc", "ss_mlp_param_count", "ss_mlp_param_offsets", "ss_mlp_workspace_bytes",
            "ss_mlp_fwd", "ss_mlp_bwd", "ss_ne_accumulate", "ss_ne_value", "ss_sync_easgd", "ss_sync_ma", "ss_sync_bmuf", "ss_shadow_start", "ss_shadow_rounds", "ss_shadow_pause", "ss_shadow_stop", "ss_to_bf16",
-           "ss_gemm_bf16", "ss_device_error", "ssh_fill_uniform", "ss_profile", "ss_profile_collect"]
+           "ss_gemm_bf16", "ss_device_error", "ss_mlp_set_flow_ctas", "ssh_fill_uniform", "ss_profile", "ss_profile_collect"]
 
 
 class SsError(RuntimeError):
@@ -91,12 +91,14 @@ def lib() -> C.CDLL:
         L.ss_to_bf16.argtypes = [vp, vp, i64, vp]
         L.ss_gemm_bf16.argtypes = [vp, i32, i64, vp, i32, i64, vp, i64, i32, i32, i32, i32, vp]
         L.ss_device_error.argtypes = [i32]
+        L.ss_mlp_set_flow_ctas.argtypes = [i32]
+        L.ss_mlp_set_flow_ctas.restype = None
         L.ss_profile.argtypes = [i32]
         L.ss_profile_collect.argtypes = [C.c_char_p, sz, C.POINTER(f32), i32]
         L.ssh_fill_uniform.argtypes = [vp, i64, C.c_uint64, C.c_uint64, f32, f32, vp]
         for name in EXPORTS:
             if name not in ("ss_status_str", "ss_last_cuda_error", "ss_num_sms", "ss_embbag_bwd_workspace_bytes",
-                            "ss_mlp_param_count", "ss_mlp_workspace_bytes", "ss_shadow_rounds"):
+                            "ss_mlp_param_count", "ss_mlp_workspace_bytes", "ss_shadow_rounds", "ss_mlp_set_flow_ctas"):
                 getattr(L, name).restype = i32
         _lib = L
     return _lib
@@ -262,6 +264,11 @@ def ss_sync_bmuf(w: Sequence[torch.Tensor], global_, delta, n, alpha, eta, mu, f
 def ss_gemm_bf16(a, a_mn_major, lda, b, b_mn_major, ldb, c, ldc, M, N, K, force_simt=0, stream=None) -> None:
     _check("ss_gemm_bf16", lib().ss_gemm_bf16(_ptr(a), int(a_mn_major), lda, _ptr(b), int(b_mn_major), ldb, _ptr(c),
                                                ldc, M, N, K, int(force_simt), _stream(stream)))
+
+
+def ss_mlp_set_flow_ctas(ctas: int) -> None:
+    """CTAs the persistent tensor-core launches of the MLP take (0 = the library's rule)."""
+    lib().ss_mlp_set_flow_ctas(int(ctas))
 
 
 def ss_device_error(clear: bool = True) -> int:

@@ -2,7 +2,7 @@
 //
 //   C[m, n] = sum_k A(m, k) * B(n, k)        m < M, n < N, k < K
 //
-// followed by one epilogue: + bias[n], ReLU, multiply by (mask[m, n] > 0) for n < mask_cols, then
+// followed by one epilogue: + bias[n], ReLU, multiply by (mask[m, n] > 0) for n < mask_cols (mask_cols > 0), then
 // columns [0, lo_cols) go to out_lo (float or bf16, leading dimension ld_lo) and columns
 // [lo_cols, N) to the float matrix out_hi at column n - lo_cols.
 #pragma once
@@ -25,6 +25,14 @@ struct Epilogue {
   int lo_cols = 0;
   float* out_hi = nullptr;
   int64_t ld_hi = 0;
+  // Tensor-core kernels only.  bits_out: besides out_lo (bf16), one bit per element "the stored value is positive",
+  // bit n % 32 of word [m * ld_bits_out + n / 32]: the ReLU-gradient mask of the backward pass at 1/16 of the bytes.
+  // mask_bits: such a word array of the producing layer; when given it is used instead of `mask` (same meaning).
+  // Both pitches are multiples of 4 words and the arrays 16-byte aligned.
+  uint32_t* bits_out = nullptr;
+  int64_t ld_bits_out = 0;
+  const uint32_t* mask_bits = nullptr;
+  int64_t ld_mask_bits = 0;
 };
 
 struct Operand {
@@ -72,6 +80,8 @@ inline size_t tc_flow_ctrl_ints(int max_rows) { return 2 + (size_t)kTcMaxFlow * 
 // ctrl == nullptr: tiles are assigned round-robin instead (only for flows without dependencies).
 // max_ctas <= 0: one CTA per SM at most.
 ss_status gemm_tc_flow(const TcJob* jobs, int n, int* ctrl, int max_rows, int max_ctas, cudaStream_t st);
+// CTAs a flow with dependencies takes when the caller gives no number (0: the built-in rule).
+void set_flow_ctas(int ctas);
 // Tensor cores when eligible, SIMT otherwise.
 ss_status gemm(int M, int N, int K, const Operand& A, const Operand& B, const Epilogue& ep, cudaStream_t st);
 // The device error flag raised by a bounded wait that ran out (0 = none); synchronises the device.

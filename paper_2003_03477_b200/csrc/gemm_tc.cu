@@ -113,13 +113,15 @@ __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
+// One try: the hardware may park the thread for up to the given time while the phase is incomplete (it is woken
+// when the phase completes), so a waiting role leaves the issue slots to the other warps of the SM.
 __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
       "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+      : "=r"(ok) : "r"(bar), "r"(parity), "r"(20000u) : "memory");
   return ok;
 }
 // Bounded wait.  Returns false when the limit is reached (records `code`) or another role has given up.
@@ -152,6 +154,7 @@ __device__ __forceinline__ bool wait_count(const int* word, int need, volatile i
         atomicCAS(err, 0, 4);
         return false;
       }
+      __nanosleep(200);
     }
   }
   // what the other CTAs stored through the generic proxy is read by TMA (async proxy) from here on
@@ -244,6 +247,18 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes,
   d |= 1ull << 46;
   d |= 2ull << 61;
   return d;
+}
+
+// Two bits for a packed pair of bf16: each "the value is positive" (sign clear and not zero).
+__device__ __forceinline__ uint32_t positive2(uint32_t packed) {
+  const uint32_t lo = packed & 0xFFFFu, hi = packed >> 16;
+  return (uint32_t)((lo & 0x8000u) == 0 && (lo & 0x7FFFu) != 0) | ((uint32_t)((hi & 0x8000u) == 0 && (hi & 0x7FFFu) != 0) << 1);
+}
+__device__ __forceinline__ uint32_t pick4(const uint4& v, int i) {
+  return (i & 2) ? ((i & 1) ? v.w : v.z) : ((i & 1) ? v.y : v.x);
+}
+__device__ __forceinline__ void put4(uint4& v, int i, uint32_t w) {
+  if (i == 0) v.x = w; else if (i == 1) v.y = w; else if (i == 2) v.z = w; else v.w = w;
 }
 
 __device__ __forceinline__ uint32_t pack2(float a, float b) {
@@ -544,7 +559,16 @@ gemm_tc_kernel(const __grid_constant__ TcFlow<NP> flow) {
           *reinterpret_cast<float4*>(s_bias + 128 * i + 4 * lane) = bv;
         }
       }
-      const bool masked = tma_out && ep.mask != nullptr;
+      // the row's mask words (one bit per column), when the producing layer left them: 16 bytes per 128 columns
+      const int64_t mrow = (int64_t)m0 + 32 * q + lane;
+      const bool use_bits = ep.mask_bits != nullptr;
+      uint4 mq0 = make_uint4(~0u, ~0u, ~0u, ~0u), mq1 = mq0;
+      if (use_bits && mrow < p.M) {
+        if (n0 < ep.mask_cols) mq0 = __ldg(reinterpret_cast<const uint4*>(ep.mask_bits + mrow * ep.ld_mask_bits + (n0 >> 5)));
+        if (kBN > 128 && n0 + 128 < ep.mask_cols)
+          mq1 = __ldg(reinterpret_cast<const uint4*>(ep.mask_bits + mrow * ep.ld_mask_bits + ((n0 + 128) >> 5)));
+      }
+      const bool masked = tma_out && ep.mask != nullptr && !use_bits;
       auto request_mask = [&](int h) {                     // the mask of columns 64 h .. 64 h + 63 of the tile, rows of this warp
         if (kMaskSlabs > 0 && lane == 0) {
           mbar_expect_tx(mask_full(2 * q + (h & 1)), kSlabBytes);
@@ -568,6 +592,7 @@ gemm_tc_kernel(const __grid_constant__ TcFlow<NP> flow) {
         const int sw = lane & 7;
         const uint32_t row_off = (uint32_t)lane * 128u;
         bool failed = false;
+        uint4 bq = make_uint4(0u, 0u, 0u, 0u);
 #pragma unroll 1
         for (int c = 0; c < kBN / 32; ++c) {
           const int nb = n0 + 32 * c;
@@ -588,6 +613,13 @@ gemm_tc_kernel(const __grid_constant__ TcFlow<NP> flow) {
           if (ep.relu) {
 #pragma unroll
             for (int j = 0; j < 32; ++j) v[j] = fmaxf(v[j], 0.f);
+          }
+          if (use_bits && nb < ep.mask_cols) {
+            uint32_t w = pick4((kBN > 128 && c >= 4) ? mq1 : mq0, c & 3);
+            if (nb + 32 > ep.mask_cols) w |= ~0u << (ep.mask_cols - nb);   // columns from mask_cols on are not masked
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+              if (!((w >> j) & 1u)) v[j] = 0.f;
           }
           if (masked && nb < ep.mask_cols) {
             // mask slab (c / 2) & 1 holds the 64 columns of this piece and its neighbour
@@ -620,12 +652,22 @@ gemm_tc_kernel(const __grid_constant__ TcFlow<NP> flow) {
               if (lane == 0) tma_store_wait_read1();       // this slab's previous contents have been read (the other may be in flight)
               __syncwarp();
             }
+            uint32_t wbits = 0;
 #pragma unroll
             for (int g = 0; g < 4; ++g) {
               uint4 o;
               o.x = pack2(v[8 * g], v[8 * g + 1]); o.y = pack2(v[8 * g + 2], v[8 * g + 3]);
               o.z = pack2(v[8 * g + 4], v[8 * g + 5]); o.w = pack2(v[8 * g + 6], v[8 * g + 7]);
               *reinterpret_cast<uint4*>(slab + row_off + ((uint32_t)((g + 4 * odd) ^ sw) << 4)) = o;
+              wbits |= (positive2(o.x) | (positive2(o.y) << 2) | (positive2(o.z) << 4) | (positive2(o.w) << 6)) << (8 * g);
+            }
+            if (ep.bits_out) {                             // the words of 128 columns leave together
+              put4(bq, c & 3, wbits);
+              if ((c & 3) == 3 || nb + 32 >= p.N) {
+                if (mrow < p.M && !*aborted)
+                  *reinterpret_cast<uint4*>(ep.bits_out + mrow * ep.ld_bits_out + ((n0 + 128 * (c >> 2)) >> 5)) = bq;
+                bq = make_uint4(0u, 0u, 0u, 0u);
+              }
             }
             if (odd || nb + 32 >= p.N || nb + 32 >= ep.lo_cols) {   // the slab is complete (or the output ends here)
               asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -681,6 +723,7 @@ gemm_tc_kernel(const __grid_constant__ TcFlow<NP> flow) {
 #pragma unroll
           for (int j = 0; j < 32; ++j) v[j] = fmaxf(v[j], 0.f);
         }
+        uint32_t dbits = 0;
 #pragma unroll
         for (int g = 0; g < 4; ++g) {
           const int n = nb + 8 * g;
@@ -702,6 +745,7 @@ gemm_tc_kernel(const __grid_constant__ TcFlow<NP> flow) {
               uint4 o;
               o.x = pack2(x[0], x[1]); o.y = pack2(x[2], x[3]); o.z = pack2(x[4], x[5]); o.w = pack2(x[6], x[7]);
               *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(ep.out_lo) + m * ep.ld_lo + n) = o;
+              dbits |= (positive2(o.x) | (positive2(o.y) << 2) | (positive2(o.z) << 4) | (positive2(o.w) << 6)) << (8 * g);
             } else {
               float4* o = reinterpret_cast<float4*>(reinterpret_cast<float*>(ep.out_lo) + (int64_t)a.z * p.split_stride + m * ep.ld_lo + n);
               o[0] = make_float4(x[0], x[1], x[2], x[3]);
@@ -713,6 +757,7 @@ gemm_tc_kernel(const __grid_constant__ TcFlow<NP> flow) {
             o[1] = make_float4(x[4], x[5], x[6], x[7]);
           }
         }
+        if (ep.bits_out && ep.lo_bf16 && nb < ep.lo_cols) ep.bits_out[m * ep.ld_bits_out + (nb >> 5)] = dbits;
       }
       }
       // the accumulator may be overwritten: this warp's reads of it are complete
@@ -910,6 +955,9 @@ static bool splits_ok(const TcJob& j) {
   return j.k_splits <= 1 || !(ep.lo_bf16 || ep.lo_cols < j.N || ep.bias || ep.relu || ep.mask);
 }
 
+static int g_flow_ctas = 0;     // 0: the rule in gemm_tc_flow
+void set_flow_ctas(int ctas) { g_flow_ctas = ctas < 0 ? 0 : ctas; }
+
 ss_status gemm_tc_flow(const TcJob* jobs, int n, int* ctrl, int max_rows, int max_ctas, cudaStream_t st) {
   if (n < 1 || n > kTcMaxFlow) return SS_ERR_SHAPE;
   bool wide = true;
@@ -965,7 +1013,7 @@ ss_status gemm_tc_flow(const TcJob* jobs, int n, int* ctrl, int max_rows, int ma
   // training: 13.9 M examples/s with a CTA on every SM, 15.6 M with 64, 15.9 M with 32, while the flows themselves
   // get slower: 55 / 63 / 81 us).  So a flow takes 64 CTAs, more only when it has more than eight tiles for each.
   int ctas = num_sms();
-  if (ctrl && max_ctas <= 0) max_ctas = total / 8 > 64 ? total / 8 : 64;
+  if (ctrl && max_ctas <= 0) max_ctas = g_flow_ctas > 0 ? g_flow_ctas : (total / 8 > 64 ? total / 8 : 64);
   if (max_ctas > 0 && max_ctas < ctas) ctas = max_ctas;
   if (pair) {
     ctas &= ~1;                                            // whole pairs
@@ -1006,6 +1054,8 @@ ss_status gemm(int M, int N, int K, const Operand& A, const Operand& B, const Ep
 extern "C" {
 
 int ss_device_error(int clear) { return ss::read_device_error(clear != 0); }
+
+void ss_mlp_set_flow_ctas(int ctas) { ss::set_flow_ctas(ctas); }
 
 ss_status ss_gemm_bf16(const void* a, int a_mn_major, int64_t lda, const void* b, int b_mn_major, int64_t ldb,
                        float* c, int64_t ldc, int M, int N, int K, int force_simt, ss_stream stream) {

@@ -424,7 +424,9 @@ constexpr int kFirstRowsMax = 32;   // most samples per block (the launch picks 
 
 __global__ void __launch_bounds__(256)
 few_inputs_layer_kernel(const float* __restrict__ x, int K, const __nv_bfloat16* __restrict__ W, const float* __restrict__ bias,
-                        int relu, int B, int N, __nv_bfloat16* __restrict__ Y, int64_t ldy, int rows_per_block) {
+                        int relu, int B, int N, __nv_bfloat16* __restrict__ Y, int64_t ldy, int rows_per_block,
+                        uint8_t* __restrict__ bits /*nullable: one bit per output "positive", rows of ld_bits bytes*/,
+                        int64_t ld_bits) {
   extern __shared__ __align__(16) __nv_bfloat16 s_w[];       // [K][N]
   __shared__ float s_x[kFirstRowsMax][kFewInputs];           // the block's samples, rounded to bf16, zero beyond K
   const int b0 = blockIdx.x * rows_per_block;
@@ -460,14 +462,19 @@ few_inputs_layer_kernel(const float* __restrict__ x, int K, const __nv_bfloat16*
     const float4 b0v = reinterpret_cast<const float4*>(bias + o)[0], b1v = reinterpret_cast<const float4*>(bias + o)[1];
     const float bv[8] = {b0v.x, b0v.y, b0v.z, b0v.w, b1v.x, b1v.y, b1v.z, b1v.w};
     uint32_t out[4];
+    uint32_t pos = 0;                                          // bit j: output o + j is positive as stored
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
       float v0 = acc[2 * j] + bv[2 * j], v1 = acc[2 * j + 1] + bv[2 * j + 1];
       if (relu) { v0 = fmaxf(v0, 0.f); v1 = fmaxf(v1, 0.f); }
       __nv_bfloat162 h = __floats2bfloat162_rn(v0, v1);
       out[j] = *reinterpret_cast<uint32_t*>(&h);
+      const uint32_t lo = out[j] & 0xFFFFu, hi = out[j] >> 16;
+      pos |= (uint32_t)((lo & 0x8000u) == 0 && (lo & 0x7FFFu) != 0) << (2 * j);
+      pos |= (uint32_t)((hi & 0x8000u) == 0 && (hi & 0x7FFFu) != 0) << (2 * j + 1);
     }
     *reinterpret_cast<uint4*>(Y + (int64_t)(b0 + r) * ldy + o) = make_uint4(out[0], out[1], out[2], out[3]);
+    if (bits) bits[(int64_t)(b0 + r) * ld_bits + (o >> 3)] = (uint8_t)pos;   // byte o / 8 of the row's little-endian words
   }
 }
 
@@ -506,6 +513,38 @@ struct FlowBuilder {
     return n++;
   }
 };
+
+// How layer l (not the last) of the forward pass is computed, and with which operands: the forward pass runs it, the
+// backward pass asks the same question to know whether the layer left the sign bits of its output (bits[l]).
+enum { FWD_FEW_INPUTS = 0, FWD_TENSOR_CORE = 1, FWD_SIMT = 2 };
+struct FwdLayer { Operand A, Bm; Epilogue ep; int how; };
+static FwdLayer describe_fwd_layer(const MlpPlan& p, int l, int B, const float* w, const void* w_bf16, const float* dense,
+                                   const float* concat_f32, const void* concat_bf16, char* ws) {
+  const LayerInfo& L = p.layer[l];
+  const int act_kind = p.bf16 ? OP_BF16 : OP_F32;
+  FwdLayer f;
+  if (l == 0) f.A = Operand{dense, p.bf16 ? OP_F32_ROUND_BF16 : OP_F32, p.n_dense, 1};
+  else if (l == p.nb) f.A = Operand{p.bf16 ? (const void*)concat_bf16 : (const void*)concat_f32, act_kind, p.W, 1};
+  else f.A = Operand{ws + p.act[l - 1], act_kind, L.in, 1};
+  f.Bm = p.bf16 ? Operand{reinterpret_cast<const __nv_bfloat16*>(w_bf16) + L.w_off, OP_BF16, L.in, 1}
+                : Operand{w + L.w_off, OP_F32, L.in, 1};
+  f.ep.bias = w + L.b_off;
+  f.ep.relu = L.relu;
+  f.ep.lo_cols = L.out;
+  if (l == p.nb - 1) {
+    f.ep.out_lo = p.bf16 ? const_cast<void*>(concat_bf16) : (void*)concat_f32; f.ep.lo_bf16 = p.bf16; f.ep.ld_lo = p.W;
+  } else {
+    f.ep.out_lo = ws + p.act[l]; f.ep.lo_bf16 = p.bf16; f.ep.ld_lo = L.out;
+  }
+  const size_t few_smem = (size_t)L.in * L.out * 2;
+  if (p.bf16 && l == 0 && L.in <= kFewInputs && few_smem <= 48 * 1024 && (f.ep.ld_lo & 7) == 0 && aligned16(f.ep.out_lo))
+    f.how = FWD_FEW_INPUTS;
+  else if (gemm_tc_eligible(B, L.out, L.in, f.A, f.Bm, f.ep))
+    f.how = FWD_TENSOR_CORE;
+  else
+    f.how = FWD_SIMT;
+  return f;
+}
 
 static ss_status check_common(const MlpPlan& p, int B, const void* concat_f32, const void* concat_bf16,
                               const void* w_bf16, void* ws, size_t ws_bytes) {
@@ -566,12 +605,10 @@ ss_status ss_mlp_fwd(const ss_mlp_desc* desc, const float* w, const void* w_bf16
 
   for (int l = 0; l < p.nl; ++l) {
     const LayerInfo& L = p.layer[l];
-    Operand A, Bm;
-    if (l == 0) A = Operand{dense, p.bf16 ? OP_F32_ROUND_BF16 : OP_F32, p.n_dense, 1};
-    else if (l == p.nb) A = Operand{p.bf16 ? (const void*)concat_bf16 : (const void*)concat_f32, act_kind, p.W, 1};
-    else A = Operand{ws + p.act[l - 1], act_kind, L.in, 1};
-    Bm = p.bf16 ? Operand{reinterpret_cast<const __nv_bfloat16*>(w_bf16) + L.w_off, OP_BF16, L.in, 1}
-                : Operand{w + L.w_off, OP_F32, L.in, 1};
+    const FwdLayer f = describe_fwd_layer(p, l, B, w, w_bf16, dense, concat_f32, concat_bf16, ws);
+    const Operand& A = f.A;
+    const Operand& Bm = f.Bm;
+    const Epilogue& ep = f.ep;
     if (l == p.nl - 1) {   // one output unit: a dot product per sample
       st = flow.flush();
       if (st != SS_OK) return st;
@@ -583,32 +620,25 @@ ss_status ss_mlp_fwd(const ss_mlp_desc* desc, const float* w, const void* w_bf16
       SS_LAUNCH_OK();
       break;
     }
-    Epilogue ep;
-    ep.bias = w + L.b_off;
-    ep.relu = L.relu;
-    ep.lo_cols = L.out;
-    if (l == p.nb - 1) {
-      ep.out_lo = p.bf16 ? concat_bf16 : (void*)concat_f32; ep.lo_bf16 = p.bf16; ep.ld_lo = p.W;
-    } else {
-      ep.out_lo = ws + p.act[l]; ep.lo_bf16 = p.bf16; ep.ld_lo = L.out;
-    }
-    const size_t few_smem = (size_t)L.in * L.out * 2;
-    if (p.bf16 && l == 0 && L.in <= kFewInputs && few_smem <= 48 * 1024 && (ep.ld_lo & 7) == 0 && aligned16(ep.out_lo)) {
+    if (f.how == FWD_FEW_INPUTS) {
       int rows = 8;                                            // every block stages the whole weight matrix
       while (rows < kFirstRowsMax && (B + rows - 1) / rows > 2 * num_sms()) rows *= 2;
       SS_TIMED("few_inputs_layer_kernel", cs);
-      few_inputs_layer_kernel<<<(B + rows - 1) / rows, 256, few_smem, cs>>>(
+      few_inputs_layer_kernel<<<(B + rows - 1) / rows, 256, (size_t)L.in * L.out * 2, cs>>>(
           dense, L.in, reinterpret_cast<const __nv_bfloat16*>(w_bf16) + L.w_off, ep.bias, ep.relu, B, L.out,
-          reinterpret_cast<__nv_bfloat16*>(ep.out_lo), ep.ld_lo, rows);
+          reinterpret_cast<__nv_bfloat16*>(ep.out_lo), ep.ld_lo, rows, reinterpret_cast<uint8_t*>(ws + p.bits[l]),
+          (int64_t)p.ld_bits[l] * 4);
       SS_LAUNCH_OK();
       continue;
     }
-    if (gemm_tc_eligible(B, L.out, L.in, A, Bm, ep)) {
+    if (f.how == FWD_TENSOR_CORE) {
       // The whole chain of tensor-core layers is ONE launch: layer l's tiles wait for the row blocks of layer l - 1
       // they read.  The first top layer reads the concat buffer, of which only the first D0 columns come from the
       // bottom MLP: it contracts the pooled embeddings first and waits for the bottom output only then.
       TcJob j;
       j.M = B; j.N = L.out; j.K = L.in; j.A = A; j.B = Bm; j.ep = ep;
+      j.ep.bits_out = reinterpret_cast<uint32_t*>(ws + p.bits[l]);   // the backward pass masks with these
+      j.ep.ld_bits_out = p.ld_bits[l];
       const int idx = flow.add(j, l - 1, 1, l == p.nb ? (p.D0 + 63) / 64 : 0);
       if (idx < 0) return (ss_status)idx;
       flow.writer[l] = idx;
@@ -712,6 +742,11 @@ ss_status ss_mlp_bwd(const ss_mlp_desc* desc, float* w, void* w_bf16, float* ada
       } else {
         ep.mask = ws + p.act[l - 1]; ep.ld_mask = L.in; ep.mask_cols = L.in;
         ep.ld_lo = L.in; ep.lo_cols = L.in;
+      }
+      // the sign bits of the producing layer's output, where its forward kernel left them
+      if (p.bf16 && describe_fwd_layer(p, l - 1, B, w, w_bf16, dense, concat_f32, concat_bf16, ws).how != FWD_SIMT) {
+        ep.mask_bits = reinterpret_cast<const uint32_t*>(ws + p.bits[l - 1]);
+        ep.ld_mask_bits = p.ld_bits[l - 1];
       }
       if (gemm_tc_eligible(B, L.in, L.out, A, Wt, ep)) {
         TcJob j;

@@ -22,6 +22,10 @@ struct MlpPlan {
   // respect to it after the ReLU mask.  The last bottom layer's output lives in the concat buffer and
   // the last top layer's in logit[], so act[] is unused for those two.
   size_t act[kMaxLayers], dact[kMaxLayers];
+  // bits[l]: one bit per element of layer l's output, "positive" (the ReLU-gradient mask of the backward pass),
+  // rows of ld_bits[l] 32-bit words (a multiple of 4); bf16 mode only
+  size_t bits[kMaxLayers];
+  int ld_bits[kMaxLayers];
   size_t grads, red_partial, gpart, loss_part, ctrl, total;   // loss_part: a ticket word, then one partial loss per 8 samples
   int ctrl_rows;          // most rows of a product that another product of a tensor-core flow may wait for
   size_t ctrl_bytes;      // control words of the tensor-core flows (directly behind the loss ticket: one memset clears both)
@@ -65,6 +69,8 @@ inline ss_status make_mlp_plan(const ss_mlp_desc* d, int B, MlpPlan* p) {
     const size_t bytes = (size_t)B * p->layer[l].out * es;
     p->act[l] = take(bytes);
     p->dact[l] = take(bytes);
+    p->ld_bits[l] = ((p->layer[l].out + 31) / 32 + 3) & ~3;
+    p->bits[l] = take(p->bf16 ? (size_t)B * p->ld_bits[l] * 4 : 0);
   }
   p->grads = take((size_t)p->P * 4);
   p->red_splits = B >= 1024 ? (B + 127) / 128 : (B >= 256 ? 8 : (B >= 64 ? 2 : 1));   // at most 128-row slices
