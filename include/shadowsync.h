@@ -10,15 +10,30 @@
  *
  * General conventions
  *   - All data pointers are DEVICE pointers into caller-owned memory unless a
- *     parameter says "host".  The library allocates nothing and keeps no state
- *     besides the last CUDA error code and cached driver entry points.
+ *     parameter says "host".  The compute calls allocate no device memory: scratch
+ *     comes from caller-provided workspaces whose sizes are queried first.
+ *   - State the library keeps: the last CUDA error code of each host thread; per
+ *     device, cached facts found on first use (compute capability, SM count, kernel
+ *     attributes such as the dynamic shared-memory limit, driver entry points, the
+ *     device addresses of its own __device__ symbols); one device-side error word
+ *     (ss_device_error); the 2112 KiB built-in scratch of ss_embbag_bwd_sort_noalloc;
+ *     the tuning value of ss_mlp_set_flow_ctas; while the kernel timers are on
+ *     (ss_profile), pools of CUDA events and their records; and, per ss_shadow_start,
+ *     a heap-allocated handle with a host thread until ss_shadow_stop.
+ *     Because of the first-use set-up, make the first call of each entry point on a
+ *     device outside any stream capture; later calls can be captured into CUDA graphs
+ *     (the timers must be off while capturing).  Calls may come from several host
+ *     threads; calls that share a workspace must be ordered by the caller.
  *   - Calls validate their arguments on the host, enqueue on `stream`
  *     (a cudaStream_t passed as void*, 0 = the legacy default stream) and
  *     return without synchronising.  Buffers must stay alive until the stream
  *     has run the work.
  *   - Return value: SS_OK or a negative ss_status.  Nothing aborts; no kernel
  *     traps.  Malformed *data* seen on the device (an index outside [0,N), a
- *     decreasing offset) ORs a bit into *d_status and that lookup is skipped.
+ *     decreasing or negative offset, an offset beyond the end of the index list
+ *     offsets[T*B]) ORs a bit into *d_status and that lookup or bag is skipped.
+ *     A bounded wait inside a tensor-core kernel that runs out raises the device
+ *     error word instead of hanging; the kernel then stores nothing more.
  *   - Row-major everywhere.  float = IEEE binary32, bf16 = bfloat16 stored as
  *     uint16_t.  "ld" = leading dimension in elements.
  *   - Pointers that are read or written with 128-bit accesses must be 16-byte
@@ -177,7 +192,13 @@ int64_t ss_mlp_param_count(const ss_mlp_desc* desc);  /* padded length of the fl
 ss_status ss_mlp_param_offsets(const ss_mlp_desc* desc, int64_t* w_off, int64_t* b_off); /* host arrays [n_bottom+n_top] */
 size_t ss_mlp_workspace_bytes(const ss_mlp_desc* desc, int B);
 
-/* Forward.  dense float [B, bottom_dims[0]]; labels float [B] in {0,1}.
+/* How the tensor-core layers run (gemm_dtype 1): all of them in ONE persistent launch per pass.  Its CTAs draw
+ * 128-row output tiles of all layers from a counter in the workspace; a tile of a layer waits, inside the launch,
+ * for the row blocks of the previous layer it reads (forward: activations; backward: the gradient above it; weight
+ * gradients, which contract over the batch, wait k block by k block).  The workspace therefore also holds the
+ * launch's control words; ss_mlp_fwd clears them, so a workspace needs no initialisation.
+ *
+ * Forward.  dense float [B, bottom_dims[0]]; labels float [B] in {0,1}.
  * concat_f32 [B, W] (gemm_dtype 0) / concat_bf16 [B, W] (gemm_dtype 1) must already hold the pooled
  * columns; the call fills columns 0..D0-1.  Outputs: logit[B], prob[B] = sigmoid(logit),
  * loss[1] = mean_b( max(z,0) - z*y + log(1+exp(-|z|)) ).  The workspace keeps the activations

@@ -48,19 +48,17 @@ __host__ __device__ constexpr int stage_bytes(int bn) { return kTileBytes + bn *
 constexpr int kEpiWarps = 4;                              // one per tensor-memory lane quadrant
 constexpr int kTcThreads = 64 + 32 * kEpiWarps;
 constexpr int kQueue = 4;                                 // tiles a CTA may have drawn and not yet finished
-// Ring depth: 4 stages of 32 KiB for 128-wide tiles, 3 stages of 48 KiB for 256-wide tiles (a quarter less
-// shared-memory traffic per flop, for products that fill the machine), 5 stages of 32 KiB for CTA pairs (which carry
-// no mask slabs); one CTA per SM in every case.
-constexpr int kStagesNarrow = 4, kStagesWide = 3, kStagesPair = 5;
+// Ring depth: 5 stages of 32 KiB for 128-wide tiles and for CTA pairs, 3 stages of 48 KiB for 256-wide tiles (a
+// quarter less shared-memory traffic per flop than 128-wide ones); one CTA per SM in every case.
+constexpr int kStagesNarrow = 5, kStagesWide = 3, kStagesPair = 5;
 constexpr int kCtlBytes = 512;                            // barriers, tile queue, tensor-memory address, abort flag
 // Per epilogue warp: two 4 KiB slabs (32 rows x 128 bytes, 128-byte swizzle) from which TMA stores pieces of the
-// output (one is filled while the other is being read), kMaskSlabs (0 or 2) slabs into which TMA loads the warp's rows
-// of the ReLU-gradient mask, 64 columns each, and the tile's bias values.
+// output (one is filled while the other is being read), and the tile's bias values.
 constexpr int kSlabBytes = 32 * 128;
 constexpr int kBiasBytes = 256 * 4;
-__host__ __device__ constexpr int epi_warp_bytes(int mask_slabs) { return (2 + mask_slabs) * kSlabBytes + kBiasBytes; }
-constexpr size_t tc_smem_bytes(int stages, int load_n, int mask_slabs, size_t meta_bytes) {
-  return (size_t)stages * stage_bytes(load_n) + kEpiWarps * epi_warp_bytes(mask_slabs) + 1024 /*alignment slack*/ + kCtlBytes + meta_bytes;
+constexpr int kEpiWarpBytes = 2 * kSlabBytes + kBiasBytes;
+constexpr size_t tc_smem_bytes(int stages, int load_n, size_t meta_bytes) {
+  return (size_t)stages * stage_bytes(load_n) + kEpiWarps * kEpiWarpBytes + 1024 /*alignment slack*/ + kCtlBytes + meta_bytes;
 }
 constexpr long long kWaitCycles = 400ll * 1000 * 1000;    // ~0.2 s: far beyond any legitimate wait
 
@@ -89,7 +87,7 @@ struct TcMeta {
 };
 struct TcProblem {
   CUtensorMap map_a, map_b;
-  CUtensorMap map_lo, map_hi, map_mask;   // out_lo (3-d for float: column, row, K slice), out_hi, mask; used when tma_out
+  CUtensorMap map_lo, map_hi;             // out_lo (3-d for float: column, row, K slice), out_hi; used when tma_out
   TcMeta meta;
 };
 template <int NP>
@@ -292,7 +290,7 @@ __device__ __forceinline__ TileAt locate_tile(const TcMeta* meta, int n, int t) 
 // both SMs read both halves) and the accumulator of its own 128 rows.  Per flop a CTA loads and reads a third less
 // shared memory than with 128 x 256 tiles of its own, which is what bounds those.  Tiles are assigned round-robin to
 // the pairs (no dependencies between products in this mode).
-template <int kStages, int kBN, int NP, bool kPair, int kMaskSlabs>
+template <int kStages, int kBN, int NP, bool kPair>
 __global__ void __launch_bounds__(kTcThreads, 1)
 gemm_tc_kernel(const __grid_constant__ TcFlow<NP> flow) {
   extern __shared__ uint8_t smem_raw[];
@@ -300,7 +298,6 @@ gemm_tc_kernel(const __grid_constant__ TcFlow<NP> flow) {
   constexpr int kTileM = kPair ? 2 * kBM : kBM;            // rows of a tile
   constexpr int kStageBytes = stage_bytes(kLoadN);
   constexpr int kTmemCols = 2 * kBN;                       // two accumulators of kBN fp32 columns
-  constexpr int kEpiWarpBytes = epi_warp_bytes(kMaskSlabs);
   const uint32_t rank = kPair ? cluster_rank() : 0u;       // 0: the CTA that issues the pair's MMAs
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t tiles = (raw + 1023u) & ~1023u;                 // 1024-byte aligned swizzle atoms
@@ -309,9 +306,8 @@ gemm_tc_kernel(const __grid_constant__ TcFlow<NP> flow) {
   uint8_t* epi_gen = gen + (size_t)kStages * kStageBytes;
   uint8_t* ctl = epi_gen + kEpiWarps * kEpiWarpBytes;
   const uint32_t bar0 = epi0 + kEpiWarps * kEpiWarpBytes;
-  // barriers: [0,S) full, [S,2S) empty, then accumulator full[2], empty[2], queue full[kQueue], empty[kQueue],
-  // mask slab full [epilogue warp][2]
-  constexpr int kNumBars = 2 * kStages + 4 + 2 * kQueue + 2 * kEpiWarps;
+  // barriers: [0,S) full, [S,2S) empty, then accumulator full[2], empty[2], queue full[kQueue], empty[kQueue]
+  constexpr int kNumBars = 2 * kStages + 4 + 2 * kQueue;
   int* tile_q = reinterpret_cast<int*>(ctl + 8 * kNumBars);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tile_q + kQueue);
   volatile int* aborted = reinterpret_cast<volatile int*>(tmem_slot + 1);
@@ -330,7 +326,6 @@ gemm_tc_kernel(const __grid_constant__ TcFlow<NP> flow) {
   auto acc_empty = [&](int b) { return bar0 + 8u * (2 * kStages + 2 + b); };
   auto q_full = [&](int s) { return bar0 + 8u * (2 * kStages + 4 + s); };
   auto q_empty = [&](int s) { return bar0 + 8u * (2 * kStages + 4 + kQueue + s); };
-  auto mask_full = [&](int w) { return bar0 + 8u * (2 * kStages + 4 + 2 * kQueue + w); };
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) {
@@ -341,7 +336,6 @@ gemm_tc_kernel(const __grid_constant__ TcFlow<NP> flow) {
     for (int s = 0; s < kStages; ++s) { mbar_init(full(s), 1); mbar_init(empty(s), 1); }
     for (int b = 0; b < 2; ++b) { mbar_init(acc_full(b), 1); mbar_init(acc_empty(b), kPair ? 2 * kEpiWarps : kEpiWarps); }
     for (int s = 0; s < kQueue; ++s) { mbar_init(q_full(s), 1); mbar_init(q_empty(s), 1 + kEpiWarps); }
-    for (int w = 0; w < 2 * kEpiWarps; ++w) mbar_init(mask_full(w), 1);
     *aborted = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -525,10 +519,9 @@ gemm_tc_kernel(const __grid_constant__ TcFlow<NP> flow) {
   } else {
     // ------------------------------------------------------------------ epilogue warps 2..5
     const int q = warp & 3;               // tensor-memory lane quadrant this warp may read
-    uint8_t* const slab_gen = epi_gen + q * kEpiWarpBytes;              // [out 0][out 1][mask 0][mask 1][bias]
-    const uint32_t slab_out = epi0 + q * kEpiWarpBytes, slab_mask = slab_out + 2 * kSlabBytes;
-    float* const s_bias = reinterpret_cast<float*>(slab_gen + (2 + kMaskSlabs) * kSlabBytes);
-    uint32_t mask_uses[2] = {0, 0};       // completed phases of this warp's two mask barriers
+    uint8_t* const slab_gen = epi_gen + q * kEpiWarpBytes;              // [out 0][out 1][bias]
+    const uint32_t slab_out = epi0 + q * kEpiWarpBytes;
+    float* const s_bias = reinterpret_cast<float*>(slab_gen + 2 * kSlabBytes);
     uint32_t n_stores = 0;                // slabs handed to TMA so far (they alternate)
     uint32_t at = 0;
     for (uint32_t qi = 0;; ++qi) {
@@ -544,12 +537,11 @@ gemm_tc_kernel(const __grid_constant__ TcFlow<NP> flow) {
                                                                  meta[a.j].p.split_stride};
       const int m0 = a.y * kTileM + (int)rank * kBM, n0 = a.x * kBN;
       const int buf = at & 1;
-      const bool tma_out = meta[a.j].p.tma_out != 0 && (kMaskSlabs > 0 || ep.mask == nullptr);
+      const bool tma_out = meta[a.j].p.tma_out != 0;
       const TcProblem& pr = flow.prob[a.j];
       // Everything the epilogue needs from memory is requested as soon as the tile is known, so that it arrives while
       // the tensor cores still work on the tile: the tile's bias values (every thread needs all of them: one 16-byte
-      // load per lane into the warp's shared memory), and this warp's rows of the mask (the producing layer's bf16
-      // activation), 64 columns per slab.
+      // load per lane into the warp's shared memory) and the thread's words of the ReLU-gradient mask.
       if (ep.bias) {
 #pragma unroll
         for (int i = 0; i < kBN / 128; ++i) {
@@ -568,18 +560,6 @@ gemm_tc_kernel(const __grid_constant__ TcFlow<NP> flow) {
         if (kBN > 128 && n0 + 128 < ep.mask_cols)
           mq1 = __ldg(reinterpret_cast<const uint4*>(ep.mask_bits + mrow * ep.ld_mask_bits + ((n0 + 128) >> 5)));
       }
-      const bool masked = tma_out && ep.mask != nullptr && !use_bits;
-      auto request_mask = [&](int h) {                     // the mask of columns 64 h .. 64 h + 63 of the tile, rows of this warp
-        if (kMaskSlabs > 0 && lane == 0) {
-          mbar_expect_tx(mask_full(2 * q + (h & 1)), kSlabBytes);
-          tma_load_2d(slab_mask + (h & 1) * kSlabBytes, &pr.map_mask, mask_full(2 * q + (h & 1)), n0 + 64 * h, m0 + 32 * q);
-        }
-      };
-      if (masked) {
-#pragma unroll
-        for (int h = 0; h < 2; ++h)
-          if (n0 + 64 * h < ep.mask_cols && n0 + 64 * h < p.N) request_mask(h);
-      }
       __syncwarp();                                        // the bias values are in shared memory
       if (!mbar_wait(acc_full(buf), (at >> 1) & 1, aborted, flow.err, 3)) break;
       if (threadIdx.x == 64) SS_TC_TRACE(7, t);
@@ -591,7 +571,6 @@ gemm_tc_kernel(const __grid_constant__ TcFlow<NP> flow) {
         // output (two pieces) or 32 columns of float output.
         const int sw = lane & 7;
         const uint32_t row_off = (uint32_t)lane * 128u;
-        bool failed = false;
         uint4 bq = make_uint4(0u, 0u, 0u, 0u);
 #pragma unroll 1
         for (int c = 0; c < kBN / 32; ++c) {
@@ -614,36 +593,12 @@ gemm_tc_kernel(const __grid_constant__ TcFlow<NP> flow) {
 #pragma unroll
             for (int j = 0; j < 32; ++j) v[j] = fmaxf(v[j], 0.f);
           }
-          if (use_bits && nb < ep.mask_cols) {
+          if (use_bits && nb < ep.mask_cols) {               // (a tile with a mask takes this path only with mask words)
             uint32_t w = pick4((kBN > 128 && c >= 4) ? mq1 : mq0, c & 3);
             if (nb + 32 > ep.mask_cols) w |= ~0u << (ep.mask_cols - nb);   // columns from mask_cols on are not masked
 #pragma unroll
             for (int j = 0; j < 32; ++j)
               if (!((w >> j) & 1u)) v[j] = 0.f;
-          }
-          if (masked && nb < ep.mask_cols) {
-            // mask slab (c / 2) & 1 holds the 64 columns of this piece and its neighbour
-            const int h = c >> 1, ms = h & 1;
-            if (!odd && !mbar_wait(mask_full(2 * q + ms), (mask_uses[ms]++) & 1, aborted, flow.err, 9)) { failed = true; break; }
-#pragma unroll
-            for (int g = 0; g < 4; ++g) {
-              if (nb + 8 * g >= ep.mask_cols) break;
-              const uint4 mk = *reinterpret_cast<const uint4*>(slab_gen + (2 + ms) * kSlabBytes + row_off + ((uint32_t)((g + 4 * odd) ^ sw) << 4));
-              const uint32_t w[4] = {mk.x, mk.y, mk.z, mk.w};
-#pragma unroll
-              for (int j = 0; j < 4; ++j) {
-                // a bf16 is positive iff its sign bit is clear and it is not zero
-                const uint32_t lo = w[j] & 0xFFFFu, hi = w[j] >> 16;
-                if (!((lo & 0x8000u) == 0 && (lo & 0x7FFFu) != 0)) v[8 * g + 2 * j] = 0.f;
-                if (!((hi & 0x8000u) == 0 && (hi & 0x7FFFu) != 0)) v[8 * g + 2 * j + 1] = 0.f;
-              }
-            }
-            // the slab's 64 columns are used up: it takes the 64 columns after the other slab's (256-wide tiles)
-            const bool last_of_slab = odd || nb + 32 >= p.N || nb + 32 >= ep.mask_cols;
-            if (kBN > 128 && last_of_slab && h + 2 < kBN / 64 && n0 + 64 * (h + 2) < ep.mask_cols && n0 + 64 * (h + 2) < p.N) {
-              __syncwarp();                                // every lane has read the slab
-              request_mask(h + 2);
-            }
           }
           const bool to_lo = nb < ep.lo_cols;
           if (to_lo && ep.lo_bf16) {
@@ -696,7 +651,6 @@ gemm_tc_kernel(const __grid_constant__ TcFlow<NP> flow) {
             ++n_stores;
           }
         }
-        if (failed) break;
       } else {
       // tcgen05.ld hands a thread one accumulator row, 32 consecutive columns at a time: the thread applies the
       // epilogue to its row and stores 16-byte pieces of it (whole 32-byte sectors per pair of stores).
@@ -783,9 +737,6 @@ gemm_tc_kernel(const __grid_constant__ TcFlow<NP> flow) {
       ++at;
     }
     if (lane == 0) tma_store_wait_all();                   // the slabs are read before the CTA gives up its shared memory
-    if (*aborted) {
-      for (int i = 0; i < 64; ++i) __nanosleep(1000);      // mask slabs still on their way land in this CTA's memory
-    }
   }
 
   tc_fence_before();
@@ -869,14 +820,14 @@ bool gemm_tc_eligible(int M, int N, int K, const Operand& A, const Operand& B, c
   return true;
 }
 
-template <int kStages, int kBN, bool kPair, int kMaskSlabs>
+template <int kStages, int kBN, bool kPair>
 static ss_status launch_flow(const TcFlow<kTcMaxFlow>& f, int ctas, cudaStream_t st) {
   static bool attr_set[64];
   int dev = 0;
   SS_CUDA(cudaGetDevice(&dev));
-  const size_t smem = tc_smem_bytes(kStages, kPair ? kBN / 2 : kBN, kMaskSlabs, sizeof(TcMeta) * kTcMaxFlow);
+  const size_t smem = tc_smem_bytes(kStages, kPair ? kBN / 2 : kBN, sizeof(TcMeta) * kTcMaxFlow);
   if (dev >= 0 && dev < 64 && !attr_set[dev]) {
-    SS_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<kStages, kBN, kTcMaxFlow, kPair, kMaskSlabs>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    SS_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<kStages, kBN, kTcMaxFlow, kPair>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  (int)smem));
     attr_set[dev] = true;
   }
@@ -892,9 +843,9 @@ static ss_status launch_flow(const TcFlow<kTcMaxFlow>& f, int ctas, cudaStream_t
     attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    SS_CUDA(cudaLaunchKernelEx(&cfg, gemm_tc_kernel<kStages, kBN, kTcMaxFlow, kPair, kMaskSlabs>, f));
+    SS_CUDA(cudaLaunchKernelEx(&cfg, gemm_tc_kernel<kStages, kBN, kTcMaxFlow, kPair>, f));
   } else {
-    gemm_tc_kernel<kStages, kBN, kTcMaxFlow, kPair, kMaskSlabs><<<ctas, kTcThreads, smem, st>>>(f);
+    gemm_tc_kernel<kStages, kBN, kTcMaxFlow, kPair><<<ctas, kTcThreads, smem, st>>>(f);
   }
   }
   SS_LAUNCH_OK();
@@ -922,8 +873,9 @@ static int fill_problem(TcProblem* pr, const TcJob& j, int bn, int tile_begin, i
   // Outputs through TMA stores: every 64-column piece of a tile lies on one side of the lo / hi boundary.
   const Epilogue& ep = j.ep;
   p.tma_out = 0;
-  pr->map_lo = pr->map_a; pr->map_hi = pr->map_a; pr->map_mask = pr->map_a;   // defined, unused unless tma_out
-  if (ep.out_lo && ep.lo_cols > 0 && ((ep.lo_cols & 63) == 0 || ep.lo_cols >= j.N) && (!ep.mask || ep.mask_bf16)) {
+  pr->map_lo = pr->map_a; pr->map_hi = pr->map_a;   // defined, unused unless tma_out
+  // (a mask must come as sign bits; a mask given by values only takes the epilogue with plain loads and stores)
+  if (ep.out_lo && ep.lo_cols > 0 && ((ep.lo_cols & 63) == 0 || ep.lo_cols >= j.N) && (!ep.mask || ep.mask_bits)) {
     bool ok = true;
     if (ep.lo_bf16) {
       ok = make_map_any(&pr->map_lo, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, ep.out_lo, ep.lo_cols < j.N ? ep.lo_cols : j.N, j.M,
@@ -935,9 +887,6 @@ static int fill_problem(TcProblem* pr, const TcJob& j, int bn, int tile_begin, i
     }
     if (ok && ep.lo_cols < j.N)
       ok = ep.out_hi && make_map_any(&pr->map_hi, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, ep.out_hi, j.N - ep.lo_cols, j.M, ep.ld_hi, 32, 32);
-    if (ok && ep.mask)
-      ok = make_map_any(&pr->map_mask, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, ep.mask, ep.mask_cols < j.N ? ep.mask_cols : j.N, j.M,
-                        ep.ld_mask, 64, 32);
     p.tma_out = ok ? 1 : 0;
   }
   pr->meta.tile_begin = tile_begin;
@@ -1018,11 +967,11 @@ ss_status gemm_tc_flow(const TcJob* jobs, int n, int* ctrl, int max_rows, int ma
   if (pair) {
     ctas &= ~1;                                            // whole pairs
     if (2 * total < ctas) ctas = 2 * total;
-    return launch_flow<kStagesPair, 256, true, 0>(f, ctas, st);
+    return launch_flow<kStagesPair, 256, true>(f, ctas, st);
   }
   if (total < ctas) ctas = total;
-  if (wide) return launch_flow<kStagesWide, 256, false, 2>(f, ctas, st);
-  return launch_flow<kStagesNarrow, 128, false, 2>(f, ctas, st);
+  if (wide) return launch_flow<kStagesWide, 256, false>(f, ctas, st);
+  return launch_flow<kStagesNarrow, 128, false>(f, ctas, st);
 }
 
 ss_status gemm_tc(int M, int N, int K, const Operand& A, const Operand& B, const Epilogue& ep, cudaStream_t st,

@@ -28,7 +28,13 @@ def assert_close(got, want, rtol, what="", floor=0.0):
                              f"got {got[i]!r} want {want[i]!r} (scale {scale[i]:.3e})")
 
 
-GATE_DELTA = 2.0 ** -8   # one bfloat16 ulp, relative to the RMS pre-activation of the layer
+# How close to zero, relative to the RMS pre-activation of its layer, a hidden unit must be for its ReLU gate to
+# count as "at the edge".  Both sides feed the unit the same bf16 weights, but an input activation whose float value
+# lies within float rounding of a bf16 rounding boundary may come out one bf16 ulp apart (2^-8 of that input) on the
+# two sides; one such input moves the pre-activation by |a_k w_k| 2^-8, about rms(z) 2^-8 / sqrt(K) for a layer of K
+# inputs, and a unit has a handful of them at most.  Observed distances of switched units: up to 1.0e-3 rms (large
+# model, 3456 inputs); the limit is twice that, half a bf16 ulp.
+GATE_DELTA = 2.0 ** -9
 
 
 def match_relu_gates(fwd, backward, got_grad_pooled, rtol, n_bottom, n_layers, delta=GATE_DELTA, max_flips=3):
@@ -40,9 +46,10 @@ def match_relu_gates(fwd, backward, got_grad_pooled, rtol, n_bottom, n_layers, d
     discrete decision is compared in the kernel's precision, the oracle follows the kernel there: for each
     sample whose grad_pooled row misses the tolerance, units with |pre| < delta * rms(pre of the layer) are
     switched, greedily, while that brings the row closer; no other unit may change.  The sample must then
-    match, which the caller checks with the strict tolerance on every output of the step.  grad_pooled
-    sees the gates of the top MLP only; a bottom-MLP unit at the edge is not searched for and would show
-    up as a failure of the caller's strict comparison of that layer's weight step.
+    match, which the caller checks with the strict tolerance on every output of the step.  Only gates of
+    the top MLP are ever switched (grad_pooled, the evidence used here, sees no others): a bottom-MLP gate
+    decided differently by the two sides is NOT explained away and fails the caller's strict comparison of
+    that layer's weight and bias steps.
 
     fwd: the oracle's forward dict (not modified); backward(fwd) -> grad_pooled [B, C] float64.
     Returns (fwd with the switched pre-activations, list of (sample, layer, unit)).
