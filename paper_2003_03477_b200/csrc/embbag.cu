@@ -35,45 +35,48 @@ __device__ __forceinline__ uint2 bf16x4(float4 v) {
 }
 
 // G lanes per bag (power of two <= 32); NV float4 slices per lane (NV*G*4 >= D).
+// Grid: x over the samples of a table (256 / G bags per block), y = table: no division finds (t, b), and all
+// addressing inside a table is 32-bit (N * D / 4 < 2^32 is checked by the host).
 template <int G, int NV>
 __global__ void __launch_bounds__(256)
-embbag_fwd_kernel(const float* __restrict__ tables, int T, int64_t N, int D,
+embbag_fwd_kernel(const float* __restrict__ tables, int T, uint32_t N, int D,
                   const int32_t* __restrict__ indices, const int32_t* __restrict__ offsets, int B,
                   float* __restrict__ out_f32, int64_t ld_f32,
                   __nv_bfloat16* __restrict__ out_bf16, int64_t ld_bf16, int col0,
                   int32_t* __restrict__ d_status) {
-  const int64_t bag = (int64_t)blockIdx.x * (256 / G) + threadIdx.x / G;
+  const int b = blockIdx.x * (256 / G) + threadIdx.x / G;
   const int lane = threadIdx.x % G;
-  if (bag >= (int64_t)T * B) return;
-  const int t = (int)(bag / B);
-  const int b = (int)(bag - (int64_t)t * B);
-  int lo = offsets[bag], hi = offsets[bag + 1];
+  const int t = blockIdx.y;
+  if (b >= B) return;
+  const int32_t* off = offsets + (int64_t)t * B + b;
+  int lo = off[0], hi = off[1];
   // the index list ends where the last bag ends; a bag that is not inside [0, L] in ascending order is treated as empty
   const int L = __ldg(offsets + (int64_t)T * B);
   int bad = 0;
   if (lo < 0 || hi < lo || hi > L) { bad |= SS_DEV_BAD_OFFSET; lo = hi = 0; }
+  const uint32_t nvec = (uint32_t)D >> 2;
   const float4* tab = reinterpret_cast<const float4*>(tables + (int64_t)t * N * D);
-  const int nvec = D >> 2;
 
   float4 acc[NV];
 #pragma unroll
   for (int v = 0; v < NV; ++v) acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
 
-  // kRows lookups per round: their indices are loaded first, then their rows
+  // kRows lookups per round: their indices are loaded first, then their rows; a lookup beyond the bag's end or with
+  // an index outside the table reads nothing and adds zeros
   constexpr int kRows = NV >= 2 ? 2 : 4;
   for (int j = lo; j < hi; j += kRows) {
-    int idx[kRows];
+    uint32_t idx[kRows];
 #pragma unroll
-    for (int u = 0; u < kRows; ++u) idx[u] = (j + u < hi) ? indices[j + u] : 0;
+    for (int u = 0; u < kRows; ++u) idx[u] = (j + u < hi) ? (uint32_t)indices[j + u] : 0xffffffffu;
     float4 rowv[kRows][NV];
 #pragma unroll
     for (int u = 0; u < kRows; ++u) {
-      const bool ok = (j + u < hi) && (idx[u] >= 0) && (idx[u] < N);
-      if (j + u < hi && !ok) bad |= SS_DEV_BAD_INDEX;
+      const bool ok = idx[u] < N;                            // one unsigned compare: negative indices are huge
+      if (!ok && j + u < hi) bad |= SS_DEV_BAD_INDEX;
 #pragma unroll
       for (int v = 0; v < NV; ++v) {
-        const int c = lane + v * G;
-        rowv[u][v] = (ok && c < nvec) ? tab[(int64_t)idx[u] * nvec + c] : make_float4(0.f, 0.f, 0.f, 0.f);
+        const uint32_t c = lane + v * G;
+        rowv[u][v] = (ok && c < nvec) ? __ldg(tab + (idx[u] * nvec + c)) : make_float4(0.f, 0.f, 0.f, 0.f);
       }
     }
 #pragma unroll
@@ -85,7 +88,7 @@ embbag_fwd_kernel(const float* __restrict__ tables, int T, int64_t N, int D,
 #pragma unroll
   for (int v = 0; v < NV; ++v) {
     const int c = lane + v * G;
-    if (c < nvec) {
+    if (c < (int)nvec) {
       const int64_t col = (int64_t)col0 + (int64_t)t * D + 4 * c;
       if (out_f32) *reinterpret_cast<float4*>(out_f32 + (int64_t)b * ld_f32 + col) = acc[v];
       if (out_bf16) *reinterpret_cast<uint2*>(out_bf16 + (int64_t)b * ld_bf16 + col) = bf16x4(acc[v]);
@@ -101,11 +104,10 @@ static void launch_fwd(const float* tables, int T, int64_t N, int D, const int32
   // rows of 65..128 floats: two float4 per lane and 16 lanes per bag (measured faster than 32 lanes with one each;
   // for narrower rows the single-float4 form is the faster one)
   constexpr int FG = (NV == 1 && G == 32) ? 16 : G, FNV = (NV == 1 && G == 32) ? 2 : NV;
-  const int64_t bags = (int64_t)T * B;
   const int per_block = 256 / FG;
-  const unsigned blocks = (unsigned)((bags + per_block - 1) / per_block);
+  const dim3 blocks((unsigned)((B + per_block - 1) / per_block), (unsigned)T);
   { SS_TIMED("embbag_fwd_kernel", st);
-  embbag_fwd_kernel<FG, FNV><<<blocks, 256, 0, st>>>(tables, T, N, D, indices, offsets, B, out_f32, ld_f32,
+  embbag_fwd_kernel<FG, FNV><<<blocks, 256, 0, st>>>(tables, T, (uint32_t)N, D, indices, offsets, B, out_f32, ld_f32,
                                                       out_bf16, ld_bf16, col0, d_status);
   }
 }
@@ -1282,7 +1284,7 @@ ss_status ss_embbag_fwd(const float* tables, int T, int64_t N, int D, const int3
   if (!tables || !indices || !offsets) return SS_ERR_NULL;
   if (!out_f32 && !out_bf16) return SS_ERR_NULL;
   if (T < 0 || B < 0 || N <= 0 || D <= 0 || D > 1024 || (D & 3) || col0 < 0) return SS_ERR_SHAPE;
-  if ((uint64_t)T * (uint64_t)N >= (1ull << 31)) return SS_ERR_SHAPE;
+  if ((uint64_t)T * (uint64_t)N >= (1ull << 31) || T > 65535 || (uint64_t)N * (uint64_t)(D / 4) >= (1ull << 32)) return SS_ERR_SHAPE;
   if (!ss::aligned16(tables) || (col0 & 3)) return SS_ERR_ALIGN;
   if (out_f32 && (!ss::aligned16(out_f32) || (ld_f32 & 3) || ld_f32 < col0 + (int64_t)T * D)) return SS_ERR_ALIGN;
   if (out_bf16 && ((reinterpret_cast<uintptr_t>(out_bf16) & 7u) || (ld_bf16 & 3) || ld_bf16 < col0 + (int64_t)T * D))
