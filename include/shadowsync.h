@@ -300,11 +300,12 @@ ss_status ss_gemm_bf16(const void* a, int a_mn_major, int64_t lda, const void* b
 int ss_device_error(int clear);
 
 /* Tuning knob, no counterpart in the paper: how many CTAs (SMs) the persistent tensor-core launch of ss_mlp_fwd /
- * ss_mlp_bwd takes.  0 (the default) lets the library choose: 64, more for passes with more than 512 tiles.  A pass
- * alone on the device is fastest with one CTA on every SM; several replicas training concurrently get more
- * throughput with fewer, because CTAs that wait for one another hold registers and shared memory meanwhile.
+ * ss_mlp_bwd takes.  0 (the default) means 32, the value with which several replicas training concurrently on one device
+ * got the most examples per second (CTAs of such a launch hold a whole SM's shared memory and wait for one another).
+ * A pass that has the device to itself is fastest with one CTA on every SM (pass the SM count).
+ * A negative value changes nothing.  Returns the number now in effect (32 while the default stands).
  * Process-wide; set it before the calls it should affect (a captured CUDA graph keeps the value it was captured with). */
-void ss_mlp_set_flow_ctas(int ctas);
+int ss_mlp_set_flow_ctas(int ctas);
 
 /* float -> bf16 (round to nearest even) of n elements; used to initialise a bf16 mirror. */
 ss_status ss_to_bf16(const float* src, void* dst_bf16, int64_t n, ss_stream stream);

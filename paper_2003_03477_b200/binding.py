@@ -92,7 +92,7 @@ def lib() -> C.CDLL:
         L.ss_gemm_bf16.argtypes = [vp, i32, i64, vp, i32, i64, vp, i64, i32, i32, i32, i32, vp]
         L.ss_device_error.argtypes = [i32]
         L.ss_mlp_set_flow_ctas.argtypes = [i32]
-        L.ss_mlp_set_flow_ctas.restype = None
+        L.ss_mlp_set_flow_ctas.restype = i32
         L.ss_profile.argtypes = [i32]
         L.ss_profile_collect.argtypes = [C.c_char_p, sz, C.POINTER(f32), i32]
         L.ssh_fill_uniform.argtypes = [vp, i64, C.c_uint64, C.c_uint64, f32, f32, vp]
@@ -266,9 +266,10 @@ def ss_gemm_bf16(a, a_mn_major, lda, b, b_mn_major, ldb, c, ldc, M, N, K, force_
                                                ldc, M, N, K, int(force_simt), _stream(stream)))
 
 
-def ss_mlp_set_flow_ctas(ctas: int) -> None:
-    """CTAs the persistent tensor-core launches of the MLP take (0 = the library's rule)."""
-    lib().ss_mlp_set_flow_ctas(int(ctas))
+def ss_mlp_set_flow_ctas(ctas: int) -> int:
+    """CTAs the persistent tensor-core launches of the MLP take (0 = the library's default, negative = leave as it
+    is); returns the number now in effect."""
+    return int(lib().ss_mlp_set_flow_ctas(int(ctas)))
 
 
 def ss_device_error(clear: bool = True) -> int:

@@ -80,8 +80,9 @@ inline size_t tc_flow_ctrl_ints(int max_rows) { return 2 + (size_t)kTcMaxFlow * 
 // ctrl == nullptr: tiles are assigned round-robin instead (only for flows without dependencies).
 // max_ctas <= 0: one CTA per SM at most.
 ss_status gemm_tc_flow(const TcJob* jobs, int n, int* ctrl, int max_rows, int max_ctas, cudaStream_t st);
-// CTAs a flow with dependencies takes when the caller gives no number (0: the built-in rule).
-void set_flow_ctas(int ctas);
+// CTAs a flow with dependencies takes when the caller gives no number (0: the built-in default, negative: no
+// change); returns the number now in effect.
+int set_flow_ctas(int ctas);
 // Tensor cores when eligible, SIMT otherwise.
 ss_status gemm(int M, int N, int K, const Operand& A, const Operand& B, const Epilogue& ep, cudaStream_t st);
 // The device error flag raised by a bounded wait that ran out (0 = none); synchronises the device.

@@ -290,8 +290,10 @@ __device__ __forceinline__ TileAt locate_tile(const TcMeta* meta, int n, int t) 
 // both SMs read both halves) and the accumulator of its own 128 rows.  Per flop a CTA loads and reads a third less
 // shared memory than with 128 x 256 tiles of its own, which is what bounds those.  Tiles are assigned round-robin to
 // the pairs (no dependencies between products in this mode).
+// 112 registers a thread (the epilogue would take 144; capped, it recomputes a few addresses and spills nothing): a
+// CTA of this kernel sits beside the blocks of other streams' kernels, which get the registers it leaves.
 template <int kStages, int kBN, int NP, bool kPair>
-__global__ void __launch_bounds__(kTcThreads, 1)
+__global__ void __maxnreg__(112)
 gemm_tc_kernel(const __grid_constant__ TcFlow<NP> flow) {
   extern __shared__ uint8_t smem_raw[];
   constexpr int kLoadN = kPair ? kBN / 2 : kBN;            // columns of B this CTA loads
@@ -904,12 +906,15 @@ static bool splits_ok(const TcJob& j) {
   return j.k_splits <= 1 || !(ep.lo_bf16 || ep.lo_cols < j.N || ep.bias || ep.relu || ep.mask);
 }
 
-static int g_flow_ctas = 0;     // 0: the rule in gemm_tc_flow
-void set_flow_ctas(int ctas) { g_flow_ctas = ctas < 0 ? 0 : ctas; }
+constexpr int kFlowCtasDefault = 32;
+static int g_flow_ctas = 0;     // 0: kFlowCtasDefault
+int set_flow_ctas(int ctas) {
+  if (ctas >= 0) g_flow_ctas = ctas;
+  return g_flow_ctas > 0 ? g_flow_ctas : kFlowCtasDefault;
+}
 
 ss_status gemm_tc_flow(const TcJob* jobs, int n, int* ctrl, int max_rows, int max_ctas, cudaStream_t st) {
   if (n < 1 || n > kTcMaxFlow) return SS_ERR_SHAPE;
-  bool wide = true;
   double flops = 0.0;
   for (int i = 0; i < n; ++i) {
     const TcJob& j = jobs[i];
@@ -917,24 +922,22 @@ ss_status gemm_tc_flow(const TcJob* jobs, int n, int* ctrl, int max_rows, int ma
     if (j.dep >= i || (j.dep >= 0 && (!ctrl || j.dep_mode < 1 || j.dep_mode > 2 || jobs[j.dep].k_splits > 1))) return SS_ERR_SHAPE;
     if (j.dep >= 0 && jobs[j.dep].M > max_rows) return SS_ERR_SHAPE;
     flops += 2.0 * j.M * j.N * j.K;
-    if (j.N < 256) wide = false;
   }
   int* err = device_error_ptr();
   if (!err) return SS_ERR_CUDA;
-  // 128 x 256 tiles where every product is at least that wide and the flow fills the SMs with them; 256 x 256 tiles on
-  // CTA pairs where, in addition, no product waits for another (tiles then go round-robin) and there is no K slicing
+  // 128 x 256 tiles where the flow fills the SMs with them (a narrower product then has one partly empty tile per row
+  // block); 256 x 256 tiles on CTA pairs where, in addition, every product is at least that wide, no product waits for
+  // another (tiles then go round-robin) and there is no K slicing
   long long t256 = 0, t_pair = 0;
-  bool pair = wide && ctrl == nullptr;
-  if (wide) {
-    for (int i = 0; i < n; ++i) {
-      const long long ks = jobs[i].k_splits < 1 ? 1 : jobs[i].k_splits;
-      t256 += (long long)((jobs[i].N + 255) / 256) * ((jobs[i].M + kBM - 1) / kBM) * ks;
-      t_pair += (long long)((jobs[i].N + 255) / 256) * ((jobs[i].M + 2 * kBM - 1) / (2 * kBM));
-      if (ks > 1 || jobs[i].dep >= 0) pair = false;
-    }
-    wide = t256 >= num_sms();
-    pair = pair && t_pair >= num_sms() / 2;
+  bool pair = ctrl == nullptr;
+  for (int i = 0; i < n; ++i) {
+    const long long ks = jobs[i].k_splits < 1 ? 1 : jobs[i].k_splits;
+    t256 += (long long)((jobs[i].N + 255) / 256) * ((jobs[i].M + kBM - 1) / kBM) * ks;
+    t_pair += (long long)((jobs[i].N + 255) / 256) * ((jobs[i].M + 2 * kBM - 1) / (2 * kBM));
+    if (ks > 1 || jobs[i].dep >= 0 || jobs[i].N < 256) pair = false;
   }
+  const bool wide = t256 >= num_sms();
+  pair = pair && wide && t_pair >= num_sms() / 2;
   const int bn = wide ? 256 : 128;
   alignas(64) TcFlow<kTcMaxFlow> f;
   f.n = n;
@@ -957,12 +960,14 @@ ss_status gemm_tc_flow(const TcJob* jobs, int n, int* ctrl, int max_rows, int ma
   f.ctrl = ctrl;
   f.rb_stride = (max_rows + kBM - 1) / kBM + 1;    // per product: one word per row block, then their total
   f.err = err;
-  // A flow with dependencies keeps CTAs waiting for one another, and a waiting CTA still holds its SM's shared
-  // memory and a third of its registers, which the other streams' kernels then lack (measured with four replicas
-  // training: 13.9 M examples/s with a CTA on every SM, 15.6 M with 64, 15.9 M with 32, while the flows themselves
-  // get slower: 55 / 63 / 81 us).  So a flow takes 64 CTAs, more only when it has more than eight tiles for each.
+  // A flow with dependencies keeps CTAs waiting for one another, and a CTA, waiting or not, holds its SM's shared
+  // memory and a third of its registers, which the other streams' kernels then lack.  Measured with all replicas of
+  // a model training at once (examples/s at 16 / 32 / 64 / 148 CTAs per flow): four replicas, batch 2048: 15.0 /
+  // 16.0 / 15.2 / 13.4 M; eight replicas, batch 1024: 13.1 / 13.6 / 12.6 / 11.8 M; sixteen replicas of a model ten
+  // times as large, batch 4096: 7.9 / 8.4 / 7.0 / 7.2 M -- while a flow alone on the device is fastest with a CTA on
+  // every SM.  So a flow takes 32 CTAs unless the caller says otherwise (set_flow_ctas).
   int ctas = num_sms();
-  if (ctrl && max_ctas <= 0) max_ctas = g_flow_ctas > 0 ? g_flow_ctas : (total / 8 > 64 ? total / 8 : 64);
+  if (ctrl && max_ctas <= 0) max_ctas = g_flow_ctas > 0 ? g_flow_ctas : kFlowCtasDefault;
   if (max_ctas > 0 && max_ctas < ctas) ctas = max_ctas;
   if (pair) {
     ctas &= ~1;                                            // whole pairs
@@ -1004,7 +1009,7 @@ extern "C" {
 
 int ss_device_error(int clear) { return ss::read_device_error(clear != 0); }
 
-void ss_mlp_set_flow_ctas(int ctas) { ss::set_flow_ctas(ctas); }
+int ss_mlp_set_flow_ctas(int ctas) { return ss::set_flow_ctas(ctas); }
 
 ss_status ss_gemm_bf16(const void* a, int a_mn_major, int64_t lda, const void* b, int b_mn_major, int64_t ldb,
                        float* c, int64_t ldc, int M, int N, int K, int force_simt, ss_stream stream) {

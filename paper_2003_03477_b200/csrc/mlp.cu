@@ -495,7 +495,7 @@ struct FlowBuilder {
   // launches what has been collected; everything it writes is complete for whatever follows on the stream
   ss_status flush() {
     if (n == 0) return SS_OK;
-    const ss_status r = gemm_tc_flow(jobs, n, ctrl, max_rows, 0, st);
+    const ss_status r = gemm_tc_flow(jobs, n, (n == 1 && jobs[0].dep < 0) ? nullptr : ctrl, max_rows, 0, st);
     n = 0;
     for (int l = 0; l < kMaxLayers; ++l) writer[l] = -1;
     return r;
