@@ -47,6 +47,7 @@ NCU_TRAFFIC = {
     "embbag_fwd_kernel": {"workload": "medium", "bytes_per_launch": 60736000, "launches_captured": 1,
         "sources": {"embbag.cu": "393cd1570c3d6da7696206835332eaba25901bf2e8746b9382dd3c7f5e5936cf"}},
     "gemm_tc_kernel": {"workload": "medium", "bytes_per_launch": 13705472, "launches_captured": 2,
+        "tensor_pipe_active_pct": {"forward flow": 19.8, "backward flow": 26.4},   # of peak, on the SMs it runs on
         "sources": {"gemm_tc.cu": "2d1ecbac35f61b388416934a76b517173601967a524e486633ac8a09f8da6f9b", "gemm.cuh": "4d6c8c9e6e5d6074538581dc140b390c97ecf03d2981f64d8c6141a64a63af34", "mlp.cu": "b822041d4f8cd57822dcb356f9b6c1cc6c848a25a244fe4ae0e58143ebfa5b2a", "mlp_plan.cuh": "5f73399683bba8691505ec8d1e6cbb83fe39a5e25044ee8f2a9823f698f03d9a"}},
     "window_apply_kernel": {"workload": "medium", "bytes_per_launch": 123754240, "launches_captured": 1,
         "sources": {"embbag.cu": "393cd1570c3d6da7696206835332eaba25901bf2e8746b9382dd3c7f5e5936cf"}},
@@ -55,9 +56,9 @@ NCU_TRAFFIC = {
 }
 
 
-def ncu_traffic(kernel, workload):
-    """Bytes per launch from the stored ncu capture, or None when it does not cover this kernel, this workload
-    or the current sources."""
+def ncu_traffic(kernel, workload, field="bytes_per_launch"):
+    """Bytes per launch (or another field) from the stored ncu capture, or None when it does not cover this
+    kernel, this workload or the current sources."""
     import hashlib
     e = NCU_TRAFFIC.get(kernel)
     if e is None or e["workload"] != workload:
@@ -70,7 +71,7 @@ def ncu_traffic(kernel, workload):
                     return None
         except OSError:
             return None
-    return e["bytes_per_launch"]
+    return e.get(field)
 
 
 def measured_peaks():
@@ -785,7 +786,8 @@ def roofline(kernels, model, host, cfg, peaks):
         from paper_2003_03477_b200 import binding as ss
         sms = torch.cuda.get_device_properties(model.center.device).multi_processor_count
         ctas = min(ss.ss_mlp_set_flow_ctas(-1), sms)
-        extra = {"ctas_per_launch": ctas, "sms": sms, "frac_of_the_peak_of_the_sms_it_takes": achieved / peak * sms / ctas}
+        extra = {"ctas_per_launch": ctas, "sms": sms, "frac_of_the_peak_of_the_sms_it_takes": achieved / peak * sms / ctas,
+                 "tensor_pipe_active_pct_ncu": ncu_traffic(name, cfg.name, "tensor_pipe_active_pct")}
     return {"kernel": name, "bound": bound, "achieved": achieved, "peak": peak, "unit": unit, "frac": achieved / peak,
             **extra, "traffic": ncu_traffic(name, cfg.name), "traffic_unit": "bytes per launch (ncu, DRAM read + write)",
             "peak_source": peaks["source"], "launches_per_replica_step": n_launch,
