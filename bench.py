@@ -798,7 +798,8 @@ def roofline(kernels, model, host, cfg, peaks):
 
 def bench_e2e(model, host, dev, graphs, cfg, K, W, args):
     """Same metric with the step's inputs in pinned host memory: every step copies its batch host->device
-    into the ring slot's device buffers, replays that slot's captured step and reads the loss back.  Host wall
+    into the ring slot's device buffers (on a copy stream, so the copy of a later step overlaps the kernels of an
+    earlier one), replays that slot's captured step once the copy has landed and reads the loss back.  Host wall
     clock around exactly K steps (ending with a synchronise of every replica stream), the region repeated until
     half of args.min_seconds has been timed; the median region gives the value."""
     import torch
@@ -810,18 +811,32 @@ def bench_e2e(model, host, dev, graphs, cfg, K, W, args):
     ring = len(dev[0])
     paced = cfg.sync_every
 
+    # A copy stream per replica prefetches: the copies of step t go out as soon as the step that used the ring slot
+    # before (t - ring) has finished, not behind step t - 1, so they overlap this replica's own kernels.
+    copy_streams = [torch.cuda.Stream(device=rep.stream.device) for rep in model.replicas]
+    slot_free = [[None] * ring for _ in range(cfg.R)]          # recorded after the step that read the slot
+    slot_ready = [[torch.cuda.Event() for _ in range(ring)] for _ in range(cfg.R)]
+
     def step(t):
         nonlocal h2d, d2h
         for r, rep in enumerate(model.replicas):
             slot = t % ring
             src, dst = pinned[r][slot], dev[r][slot]
-            with torch.cuda.stream(rep.stream):
+            with torch.cuda.stream(copy_streams[r]):
+                if slot_free[r][slot] is not None:
+                    copy_streams[r].wait_event(slot_free[r][slot])
                 dst.indices.copy_(src[0], non_blocking=True)
                 dst.offsets.copy_(src[1], non_blocking=True)
                 dst.dense.copy_(src[2], non_blocking=True)
                 dst.labels.copy_(src[3], non_blocking=True)
+                slot_ready[r][slot].record(copy_streams[r])
+            with torch.cuda.stream(rep.stream):
+                rep.stream.wait_event(slot_ready[r][slot])
                 graphs[r][slot].replay()
                 loss_host[r].copy_(rep.loss, non_blocking=True)
+                if slot_free[r][slot] is None:
+                    slot_free[r][slot] = torch.cuda.Event()
+                slot_free[r][slot].record(rep.stream)
             h2d += sum(x.numel() * x.element_size() for x in src)
             d2h += 4
         if paced and (t + 1) % paced == 0:
