@@ -925,9 +925,19 @@ ss_status gemm_tc_flow(const TcJob* jobs, int n, int* ctrl, int max_rows, int ma
   }
   int* err = device_error_ptr();
   if (!err) return SS_ERR_CUDA;
-  // 128 x 256 tiles where the flow fills the SMs with them (a narrower product then has one partly empty tile per row
-  // block); 256 x 256 tiles on CTA pairs where, in addition, every product is at least that wide, no product waits for
-  // another (tiles then go round-robin) and there is no K slicing
+  // A flow with dependencies keeps CTAs waiting for one another, and a CTA, waiting or not, holds its SM's shared
+  // memory and a third of its registers, which the other streams' kernels then lack.  Measured with all replicas of
+  // a model training at once (examples/s at 16 / 32 / 64 / 148 CTAs per flow): four replicas, batch 2048: 15.0 /
+  // 16.0 / 15.2 / 13.4 M; eight replicas, batch 1024: 13.1 / 13.6 / 12.6 / 11.8 M; sixteen replicas of a model ten
+  // times as large, batch 4096: 7.9 / 8.4 / 7.0 / 7.2 M -- while a flow alone on the device is fastest with a CTA on
+  // every SM.  So a flow takes 32 CTAs unless the caller says otherwise (set_flow_ctas).
+  int ctas = num_sms();
+  if (ctrl && max_ctas <= 0) max_ctas = g_flow_ctas > 0 ? g_flow_ctas : kFlowCtasDefault;
+  if (max_ctas > 0 && max_ctas < ctas) ctas = max_ctas;
+  // 128 x 256 tiles where the flow has at least one of them for each of its CTAs (a third less shared-memory traffic
+  // per flop than 128 x 128; a narrower product then has one partly empty tile per row block); 256 x 256 tiles on
+  // CTA pairs where, in addition, every product is at least that wide, no product waits for another (tiles then go
+  // round-robin) and there is no K slicing
   long long t256 = 0, t_pair = 0;
   bool pair = ctrl == nullptr;
   for (int i = 0; i < n; ++i) {
@@ -936,7 +946,7 @@ ss_status gemm_tc_flow(const TcJob* jobs, int n, int* ctrl, int max_rows, int ma
     t_pair += (long long)((jobs[i].N + 255) / 256) * ((jobs[i].M + 2 * kBM - 1) / (2 * kBM));
     if (ks > 1 || jobs[i].dep >= 0 || jobs[i].N < 256) pair = false;
   }
-  const bool wide = t256 >= num_sms();
+  const bool wide = t256 >= ctas;
   pair = pair && wide && t_pair >= num_sms() / 2;
   const int bn = wide ? 256 : 128;
   alignas(64) TcFlow<kTcMaxFlow> f;
@@ -960,15 +970,6 @@ ss_status gemm_tc_flow(const TcJob* jobs, int n, int* ctrl, int max_rows, int ma
   f.ctrl = ctrl;
   f.rb_stride = (max_rows + kBM - 1) / kBM + 1;    // per product: one word per row block, then their total
   f.err = err;
-  // A flow with dependencies keeps CTAs waiting for one another, and a CTA, waiting or not, holds its SM's shared
-  // memory and a third of its registers, which the other streams' kernels then lack.  Measured with all replicas of
-  // a model training at once (examples/s at 16 / 32 / 64 / 148 CTAs per flow): four replicas, batch 2048: 15.0 /
-  // 16.0 / 15.2 / 13.4 M; eight replicas, batch 1024: 13.1 / 13.6 / 12.6 / 11.8 M; sixteen replicas of a model ten
-  // times as large, batch 4096: 7.9 / 8.4 / 7.0 / 7.2 M -- while a flow alone on the device is fastest with a CTA on
-  // every SM.  So a flow takes 32 CTAs unless the caller says otherwise (set_flow_ctas).
-  int ctas = num_sms();
-  if (ctrl && max_ctas <= 0) max_ctas = g_flow_ctas > 0 ? g_flow_ctas : kFlowCtasDefault;
-  if (max_ctas > 0 && max_ctas < ctas) ctas = max_ctas;
   if (pair) {
     ctas &= ~1;                                            // whole pairs
     if (2 * total < ctas) ctas = 2 * total;
