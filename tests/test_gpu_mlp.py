@@ -112,6 +112,29 @@ def test_mlp_bf16_medium_shapes_reduced_batch():
     _check(cfg, seed=5)
 
 
+def test_mlp_results_do_not_depend_on_how_many_ctas_the_persistent_launches_take():
+    """All tensor-core products of a pass run in one launch whose CTAs draw tiles in ticket order and wait, inside the
+    launch, for the tiles they depend on.  A tile's arithmetic is fixed, so the outputs are bit-identical whether one
+    CTA works through all tickets (every dependency is then on the same CTA's own earlier tiles), a handful do, or
+    one per SM; no wait runs out."""
+    cfg = synth.scaled(synth.CONFIGS["medium"], B=1000)      # eight row blocks, the last one ragged
+    layers, dense, pooled, labels = _setup(cfg, seed=11)
+    ref = None
+    try:
+        for ctas in (1, 3, 32, 1000):
+            assert ss.ss_mlp_set_flow_ctas(ctas) == ctas
+            g = _gpu_fwd_bwd(cfg, layers, dense, pooled, labels, apply_update=0)
+            assert ss.ss_device_error() == 0
+            if ref is None:
+                ref = g
+                continue
+            for k in ("logit", "prob", "concat", "grads", "gp"):
+                assert np.array_equal(ref[k], g[k]), f"{k} differs between 1 CTA and {ctas}"
+            assert ref["loss"] == g["loss"]
+    finally:
+        assert ss.ss_mlp_set_flow_ctas(0) == 32               # back to the library's default
+
+
 def test_mlp_bf16_large_shapes_full_batch():
     """Configuration 4's MLP at its full batch of 4096: products of 2^33 flop and more take the 128 x 256 tiles, as
     single launches (forward, input gradients) and as the grouped weight-gradient launch.
