@@ -804,8 +804,7 @@ def bench_e2e(model, host, dev, graphs, cfg, K, W, args):
     half of args.min_seconds has been timed; the median region gives the value."""
     import torch
     from paper_2003_03477_b200 import trainer
-    pinned = [[tuple(torch.from_numpy(np.ascontiguousarray(a)).pin_memory() for a in
-                     (b.indices, b.offsets, b.dense, b.labels)) for b in bs] for bs in host]
+    pinned = [[trainer.DeviceBatch.pack_host(b.indices, b.offsets, b.dense, b.labels) for b in bs] for bs in host]
     loss_host = [torch.zeros(1).pin_memory() for _ in range(cfg.R)]
     h2d = d2h = 0
     ring = len(dev[0])
@@ -825,10 +824,7 @@ def bench_e2e(model, host, dev, graphs, cfg, K, W, args):
             with torch.cuda.stream(copy_streams[r]):
                 if slot_free[r][slot] is not None:
                     copy_streams[r].wait_event(slot_free[r][slot])
-                dst.indices.copy_(src[0], non_blocking=True)
-                dst.offsets.copy_(src[1], non_blocking=True)
-                dst.dense.copy_(src[2], non_blocking=True)
-                dst.labels.copy_(src[3], non_blocking=True)
+                dst.storage.copy_(src, non_blocking=True)    # indices, offsets, dense features and labels in one copy
                 slot_ready[r][slot].record(copy_streams[r])
             with torch.cuda.stream(rep.stream):
                 rep.stream.wait_event(slot_ready[r][slot])
@@ -837,7 +833,7 @@ def bench_e2e(model, host, dev, graphs, cfg, K, W, args):
                 if slot_free[r][slot] is None:
                     slot_free[r][slot] = torch.cuda.Event()
                 slot_free[r][slot].record(rep.stream)
-            h2d += sum(x.numel() * x.element_size() for x in src)
+            h2d += src.numel()
             d2h += 4
         if paced and (t + 1) % paced == 0:
             model.sync(**sync_args(cfg))

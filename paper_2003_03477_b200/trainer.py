@@ -20,17 +20,47 @@ from . import binding as ss
 
 
 class DeviceBatch:
-    """One batch resident on the device."""
+    """One batch resident on the device.  The four arrays are views of ONE device buffer (`storage`, each array on a
+    256-byte boundary), so a batch staged on the host in the same layout (`pack_host`) arrives with a single copy."""
+
+    FIELDS = (("indices", torch.int32), ("offsets", torch.int32), ("dense", torch.float32), ("labels", torch.float32))
+
+    @staticmethod
+    def _layout(arrays):
+        offs, o = [], 0
+        for a in arrays:
+            offs.append(o)
+            o += (a.numel() * a.element_size() + 255) // 256 * 256
+        return offs, o
+
+    @classmethod
+    def _as_tensors(cls, indices, offsets, dense, labels):
+        out = []
+        for a, (_, dt) in zip((indices, offsets, dense, labels), cls.FIELDS):
+            t = a if isinstance(a, torch.Tensor) else torch.from_numpy(np.ascontiguousarray(a))
+            out.append(t.to(dtype=dt).contiguous())
+        return out
+
+    @classmethod
+    def pack_host(cls, indices, offsets, dense, labels):
+        """The batch in the layout of `storage`, in pinned host memory."""
+        ts = cls._as_tensors(indices, offsets, dense, labels)
+        offs, total = cls._layout(ts)
+        buf = torch.zeros(total, dtype=torch.uint8).pin_memory()
+        for t, o in zip(ts, offs):
+            n = t.numel() * t.element_size()
+            buf[o:o + n] = t.cpu().reshape(-1).view(torch.uint8)
+        return buf
 
     def __init__(self, indices, offsets, dense, labels, device="cuda"):
-        def dev(a, dt):
-            if isinstance(a, torch.Tensor):
-                return a.to(device=device, dtype=dt, non_blocking=True)
-            return torch.from_numpy(np.ascontiguousarray(a)).to(device=device, dtype=dt)
-        self.indices = dev(indices, torch.int32)
-        self.offsets = dev(offsets, torch.int32)
-        self.dense = dev(dense, torch.float32)
-        self.labels = dev(labels, torch.float32)
+        ts = self._as_tensors(indices, offsets, dense, labels)
+        offs, total = self._layout(ts)
+        self.storage = torch.zeros(total, dtype=torch.uint8, device=device)
+        for t, o, (name, dt) in zip(ts, offs, self.FIELDS):
+            n = t.numel() * t.element_size()
+            view = self.storage[o:o + n].view(dt).view(t.shape)
+            view.copy_(t.to(device=device, non_blocking=True) if t.device != view.device else t)
+            setattr(self, name, view)
         self.L = int(self.indices.numel())
 
 
