@@ -1029,9 +1029,11 @@ combine_rows_kernel(const int32_t* __restrict__ seg, const int32_t* __restrict__
   if (!ws_matches(scalars, L, sentinel, nullptr)) return;
   const int n = min(scalars[1], nwin);
   // Spans of up to kShort windows: one lane group per row, which requests kBatch partials at a time and adds them in
-  // window order.  Only the few rows with longer spans (the hottest of a skewed table) take a whole block each: a
-  // block works through its rows one after the other, so that path must stay short.
-  constexpr int kShort = 32;
+  // window order.  Only the rows with longer spans (the hottest of a skewed table) take a whole block each: a
+  // block works through its rows one after the other, so that path must stay short -- but a lane group walking a
+  // long span is a chain of dependent rounds at the kernel's tail: of 2 / 4 / 8 / 32 / 128 windows, 8 was the
+  // fastest (the call 66.7 us against 69.5 with 32 and 89.8 with 128).
+  constexpr int kShort = 8;
   constexpr int kBatch = NV <= 1 ? 8 : (NV <= 2 ? 4 : 2);
   // phase A
   for (int i = blockIdx.x * kGroups + grp; i < n; i += gridDim.x * kGroups) {
