@@ -1035,8 +1035,17 @@ combine_rows_kernel(const int32_t* __restrict__ seg, const int32_t* __restrict__
   // fastest (the call 66.7 us against 69.5 with 32 and 89.8 with 128).
   constexpr int kShort = 8;
   constexpr int kBatch = NV <= 1 ? 8 : (NV <= 2 ? 4 : 2);
+  // The two phases are two chains of dependent loads; with enough blocks the first half of the grid takes the long
+  // spans (phase B) and the second half the short ones (phase A), so that the chains run side by side instead of
+  // one after the other.  A small grid does both in every block.
+  const int nb_long = gridDim.x >= 4 ? (int)gridDim.x / 2 : 0;
+  const bool do_short = nb_long == 0 || (int)blockIdx.x >= nb_long;
+  const bool do_long = nb_long == 0 || (int)blockIdx.x < nb_long;
+  const int a_blk = nb_long == 0 ? (int)blockIdx.x : (int)blockIdx.x - nb_long;
+  const int a_blocks = nb_long == 0 ? (int)gridDim.x : (int)gridDim.x - nb_long;
+  const int b_blocks = nb_long == 0 ? (int)gridDim.x : nb_long;
   // phase A
-  for (int i = blockIdx.x * kGroups + grp; i < n; i += gridDim.x * kGroups) {
+  for (int i = a_blk * kGroups + grp; do_short && i < n; i += a_blocks * kGroups) {
     const int u = long_list[i];
     if (u < 0 || u >= umax) continue;
     const int s0 = seg[u], s1 = seg[u + 1];
@@ -1081,11 +1090,11 @@ combine_rows_kernel(const int32_t* __restrict__ seg, const int32_t* __restrict__
   // its threads look at 256 of them at a time (one round of loads) and queue the long ones.
   __shared__ int s_long[256];
   __shared__ int s_nlong;
-  for (int64_t base = 0; (int64_t)blockIdx.x + base * gridDim.x < n; base += 256) {
+  for (int64_t base = 0; do_long && (int64_t)blockIdx.x + base * b_blocks < n; base += 256) {
     if (threadIdx.x == 0) s_nlong = 0;
     __syncthreads();
     {
-      const int64_t i = (int64_t)blockIdx.x + (base + threadIdx.x) * gridDim.x;
+      const int64_t i = (int64_t)blockIdx.x + (base + threadIdx.x) * b_blocks;
       if (i < n) {
         const int u = long_list[i];
         if (u >= 0 && u < umax) {
